@@ -1,0 +1,227 @@
+/*
+ * gear.h -- C ABI of libgear: the sparse-part training step of Gear Training
+ * (arXiv 1806.03925) on one NVIDIA B200 (sm_100a), with the Dense Part replaced
+ * by a table of cached Dense Feature Vectors (DFVs).
+ *
+ * The calls follow the paper's Section 3 event list (events 1-6) and the two
+ * cache rules of Section 1 ("inference expired time", "accumulated to M"):
+ *
+ *   gear_init_tables          cluster start-up: the DFV cache, the gradient
+ *                             store and the embedding tables exist and are warm.
+ *   gear_forward_backward     events 1, 3, 4: fetch DFVs by Image ID, Sparse
+ *                             Part forward to the loss, backward through the
+ *                             Sparse Part only, stopping at dLoss/dDFV (Eq. 1,
+ *                             left factor); apply the embedding gradients.
+ *   gear_accumulate_dfv_grad  event 5 and the first half of event 6: (Image
+ *                             ID, gradient) pairs arrive and are summed per
+ *                             image; every M-th arrival completes a group.
+ *   gear_collect_ready        event 6: hand over the averaged gradient of
+ *                             every completed group.
+ *   gear_collect_expired      Section 1 / Section 3: cached inference results
+ *                             older than the inference-expired time.
+ *
+ * General rules
+ *   - Every function returns GEAR_OK (0) or a negative GEAR_ERR_* code.  None
+ *     throws, exits or traps the device.
+ *   - All device work is enqueued on the caller's stream (`stream` is a
+ *     cudaStream_t passed as void*; NULL is the default stream).  A call
+ *     blocks the host only when a host out-pointer (h_n) is non-NULL, in
+ *     gear_status, and in gear_init_tables / gear_destroy.
+ *   - Ownership: every table, every input and output array and the workspace
+ *     are DEVICE memory allocated and owned by the caller.  The library
+ *     allocates no device memory.  The gear_ctx is host memory owned by the
+ *     library and released by gear_destroy.  Structs passed by pointer are
+ *     HOST memory and are copied during the call.
+ *   - Layout: all matrices are row-major and dense unless a leading dimension
+ *     is given.  IDs are int32; an ID outside [0, vocab) is ignored (its row
+ *     counts as zeros / its gradient is dropped) and raises the sticky
+ *     GEAR_DEV_BAD_ID bit of the device status word.
+ *   - Calls on one ctx must be issued from one host thread at a time and on
+ *     one stream (or on streams the caller orders with events).
+ */
+#ifndef GEAR_H
+#define GEAR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    GEAR_OK = 0,
+    GEAR_ERR_ARG = -1,       /* NULL pointer, bad dimension, misaligned buffer, batch larger than configured */
+    GEAR_ERR_CAPACITY = -2,  /* an output list or the ready queue is too small; nothing was consumed */
+    GEAR_ERR_BAD_ID = -3,    /* an out-of-range ID was met (reported by gear_status; the row was skipped) */
+    GEAR_ERR_CUDA = -4,      /* a CUDA runtime or driver call failed */
+    GEAR_ERR_STATE = -5      /* call order violated (e.g. ctx destroyed) */
+};
+
+/* element types of tables and of the head's matrix-product operands */
+enum { GEAR_F32 = 0, GEAR_BF16 = 1 };
+
+/* how gear_accumulate_dfv_grad combines rows that share an Image ID */
+enum {
+    GEAR_ACC_SORT = 0,       /* stable key sort + segmented reduction: groups split exactly at every
+                                M-th arrival in row order; deterministic */
+    GEAR_ACC_ATOMIC = 1      /* fp32 atomic adds on the accumulator rows: arrival order (hence group
+                                membership) is whatever the hardware makes it; counts and emission
+                                counts still match the sorted path */
+};
+
+/* bits of the device status word (sticky until gear_status clears them) */
+enum {
+    GEAR_DEV_BAD_ID = 1,         /* an ID outside [0, vocab) was skipped */
+    GEAR_DEV_READY_OVERFLOW = 2, /* an accumulate call would have overflowed the ready queue and was dropped whole */
+    GEAR_DEV_OUT_CAPACITY = 4,   /* a collect call found cap too small and left everything in place */
+    GEAR_DEV_BAD_CSR = 8         /* img_off not non-decreasing / not ending at nnz */
+};
+
+/* tags of the procedural table fill (SplitMix64 streams, see gear_fill_uniform) */
+enum { GEAR_TAG_USER = 1, GEAR_TAG_URL = 2, GEAR_TAG_DFV = 3, GEAR_TAG_TS = 4, GEAR_TAG_GRAD = 5 };
+
+typedef struct gear_ctx gear_ctx;
+
+/* Static description of one model + store.  Validated by gear_init_tables. */
+typedef struct {
+    int64_t user_vocab, url_vocab, img_vocab; /* each in [1, 2^31 - 2] */
+    int32_t emb_dim;       /* columns of the user and URL-hash tables (fp32); multiple of 4, <= 1024 */
+    int32_t dfv_dim;       /* columns of the DFV table; multiple of 8, <= 1024 */
+    int32_t dfv_dtype;     /* GEAR_F32 | GEAR_BF16: storage type of the DFV table */
+    int32_t head_dtype;    /* GEAR_F32: fp32 FMA head.  GEAR_BF16: operands of the head's matrix products
+                              (head input, weights, hidden activations, activation gradients) are rounded
+                              to bfloat16 (nearest-even); products accumulate in fp32 */
+    int32_t n_hidden;      /* 1 or 2 hidden ReLU layers; the output layer is one logistic unit */
+    int32_t hidden[2];     /* widths; multiples of 8 (GEAR_F32) or 64 (GEAR_BF16), <= 1024 */
+    int32_t M;             /* gradients per image per emitted average, >= 1 */
+    int64_t expire;        /* inference-expired time, >= 0, in the caller's time unit */
+    int32_t max_batch;     /* largest B of any gear_forward_backward call */
+    int64_t max_nnz;       /* largest number of rows of any forward_backward / accumulate call */
+    int64_t ready_cap;     /* rows of the ready queue (averages waiting for gear_collect_ready);
+                              0 = max_nnz, which can never overflow if every accumulate call is
+                              followed by a collect */
+    int32_t accum_mode;    /* GEAR_ACC_SORT | GEAR_ACC_ATOMIC */
+} gear_config;
+
+/* Caller-owned device buffers that persist across calls. */
+typedef struct {
+    float*    user_emb;     /* [user_vocab][emb_dim] fp32 */
+    float*    url_emb;      /* [url_vocab][emb_dim]  fp32 */
+    void*     dfv;          /* [img_vocab][dfv_dim]  dfv_dtype; rows 16-byte aligned */
+    float*    dfv_gsum;     /* [img_vocab][dfv_dim]  fp32 running sum of the open group of each image */
+    int32_t*  dfv_gcnt;     /* [img_vocab]           arrivals in the open group, always in [0, M) */
+    int64_t*  dfv_ts;       /* [img_vocab]           time the cached DFV was computed */
+    float*    head_params;  /* packed fp32: per hidden layer W[in][out] then b[out]; then w_out[in], b_out.
+                               Read at every gear_forward_backward; never written by the library */
+    void*     workspace;    /* scratch, 256-byte aligned, >= gear_workspace_bytes; contents belong to the ctx */
+    size_t    workspace_bytes;
+} gear_buffers;
+
+/* One batch of page views (Table 1 of the paper) in CSR form; device pointers. */
+typedef struct {
+    int32_t B;                 /* views, 0 <= B <= max_batch */
+    int64_t nnz;               /* image occurrences, = img_off[B], <= max_nnz */
+    const int32_t* user_id;    /* [B] */
+    const int32_t* url_id;     /* [B]  URL already hashed to a bucket */
+    const int32_t* img_off;    /* [B+1] img_off[0] = 0, non-decreasing, img_off[B] = nnz */
+    const int32_t* img_id;     /* [nnz] view-major, slot-minor */
+    const float*   label;      /* [B]  0 or 1 */
+} gear_batch;
+
+/* Outputs of one step; device pointers.  "optional" ones may be NULL. */
+typedef struct {
+    float* loss;        /* [1]  mean binary cross-entropy over the batch */
+    float* prob;        /* [B]  sigmoid of the logit; optional */
+    float* head_grad;   /* packed like head_params: dLoss/dparams (not applied by the library) */
+    float* dX;          /* [B][2*emb_dim + dfv_dim] dLoss/d(head input).  Columns [2*emb_dim, ...) are
+                           dLoss/d(pooled DFV) of each view: pass dX + 2*emb_dim with ld = 2*emb_dim + dfv_dim
+                           to gear_accumulate_dfv_grad */
+    int32_t* row_view;  /* [nnz] view index of every image occurrence (the src_row of accumulate); optional */
+    float*   inv_n;     /* [B]   1/n_b, the mean-pool weight (the scale of accumulate); optional */
+    void*  x_debug;     /* [B][2*emb_dim + dfv_dim] copy of the head input in head_dtype; optional */
+    float* user_grad;   /* [user_vocab][emb_dim] optional: the summed embedding gradient is ADDED here and the */
+    float* url_grad;    /* [url_vocab][emb_dim]  table is left untouched (both or neither) */
+} gear_step_out;
+
+/* Bytes of workspace a ctx with this configuration needs.  Host-only. */
+int gear_workspace_bytes(const gear_config* cfg, size_t* out_bytes);
+
+/*
+ * Create a ctx.  fill = 0: keep the caller's table contents (dfv_gcnt must be
+ * in [0, M)).  fill = 1: user/url/DFV tables get the procedural uniform fill
+ * with standard deviation 0.1 (the paper's initial value for all variables),
+ * tags GEAR_TAG_USER/URL/DFV; dfv_gsum and dfv_gcnt are zeroed; dfv_ts[id] =
+ * now - (draw(seed, GEAR_TAG_TS, id) mod max(expire, 1)).  The workspace is
+ * initialised in both cases.  Synchronises the stream before returning.
+ */
+int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buffers* buf,
+                     uint64_t seed, int fill, int64_t now, void* stream);
+
+/*
+ * Events 1, 3, 4.  X[b] = [user_emb[user_id[b]] | url_emb[url_id[b]] | mean_j DFV[img_id[j]]] (fp32 sum
+ * in slot order, divided by n_b; zeros for n_b = 0); hidden layers h = ReLU(h W + b); z = h . w_out + b_out;
+ * p = sigmoid(z); loss = mean_b BCE(p_b, label_b).  Backward yields head_grad and dX.  Then, per
+ * embedding table, rows of views sharing an ID are summed and table[id] -= lr * sum (or the sums are
+ * added to user_grad / url_grad when those are given).
+ */
+int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, const gear_step_out* out,
+                          void* stream);
+
+/*
+ * Event 5 + 6a.  Row r (0 <= r < n) carries Image ID img_id[r] and the gradient
+ *     g_r[c] = grads[s * ld + c] * (scale ? scale[s] : 1),  s = src_row ? src_row[r] : r,  c < dfv_dim.
+ * Rows are taken to arrive in index order.  Per image: dfv_gsum += g_r, dfv_gcnt += 1; when the count
+ * reaches M the group's average (sum / M, fp32) joins the ready queue and sum and count restart at 0;
+ * a call may complete several groups of one image.  grads rows must be 16-byte aligned (ld multiple of 4).
+ * If the queue cannot take every group the call completes, the whole call is dropped and
+ * GEAR_DEV_READY_OVERFLOW is raised.
+ */
+int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* grads, int64_t ld,
+                             const int32_t* src_row, const float* scale, int64_t n, void* stream);
+
+/*
+ * Event 6b.  Moves the ready queue to (ids[k], seq[k], avg[k][dfv_dim]), k < n, sorted by (id, seq);
+ * seq numbers the emissions of one image since the previous collect, in arrival order.  The count is
+ * written to *d_n (device, optional) and *h_n (host, optional: the call then synchronises).  If the queue
+ * holds more than cap entries nothing is moved, the required count is reported, GEAR_DEV_OUT_CAPACITY is
+ * raised and (when h_n is given) GEAR_ERR_CAPACITY is returned.
+ */
+int gear_collect_ready(gear_ctx* ctx, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
+                       int64_t* d_n, int64_t* h_n, void* stream);
+
+/*
+ * Expiry scan.  Lists, in ascending order, every image with now - dfv_ts[id] >= expire; with
+ * restamp != 0 the listed entries get dfv_ts[id] = now (a refresh has been requested).  Count and
+ * capacity behaviour as in gear_collect_ready (too small: nothing listed, nothing restamped).
+ */
+int gear_collect_expired(gear_ctx* ctx, int64_t now, int restamp, int32_t* ids, int64_t cap,
+                         int64_t* d_n, int64_t* h_n, void* stream);
+
+/*
+ * Synchronises the stream last used; returns the device status word (GEAR_DEV_* bits, then cleared) and
+ * the number of averages waiting in the ready queue.  Either out-pointer may be NULL.  Returns
+ * GEAR_ERR_BAD_ID if GEAR_DEV_BAD_ID was set, GEAR_ERR_CAPACITY for the two capacity bits, else GEAR_OK.
+ */
+int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready);
+
+/* Releases the ctx (host memory only).  Synchronises the stream last used. */
+int gear_destroy(gear_ctx* ctx);
+
+/*
+ * Procedural fill used by gear_init_tables, exposed for building synthetic inputs on the device.
+ * Element (r, c) of a [n_rows][dim] array is  float(k - 2^23) * float(amp / 2^23)  with
+ * k = top 24 bits of draw(seed, tag, r * dim + c), draw(seed, tag, i) = mix(mix(seed + G*(tag+1)) + G*(i+1)),
+ * mix = the SplitMix64 finaliser and G = 0x9e3779b97f4a7c15 (Steele, Lea, Flood 2014); bf16 output is
+ * the nearest-even rounding of that float.  Not part of the paper.  dst: device, 16-byte aligned.
+ */
+int gear_fill_uniform(void* dst, int32_t dtype, int64_t n_rows, int32_t dim, uint64_t seed, uint64_t tag,
+                      double amp, void* stream);
+
+/* Last CUDA error string seen by the library on this thread ("" if none).  Host-only. */
+const char* gear_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GEAR_H */

@@ -143,6 +143,8 @@ class GearOracle:
     def __init__(self, user_emb: np.ndarray, url_emb: np.ndarray, dfv: np.ndarray,
                  hidden: Sequence[int], M: int, expire: int, round_bf16: bool = False,
                  ts: Optional[np.ndarray] = None):
+        """ts may be longer than the DFV table: a test that keeps only the touched rows of a huge
+        table still scans every timestamp."""
         self.user_emb = np.ascontiguousarray(user_emb)
         self.url_emb = np.ascontiguousarray(url_emb)
         self.dfv = np.ascontiguousarray(dfv)
@@ -254,8 +256,8 @@ class GearOracle:
 
     # -- expiry -----------------------------------------------------------------
     def collect_expired(self, now: int, restamp: bool = True) -> np.ndarray:
-        out = np.zeros(self.V, dtype=np.int32)
-        n = lib().orc_collect_expired(_ptr(self.ts), self.V, int(now), self.expire, 1 if restamp else 0,
+        out = np.zeros(len(self.ts), dtype=np.int32)
+        n = lib().orc_collect_expired(_ptr(self.ts), len(self.ts), int(now), self.expire, 1 if restamp else 0,
                                       _ptr(out))
         return out[:n].copy()
 

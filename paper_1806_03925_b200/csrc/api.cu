@@ -1,0 +1,285 @@
+// The C ABI of libgear (see include/gear.h): argument validation, workspace planning and the
+// order in which the kernels of each call are enqueued.  No device memory is allocated here.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace gear {
+
+static thread_local char g_last_error[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* where) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s: %s", where, cudaGetErrorString(e));
+    return GEAR_ERR_CUDA;
+}
+static int arg_fail(const char* what) {
+    snprintf(g_last_error, sizeof(g_last_error), "bad argument: %s", what);
+    return GEAR_ERR_ARG;
+}
+
+static int validate_config(const gear_config& c) {
+    const int64_t vmax = 2147483646ll;
+    if (c.user_vocab < 1 || c.user_vocab > vmax || c.url_vocab < 1 || c.url_vocab > vmax || c.img_vocab < 1 ||
+        c.img_vocab > vmax)
+        return arg_fail("vocabulary sizes must be in [1, 2^31 - 2]");
+    if (c.emb_dim < 4 || c.emb_dim % 4 || c.emb_dim > 1024) return arg_fail("emb_dim: multiple of 4 in [4, 1024]");
+    if (c.dfv_dim < 8 || c.dfv_dim % 8 || c.dfv_dim > 1024) return arg_fail("dfv_dim: multiple of 8 in [8, 1024]");
+    if (c.dfv_dtype != GEAR_F32 && c.dfv_dtype != GEAR_BF16) return arg_fail("dfv_dtype");
+    if (c.head_dtype != GEAR_F32 && c.head_dtype != GEAR_BF16) return arg_fail("head_dtype");
+    if (c.n_hidden < 1 || c.n_hidden > MAX_LAYERS) return arg_fail("n_hidden must be 1 or 2");
+    for (int l = 0; l < c.n_hidden; ++l) {
+        const int mult = c.head_dtype == GEAR_BF16 ? 64 : 8;
+        if (c.hidden[l] < mult || c.hidden[l] % mult || c.hidden[l] > 1024)
+            return arg_fail("hidden widths: multiples of 8 (fp32 head) or 64 (bf16 head), at most 1024");
+    }
+    if (c.M < 1) return arg_fail("M >= 1");
+    if (c.expire < 0) return arg_fail("expire >= 0");
+    if (c.max_batch < 1) return arg_fail("max_batch >= 1");
+    if (c.max_nnz < 1 || c.max_nnz > vmax) return arg_fail("max_nnz in [1, 2^31 - 2]");
+    if (c.ready_cap < 0 || c.ready_cap > vmax) return arg_fail("ready_cap in [0, 2^31 - 2]");
+    if (c.accum_mode != GEAR_ACC_SORT && c.accum_mode != GEAR_ACC_ATOMIC) return arg_fail("accum_mode");
+    return GEAR_OK;
+}
+
+int plan_workspace(const gear_config& c, WsPlan* p) {
+    memset(p, 0, sizeof(*p));
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
+    const size_t hsz = c.head_dtype == GEAR_BF16 ? 2 : 4;
+    const int d_in = 2 * c.emb_dim + c.dfv_dim;
+    const size_t B = (size_t)c.max_batch;
+    p->ready_cap = c.ready_cap > 0 ? c.ready_cap : c.max_nnz;
+    p->sort_cap = c.max_nnz;
+    if (p->sort_cap < c.max_batch) p->sort_cap = c.max_batch;
+    if (p->sort_cap < p->ready_cap) p->sort_cap = p->ready_cap;
+    p->loss_blocks = (int)ceil_div(c.max_batch, 8);
+    if (p->loss_blocks > 592) p->loss_blocks = 592;
+
+    p->state = take(sizeof(DevState));
+    p->x = take(B * d_in * hsz);
+    int fan = d_in;
+    for (int l = 0; l < c.n_hidden; ++l) {
+        p->h[l] = take(B * c.hidden[l] * hsz);
+        p->da[l] = take(B * c.hidden[l] * hsz);
+        p->wb[l] = take((size_t)fan * c.hidden[l] * 2);
+        p->wbt[l] = take((size_t)fan * c.hidden[l] * 2);
+        fan = c.hidden[l];
+    }
+    p->dz = take(B * 4);
+    p->loss_part = take((size_t)p->loss_blocks * 4);
+    for (int i = 0; i < 2; ++i) {
+        p->sort_keys[i] = take((size_t)p->sort_cap * 4);
+        p->sort_vals[i] = take((size_t)p->sort_cap * 4);
+    }
+    p->sort_hist = take((size_t)RS_BUCKETS * sort_tiles(p->sort_cap) * 4);
+    p->sort_tot = take(RS_BUCKETS * 4);
+    p->tile_cnt = take((size_t)(ceil_div(c.max_nnz, 1024) + 1) * sizeof(uint2));
+    p->grp_start = take((size_t)c.max_nnz * 4);
+    p->grp_slot = take((size_t)c.max_nnz * 4);
+    p->q_id = take((size_t)p->ready_cap * 4);
+    p->q_avg = take((size_t)p->ready_cap * c.dfv_dim * 4);
+    p->exp_bits = take((size_t)ceil_div(c.img_vocab, 32) * 4);
+    p->exp_cnt = take((size_t)(ceil_div(c.img_vocab, EXP_TILE) + 1) * sizeof(uint2));
+    p->total = off;
+    return GEAR_OK;
+}
+
+static int64_t param_count(const gear_config& c) {
+    int64_t n = 0, fan = 2 * c.emb_dim + c.dfv_dim;
+    for (int l = 0; l < c.n_hidden; ++l) { n += fan * c.hidden[l] + c.hidden[l]; fan = c.hidden[l]; }
+    return n + fan + 1;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace gear
+
+using namespace gear;
+
+struct gear_ctx { gear_ctx_impl impl; };
+
+extern "C" {
+
+const char* gear_last_error(void) { return g_last_error; }
+
+int gear_workspace_bytes(const gear_config* cfg, size_t* out_bytes) {
+    if (!cfg || !out_bytes) return arg_fail("NULL pointer");
+    int rc = validate_config(*cfg);
+    if (rc != GEAR_OK) return rc;
+    WsPlan p;
+    plan_workspace(*cfg, &p);
+    *out_bytes = p.total;
+    return GEAR_OK;
+}
+
+int gear_fill_uniform(void* dst, int32_t dtype, int64_t n_rows, int32_t dim, uint64_t seed, uint64_t tag, double amp,
+                      void* stream) {
+    if (!dst || n_rows < 0 || dim < 1 || !aligned16(dst)) return arg_fail("gear_fill_uniform");
+    if (dtype != GEAR_F32 && dtype != GEAR_BF16) return arg_fail("dtype");
+    cudaError_t e = launch_fill_uniform(dst, dtype, n_rows * dim, seed, tag, amp, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "gear_fill_uniform");
+}
+
+int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buffers* buf, uint64_t seed, int fill,
+                     int64_t now, void* stream) {
+    if (!out_ctx || !cfg || !buf) return arg_fail("NULL pointer");
+    *out_ctx = nullptr;
+    int rc = validate_config(*cfg);
+    if (rc != GEAR_OK) return rc;
+    if (!buf->user_emb || !buf->url_emb || !buf->dfv || !buf->dfv_gsum || !buf->dfv_gcnt || !buf->dfv_ts ||
+        !buf->head_params || !buf->workspace)
+        return arg_fail("NULL buffer");
+    if (!aligned16(buf->user_emb) || !aligned16(buf->url_emb) || !aligned16(buf->dfv) || !aligned16(buf->dfv_gsum) ||
+        (reinterpret_cast<uintptr_t>(buf->workspace) & 255u))
+        return arg_fail("tables must be 16-byte aligned, the workspace 256-byte aligned");
+    gear_ctx* ctx = new (std::nothrow) gear_ctx;
+    if (!ctx) return arg_fail("out of host memory");
+    gear_ctx_impl& c = ctx->impl;
+    c.cfg = *cfg;
+    c.buf = *buf;
+    plan_workspace(*cfg, &c.ws);
+    if (buf->workspace_bytes < c.ws.total) { delete ctx; return arg_fail("workspace too small"); }
+    c.d_in = 2 * cfg->emb_dim + cfg->dfv_dim;
+    c.n_params = param_count(*cfg);
+    c.alive = true;
+    c.tc_state = nullptr;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.last_stream = st;
+
+    cudaError_t e = cudaMemsetAsync(c.state(), 0, sizeof(DevState), st);
+    if (e == cudaSuccess && fill) {
+        const double amp = 0.17320508075688773;   // uniform half-width for standard deviation 0.1
+        e = launch_fill_uniform(buf->user_emb, GEAR_F32, cfg->user_vocab * cfg->emb_dim, seed, GEAR_TAG_USER, amp, st);
+        if (e == cudaSuccess)
+            e = launch_fill_uniform(buf->url_emb, GEAR_F32, cfg->url_vocab * cfg->emb_dim, seed, GEAR_TAG_URL, amp, st);
+        if (e == cudaSuccess)
+            e = launch_fill_uniform(buf->dfv, cfg->dfv_dtype, cfg->img_vocab * cfg->dfv_dim, seed, GEAR_TAG_DFV, amp, st);
+        if (e == cudaSuccess)
+            e = cudaMemsetAsync(buf->dfv_gsum, 0, sizeof(float) * (size_t)cfg->img_vocab * cfg->dfv_dim, st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(buf->dfv_gcnt, 0, sizeof(int32_t) * (size_t)cfg->img_vocab, st);
+        if (e == cudaSuccess) e = launch_fill_ts(buf->dfv_ts, cfg->img_vocab, seed, cfg->expire, now, st);
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { delete ctx; return cuda_fail(e, "gear_init_tables"); }
+    *out_ctx = ctx;
+    return GEAR_OK;
+}
+
+int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, const gear_step_out* out, void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    if (!batch || !out) return arg_fail("NULL pointer");
+    gear_ctx_impl& c = ctx->impl;
+    const gear_batch& b = *batch;
+    const gear_step_out& o = *out;
+    if (b.B < 0 || b.B > c.cfg.max_batch) return arg_fail("B outside [0, max_batch]");
+    if (b.nnz < 0 || b.nnz > c.cfg.max_nnz) return arg_fail("nnz outside [0, max_nnz]");
+    if (b.B > 0 && (!b.user_id || !b.url_id || !b.img_off || !b.label)) return arg_fail("NULL batch array");
+    if (b.nnz > 0 && !b.img_id) return arg_fail("NULL img_id");
+    if (!o.loss || !o.head_grad || !o.dX) return arg_fail("loss, head_grad and dX are required outputs");
+    if ((o.user_grad == nullptr) != (o.url_grad == nullptr)) return arg_fail("user_grad and url_grad: both or neither");
+    if (!aligned16(o.dX) || (o.x_debug && !aligned16(o.x_debug)) || (o.user_grad && !aligned16(o.user_grad)) ||
+        (o.url_grad && !aligned16(o.url_grad)))
+        return arg_fail("dX, x_debug, user_grad, url_grad must be 16-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.last_stream = st;
+
+    cudaError_t e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
+    if (e != cudaSuccess) return cuda_fail(e, "gather");
+    e = launch_head_simt(c, b, o, st);
+    if (e != cudaSuccess) return cuda_fail(e, "head");
+    const int E = c.cfg.emb_dim;
+    float* ut = o.user_grad ? o.user_grad : c.buf.user_emb;
+    float* ht = o.url_grad ? o.url_grad : c.buf.url_emb;
+    const float alpha = o.user_grad ? 1.0f : -lr;
+    e = launch_emb_scatter(c, b.user_id, b.B, c.cfg.user_vocab, ut, o.dX, c.d_in, 0, alpha, st);
+    if (e != cudaSuccess) return cuda_fail(e, "user embedding scatter");
+    e = launch_emb_scatter(c, b.url_id, b.B, c.cfg.url_vocab, ht, o.dX, c.d_in, E, alpha, st);
+    if (e != cudaSuccess) return cuda_fail(e, "url embedding scatter");
+    return GEAR_OK;
+}
+
+int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* grads, int64_t ld,
+                             const int32_t* src_row, const float* scale, int64_t n, void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (n < 0 || n > c.cfg.max_nnz) return arg_fail("n outside [0, max_nnz]");
+    if (n == 0) return GEAR_OK;
+    if (!img_id || !grads) return arg_fail("NULL pointer");
+    if (ld < c.cfg.dfv_dim || ld % 4 || !aligned16(grads)) return arg_fail("grads rows must be 16-byte aligned, ld >= dfv_dim");
+    if (c.cfg.accum_mode != GEAR_ACC_SORT) return arg_fail("accum_mode not available");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.last_stream = st;
+    cudaError_t e = launch_accumulate(c, img_id, grads, ld, src_row, scale, n, st);
+    return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "accumulate");
+}
+
+static int finish_count(gear_ctx_impl& c, const int64_t* d_src, int64_t cap, int64_t* h_n, cudaStream_t st) {
+    if (!h_n) return GEAR_OK;
+    cudaError_t e = cudaMemcpyAsync(h_n, d_src, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "read count");
+    if (*h_n > cap) {
+        snprintf(g_last_error, sizeof(g_last_error), "capacity %lld too small, %lld entries waiting", (long long)cap,
+                 (long long)*h_n);
+        return GEAR_ERR_CAPACITY;
+    }
+    return GEAR_OK;
+}
+
+int gear_collect_ready(gear_ctx* ctx, int32_t* ids, int32_t* seq, float* avg, int64_t cap, int64_t* d_n, int64_t* h_n,
+                       void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (cap < 0 || (cap > 0 && (!ids || !seq || !avg))) return arg_fail("NULL output with cap > 0");
+    if (avg && !aligned16(avg)) return arg_fail("avg must be 16-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.last_stream = st;
+    // the count is staged in the device state so that h_n can be served even when d_n is NULL
+    int64_t* d_cnt = d_n ? d_n : &c.state()->pad[0];
+    cudaError_t e = launch_collect_ready(c, ids, seq, avg, cap, d_cnt, st);
+    if (e != cudaSuccess) return cuda_fail(e, "collect_ready");
+    return finish_count(c, d_cnt, cap, h_n, st);
+}
+
+int gear_collect_expired(gear_ctx* ctx, int64_t now, int restamp, int32_t* ids, int64_t cap, int64_t* d_n,
+                         int64_t* h_n, void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (cap < 0 || (cap > 0 && !ids)) return arg_fail("NULL output with cap > 0");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.last_stream = st;
+    int64_t* d_cnt = d_n ? d_n : &c.state()->pad[1];
+    cudaError_t e = launch_collect_expired(c, now, restamp, ids, cap, d_cnt, st);
+    if (e != cudaSuccess) return cuda_fail(e, "collect_expired");
+    return finish_count(c, d_cnt, cap, h_n, st);
+}
+
+int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    DevState h;
+    cudaError_t e = cudaStreamSynchronize(c.last_stream);
+    if (e == cudaSuccess) e = cudaMemcpy(&h, c.state(), sizeof(DevState), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && h.status != 0) e = cudaMemset(&c.state()->status, 0, sizeof(int32_t));
+    if (e != cudaSuccess) return cuda_fail(e, "gear_status");
+    if (device_status) *device_status = h.status;
+    if (pending_ready) *pending_ready = h.q_count;
+    if (h.status & GEAR_DEV_BAD_ID) return GEAR_ERR_BAD_ID;
+    if (h.status & (GEAR_DEV_READY_OVERFLOW | GEAR_DEV_OUT_CAPACITY)) return GEAR_ERR_CAPACITY;
+    if (h.status & GEAR_DEV_BAD_CSR) return GEAR_ERR_ARG;
+    return GEAR_OK;
+}
+
+int gear_destroy(gear_ctx* ctx) {
+    if (!ctx) return GEAR_OK;
+    if (!ctx->impl.alive) return GEAR_ERR_STATE;
+    cudaStreamSynchronize(ctx->impl.last_stream);
+    ctx->impl.alive = false;
+    delete ctx;
+    return GEAR_OK;
+}
+
+}  // extern "C"

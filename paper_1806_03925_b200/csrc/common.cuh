@@ -1,0 +1,120 @@
+// Shared device helpers and the internal host-side declarations of libgear.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/gear.h"
+
+namespace gear {
+
+// ---------------------------------------------------------------- device state
+// Lives at the start of the workspace.  Counters are device-resident so that no
+// call has to synchronise to learn a size produced by an earlier kernel.
+struct DevState {
+    int32_t status;        // GEAR_DEV_* bits, sticky
+    int32_t drop_call;     // set by the accumulate planner when the ready queue would overflow
+    int64_t q_count;       // averages waiting in the ready queue
+    int64_t n_valid;       // accumulate: rows with an in-range ID (sorted prefix length)
+    int64_t n_groups;      // accumulate: groups found in this call
+    int64_t n_complete;    // accumulate: groups of this call that reached M
+    int64_t exp_total;     // expiry scan: entries found
+    int64_t collect_n;     // collect_ready: entries moved by the running call
+    int64_t pad[9];
+};
+static_assert(sizeof(DevState) == 128, "DevState layout");
+
+// ---------------------------------------------------------------- small helpers
+__host__ __device__ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+__device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ uint32_t warp_inclusive_scan(uint32_t v) {
+    const unsigned lane = lane_id();
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= (unsigned)o) v += t;
+    }
+    return v;
+}
+
+// Exclusive scan over the threads of a block (blockDim.x a multiple of 32, <= 1024).
+// `scratch` needs 33 words of shared memory.  Returns the exclusive prefix; *total gets the block sum.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch, uint32_t* total) {
+    const unsigned lane = lane_id(), warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    uint32_t inc = warp_inclusive_scan(v);
+    if (lane == 31) scratch[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = lane < nwarp ? scratch[lane] : 0u;
+        uint32_t winc = warp_inclusive_scan(w);
+        scratch[lane] = winc - w;
+        if (lane == 31) scratch[32] = winc;
+    }
+    __syncthreads();
+    uint32_t res = scratch[warp] + inc - v;
+    if (total) *total = scratch[32];
+    __syncthreads();
+    return res;
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+
+__device__ __forceinline__ float4 ld_f4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ void st_f4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+
+// 128-bit load that does not allocate in L1 (streamed data read once)
+__device__ __forceinline__ float4 ld_stream_f4(const float* p) {
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
+// vector reduction: *p += v without a return value (sm_90+)
+__device__ __forceinline__ void red_add_f4(float* p, float4 v) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+
+// ---------------------------------------------------------------- radix sort / scans (prims.cu)
+constexpr int RS_THREADS = 256;
+constexpr int RS_ITEMS = 16;
+constexpr int RS_TILE = RS_THREADS * RS_ITEMS;
+constexpr int RS_BUCKETS = 256;
+
+struct SortBufs {
+    uint32_t* keys[2];
+    uint32_t* vals[2];
+    uint32_t* hist;     // [256][n_tiles(n_max)]
+    uint32_t* tot;      // [256]
+};
+
+inline int64_t sort_tiles(int64_t n_max) { return n_max > 0 ? ceil_div(n_max, RS_TILE) : 1; }
+
+// Stable LSD radix sort of (key, value) pairs on the low `bits` bits of the key.  Input pairs are in
+// bufs.keys[0] / bufs.vals[0]; with identity_vals the first pass uses the element index as value.
+// n_dev (optional, device) caps the element count at min(*n_dev, n_max).  Returns the index (0 or 1)
+// of the buffer pair that holds the sorted result.
+int radix_sort_pairs(const SortBufs& bufs, int64_t n_max, const int64_t* n_dev, int bits, bool identity_vals,
+                     cudaStream_t st);
+
+// In-place exclusive scan of m (a, b) counter pairs by one block; the totals go to total[0..1].
+void scan_pairs(uint2* data, int64_t m, uint2* total, cudaStream_t st);
+
+inline int bits_for(int64_t max_key_inclusive) {
+    int b = 1;
+    while (b < 32 && (int64_t(1) << b) <= max_key_inclusive) ++b;
+    return b;
+}
+
+}  // namespace gear

@@ -1,0 +1,286 @@
+// The Sparse Part's head (event 4) with fp32 FMA matrix products.
+//
+// Used for GEAR_F32 heads, where the 1e-5 tolerance rules out tf32/bf16 tensor-core products, and as the
+// plain-ALU version of the GEAR_BF16 head (operands rounded to bf16, fp32 accumulation).  One generic
+// shared-memory tiled GEMM with strided operands covers the three product shapes of the step:
+//   forward        H_l    = ReLU(H_{l-1} W_l + b_l)
+//   input gradient dH_{l-1} = (dA_l W_l^T) masked by H_{l-1} > 0
+//   weight gradient dW_l  = H_{l-1}^T dA_l           (reduction over the batch, split over blocks)
+#include <type_traits>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace gear {
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+enum { EPI_NONE = 0, EPI_BIAS_RELU = 1, EPI_MASK = 2, EPI_ATOMIC = 3 };
+
+constexpr int GT = 64;    // tile edge in M and N
+constexpr int GK = 16;    // tile depth
+
+// C[m][n] (+)= epi( sum_k A(m,k) * B(k,n) ),  A(m,k) = A[m*sam + k*sak],  B(k,n) = B[k*sbk + n*sbn].
+// blockIdx.z selects a k-range of k_chunk elements (EPI_ATOMIC adds the partial products into C).
+template <typename TA, typename TB, typename TC, typename TM, int EPI>
+__global__ void __launch_bounds__(256)
+gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sam, int64_t sak,
+            const TB* __restrict__ Bm, int64_t sbk, int64_t sbn, TC* __restrict__ C, int64_t ldc,
+            const float* __restrict__ bias, const TM* __restrict__ mask, int64_t ldm, int k_chunk) {
+    __shared__ float As[GK][GT + 4];
+    __shared__ float Bs[GK][GT + 4];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int m0 = blockIdx.y * GT, n0 = blockIdx.x * GT;
+    const int k_begin = blockIdx.z * k_chunk, k_end = min(K, k_begin + k_chunk);
+    const bool a_kfast = (sak == 1), b_kfast = (sbk == 1);
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = k_begin; k0 < k_end; k0 += GK) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int idx = tid + r * 256;
+            int m, k;
+            if (a_kfast) { m = idx >> 4; k = idx & 15; } else { k = idx >> 6; m = idx & 63; }
+            const int gm = m0 + m, gk = k0 + k;
+            As[k][m] = (gm < M && gk < k_end) ? to_f(A[gm * sam + gk * sak]) : 0.f;
+            int n, kb;
+            if (b_kfast) { n = idx >> 4; kb = idx & 15; } else { kb = idx >> 6; n = idx & 63; }
+            const int gn = n0 + n, gkb = k0 + kb;
+            Bs[kb][n] = (gn < N && gkb < k_end) ? to_f(Bm[gkb * sbk + gn * sbn]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < GK; ++k) {
+            const float4 a4 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+            const float4 b4 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+            const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int gm = m0 + ty * 4 + i;
+        if (gm >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int gn = n0 + tx * 4 + j;
+            if (gn >= N) continue;
+            float v = acc[i][j];
+            if (EPI == EPI_BIAS_RELU) v = fmaxf(v + bias[gn], 0.f);
+            if (EPI == EPI_MASK) v = to_f(mask[gm * ldm + gn]) > 0.f ? v : 0.f;
+            if (EPI == EPI_ATOMIC) atomicAdd(reinterpret_cast<float*>(C) + gm * ldc + gn, v);
+            else C[gm * ldc + gn] = from_f<TC>(v);
+        }
+    }
+}
+
+template <typename TA, typename TB, typename TC, typename TM, int EPI>
+static void launch_gemm(int M, int N, int K, const TA* A, int64_t sam, int64_t sak, const TB* B, int64_t sbk,
+                        int64_t sbn, TC* C, int64_t ldc, const float* bias, const TM* mask, int64_t ldm,
+                        int splits, cudaStream_t st) {
+    if (M <= 0 || N <= 0 || K <= 0) return;
+    int k_chunk = (int)ceil_div(ceil_div(K, splits), GK) * GK;
+    splits = (int)ceil_div(K, k_chunk);
+    dim3 grid((unsigned)ceil_div(N, GT), (unsigned)ceil_div(M, GT), (unsigned)splits);
+    gemm_kernel<TA, TB, TC, TM, EPI><<<grid, 256, 0, st>>>(M, N, K, A, sam, sak, B, sbk, sbn, C, ldc, bias, mask,
+                                                          ldm, k_chunk);
+}
+
+// Output unit, loss and the gradient at the top hidden layer.  One warp per view.
+//   z = h . w_out + b_out;  p = sigmoid(z);  BCE in its overflow-safe form;  dz = (p - y) / B
+//   dA_top[b][j] = dz * w_out[j] where h[b][j] > 0, else 0
+template <typename TX>
+__global__ void __launch_bounds__(256)
+head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict__ w_out,
+                const float* __restrict__ b_out, const float* __restrict__ label, float* __restrict__ prob,
+                float* __restrict__ dz, TX* __restrict__ dA, float* __restrict__ loss_part) {
+    __shared__ float part[8];
+    const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
+    float local = 0.f;
+    for (int b = blockIdx.x * 8 + warp; b < B; b += gridDim.x * 8) {
+        const TX* row = h + (int64_t)b * H;
+        float z = 0.f;
+        for (int j = lane; j < H; j += 32) z = fmaf(to_f(row[j]), w_out[j], z);
+        z = warp_sum(z) + b_out[0];
+        const float y = label[b];
+        const float p = 1.0f / (1.0f + expf(-z));
+        const float g = (p - y) / (float)B;
+        if (lane == 0) {
+            local += fmaxf(z, 0.f) - z * y + log1pf(expf(-fabsf(z)));
+            if (prob) prob[b] = p;
+            dz[b] = g;
+        }
+        TX* drow = dA + (int64_t)b * H;
+        for (int j = lane; j < H; j += 32) drow[j] = from_f<TX>(to_f(row[j]) > 0.f ? g * w_out[j] : 0.f);
+    }
+    if (lane == 0) part[warp] = local;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int w = 0; w < 8; ++w) s += part[w];
+        loss_part[blockIdx.x] = s;
+    }
+}
+
+__global__ void loss_final_kernel(const float* __restrict__ part, int n, int B, float* __restrict__ loss) {
+    __shared__ float sm[32];
+    float s = 0.f;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) s += part[i];
+    s = warp_sum(s);
+    if (lane_id() == 0) sm[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float t = threadIdx.x < (blockDim.x >> 5) ? sm[threadIdx.x] : 0.f;
+        t = warp_sum(t);
+        if (threadIdx.x == 0) loss[0] = B > 0 ? t / (float)B : 0.f;
+    }
+}
+
+// out[n] += sum_b A[b][n] * (w ? w[b] : 1): bias gradients and the output-weight gradient.
+template <typename TA>
+__global__ void __launch_bounds__(256)
+colsum_kernel(int B, int N, const TA* __restrict__ A, const float* __restrict__ w, float* __restrict__ out,
+              int rows_per_block) {
+    const int b0 = blockIdx.x * rows_per_block, b1 = min(B, b0 + rows_per_block);
+    for (int n = threadIdx.x; n < N; n += blockDim.x) {
+        float s = 0.f;
+        for (int b = b0; b < b1; ++b) s = fmaf(to_f(A[(int64_t)b * N + n]), w ? w[b] : 1.f, s);
+        atomicAdd(out + n, s);
+    }
+}
+
+__global__ void sum_vec_kernel(int n, const float* __restrict__ v, float* __restrict__ out) {
+    __shared__ float sm[32];
+    float s = 0.f;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) s += v[i];
+    s = warp_sum(s);
+    if (lane_id() == 0) sm[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float t = threadIdx.x < (blockDim.x >> 5) ? sm[threadIdx.x] : 0.f;
+        t = warp_sum(t);
+        if (threadIdx.x == 0) out[0] = t;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+round_weights_kernel(int fan_in, int fan_out, const float* __restrict__ W, __nv_bfloat16* __restrict__ wb,
+                     __nv_bfloat16* __restrict__ wbt) {
+    const int64_t n = (int64_t)fan_in * fan_out;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const __nv_bfloat16 v = __float2bfloat16_rn(W[i]);
+        wb[i] = v;
+        const int r = (int)(i / fan_out), c = (int)(i % fan_out);
+        wbt[(int64_t)c * fan_in + r] = v;
+    }
+}
+
+struct HeadParams {
+    const float* W[MAX_LAYERS]; const float* b[MAX_LAYERS];
+    float* gW[MAX_LAYERS]; float* gb[MAX_LAYERS];
+    const float* w_out; const float* b_out; float* gw_out; float* gb_out;
+    int fan[MAX_LAYERS + 1];
+};
+
+static HeadParams split_params(const gear_ctx_impl& c, float* grad) {
+    HeadParams p;
+    const float* base = c.buf.head_params;
+    int64_t pos = 0;
+    p.fan[0] = c.d_in;
+    for (int l = 0; l < c.cfg.n_hidden; ++l) {
+        const int h = c.cfg.hidden[l];
+        p.W[l] = base + pos; p.gW[l] = grad + pos; pos += (int64_t)p.fan[l] * h;
+        p.b[l] = base + pos; p.gb[l] = grad + pos; pos += h;
+        p.fan[l + 1] = h;
+    }
+    p.w_out = base + pos; p.gw_out = grad + pos; pos += p.fan[c.cfg.n_hidden];
+    p.b_out = base + pos; p.gb_out = grad + pos;
+    return p;
+}
+
+static int splits_for(int M, int N, int K) {
+    const int64_t tiles = ceil_div(M, GT) * ceil_div(N, GT);
+    int64_t s = ceil_div(148 * 4, tiles);
+    const int64_t max_s = ceil_div(K, 256);
+    if (s > max_s) s = max_s;
+    return (int)(s < 1 ? 1 : s);
+}
+
+template <typename TX>
+static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const gear_step_out& o, cudaStream_t st) {
+    constexpr bool BF = !std::is_same<TX, float>::value;
+    const int L = c.cfg.n_hidden, B = bt.B;
+    HeadParams p = split_params(c, o.head_grad);
+    cudaError_t err = cudaMemsetAsync(o.head_grad, 0, sizeof(float) * c.n_params, st);
+    if (err != cudaSuccess) return err;
+    if (B <= 0) return cudaMemsetAsync(o.loss, 0, sizeof(float), st);
+
+    TX* H[MAX_LAYERS + 1];
+    TX* dA[MAX_LAYERS + 1];
+    H[0] = c.at<TX>(c.ws.x);
+    dA[0] = nullptr;
+    for (int l = 0; l < L; ++l) { H[l + 1] = c.at<TX>(c.ws.h[l]); dA[l + 1] = c.at<TX>(c.ws.da[l]); }
+    float* dz = c.at<float>(c.ws.dz);
+    float* loss_part = c.at<float>(c.ws.loss_part);
+
+    // weights as the products see them
+    const void* Wop[MAX_LAYERS];
+    for (int l = 0; l < L; ++l) {
+        if (BF) {
+            __nv_bfloat16* wb = c.at<__nv_bfloat16>(c.ws.wb[l]);
+            round_weights_kernel<<<64, 256, 0, st>>>(p.fan[l], p.fan[l + 1], p.W[l], wb,
+                                                     c.at<__nv_bfloat16>(c.ws.wbt[l]));
+            Wop[l] = wb;
+        } else {
+            Wop[l] = p.W[l];
+        }
+    }
+    // forward
+    for (int l = 0; l < L; ++l) {
+        const int K = p.fan[l], N = p.fan[l + 1];
+        launch_gemm<TX, TX, TX, TX, EPI_BIAS_RELU>(B, N, K, H[l], K, 1, static_cast<const TX*>(Wop[l]), N, 1,
+                                                    H[l + 1], N, p.b[l], (const TX*)nullptr, 0, 1, st);
+    }
+    const int HT = p.fan[L];
+    head_out_kernel<TX><<<c.ws.loss_blocks, 256, 0, st>>>(B, HT, H[L], p.w_out, p.b_out, bt.label, o.prob, dz, dA[L],
+                                                          loss_part);
+    loss_final_kernel<<<1, 256, 0, st>>>(loss_part, c.ws.loss_blocks, B, o.loss);
+    // backward
+    const int rows = 128;
+    colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, HT, H[L], dz, p.gw_out, rows);
+    sum_vec_kernel<<<1, 1024, 0, st>>>(B, dz, p.gb_out);
+    for (int l = L - 1; l >= 0; --l) {
+        const int K = p.fan[l], N = p.fan[l + 1];
+        // dW_l = H_l^T dA_{l+1}
+        launch_gemm<TX, TX, float, TX, EPI_ATOMIC>(K, N, B, H[l], 1, K, dA[l + 1], N, 1, p.gW[l], N, nullptr,
+                                                   (const TX*)nullptr, 0, splits_for(K, N, B), st);
+        colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, N, dA[l + 1], nullptr, p.gb[l], rows);
+        if (l > 0) {
+            launch_gemm<TX, TX, TX, TX, EPI_MASK>(B, K, N, dA[l + 1], N, 1, static_cast<const TX*>(Wop[l]), 1, N,
+                                                  dA[l], K, nullptr, H[l], K, 1, st);
+        } else {
+            launch_gemm<TX, TX, float, TX, EPI_NONE>(B, K, N, dA[l + 1], N, 1, static_cast<const TX*>(Wop[l]), 1, N,
+                                                     o.dX, K, nullptr, (const TX*)nullptr, 0, 1, st);
+        }
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_head_simt(const gear_ctx_impl& c, const gear_batch& b, const gear_step_out& o, cudaStream_t st) {
+    if (c.cfg.head_dtype == GEAR_BF16) return run_head<__nv_bfloat16>(c, b, o, st);
+    return run_head<float>(c, b, o, st);
+}
+
+}  // namespace gear

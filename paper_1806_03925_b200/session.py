@@ -1,0 +1,134 @@
+"""Device-memory plumbing around the C calls: allocates the tables, the
+workspace and the per-step outputs as torch tensors and issues the calls of one
+step in order.  No arithmetic of the method happens here.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+from . import binding as gb
+from .workloads import BF16, Batch, GearPreset
+
+
+@dataclass
+class DeviceBatch:
+    user_id: torch.Tensor
+    url_id: torch.Tensor
+    img_off: torch.Tensor
+    img_id: torch.Tensor
+    label: torch.Tensor
+    B: int
+    nnz: int
+
+    @staticmethod
+    def from_host(b: Batch, device="cuda") -> "DeviceBatch":
+        f = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
+        return DeviceBatch(f(b.user_id), f(b.url_id), f(b.img_off), f(b.img_id), f(b.label), b.B, b.nnz)
+
+
+class GearSession:
+    """Tables + ctx + output buffers for one configuration on one GPU."""
+
+    def __init__(self, p: GearPreset, head_params: np.ndarray, max_batch: Optional[int] = None,
+                 max_nnz: Optional[int] = None, seed: int = 0, fill: bool = True, now: int = 0,
+                 tables: Optional[Dict[str, np.ndarray]] = None, ready_cap: int = 0, device: str = "cuda",
+                 want_emb_grad: bool = False, want_debug: bool = False, expired_cap: Optional[int] = None):
+        gb.load()
+        self.p = p
+        self.dev = torch.device(device)
+        self.max_batch = int(max_batch or p.batch)
+        self.max_nnz = int(max_nnz or self.max_batch * p.img_hi)
+        self.d_in = p.d_in
+        dfv_t = torch.bfloat16 if p.dfv_dtype == BF16 else torch.float32
+        self.cfg = gb.make_config(p.user_vocab, p.url_vocab, p.img_vocab, p.emb_dim, p.dfv_dim,
+                                  gb.GEAR_BF16 if p.dfv_dtype == BF16 else gb.GEAR_F32,
+                                  gb.GEAR_BF16 if p.head_dtype == BF16 else gb.GEAR_F32,
+                                  list(p.hidden), p.M, p.expire, self.max_batch, self.max_nnz, ready_cap)
+        dev = self.dev
+        if tables is None:
+            self.user_emb = torch.empty((p.user_vocab, p.emb_dim), dtype=torch.float32, device=dev)
+            self.url_emb = torch.empty((p.url_vocab, p.emb_dim), dtype=torch.float32, device=dev)
+            self.dfv = torch.empty((p.img_vocab, p.dfv_dim), dtype=dfv_t, device=dev)
+            self.dfv_ts = torch.zeros(p.img_vocab, dtype=torch.int64, device=dev)
+        else:
+            fill = False
+            self.user_emb = torch.from_numpy(tables["user_emb"]).to(dev)
+            self.url_emb = torch.from_numpy(tables["url_emb"]).to(dev)
+            dfv = tables["dfv"]
+            if dfv.dtype == np.uint16:
+                self.dfv = torch.from_numpy(dfv.view(np.int16)).to(dev).view(torch.bfloat16)
+            else:
+                self.dfv = torch.from_numpy(dfv).to(dev)
+            assert self.dfv.dtype == dfv_t
+            self.dfv_ts = torch.from_numpy(tables["ts"]).to(dev)
+        self.dfv_gsum = torch.zeros((p.img_vocab, p.dfv_dim), dtype=torch.float32, device=dev)
+        self.dfv_gcnt = torch.zeros(p.img_vocab, dtype=torch.int32, device=dev)
+        self.head_params = torch.from_numpy(np.ascontiguousarray(head_params, dtype=np.float32)).to(dev)
+        assert self.head_params.numel() == p.n_params
+        self.workspace = torch.empty(gb.gear_workspace_bytes(self.cfg), dtype=torch.uint8, device=dev)
+        self.ctx = gb.gear_init_tables(self.cfg, self.user_emb, self.url_emb, self.dfv, self.dfv_gsum, self.dfv_gcnt,
+                                       self.dfv_ts, self.head_params, self.workspace, seed=seed, fill=fill, now=now)
+        B, nnz = self.max_batch, self.max_nnz
+        self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
+        self.prob = torch.zeros(B, dtype=torch.float32, device=dev)
+        self.head_grad = torch.zeros(p.n_params, dtype=torch.float32, device=dev)
+        self.dX = torch.zeros((B, self.d_in), dtype=torch.float32, device=dev)
+        self.row_view = torch.zeros(nnz, dtype=torch.int32, device=dev)
+        self.inv_n = torch.zeros(B, dtype=torch.float32, device=dev)
+        self.x_debug = (torch.zeros((B, self.d_in), dtype=torch.bfloat16 if p.head_dtype == BF16 else torch.float32,
+                                    device=dev) if want_debug else None)
+        self.user_grad = torch.zeros_like(self.user_emb) if want_emb_grad else None
+        self.url_grad = torch.zeros_like(self.url_emb) if want_emb_grad else None
+        self.ready_cap = int(ready_cap or nnz)
+        self.ready_ids = torch.zeros(self.ready_cap, dtype=torch.int32, device=dev)
+        self.ready_seq = torch.zeros(self.ready_cap, dtype=torch.int32, device=dev)
+        self.ready_avg = torch.zeros((self.ready_cap, p.dfv_dim), dtype=torch.float32, device=dev)
+        self.expired_cap = int(expired_cap if expired_cap is not None else p.img_vocab)
+        self.expired_ids = torch.zeros(self.expired_cap, dtype=torch.int32, device=dev)
+        self.d_counts = torch.zeros(2, dtype=torch.int64, device=dev)
+
+    # ---- the four calls of a step ---------------------------------------------------------------
+    def forward_backward(self, b: DeviceBatch, lr: Optional[float] = None):
+        return gb.gear_forward_backward(self.ctx, b.user_id, b.url_id, b.img_off, b.img_id, b.label,
+                                        self.p.lr if lr is None else lr, self.loss, self.head_grad, self.dX,
+                                        prob=self.prob, row_view=self.row_view, inv_n=self.inv_n,
+                                        x_debug=self.x_debug, user_grad=self.user_grad, url_grad=self.url_grad,
+                                        B=b.B, nnz=b.nnz)
+
+    def accumulate_from_step(self, b: DeviceBatch):
+        """Event 5 in its indirect form: row r of the batch is dX[row_view[r], 2E:] * inv_n[row_view[r]]."""
+        ptr = self.dX.data_ptr() + 4 * 2 * self.p.emb_dim
+        return gb.gear_accumulate_dfv_grad(self.ctx, b.img_id, ptr, self.d_in, self.row_view, self.inv_n, b.nnz)
+
+    def accumulate_rows(self, img_id: torch.Tensor, grads: torch.Tensor):
+        assert grads.dtype == torch.float32 and grads.shape[1] == self.p.dfv_dim
+        return gb.gear_accumulate_dfv_grad(self.ctx, img_id, grads.data_ptr(), grads.stride(0), None, None,
+                                           int(img_id.shape[0]))
+
+    def collect_ready(self, sync: bool = True):
+        return gb.gear_collect_ready(self.ctx, self.ready_ids, self.ready_seq, self.ready_avg, self.ready_cap,
+                                     d_n=self.d_counts[0:1], sync=sync)
+
+    def collect_expired(self, now: int, restamp: bool = True, sync: bool = True):
+        return gb.gear_collect_expired(self.ctx, now, restamp, self.expired_ids, self.expired_cap,
+                                       d_n=self.d_counts[1:2], sync=sync)
+
+    def step(self, b: DeviceBatch, now: int, sync: bool = False):
+        """One pass of the whole hot path over one batch."""
+        self.forward_backward(b)
+        self.accumulate_from_step(b)
+        n_ready = self.collect_ready(sync=sync)
+        n_exp = self.collect_expired(now, restamp=True, sync=sync)
+        return n_ready, n_exp
+
+    def status(self):
+        return gb.gear_status(self.ctx)
+
+    def close(self):
+        if self.ctx is not None:
+            gb.gear_destroy(self.ctx)
+            self.ctx = None

@@ -1,0 +1,206 @@
+"""Runs the CUDA library and the CPU oracle side by side on the same seeded inputs.
+
+The oracle never sees anything the GPU produced: both sides get the batches from
+the workload generators and the tables either from host-built arrays or, for the
+procedural fill, each from its own implementation of the generator.
+
+For vocabularies too large for dense host tables the oracle works on a compact
+problem: only the rows the batches touch are generated (row by row, from the
+procedural definition) and the IDs are renumbered; GPU results are read back at
+those rows.  The timestamp table is always kept in full.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+import oracle
+from oracle import GearOracle
+from paper_1806_03925_b200 import workloads
+from paper_1806_03925_b200.session import DeviceBatch, GearSession
+from paper_1806_03925_b200.workloads import BF16, Batch, GearPreset
+
+TOL_F32 = 1e-5      # relative tolerance for fp32 configurations (normwise: against the largest reference entry)
+TOL_BF16 = 1e-2     # for configurations whose DFVs / head operands are bfloat16
+
+
+def tol_of(p: GearPreset) -> float:
+    return TOL_BF16 if (p.head_dtype == BF16 or p.dfv_dtype == BF16) else TOL_F32
+
+
+def assert_close(got, want, tol, what=""):
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    assert got.shape == want.shape, (what, got.shape, want.shape)
+    if want.size == 0:
+        return
+    scale = max(np.abs(want).max(), 1e-30)
+    err = np.abs(got - want).max()
+    assert err <= tol * scale, "%s: max abs error %.3e > %.1e * %.3e" % (what, err, tol, scale)
+
+
+def _rows(t: torch.Tensor, rows: np.ndarray) -> np.ndarray:
+    return _np(t[torch.from_numpy(rows).to(t.device)])
+
+
+def _np(t: torch.Tensor) -> np.ndarray:
+    if t.dtype == torch.bfloat16:
+        return t.float().cpu().numpy()
+    return t.cpu().numpy()
+
+
+class Remap:
+    """Renumbering of the IDs that occur (sorted) to 0..n-1; out-of-range IDs map to -1."""
+
+    def __init__(self, ids: np.ndarray, vocab: int, dense: bool):
+        self.vocab = vocab
+        if dense:
+            self.rows = np.arange(vocab, dtype=np.int64)
+        else:
+            ok = ids[(ids >= 0) & (ids < vocab)]
+            self.rows = np.unique(ok).astype(np.int64)
+        self.dense = dense
+
+    def __call__(self, ids: np.ndarray) -> np.ndarray:
+        ids = np.asarray(ids)
+        ok = (ids >= 0) & (ids < self.vocab)
+        out = np.full(ids.shape, -1, dtype=np.int32)
+        if self.dense:
+            out[ok] = ids[ok]
+        else:
+            out[ok] = np.searchsorted(self.rows, ids[ok]).astype(np.int32)
+        return out
+
+    @property
+    def n(self) -> int:
+        return len(self.rows)
+
+
+class Pair:
+    """A GearSession on the GPU and a GearOracle on the CPU over the same problem."""
+
+    def __init__(self, p: GearPreset, batches: List[Batch], seed: int = 0, dense: Optional[bool] = None,
+                 now0: int = 0, ready_cap: int = 0, want_emb_grad: bool = False, extra_img_ids=None):
+        self.p, self.seed = p, seed
+        if dense is None:
+            dense = max(p.user_vocab, p.url_vocab, p.img_vocab) <= 200_000
+        cat = lambda k: np.concatenate([getattr(b, k) for b in batches]) if batches else np.zeros(0, np.int32)
+        img_all = cat("img_id")
+        if extra_img_ids is not None:
+            img_all = np.concatenate([img_all, extra_img_ids])
+        self.ru = Remap(cat("user_id"), p.user_vocab, dense)
+        self.rh = Remap(cat("url_id"), p.url_vocab, dense)
+        self.ri = Remap(img_all, p.img_vocab, dense)
+        self.params = workloads.head_params(p, seed)
+        max_b = max([b.B for b in batches] + [1])
+        max_nnz = max([b.nnz for b in batches] + [1])
+        if extra_img_ids is not None:
+            max_nnz = max(max_nnz, len(extra_img_ids))
+        self.gpu = GearSession(p, self.params, max_batch=max_b, max_nnz=max_nnz, seed=seed, fill=True, now=now0,
+                               ready_cap=ready_cap, want_emb_grad=want_emb_grad, want_debug=True)
+        dfv_np = np.uint16 if p.dfv_dtype == BF16 else np.float32
+        self.cpu = GearOracle(
+            oracle.fill_rows(seed, oracle.TAG_USER, p.emb_dim, self.ru.rows, self.ru.n, np.float32),
+            oracle.fill_rows(seed, oracle.TAG_URL, p.emb_dim, self.rh.rows, self.rh.n, np.float32),
+            oracle.fill_rows(seed, oracle.TAG_DFV, p.dfv_dim, self.ri.rows, self.ri.n, dfv_np),
+            p.hidden, p.M, p.expire, round_bf16=(p.head_dtype == BF16),
+            ts=oracle.fill_ts(seed, p.expire, now0, None, p.img_vocab))
+        self.tol = tol_of(p)
+        self.want_emb_grad = want_emb_grad
+        self.status_bits = 0       # device status bits seen so far (reading the word clears it)
+        self.status_rc = 0
+
+    def status(self):
+        rc, bits, pending = self.gpu.status()
+        self.status_bits |= bits
+        if rc != 0 and self.status_rc == 0:
+            self.status_rc = rc
+        return pending
+
+    # ---- one full step on both sides, compared call by call ------------------------------------
+    def step_and_compare(self, b: Batch, now: int, lr: Optional[float] = None, check_tables: bool = True):
+        p, gpu, cpu, tol = self.p, self.gpu, self.cpu, self.tol
+        lr = p.lr if lr is None else lr
+        E, D = p.emb_dim, p.dfv_dim
+        db = DeviceBatch.from_host(b)
+        gpu.forward_backward(db, lr)
+        uid, hid, img = self.ru(b.user_id), self.rh(b.url_id), self.ri(b.img_id)
+        r = cpu.forward_backward(self.params.astype(np.float64), uid, hid, b.img_off, img, b.label)
+
+        B = b.B
+        X = _np(gpu.x_debug[:B])
+        # gathered rows are copies: bit-exact (after the same bf16 rounding for bf16 heads)
+        assert np.array_equal(X[:, :2 * E].astype(np.float64), r.X[:, :2 * E]), "embedding rows"
+        n_b = np.diff(b.img_off)
+        single = (n_b == 1)
+        assert np.array_equal(X[single, 2 * E:].astype(np.float64), r.X[single, 2 * E:]), "single-image pooled rows"
+        assert_close(X, r.X, tol, "head input")
+        assert_close(_np(gpu.prob[:B]), r.prob, tol, "prob")
+        assert_close(_np(gpu.loss), [r.loss], tol, "loss")
+        assert_close(_np(gpu.head_grad), r.head_grad, tol, "head_grad")
+        assert_close(_np(gpu.dX[:B]), r.dX, tol, "dX")
+        view_of = np.repeat(np.arange(B, dtype=np.int32), n_b)
+        assert np.array_equal(_np(gpu.row_view[:b.nnz]), view_of), "row_view"
+        inv = np.where(n_b > 0, 1.0 / np.maximum(n_b, 1), 0.0)
+        assert_close(_np(gpu.inv_n[:B]), inv, 1e-7, "inv_n")
+
+        # embedding gradients / in-place update
+        if self.want_emb_grad:
+            gu = cpu.emb_grad("user", uid, r.dX)
+            gh = cpu.emb_grad("url", hid, r.dX)
+            assert_close(_rows(gpu.user_grad, self.ru.rows), gu, tol, "user_grad")
+            assert_close(_rows(gpu.url_grad, self.rh.rows), gh, tol, "url_grad")
+            gpu.user_grad.zero_()
+            gpu.url_grad.zero_()
+        else:
+            cpu.emb_apply("user", uid, r.dX, -lr)
+            cpu.emb_apply("url", hid, r.dX, -lr)
+            if check_tables:
+                assert_close(_rows(gpu.user_emb, self.ru.rows), cpu.user_emb, tol, "user_emb after update")
+                assert_close(_rows(gpu.url_emb, self.rh.rows), cpu.url_emb, tol, "url_emb after update")
+
+        # event 5 + 6
+        gpu.accumulate_from_step(db)
+        cpu.accumulate(img, cpu.dfv_grad_rows(b.img_off, r.dX))
+        self.compare_store(check_tables)
+        n_ready = self.collect_and_compare()
+        n_exp = self.expire_and_compare(now)
+        assert self.status() == 0
+        out = dict(loss=r.loss, n_ready=n_ready, n_expired=n_exp, status=self.status_bits, rc=self.status_rc,
+                   bad=r.bad_ids)
+        self.status_bits = self.status_rc = 0
+        return out
+
+    def compare_store(self, check_tables: bool = True):
+        gpu, cpu = self.gpu, self.cpu
+        rows = torch.from_numpy(self.ri.rows).to(gpu.dev)
+        assert np.array_equal(_np(gpu.dfv_gcnt[rows]), cpu.gcnt), "open-group counts"
+        assert int(gpu.dfv_gcnt.sum().item()) == int(cpu.gcnt.sum()), "counts outside the touched rows"
+        if check_tables:
+            assert_close(_np(gpu.dfv_gsum[rows]), cpu.gsum, self.tol, "open-group sums")
+
+    def collect_and_compare(self) -> int:
+        gpu, cpu = self.gpu, self.cpu
+        assert self.status() == cpu.pending_ready, "pending ready count"
+        n = gpu.collect_ready()
+        eid, eseq, eavg = oracle.sort_emissions(*cpu.collect_ready())
+        assert n == len(eid), "number of emissions"
+        gid = _np(gpu.ready_ids[:n])
+        assert np.array_equal(self.ri(gid), eid), "emitted ids"
+        assert np.array_equal(_np(gpu.ready_seq[:n]), eseq), "emission numbers"
+        assert_close(_np(gpu.ready_avg[:n]), eavg, self.tol, "averaged gradients")
+        return n
+
+    def expire_and_compare(self, now: int, restamp: bool = True) -> int:
+        gpu, cpu = self.gpu, self.cpu
+        n = gpu.collect_expired(now, restamp)
+        want = cpu.collect_expired(now, restamp)
+        assert n == len(want), "number of expired entries"
+        assert np.array_equal(_np(gpu.expired_ids[:n]), want), "expired ids"
+        assert np.array_equal(_np(gpu.dfv_ts), cpu.ts), "timestamps after the scan"
+        return n
+
+    def close(self):
+        self.gpu.close()

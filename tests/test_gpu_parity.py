@@ -1,0 +1,330 @@
+"""GPU-vs-oracle parity through the C ABI (run with -m gpu on a B200).
+
+Bit-exact: gathered rows, counts, ready / expired ID lists, emission numbers after sorting by (id, seq),
+timestamps, procedural table fill.  Within tolerance (normwise, 1e-5 for fp32 configurations, 1e-2 where
+DFVs or head operands are bfloat16): head input, probabilities, loss, head gradients, dX, embedding
+gradients and updated tables, open-group sums, averaged gradients.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1806_03925_b200 import workloads
+from paper_1806_03925_b200.workloads import BF16, F32, PRESETS, Batch, BatchSource
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_1806_03925_b200 import binding
+    binding.load()
+    return binding
+
+
+def _pair(*a, **k):
+    from gpu_harness import Pair
+    return Pair(*a, **k)
+
+
+# ------------------------------------------------------------------ procedural fill
+def test_procedural_fill_is_bit_identical(gb):
+    for dtype, np_dt, dim, rows in ((torch.float32, np.float32, 20, 1000), (torch.bfloat16, np.uint16, 24, 777),
+                                    (torch.float32, np.float32, 3, 5)):
+        t = torch.empty((rows, dim), dtype=dtype, device="cuda")
+        gb.gear_fill_uniform(t, seed=11, tag=gb.GEAR_TAG_DFV)
+        want = oracle.fill_rows(11, oracle.TAG_DFV, dim, None, rows, np_dt)
+        got = t.view(torch.int16).cpu().numpy().view(np.uint16) if dtype == torch.bfloat16 else t.cpu().numpy()
+        assert np.array_equal(got, want)
+
+
+# ------------------------------------------------------------------ whole step, every configuration (reduced where needed)
+def _run_steps(p, steps, seed=0, want_emb_grad=False, B=None, dense=None):
+    src = BatchSource(p, seed)
+    batches = [src.batch(s, B) for s in range(steps)]
+    pair = _pair(p, batches, seed=seed, want_emb_grad=want_emb_grad, dense=dense)
+    out = []
+    try:
+        for s, b in enumerate(batches):
+            out.append(pair.step_and_compare(b, now=s + 1))
+    finally:
+        pair.close()
+    return out
+
+
+def test_tiny_config_all_steps(gb):
+    p = PRESETS["tiny"]
+    out = _run_steps(p, p.steps)
+    assert all(o["status"] == 0 for o in out)
+    assert sum(o["n_ready"] for o in out) > 0 and sum(o["n_expired"] for o in out) > 0
+
+
+def test_tiny_config_embedding_gradients(gb):
+    _run_steps(PRESETS["tiny"], 3, want_emb_grad=True)
+
+
+def test_medium_config_two_steps(gb):
+    # full medium shapes (1M-row tables, bf16 DFVs, 192-256-128-1 head); the oracle keeps the touched rows only
+    p = PRESETS["medium"]
+    out = _run_steps(p, 2, dense=False)
+    assert out[-1]["n_ready"] > 0
+
+
+def test_medium_shapes_ragged_batch(gb):
+    p = PRESETS["medium"].scaled(user_vocab=50_000, url_vocab=30_000, img_vocab=20_000)
+    _run_steps(p, 2, B=1237, want_emb_grad=True)
+
+
+@pytest.mark.parametrize("M", [1, 64, 1024])
+def test_skew_config_reduced(gb, M):
+    # skew shapes with a smaller batch and image table; Zipf 1.3 keeps most rows on a handful of images
+    p = PRESETS["skew"].scaled(M=M, img_vocab=100_000, user_vocab=100_000, url_vocab=100_000)
+    out = _run_steps(p, 3, B=4096)
+    if M == 1:
+        assert out[0]["n_ready"] > 4096
+
+
+def test_large_shapes_reduced(gb):
+    # large-table head (384-512-256-1, bf16 DFV dim 256, E 64, M 32) on small tables and 1536 views
+    p = PRESETS["large"].scaled(user_vocab=80_000, url_vocab=60_000, img_vocab=40_000)
+    _run_steps(p, 2, B=1536)
+
+
+# ------------------------------------------------------------------ accumulate-only (micro-benchmark shapes, reduced)
+@pytest.mark.parametrize("zipf_s,M", [(0.0, 8), (1.1, 8), (1.1, 64)])
+def test_accumulate_only_reduced(gb, zipf_s, M):
+    from gpu_harness import assert_close, _np
+    V, D, n = 50_000, 128, 200_003
+    p = PRESETS["skew"].scaled(img_vocab=V, dfv_dim=D, M=M, user_vocab=16, url_vocab=16, expire=1 << 40)
+    mp = workloads.MicroPreset("t", n, V, D, M, zipf_s)
+    ids = workloads.micro_ids(mp, seed=3)
+    pair = _pair(p, [], seed=3, dense=True, extra_img_ids=ids, ready_cap=n)
+    try:
+        g = torch.empty((n, D), dtype=torch.float32, device="cuda")
+        gb.gear_fill_uniform(g, seed=3, tag=gb.GEAR_TAG_GRAD, amp=1.0)
+        g_cpu = oracle.fill_rows(3, oracle.TAG_GRAD, D, None, n, np.float32, amp=1.0).astype(np.float64)
+        ids_t = torch.from_numpy(ids).cuda()
+        half = n // 2 + 1
+        for lo, hi in ((0, half), (half, n)):       # two calls before one collect: emission numbers continue
+            pair.gpu.accumulate_rows(ids_t[lo:hi], g[lo:hi])
+            pair.cpu.accumulate(ids[lo:hi], g_cpu[lo:hi])
+            pair.compare_store()
+        n_ready = pair.collect_and_compare()
+        k = np.bincount(ids, minlength=V)
+        assert n_ready == int((k // M).sum())
+        pair.status()
+        assert pair.status_bits == 0
+    finally:
+        pair.close()
+
+
+# ------------------------------------------------------------------ edge cases
+def _tiny_pair(batches, **kw):
+    p = PRESETS["tiny"].scaled(user_vocab=500, url_vocab=400, img_vocab=300, **kw.pop("preset", {}))
+    return p, _pair(p, batches, dense=True, **kw)
+
+
+def _manual_batch(uid, hid, imgs, labels):
+    n = [len(v) for v in imgs]
+    off = np.concatenate([[0], np.cumsum(n)]).astype(np.int32)
+    flat = np.array([i for v in imgs for i in v], dtype=np.int32)
+    return Batch(np.array(uid, np.int32), np.array(hid, np.int32), off, flat, np.array(labels, np.float32))
+
+
+def test_empty_views_repeated_images_and_bad_ids(gb):
+    b = _manual_batch([1, 2, 2, 499, 7], [0, 399, 5, 5, 1000],          # url 1000 is out of range
+                      [[5, 5, 5], [], [299], [-3, 10, 10, 7], [12]],    # empty view, repeats, a negative image id
+                      [1, 0, 0, 1, 0])
+    p, pair = _tiny_pair([b], preset=dict(M=2))
+    try:
+        out = pair.step_and_compare(b, now=1)
+        assert out["bad"] == 2
+        assert out["status"] & 1 and out["rc"] == -3        # GEAR_DEV_BAD_ID, GEAR_ERR_BAD_ID
+        assert pair.gpu.status()[1] == 0                    # the status word is cleared once read
+    finally:
+        pair.close()
+
+
+def test_single_view_and_batch_of_one_image(gb):
+    b = _manual_batch([3], [4], [[8]], [1])
+    p, pair = _tiny_pair([b], preset=dict(M=1))
+    try:
+        out = pair.step_and_compare(b, now=1)
+        assert out["n_ready"] == 1
+    finally:
+        pair.close()
+
+
+def test_zero_sized_calls_are_accepted(gb):
+    b = _manual_batch([3], [4], [[8]], [1])
+    p, pair = _tiny_pair([b])
+    try:
+        g = pair.gpu
+        empty_i = torch.zeros(0, dtype=torch.int32, device="cuda")
+        g.accumulate_rows(empty_i, torch.zeros((0, p.dfv_dim), device="cuda"))
+        assert g.collect_ready() == 0
+        from paper_1806_03925_b200.session import DeviceBatch
+        eb = Batch(np.zeros(0, np.int32), np.zeros(0, np.int32), np.zeros(1, np.int32), np.zeros(0, np.int32),
+                   np.zeros(0, np.float32))
+        g.forward_backward(DeviceBatch.from_host(eb))
+        assert g.status()[0] == 0
+        assert float(g.loss.item()) == 0.0 and not g.head_grad.any().item()
+    finally:
+        pair.close()
+
+
+def test_ready_capacity_too_small_consumes_nothing(gb):
+    from gpu_harness import _np
+    rng = np.random.default_rng(5)
+    b = _manual_batch(rng.integers(0, 500, 64), rng.integers(0, 400, 64), [[int(i)] for i in rng.integers(0, 20, 64)],
+                      rng.integers(0, 2, 64))
+    p, pair = _tiny_pair([b], preset=dict(M=2))
+    try:
+        g, c = pair.gpu, pair.cpu
+        from paper_1806_03925_b200.session import DeviceBatch
+        db = DeviceBatch.from_host(b)
+        g.forward_backward(db)
+        g.accumulate_from_step(db)
+        pending = g.status()[2]
+        assert pending > 1
+        with pytest.raises(gb.GearError) as e:
+            gb.gear_collect_ready(g.ctx, g.ready_ids, g.ready_seq, g.ready_avg, pending - 1)
+        assert e.value.code == gb.GEAR_ERR_CAPACITY
+        rc, status, still = g.status()
+        assert still == pending and status & gb.GEAR_DEV_OUT_CAPACITY
+        assert g.collect_ready() == pending                 # a large enough list gets everything
+    finally:
+        pair.close()
+
+
+def test_expired_capacity_too_small_lists_and_restamps_nothing(gb):
+    b = _manual_batch([3], [4], [[8]], [1])
+    p, pair = _tiny_pair([b], preset=dict(expire=10))
+    try:
+        g = pair.gpu
+        before = g.dfv_ts.clone()
+        with pytest.raises(gb.GearError) as e:
+            gb.gear_collect_expired(g.ctx, 5, True, g.expired_ids, 3)
+        assert e.value.code == gb.GEAR_ERR_CAPACITY
+        assert torch.equal(before, g.dfv_ts)
+        g.status()
+        pair.expire_and_compare(5)
+        pair.expire_and_compare(5)                          # restamped: nothing is expired any more
+        pair.expire_and_compare(14, restamp=False)
+        pair.expire_and_compare(15, restamp=False)
+    finally:
+        pair.close()
+
+
+def test_ready_queue_overflow_drops_the_call(gb):
+    p = PRESETS["tiny"].scaled(user_vocab=16, url_vocab=16, img_vocab=64, M=1)
+    ids = np.arange(40, dtype=np.int32) % 64
+    pair = _pair(p, [], dense=True, extra_img_ids=ids, ready_cap=50)
+    try:
+        g = pair.gpu
+        rows = torch.ones((40, p.dfv_dim), device="cuda")
+        ids_t = torch.from_numpy(ids).cuda()
+        g.accumulate_rows(ids_t, rows)
+        g.accumulate_rows(ids_t, rows)                      # 80 > 50: dropped whole
+        rc, status, pending = g.status()
+        assert pending == 40 and status & gb.GEAR_DEV_READY_OVERFLOW and rc == gb.GEAR_ERR_CAPACITY
+        assert g.collect_ready() == 40
+    finally:
+        pair.close()
+
+
+def test_bad_arguments_are_refused_on_the_host(gb):
+    p = PRESETS["tiny"]
+    cfg = gb.make_config(p.user_vocab, p.url_vocab, p.img_vocab, 15, p.dfv_dim, 0, 0, [64], 4, 0, 16, 64)
+    with pytest.raises(gb.GearError) as e:
+        gb.gear_workspace_bytes(cfg)
+    assert e.value.code == gb.GEAR_ERR_ARG
+    b = _manual_batch([3], [4], [[8]], [1])
+    _, pair = _tiny_pair([b])
+    try:
+        g = pair.gpu
+        from paper_1806_03925_b200.session import DeviceBatch
+        big = BatchSource(PRESETS["tiny"].scaled(user_vocab=500, url_vocab=400, img_vocab=300), 0).batch(0, 64)
+        with pytest.raises(gb.GearError):
+            g.forward_backward(DeviceBatch.from_host(big))          # B > max_batch
+    finally:
+        pair.close()
+
+
+# ------------------------------------------------------------------ full size: the large-table configuration
+def test_large_tables_full_size_sampled(gb):
+    """The 48.9 GB large-table configuration as bench.py runs it.  The oracle cannot run 65536 views
+    through the head in seconds, so it checks (a) the gather, forward and per-view backward of a sample
+    of views (per-view results do not depend on the other views except through the 1/B factor),
+    (b) the full-size accumulate / collect on procedurally generated gradient rows, (c) the expiry scan."""
+    from gpu_harness import assert_close, _np, Remap, TOL_BF16
+    from oracle import GearOracle
+    from paper_1806_03925_b200.session import DeviceBatch, GearSession
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * 2**30:
+        pytest.skip("needs about 60 GB of device memory")
+    p = PRESETS["large"]
+    src = BatchSource(p, 0)
+    b = src.batch(0)
+    params = workloads.head_params(p, 0)
+    g = GearSession(p, params, seed=0, fill=True, now=0, want_debug=True)
+    try:
+        db = DeviceBatch.from_host(b)
+        g.forward_backward(db, lr=0.0)                      # lr 0: tables stay as generated
+        # (a) sample of views
+        rng = np.random.default_rng(0)
+        views = np.sort(rng.choice(b.B, 384, replace=False))
+        n_b = np.diff(b.img_off)
+        off_s = np.concatenate([[0], np.cumsum(n_b[views])]).astype(np.int32)
+        img_s = np.concatenate([b.img_id[b.img_off[v]:b.img_off[v + 1]] for v in views])
+        ru, rh, ri = (Remap(b.user_id[views], p.user_vocab, False), Remap(b.url_id[views], p.url_vocab, False),
+                      Remap(img_s, p.img_vocab, False))
+        cpu = GearOracle(oracle.fill_rows(0, oracle.TAG_USER, p.emb_dim, ru.rows, ru.n, np.float32),
+                         oracle.fill_rows(0, oracle.TAG_URL, p.emb_dim, rh.rows, rh.n, np.float32),
+                         oracle.fill_rows(0, oracle.TAG_DFV, p.dfv_dim, ri.rows, ri.n, np.uint16),
+                         p.hidden, p.M, p.expire, round_bf16=True)
+        r = cpu.forward_backward(params.astype(np.float64), ru(b.user_id[views]), rh(b.url_id[views]), off_s,
+                                 ri(img_s), b.label[views])
+        vt = torch.from_numpy(views).cuda()
+        X = _np(g.x_debug[vt])
+        E = p.emb_dim
+        assert np.array_equal(X[:, :2 * E].astype(np.float64), r.X[:, :2 * E])
+        one = n_b[views] == 1
+        assert np.array_equal(X[one, 2 * E:].astype(np.float64), r.X[one, 2 * E:])
+        assert_close(X, r.X, TOL_BF16, "head input")
+        assert_close(_np(g.prob[vt]), r.prob, TOL_BF16, "prob")
+        assert_close(_np(g.dX[vt]) * (b.B / len(views)), r.dX, TOL_BF16, "dX of the sampled views")
+        assert np.isfinite(g.loss.item()) and abs(g.loss.item() - np.log(2)) < 0.5
+        # (b) full-size accumulate on procedural rows, twice, then collect
+        n, D = b.nnz, p.dfv_dim
+        grads = torch.empty((n, D), dtype=torch.float32, device="cuda")
+        gb.gear_fill_uniform(grads, seed=9, tag=gb.GEAR_TAG_GRAD, amp=1.0)
+        g_cpu = oracle.fill_rows(9, oracle.TAG_GRAD, D, None, n, np.float32, amp=1.0).astype(np.float64)
+        ria = Remap(b.img_id, p.img_vocab, False)
+        acc = GearOracle(np.zeros((1, 4), np.float32), np.zeros((1, 4), np.float32), np.zeros((ria.n, D), np.float32),
+                         (8,), p.M, p.expire, ts=oracle.fill_ts(0, p.expire, 0, None, p.img_vocab))
+        ids_c = ria(b.img_id)
+        rows_t = torch.from_numpy(ria.rows).cuda()
+        for _ in range(2):
+            g.accumulate_rows(db.img_id, grads)
+            acc.accumulate(ids_c, g_cpu)
+            assert np.array_equal(_np(g.dfv_gcnt[rows_t]), acc.gcnt)
+        assert int(g.dfv_gcnt.sum().item()) == int(acc.gcnt.sum())
+        assert_close(_np(g.dfv_gsum[rows_t]), acc.gsum, 1e-5, "open-group sums")
+        n_ready = g.collect_ready()
+        eid, eseq, eavg = oracle.sort_emissions(*acc.collect_ready())
+        assert n_ready == len(eid)
+        assert np.array_equal(ria(_np(g.ready_ids[:n_ready])), eid)
+        assert np.array_equal(_np(g.ready_seq[:n_ready]), eseq)
+        assert_close(_np(g.ready_avg[:n_ready]), eavg, 1e-5, "averaged gradients")
+        # (c) expiry over all 20M timestamps
+        for now in (1, 2, 60):
+            k = g.collect_expired(now, True)
+            want = acc.collect_expired(now, True)
+            assert k == len(want) and np.array_equal(_np(g.expired_ids[:k]), want)
+        assert g.status()[1] == 0
+    finally:
+        g.close()
