@@ -66,7 +66,8 @@ def lib():
         L.orc_head_param_count.argtypes = [C.POINTER(_Model)]
         L.orc_forward_backward.restype = i64
         L.orc_forward_backward.argtypes = [C.POINTER(_Model), vp, C.c_int, vp, C.c_int, vp, C.c_int, vp,
-                                           i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+                                           i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                           dbl, vp, i64, vp, vp, i64]
         L.orc_emb_apply.restype = i64
         L.orc_emb_apply.argtypes = [vp, C.c_int, i64, i32, vp, i32, vp, i32, i32, dbl, vp]
         L.orc_dfv_grad_rows.restype = None
@@ -131,6 +132,14 @@ class StepResult:
     head_grad: Optional[np.ndarray]
     dX: Optional[np.ndarray]
     bad_ids: int
+    near_units: Optional[np.ndarray] = None   # coded (layer * B + view) * 1024 + column
+
+
+def decode_unit(code: int, B: int) -> Tuple[int, int, int]:
+    """(layer, view, column) of a unit code of forward_backward's near_units list."""
+    j = int(code) % 1024
+    lb = int(code) // 1024
+    return lb // B, lb % B, j
 
 
 class GearOracle:
@@ -174,7 +183,8 @@ class GearOracle:
 
     # -- events 1, 3, 4 -----------------------------------------------------
     def forward_backward(self, params: np.ndarray, user_id, url_id, img_off, img_id, label,
-                         backward: bool = True) -> StepResult:
+                         backward: bool = True, relu_margin: Optional[float] = None,
+                         flip_units: Optional[Sequence[int]] = None) -> StepResult:
         B = int(len(user_id))
         params = _c(params, np.float64)
         assert params.shape[0] == self.n_params
@@ -186,12 +196,20 @@ class GearOracle:
         loss = C.c_double(0.0)
         hg = np.zeros(self.n_params, dtype=np.float64) if backward else None
         dX = np.zeros((B, self.d_in), dtype=np.float64) if backward else None
+        near = np.zeros(65536, dtype=np.int64) if relu_margin is not None else None
+        n_near = C.c_int64(0)
+        flips = _c(flip_units, np.int64) if flip_units is not None and len(flip_units) else None
         bad = lib().orc_forward_backward(
             C.byref(self.model), _ptr(self.user_emb), _dtype_tag(self.user_emb),
             _ptr(self.url_emb), _dtype_tag(self.url_emb), _ptr(self.dfv), _dtype_tag(self.dfv),
             _ptr(params), B, _ptr(uid), _ptr(hid), _ptr(off), _ptr(img), _ptr(y),
-            _ptr(X), _ptr(prob), C.byref(loss), _ptr(hg), _ptr(dX))
-        return StepResult(X, prob, loss.value, hg, dX, int(bad))
+            _ptr(X), _ptr(prob), C.byref(loss), _ptr(hg), _ptr(dX),
+            0.0 if relu_margin is None else float(relu_margin), _ptr(near), 0 if near is None else len(near),
+            C.byref(n_near), _ptr(flips), 0 if flips is None else len(flips))
+        if near is not None:
+            assert n_near.value <= len(near), "near-zero unit list overflowed"
+            near = near[:n_near.value].copy()
+        return StepResult(X, prob, loss.value, hg, dX, int(bad), near)
 
     def emb_grad(self, which: str, ids, dX: np.ndarray) -> np.ndarray:
         """Dense summed gradient G[vocab, E] of one embedding table."""

@@ -170,6 +170,17 @@ int64_t orc_head_param_count(const orc_model* m) { return head_param_count(m); }
  *          head_grad   dLoss/dparams, packed like params
  *          dX[B][Din]  dLoss/dX; its last dfv_dim columns are dLoss/d(pooled DFV)
  * Any output pointer except X and loss may be NULL (forward only).
+ *
+ * The derivative of ReLU is decided by the sign of a floating-point number.  A
+ * pre-activation within rounding distance of zero may fall on the other side
+ * on a machine that sums in another order or precision, and either decision is
+ * then a correct evaluation of the method.  So that a comparison can accept
+ * both decisions there and nowhere else, the units (layer l, view b, column j)
+ * with |pre-activation| <= relu_margin are listed in near_units (coded
+ * (l * B + b) * 1024 + j; *n_near receives their number, near_cap bounds the
+ * list; near_units may be NULL), and the units named in flip_units take the
+ * other branch in the backward pass (their forward value is left as computed).
+ *
  * Returns the number of out-of-range IDs met (their rows count as zeros).
  */
 int64_t orc_forward_backward(const orc_model* m,
@@ -180,11 +191,14 @@ int64_t orc_forward_backward(const orc_model* m,
                              int32_t B, const int32_t* user_id, const int32_t* url_id,
                              const int32_t* img_off, const int32_t* img_id, const double* label,
                              double* X, double* prob, double* loss,
-                             double* head_grad, double* dX) {
+                             double* head_grad, double* dX,
+                             double relu_margin, int64_t* near_units, int64_t near_cap, int64_t* n_near,
+                             const int64_t* flip_units, int64_t n_flip) {
     const int E = m->emb_dim, D = m->dfv_dim, Din = 2 * E + D;
     const int L = m->n_hidden;
     const int rb = m->round_bf16;
     int64_t bad = 0;
+    if (n_near) *n_near = 0;
 
     /* parameter views */
     const double* W[2] = {0, 0}; const double* bias[2] = {0, 0};
@@ -245,6 +259,10 @@ int64_t orc_forward_backward(const orc_model* m,
             }
             for (int j = 0; j < N; ++j) {
                 double a = out[j] + bias[l][j];
+                if (near_units && fabs(a) <= relu_margin) {
+                    if (*n_near < near_cap) near_units[*n_near] = ((int64_t)l * B + b) * 1024 + j;
+                    ++*n_near;
+                }
                 a = a > 0.0 ? a : 0.0;
                 out[j] = rb ? round_bf16(a) : a;
             }
@@ -289,7 +307,10 @@ int64_t orc_forward_backward(const orc_model* m,
                 const double* out = H[l + 1] + (int64_t)b * N;
                 /* through the ReLU (derivative 0 at 0); operand rounding for bf16 heads */
                 for (int j = 0; j < N; ++j) {
-                    double g = out[j] > 0.0 ? d_hi[j] : 0.0;
+                    int active = out[j] > 0.0;
+                    for (int64_t q = 0; q < n_flip; ++q)
+                        if (flip_units[q] == ((int64_t)l * B + b) * 1024 + j) active = !active;
+                    double g = active ? d_hi[j] : 0.0;
                     d_hi[j] = rb ? round_bf16(g) : g;
                     gb[l][j] += d_hi[j];
                 }

@@ -109,6 +109,9 @@ class Pair:
             ts=oracle.fill_ts(seed, p.expire, now0, None, p.img_vocab))
         self.tol = tol_of(p)
         self.want_emb_grad = want_emb_grad
+        self.updated_user = np.zeros(0, np.int32)
+        self.updated_url = np.zeros(0, np.int32)
+        self.relu_flips_accepted = 0
         self.status_bits = 0       # device status bits seen so far (reading the word clears it)
         self.status_rc = 0
 
@@ -127,18 +130,26 @@ class Pair:
         db = DeviceBatch.from_host(b)
         gpu.forward_backward(db, lr)
         uid, hid, img = self.ru(b.user_id), self.rh(b.url_id), self.ri(b.img_id)
-        r = cpu.forward_backward(self.params.astype(np.float64), uid, hid, b.img_off, img, b.label)
+        params64 = self.params.astype(np.float64)
+        margin = 2e-6 if tol == TOL_F32 else 1e-4
+        r = cpu.forward_backward(params64, uid, hid, b.img_off, img, b.label, relu_margin=margin)
 
         B = b.B
         X = _np(gpu.x_debug[:B])
-        # gathered rows are copies: bit-exact (after the same bf16 rounding for bf16 heads)
-        assert np.array_equal(X[:, :2 * E].astype(np.float64), r.X[:, :2 * E]), "embedding rows"
+        # gathered rows are copies: bit-exact (after the same bf16 rounding for bf16 heads) for every row
+        # of a table that no earlier step has updated (an updated row agrees to rounding only)
+        fresh_u = ~np.isin(uid, self.updated_user)
+        fresh_h = ~np.isin(hid, self.updated_url)
+        assert np.array_equal(X[fresh_u, :E].astype(np.float64), r.X[fresh_u, :E]), "user embedding rows"
+        assert np.array_equal(X[fresh_h, E:2 * E].astype(np.float64), r.X[fresh_h, E:2 * E]), "url embedding rows"
         n_b = np.diff(b.img_off)
         single = (n_b == 1)
         assert np.array_equal(X[single, 2 * E:].astype(np.float64), r.X[single, 2 * E:]), "single-image pooled rows"
         assert_close(X, r.X, tol, "head input")
         assert_close(_np(gpu.prob[:B]), r.prob, tol, "prob")
         assert_close(_np(gpu.loss), [r.loss], tol, "loss")
+        r = self._resolve_relu_decisions(r, lambda flips: cpu.forward_backward(
+            params64, uid, hid, b.img_off, img, b.label, flip_units=flips), B)
         assert_close(_np(gpu.head_grad), r.head_grad, tol, "head_grad")
         assert_close(_np(gpu.dX[:B]), r.dX, tol, "dX")
         view_of = np.repeat(np.arange(B, dtype=np.int32), n_b)
@@ -157,6 +168,9 @@ class Pair:
         else:
             cpu.emb_apply("user", uid, r.dX, -lr)
             cpu.emb_apply("url", hid, r.dX, -lr)
+            if lr != 0.0:
+                self.updated_user = np.union1d(self.updated_user, uid)
+                self.updated_url = np.union1d(self.updated_url, hid)
             if check_tables:
                 assert_close(_rows(gpu.user_emb, self.ru.rows), cpu.user_emb, tol, "user_emb after update")
                 assert_close(_rows(gpu.url_emb, self.rh.rows), cpu.url_emb, tol, "url_emb after update")
@@ -172,6 +186,38 @@ class Pair:
                    bad=r.bad_ids)
         self.status_bits = self.status_rc = 0
         return out
+
+    def _resolve_relu_decisions(self, r, rerun, B):
+        """The backward pass depends on the sign of every hidden pre-activation.  Where the oracle's own
+        pre-activation is within rounding distance of zero (r.near_units) the device may validly have taken
+        the other branch.  If the strict comparison fails, the expected values are recomputed BY THE ORACLE
+        with some of those units on the other branch; units outside that list are never touched."""
+        import itertools
+        from oracle import decode_unit
+        got_dx, got_hg = _np(self.gpu.dX[:B]), _np(self.gpu.head_grad)
+
+        def ok(res):
+            try:
+                assert_close(got_hg, res.head_grad, self.tol)
+                assert_close(got_dx, res.dX, self.tol)
+                return True
+            except AssertionError:
+                return False
+
+        if ok(r) or r.near_units is None or len(r.near_units) == 0:
+            return r
+        row_rel = np.abs(got_dx - r.dX).max(1) / np.maximum(np.abs(r.dX).max(1), 1e-30)
+        thr = 1e-4 if self.tol == TOL_F32 else 2e-2
+        cand = [int(c) for c in r.near_units if row_rel[decode_unit(c, B)[1]] > thr]
+        cand.sort(key=lambda c: -row_rel[decode_unit(c, B)[1]])
+        cand = cand[:10]
+        for k in range(1, min(3, len(cand)) + 1):
+            for flips in itertools.combinations(cand, k):
+                res = rerun(np.array(flips, dtype=np.int64))
+                if ok(res):
+                    self.relu_flips_accepted += k
+                    return res
+        return r        # the strict asserts that follow report the mismatch
 
     def compare_store(self, check_tables: bool = True):
         gpu, cpu = self.gpu, self.cpu

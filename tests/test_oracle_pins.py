@@ -516,3 +516,31 @@ def test_restamp_makes_an_id_reappear_exactly_T_later():
         assert seen[i] == list(range(i + T, 20, T))
     keep = _expiry_oracle(np.array([0], dtype=np.int64), 2)
     assert [len(keep.collect_expired(now, restamp=False)) for now in range(4)] == [0, 0, 1, 1]
+
+
+# ----------------------------------------------------------------------------
+# units whose ReLU decision is within rounding distance of zero
+# ----------------------------------------------------------------------------
+def test_near_zero_units_are_listed_and_can_take_the_other_branch():
+    from oracle import decode_unit
+    orc = GearOracle(np.array([[1.0]]), np.array([[1.0]]), np.array([[2.0]]), (2,), 1, 0)
+    # unit 0: pre-activation 1 + 1 - 2 = 0 exactly; unit 1: clearly active
+    params = np.array([1.0, 0.5, 1.0, 0.5, -1.0, 0.5, 0.0, 0.25, 1.0, -2.0, 0.3])
+    args = ([0], [0], [0, 1], [0], [1.0])
+    r = orc.forward_backward(params, *args, relu_margin=1e-12)
+    assert [decode_unit(c, 1) for c in r.near_units] == [(0, 0, 0)]
+    flipped = orc.forward_backward(params, *args, flip_units=r.near_units)
+    assert flipped.loss == r.loss and np.array_equal(flipped.prob, r.prob)
+    # the other branch is the network whose ReLU has derivative 1 at 0: check against the autodiff library
+    X = torch.tensor(r.X, requires_grad=True)
+    p = torch.tensor(params, requires_grad=True)
+    (W, b), = split_params(p, 3, (2,))[0]
+    a = X @ W + b
+    h = torch.where(a >= 0, a, torch.zeros_like(a))
+    z = h @ p[8:10] + p[10]
+    loss = torch.nn.functional.binary_cross_entropy_with_logits(z, torch.tensor([1.0], dtype=torch.float64))
+    loss.backward()
+    np.testing.assert_allclose(flipped.head_grad, p.grad.numpy(), atol=1e-15)
+    np.testing.assert_allclose(flipped.dX, X.grad.numpy(), atol=1e-15)
+    assert np.any(flipped.dX != r.dX)
+    assert len(orc.forward_backward(params, *args, relu_margin=0.5).near_units) == 1      # |0.25 + ...| unit stays out
