@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Throughput of the Gear Training sparse-part step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload large|medium|tiny]
+
+One "step" is one pass of the whole hot path over one batch of synthetic page views:
+gear_forward_backward (gather, head forward/backward, embedding scatter), gear_accumulate_dfv_grad,
+gear_collect_ready and gear_collect_expired.  Prints ONE JSON line (rank 0).
+
+value      page views/s with the batches already resident in HBM (device-timed, max over ranks)
+e2e        the same with the batch arrays in pinned HOST memory, copied in inside the timed region, and
+           the loss and the two counts read back every step
+roofline   the kernel with the largest share of the step, timed per launch with CUDA events inside the
+           library (a second pass of K steps with profiling on), against the measured machine peaks
+cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload (rank 0, N=1)
+
+With --gpus N > 1 (launched under torchrun) every rank runs an independent replica on its own GPU: the
+path has no exchange step on one GPU and the multi-GPU sharding is not built, so scaling is "weak".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "page views/sec per step (1 B200); gather+accumulate HBM GB/s vs ~8 TB/s peak"
+UNIT = "page views/s"
+N_BATCHES = 8          # distinct pre-generated batches the timed loop cycles through
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], bf16_sustained=d.get("bf16_tflops_sustained"),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# fp32 FMA peak of the plain-ALU head: 148 SMs x 128 lanes x 2 flop x max SM clock
+ALU_F32_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def preset_for(name: str):
+    from paper_1806_03925_b200.workloads import PRESETS
+    return PRESETS[name]
+
+
+# ---------------------------------------------------------------------------------------------
+# algorithmic work per launch of each kernel (bytes the method must move, or flops)
+# ---------------------------------------------------------------------------------------------
+def kernel_models(p, stats):
+    """name -> (bound, work per launch, unit).  stats: per-step means measured on the generated batches."""
+    B, nnz = stats["B"], stats["nnz"]
+    E, D, Din = p.emb_dim, p.dfv_dim, p.d_in
+    dsz = 2 if p.dfv_dtype == "bf16" else 4
+    xsz = 2 if p.head_dtype == "bf16" else 4
+    m = {}
+    m["gather_pool"] = ("hbm", B * 2 * E * 4 + nnz * D * dsz + B * Din * xsz + (3 * B + 1 + 2 * nnz) * 4 + B * 4)
+    # gradient rows: the B pooled-gradient rows are read (each once from HBM; repeats hit L2), one accumulator row
+    # is read (if open) and written per distinct image, complete groups write one averaged row
+    m["acc_reduce"] = ("hbm", B * D * 4 + nnz * 8 + stats["uniq_img"] * (D * 4 + 4) * 2 + stats["n_ready"] * (D * 4 + 4))
+    m["expiry_mark"] = ("hbm", p.img_vocab * 8 + p.img_vocab // 8)
+    m["emb_reduce"] = ("hbm", B * E * 4 + B * 8 + stats["uniq_emb"] * E * 4 * 2)
+    m["collect_move"] = ("hbm", stats["n_ready"] * (D * 4 * 2 + 16))
+    fan = [Din] + list(p.hidden)
+    for l in range(len(p.hidden)):
+        m.setdefault("gemm_flops", []).append(2 * B * fan[l] * fan[l + 1])
+    return m
+
+
+def roofline_for(name, ms_per_launch, p, stats, peaks):
+    """Roofline object of one kernel from its live per-launch time."""
+    models = kernel_models(p, stats)
+    B = stats["B"]
+    fan = [p.d_in] + list(p.hidden)
+    gemm_flops_fwd = sum(2 * B * fan[l] * fan[l + 1] for l in range(len(p.hidden)))
+    sec = ms_per_launch * 1e-3
+    if name in models and isinstance(models[name], tuple):
+        work = models[name][1]
+        ach = work / sec / 1e9
+        return {"kernel": name, "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": None, "peak_source": peaks["source"],
+                "work_per_launch": work}
+    if name.startswith("simt_gemm") or name.startswith("tc_gemm"):
+        # launches of one name share the step's products of that kind evenly
+        per_launch = gemm_flops_fwd / max(len(p.hidden), 1)
+        if name.endswith("dx") or name.endswith("dh"):
+            per_launch = gemm_flops_fwd / max(len(p.hidden), 1)
+        ach = per_launch / sec / 1e12
+        if name.startswith("tc_gemm"):
+            peak, bound = peaks["bf16_sustained"] or peaks["bf16_tflops"], "tensor"
+        else:
+            peak, bound = ALU_F32_TFLOPS, "alu"
+        return {"kernel": name, "bound": bound, "achieved": round(ach, 2), "peak": round(peak, 1), "unit": "TFLOP/s",
+                "frac": round(ach / peak, 4), "traffic": None, "peak_source": peaks["source"] if bound == "tensor"
+                else "148 SMs x 128 FMA lanes x 2 x 1.965 GHz", "work_per_launch": per_launch}
+    return {"kernel": name, "bound": "latency", "achieved": None, "peak": None, "unit": None, "frac": None,
+            "traffic": None}
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle
+# ---------------------------------------------------------------------------------------------
+def oracle_sample_run(p, src, sample_views: int, step: int = 0, seed: int = 0):
+    """One bounded sample of a step on the CPU oracle.  Returns (seconds for the per-view part on the sample,
+    seconds for the expiry scan of the whole timestamp table, views in the sample)."""
+    import oracle
+    from oracle import GearOracle
+    b = src.batch(step)
+    views = slice(0, min(sample_views, b.B))
+    nv = views.stop
+    off = b.img_off[:nv + 1].astype(np.int32)
+    img = b.img_id[:off[-1]]
+    uid, hid = b.user_id[:nv], b.url_id[:nv]
+    ru, iu = np.unique(uid, return_inverse=True)
+    rh, ih = np.unique(hid, return_inverse=True)
+    ri, ii = np.unique(img, return_inverse=True)
+    dfv_np = np.uint16 if p.dfv_dtype == "bf16" else np.float32
+    orc = GearOracle(oracle.fill_rows(seed, oracle.TAG_USER, p.emb_dim, ru, len(ru), np.float32),
+                     oracle.fill_rows(seed, oracle.TAG_URL, p.emb_dim, rh, len(rh), np.float32),
+                     oracle.fill_rows(seed, oracle.TAG_DFV, p.dfv_dim, ri, len(ri), dfv_np),
+                     p.hidden, p.M, p.expire, round_bf16=(p.head_dtype == "bf16"),
+                     ts=oracle.fill_ts(seed, p.expire, 0, None, p.img_vocab))
+    from paper_1806_03925_b200 import workloads
+    params = workloads.head_params(p, seed).astype(np.float64)
+    t0 = time.perf_counter()
+    r = orc.forward_backward(params, iu.astype(np.int32), ih.astype(np.int32), off, ii.astype(np.int32), b.label[:nv])
+    orc.emb_apply("user", iu.astype(np.int32), r.dX, -p.lr)
+    orc.emb_apply("url", ih.astype(np.int32), r.dX, -p.lr)
+    orc.accumulate(ii.astype(np.int32), orc.dfv_grad_rows(off, r.dX))
+    orc.collect_ready()
+    t1 = time.perf_counter()
+    orc.collect_expired(step + 1, True)
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1, nv
+
+
+def cpu_baseline(p, src, sample_views: int):
+    t_views, t_exp, nv = oracle_sample_run(p, src, sample_views)
+    step_s = t_views * (p.batch / nv) + t_exp
+    return {"value": round(p.batch / step_s, 1), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "first %d of the %d views of one %s step (gather, head, embedding apply, accumulate, collect) "
+                      "scaled to the full batch, plus one expiry scan of all %d timestamps; %.1f s of CPU time"
+                      % (nv, p.batch, p.name, p.img_vocab, t_views + t_exp)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_1806_03925_b200.workloads import BatchSource
+    p = preset_for(args.workload)
+    src = BatchSource(p, 0)
+    sample = {"large": 1024, "medium": 1024, "tiny": 256}.get(args.workload, 512)
+    times = []
+    for s in range(args.warmup + args.steps):
+        t_views, t_exp, nv = oracle_sample_run(p, src, sample, step=s % 2)
+        if s >= args.warmup:
+            times.append(t_views * (p.batch / nv) + t_exp)
+    step_s = float(np.mean(times))
+    value = p.batch / step_s
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(step_s * 1e3, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "%s tables" % p.name if p.name == "large" else p.name, "batch": p.batch,
+                       "note": "CPU oracle, one thread; each step is a sample of %d views scaled to the batch" % sample},
+            "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": "%d views per step scaled to %d, plus the full expiry scan" % (sample, p.batch)},
+            "e2e": {"value": round(value, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1806_03925_b200 import binding as gb
+    from paper_1806_03925_b200 import workloads
+    from paper_1806_03925_b200.session import DeviceBatch, GearSession
+    from paper_1806_03925_b200.workloads import BatchSource
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libgear has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    gb.load()
+    p = preset_for(args.workload)
+    K, W = args.steps, args.warmup
+    seed = rank                                   # every replica draws its own tables and batches
+    src = BatchSource(p, seed)
+    host_batches = [src.batch(s) for s in range(N_BATCHES)]
+    max_nnz = max(b.nnz for b in host_batches)
+    sess = GearSession(p, workloads.head_params(p, seed), max_batch=p.batch, max_nnz=max_nnz, seed=seed, fill=True,
+                       now=0, expired_cap=p.img_vocab)
+    dev_batches = [DeviceBatch.from_host(b) for b in host_batches]
+    pinned = [[torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in
+               (b.user_id, b.url_id, b.img_off, b.img_id, b.label)] for b in host_batches]
+    h2d_bytes = int(np.mean([sum(t.numel() * t.element_size() for t in pb) for pb in pinned]))
+    stats = {"B": p.batch, "nnz": float(np.mean([b.nnz for b in host_batches])),
+             "uniq_img": float(np.mean([len(np.unique(b.img_id)) for b in host_batches])),
+             "uniq_emb": float(np.mean([(len(np.unique(b.user_id)) + len(np.unique(b.url_id))) / 2 for b in host_batches]))}
+
+    stream = torch.cuda.current_stream()
+    now = [0]
+
+    def one_step(db):
+        now[0] += 1
+        sess.step(db, now[0], sync=False)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record(stream)
+        for s in range(steps):
+            fn(s)
+        ev1.record(stream)
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    # ---- device-resident throughput
+    for s in range(W):
+        one_step(dev_batches[s % N_BATCHES])
+    launches0 = gb.gear_launch_count(sess.ctx)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms = timed(lambda s: one_step(dev_batches[s % N_BATCHES]), K)
+    clocks = sampler.stop()
+    launches = gb.gear_launch_count(sess.ctx) - launches0
+    rc, status, _ = sess.status()
+    n_ready_mean = None
+
+    # ---- end to end: host batches in, loss and counts out, every step
+    stage = DeviceBatch(*(torch.empty_like(t, device="cuda") for t in
+                          (dev_batches[0].user_id, dev_batches[0].url_id, dev_batches[0].img_off,
+                           torch.empty(max_nnz, dtype=torch.int32), dev_batches[0].label)), B=p.batch, nnz=0)
+    host_out = torch.zeros(4, dtype=torch.float32).pin_memory()
+    host_cnt = torch.zeros(2, dtype=torch.int64).pin_memory()
+
+    def e2e_step(s):
+        pb, hb = pinned[s % N_BATCHES], host_batches[s % N_BATCHES]
+        stage.user_id.copy_(pb[0], non_blocking=True)
+        stage.url_id.copy_(pb[1], non_blocking=True)
+        stage.img_off.copy_(pb[2], non_blocking=True)
+        stage.img_id[:hb.nnz].copy_(pb[3], non_blocking=True)
+        stage.label.copy_(pb[4], non_blocking=True)
+        stage.nnz = hb.nnz
+        one_step(stage)
+        host_out[0:1].copy_(sess.loss, non_blocking=True)
+        host_cnt.copy_(sess.d_counts, non_blocking=True)
+        stream.synchronize()                       # the caller reads the loss and the counts of this step
+
+    for s in range(min(W, 3)):
+        e2e_step(s)
+    ms_e2e = timed(e2e_step, K)
+    d2h_bytes = 4 + 16
+
+    # ---- per-kernel timing pass (profiling on; not part of the throughput numbers)
+    ready_counts = []
+    gb.gear_profile_enable(sess.ctx, True)
+    for s in range(K):
+        one_step(dev_batches[s % N_BATCHES])
+        ready_counts.append(int(sess.d_counts[0].item()))
+    prof = gb.gear_profile_read(sess.ctx, 64)
+    gb.gear_profile_enable(sess.ctx, False)
+    stats["n_ready"] = float(np.mean(ready_counts)) if ready_counts else 0.0
+    total_ms = sum(v[0] for v in prof.values()) or 1.0
+    kernels = sorted(({"name": k, "launches_per_step": v[1] / K, "ms_per_step": v[0] / K, "share": v[0] / total_ms,
+                       "ms_per_launch": v[0] / v[1]} for k, v in prof.items()), key=lambda d: -d["ms_per_step"])
+    peaks = measured_peaks()
+    top = kernels[0]
+    roof = roofline_for(top["name"], top["ms_per_launch"], p, stats, peaks)
+    hbm_kernels = []
+    for kd in kernels:
+        r = roofline_for(kd["name"], kd["ms_per_launch"], p, stats, peaks)
+        if r["bound"] == "hbm":
+            hbm_kernels.append({"kernel": kd["name"], "GB/s": r["achieved"], "frac_of_measured": r["frac"],
+                                "frac_of_8TBs": round(r["achieved"] / 8000.0, 4), "ms": round(kd["ms_per_launch"], 4)})
+
+    views = p.batch * K * world
+    line = {"metric": METRIC, "value": round(views / (ms * 1e-3), 1), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if p.head_dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": "large tables" if p.name == "large" else p.name, "batch": p.batch,
+                       "tables_gb": round((p.user_vocab + p.url_vocab) * p.emb_dim * 4 / 1e9 + p.img_vocab * p.dfv_dim *
+                                          ((2 if p.dfv_dtype == "bf16" else 4) + 4) / 1e9 + p.img_vocab * 12 / 1e9, 1),
+                       "M": p.M, "expire": p.expire, "mean_nnz": round(stats["nnz"], 1),
+                       "l2": "tables far exceed the 126 MB L2 and rows are Zipf-random; %d pre-generated batches cycle; "
+                             "no explicit flush" % N_BATCHES,
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks,
+            "e2e": {"value": round(views / (ms_e2e * 1e-3), 1), "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,
+                    "d2h_bytes_per_step": d2h_bytes, "ms_per_step": round(ms_e2e / K, 4)},
+            "gpu_launches": int(launches),
+            "roofline": roof,
+            "kernels": [{"name": k["name"], "ms_per_step": round(k["ms_per_step"], 4), "share": round(k["share"], 4),
+                         "launches_per_step": round(k["launches_per_step"], 2)} for k in kernels[:12]],
+            "hbm_kernels": hbm_kernels,
+            "device_status": status}
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            sample = {"large": 4096, "medium": 4096, "tiny": 256}.get(args.workload, 1024)
+            line["cpu_baseline"] = cpu_baseline(p, BatchSource(p, 0), sample)
+        else:
+            line["cpu_baseline"] = None
+        print(json.dumps(line), flush=True)
+    sess.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=["large", "medium", "tiny", "skew"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -218,6 +218,18 @@ int gear_destroy(gear_ctx* ctx);
 int gear_fill_uniform(void* dst, int32_t dtype, int64_t n_rows, int32_t dim, uint64_t seed, uint64_t tag,
                       double amp, void* stream);
 
+/*
+ * Per-kernel timing (not part of the paper).  While enabled, every kernel the library launches for this
+ * ctx is bracketed by a pair of CUDA events on the caller's stream.  gear_profile_read synchronises,
+ * sums the elapsed time and the launch count per kernel name since the last read or enable, writes up to
+ * cap entries (names: cap rows of 64 chars, NUL-terminated; total_ms, launches: cap entries) and clears
+ * the records.  Event records cost a few microseconds each: do not time throughput with profiling on.
+ * gear_launch_count returns the number of kernels this ctx has launched since it was created.
+ */
+int gear_profile_enable(gear_ctx* ctx, int on);
+int gear_profile_read(gear_ctx* ctx, char* names, float* total_ms, int32_t* launches, int32_t cap, int32_t* n_out);
+int gear_launch_count(gear_ctx* ctx, int64_t* n_launches);
+
 /* Last CUDA error string seen by the library on this thread ("" if none).  Host-only. */
 const char* gear_last_error(void);
 

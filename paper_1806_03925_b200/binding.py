@@ -24,7 +24,7 @@ GEAR_TAG_USER, GEAR_TAG_URL, GEAR_TAG_DFV, GEAR_TAG_TS, GEAR_TAG_GRAD = 1, 2, 3,
 
 EXPORTS = ("gear_workspace_bytes", "gear_init_tables", "gear_forward_backward", "gear_accumulate_dfv_grad",
            "gear_collect_ready", "gear_collect_expired", "gear_status", "gear_destroy", "gear_fill_uniform",
-           "gear_last_error")
+           "gear_last_error", "gear_profile_enable", "gear_profile_read", "gear_launch_count")
 
 
 class GearError(RuntimeError):
@@ -89,6 +89,12 @@ def load() -> C.CDLL:
     L.gear_destroy.argtypes = [vp]
     L.gear_fill_uniform.restype = C.c_int
     L.gear_fill_uniform.argtypes = [vp, i32, i64, i32, u64, u64, C.c_double, vp]
+    L.gear_profile_enable.restype = C.c_int
+    L.gear_profile_enable.argtypes = [vp, C.c_int]
+    L.gear_profile_read.restype = C.c_int
+    L.gear_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_float), C.POINTER(i32), i32, C.POINTER(i32)]
+    L.gear_launch_count.restype = C.c_int
+    L.gear_launch_count.argtypes = [vp, C.POINTER(i64)]
     L.gear_last_error.restype = C.c_char_p
     L.gear_last_error.argtypes = []
     _lib = L
@@ -210,3 +216,27 @@ def gear_status(ctx, raise_on_error: bool = False):
 
 def gear_destroy(ctx):
     return _check(load().gear_destroy(ctx), "gear_destroy")
+
+
+def gear_profile_enable(ctx, on: bool):
+    return _check(load().gear_profile_enable(ctx, 1 if on else 0), "gear_profile_enable")
+
+
+def gear_profile_read(ctx, cap: int = 64):
+    """{kernel name: (total ms, launches)} since the last read; synchronises."""
+    names = C.create_string_buffer(64 * cap)
+    ms = (C.c_float * cap)()
+    cnt = (C.c_int32 * cap)()
+    n = C.c_int32(0)
+    _check(load().gear_profile_read(ctx, names, ms, cnt, cap, C.byref(n)), "gear_profile_read")
+    out = {}
+    for k in range(n.value):
+        name = names.raw[64 * k:64 * (k + 1)].split(b"\0", 1)[0].decode()
+        out[name] = (float(ms[k]), int(cnt[k]))
+    return out
+
+
+def gear_launch_count(ctx) -> int:
+    n = C.c_int64(0)
+    _check(load().gear_launch_count(ctx, C.byref(n)), "gear_launch_count")
+    return n.value

@@ -322,29 +322,34 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     const int D = c.cfg.dfv_dim, M = c.cfg.M;
     SortBufs sb = c.sort_bufs();
     DevState* state = c.state();
-    acc_keys_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(img_id, n, vocab, sb.keys[0], state);
-    const int cur = radix_sort_pairs(sb, n, nullptr, bits_for(vocab), true, st);
+    { KernelScope ks(&c.prof, "acc_keys", st);
+    acc_keys_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(img_id, n, vocab, sb.keys[0], state); }
+    const int cur = radix_sort_pairs(sb, n, nullptr, bits_for(vocab), true, st, &c.prof);
     const uint32_t* ks = sb.keys[cur];
     const int64_t n_tiles = ceil_div(n, AF_TILE);
     uint2* tile_cnt = c.at<uint2>(c.ws.tile_cnt);
-    acc_flag_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt, state);
-    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st);
+    { KernelScope k(&c.prof, "acc_flag", st);
+    acc_flag_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt, state); }
+    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, &c.prof);
     uint32_t* grp_start = c.at<uint32_t>(c.ws.grp_start);
     int32_t* grp_slot = c.at<int32_t>(c.ws.grp_slot);
+    { KernelScope k(&c.prof, "acc_plan", st);
     acc_plan_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt,
-                                                            grp_start, grp_slot, state);
+                                                            grp_start, grp_slot, state); }
     RowSource rs{sb.vals[cur], grads, ld, src_row, scale};
     const int nq = (int)ceil_div(D / 4, 32);
     int64_t want = ceil_div(n, 8);
     const int grid = (int)(want < reduce_grid() ? (want < 1 ? 1 : want) : reduce_grid());
 #define GEAR_ACC_LAUNCH(NQ) acc_reduce_kernel<NQ><<<grid, 256, 0, st>>>(ks, rs, D, M, n_tiles, c.ws.ready_cap, tile_cnt, \
         grp_start, grp_slot, c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id), c.at<float>(c.ws.q_avg), state)
+    { KernelScope k(&c.prof, "acc_reduce", st);
     if (nq <= 1) GEAR_ACC_LAUNCH(1);
     else if (nq <= 2) GEAR_ACC_LAUNCH(2);
     else if (nq <= 4) GEAR_ACC_LAUNCH(4);
-    else GEAR_ACC_LAUNCH(8);
+    else GEAR_ACC_LAUNCH(8); }
 #undef GEAR_ACC_LAUNCH
-    acc_commit_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, c.ws.ready_cap, state);
+    { KernelScope k(&c.prof, "acc_commit", st);
+    acc_commit_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, c.ws.ready_cap, state); }
     return cudaGetLastError();
 }
 
@@ -397,16 +402,20 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     DevState* state = c.state();
     SortBufs sb = c.sort_bufs();
     const int64_t n_max = c.ws.ready_cap;
-    collect_begin_kernel<<<1, 1, 0, st>>>(state, cap, d_n);
+    { KernelScope k(&c.prof, "collect_begin", st);
+    collect_begin_kernel<<<1, 1, 0, st>>>(state, cap, d_n); }
     int64_t blocks = ceil_div(n_max, 256);
+    { KernelScope k(&c.prof, "collect_keys", st);
     collect_keys_kernel<<<(unsigned)(blocks > 1184 ? 1184 : blocks), 256, 0, st>>>(c.at<int32_t>(c.ws.q_id), state,
-                                                                                 sb.keys[0]);
-    const int cur = radix_sort_pairs(sb, n_max, &state->collect_n, bits_for(c.cfg.img_vocab), true, st);
+                                                                                 sb.keys[0]); }
+    const int cur = radix_sort_pairs(sb, n_max, &state->collect_n, bits_for(c.cfg.img_vocab), true, st, &c.prof);
     int64_t want = ceil_div(n_max, 8);
+    { KernelScope k(&c.prof, "collect_move", st);
     collect_move_kernel<<<(unsigned)(want > 1184 ? 1184 : want), 256, 0, st>>>(sb.keys[cur], sb.vals[cur],
                                                                             c.at<float>(c.ws.q_avg), c.cfg.dfv_dim,
-                                                                            state, ids, seq, avg);
-    collect_end_kernel<<<1, 1, 0, st>>>(state);
+                                                                            state, ids, seq, avg); }
+    { KernelScope k(&c.prof, "collect_end", st);
+    collect_end_kernel<<<1, 1, 0, st>>>(state); }
     return cudaGetLastError();
 }
 

@@ -273,6 +273,50 @@ int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready) {
     return GEAR_OK;
 }
 
+int gear_profile_enable(gear_ctx* ctx, int on) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    cudaStreamSynchronize(ctx->impl.last_stream);
+    ctx->impl.prof.clear();
+    ctx->impl.prof.on = on != 0;
+    return GEAR_OK;
+}
+
+int gear_profile_read(gear_ctx* ctx, char* names, float* total_ms, int32_t* launches, int32_t cap, int32_t* n_out) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    if (!n_out || cap < 0 || (cap > 0 && (!names || !total_ms || !launches))) return arg_fail("gear_profile_read");
+    gear_ctx_impl& c = ctx->impl;
+    cudaError_t e = cudaStreamSynchronize(c.last_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "gear_profile_read");
+    int n = 0;
+    for (const auto& r : c.prof.recs) {
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, r.start, r.stop);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventElapsedTime");
+        int k = 0;
+        while (k < n && strncmp(names + 64 * k, r.name, 63) != 0) ++k;
+        if (k == n) {
+            if (n >= cap) continue;
+            strncpy(names + 64 * k, r.name, 63);
+            names[64 * k + 63] = 0;
+            total_ms[k] = 0.f;
+            launches[k] = 0;
+            ++n;
+        }
+        total_ms[k] += ms;
+        launches[k] += 1;
+    }
+    *n_out = n;
+    c.prof.clear();
+    return GEAR_OK;
+}
+
+int gear_launch_count(gear_ctx* ctx, int64_t* n_launches) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    if (!n_launches) return arg_fail("NULL pointer");
+    *n_launches = ctx->impl.prof.launches;
+    return GEAR_OK;
+}
+
 int gear_destroy(gear_ctx* ctx) {
     if (!ctx) return GEAR_OK;
     if (!ctx->impl.alive) return GEAR_ERR_STATE;

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "../../include/gear.h"
 
 namespace gear {
@@ -86,6 +88,46 @@ __device__ __forceinline__ void red_add_f4(float* p, float4 v) {
                  :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
+// ---------------------------------------------------------------- launch accounting / per-kernel timing
+// Every kernel launch of the library goes through a KernelScope: it counts the launch and, when profiling
+// is on, brackets it with a pair of CUDA events on the caller's stream (read back by gear_profile_read).
+struct Profiler {
+    struct Rec { const char* name; cudaEvent_t start, stop; };
+    bool on = false;
+    int64_t launches = 0;
+    std::vector<Rec> recs;
+    std::vector<cudaEvent_t> pool;
+    cudaEvent_t get() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+    void clear() {
+        for (auto& r : recs) { pool.push_back(r.start); pool.push_back(r.stop); }
+        recs.clear();
+    }
+    ~Profiler() {
+        clear();
+        for (auto e : pool) cudaEventDestroy(e);
+    }
+};
+
+struct KernelScope {
+    Profiler* p; cudaStream_t st; cudaEvent_t stop = nullptr;
+    KernelScope(Profiler* prof, const char* name, cudaStream_t s) : p(prof), st(s) {
+        if (!p) return;
+        ++p->launches;
+        if (p->on) {
+            Profiler::Rec r{name, p->get(), p->get()};
+            stop = r.stop;
+            cudaEventRecord(r.start, st);
+            p->recs.push_back(r);
+        }
+    }
+    ~KernelScope() { if (stop) cudaEventRecord(stop, st); }
+};
+
 // ---------------------------------------------------------------- radix sort / scans (prims.cu)
 constexpr int RS_THREADS = 256;
 constexpr int RS_ITEMS = 16;
@@ -106,10 +148,10 @@ inline int64_t sort_tiles(int64_t n_max) { return n_max > 0 ? ceil_div(n_max, RS
 // n_dev (optional, device) caps the element count at min(*n_dev, n_max).  Returns the index (0 or 1)
 // of the buffer pair that holds the sorted result.
 int radix_sort_pairs(const SortBufs& bufs, int64_t n_max, const int64_t* n_dev, int bits, bool identity_vals,
-                     cudaStream_t st);
+                     cudaStream_t st, Profiler* prof);
 
 // In-place exclusive scan of m (a, b) counter pairs by one block; the totals go to total[0..1].
-void scan_pairs(uint2* data, int64_t m, uint2* total, cudaStream_t st);
+void scan_pairs(uint2* data, int64_t m, uint2* total, cudaStream_t st, Profiler* prof);
 
 inline int bits_for(int64_t max_key_inclusive) {
     int b = 1;

@@ -79,8 +79,9 @@ cudaError_t launch_emb_scatter(const gear_ctx_impl& c, const int32_t* ids, int32
                                const float* dX, int ldx, int col0, float alpha, cudaStream_t st) {
     if (B <= 0) return cudaSuccess;
     SortBufs sb = c.sort_bufs();
-    emb_keys_kernel<<<(unsigned)ceil_div(B, 256), 256, 0, st>>>(ids, B, vocab, sb.keys[0]);
-    const int cur = radix_sort_pairs(sb, B, nullptr, bits_for(vocab), true, st);
+    { KernelScope ks(&c.prof, "emb_keys", st);
+    emb_keys_kernel<<<(unsigned)ceil_div(B, 256), 256, 0, st>>>(ids, B, vocab, sb.keys[0]); }
+    const int cur = radix_sort_pairs(sb, B, nullptr, bits_for(vocab), true, st, &c.prof);
     const int E = c.cfg.emb_dim, n_chunks = E / 4;
     int lpr = 1;
     while (lpr < n_chunks && lpr < 32) lpr <<= 1;
@@ -89,6 +90,7 @@ cudaError_t launch_emb_scatter(const gear_ctx_impl& c, const int32_t* ids, int32
     const unsigned grid = (unsigned)ceil_div(groups * lpr, 256);
 #define GEAR_ES_LAUNCH(NQ) emb_reduce_kernel<NQ><<<grid, 256, 0, st>>>(sb.keys[cur], sb.vals[cur], B, (uint32_t)vocab, \
                                                                         E, lpr, dX, ldx, col0, table, alpha)
+    KernelScope ks(&c.prof, "emb_reduce", st);
     if (nq <= 1) GEAR_ES_LAUNCH(1);
     else if (nq <= 2) GEAR_ES_LAUNCH(2);
     else if (nq <= 4) GEAR_ES_LAUNCH(4);

@@ -77,11 +77,14 @@ cudaError_t launch_collect_expired(const gear_ctx_impl& c, int64_t now, int rest
     const int64_t n_tiles = ceil_div(vocab, EXP_TILE);
     uint32_t* bits = c.at<uint32_t>(c.ws.exp_bits);
     uint2* tile_cnt = c.at<uint2>(c.ws.exp_cnt);
-    expiry_mark_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(c.buf.dfv_ts, vocab, now, c.cfg.expire, bits, tile_cnt);
-    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st);
-    expiry_check_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, cap, d_n, c.state());
+    { KernelScope k(&c.prof, "expiry_mark", st);
+    expiry_mark_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(c.buf.dfv_ts, vocab, now, c.cfg.expire, bits, tile_cnt); }
+    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, &c.prof);
+    { KernelScope k(&c.prof, "expiry_check", st);
+    expiry_check_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, cap, d_n, c.state()); }
+    { KernelScope k(&c.prof, "expiry_write", st);
     expiry_write_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(bits, vocab, tile_cnt, c.state(), now, restamp,
-                                                                  c.buf.dfv_ts, ids);
+                                                                  c.buf.dfv_ts, ids); }
     return cudaGetLastError();
 }
 

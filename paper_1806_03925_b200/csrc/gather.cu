@@ -145,13 +145,14 @@ gather_pool_kernel(const GatherArgs a) {
 }
 
 template <typename TD, typename TX>
-static cudaError_t dispatch_nq(const GatherArgs& a, cudaStream_t st) {
+static cudaError_t dispatch_nq(const GatherArgs& a, cudaStream_t st, Profiler* prof) {
     constexpr int PER = Chunk<TD>::PER;
     const int n_chunks = a.D / PER;
     const int nq = (n_chunks + 31) / 32;
     const int warps = 8;
     int grid = (int)ceil_div(a.B, warps);
     if (grid < 1) grid = 1;
+    KernelScope ks(prof, "gather_pool", st);
     if (nq <= 1) gather_pool_kernel<TD, TX, 1><<<grid, warps * 32, 0, st>>>(a);
     else if (nq <= 2) gather_pool_kernel<TD, TX, 2><<<grid, warps * 32, 0, st>>>(a);
     else if (nq <= 4) gather_pool_kernel<TD, TX, 4><<<grid, warps * 32, 0, st>>>(a);
@@ -170,10 +171,10 @@ cudaError_t launch_gather(const gear_ctx_impl& c, const gear_batch& b, int32_t* 
     a.X = c.at<void>(c.ws.x); a.x_debug = x_debug; a.row_view = row_view; a.inv_n = inv_n;
     a.state = c.state();
     const bool dbf = c.cfg.dfv_dtype == GEAR_BF16, xbf = c.cfg.head_dtype == GEAR_BF16;
-    if (dbf && xbf) return dispatch_nq<__nv_bfloat16, __nv_bfloat16>(a, st);
-    if (dbf && !xbf) return dispatch_nq<__nv_bfloat16, float>(a, st);
-    if (!dbf && xbf) return dispatch_nq<float, __nv_bfloat16>(a, st);
-    return dispatch_nq<float, float>(a, st);
+    if (dbf && xbf) return dispatch_nq<__nv_bfloat16, __nv_bfloat16>(a, st, &c.prof);
+    if (dbf && !xbf) return dispatch_nq<__nv_bfloat16, float>(a, st, &c.prof);
+    if (!dbf && xbf) return dispatch_nq<float, __nv_bfloat16>(a, st, &c.prof);
+    return dispatch_nq<float, float>(a, st, &c.prof);
 }
 
 }  // namespace gear

@@ -89,8 +89,9 @@ gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sam, int64_t 
 template <typename TA, typename TB, typename TC, typename TM, int EPI>
 static void launch_gemm(int M, int N, int K, const TA* A, int64_t sam, int64_t sak, const TB* B, int64_t sbk,
                         int64_t sbn, TC* C, int64_t ldc, const float* bias, const TM* mask, int64_t ldm,
-                        int splits, cudaStream_t st) {
+                        int splits, cudaStream_t st, Profiler* prof, const char* name) {
     if (M <= 0 || N <= 0 || K <= 0) return;
+    KernelScope ks(prof, name, st);
     int k_chunk = (int)ceil_div(ceil_div(K, splits), GK) * GK;
     splits = (int)ceil_div(K, k_chunk);
     dim3 grid((unsigned)ceil_div(N, GT), (unsigned)ceil_div(M, GT), (unsigned)splits);
@@ -240,6 +241,7 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
     for (int l = 0; l < L; ++l) {
         if (BF) {
             __nv_bfloat16* wb = c.at<__nv_bfloat16>(c.ws.wb[l]);
+            KernelScope ks(&c.prof, "round_weights", st);
             round_weights_kernel<<<64, 256, 0, st>>>(p.fan[l], p.fan[l + 1], p.W[l], wb,
                                                      c.at<__nv_bfloat16>(c.ws.wbt[l]));
             Wop[l] = wb;
@@ -251,28 +253,34 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
     for (int l = 0; l < L; ++l) {
         const int K = p.fan[l], N = p.fan[l + 1];
         launch_gemm<TX, TX, TX, TX, EPI_BIAS_RELU>(B, N, K, H[l], K, 1, static_cast<const TX*>(Wop[l]), N, 1,
-                                                    H[l + 1], N, p.b[l], (const TX*)nullptr, 0, 1, st);
+                                                    H[l + 1], N, p.b[l], (const TX*)nullptr, 0, 1, st, &c.prof,
+                                                    "simt_gemm_fwd");
     }
     const int HT = p.fan[L];
+    { KernelScope ks(&c.prof, "head_out", st);
     head_out_kernel<TX><<<c.ws.loss_blocks, 256, 0, st>>>(B, HT, H[L], p.w_out, p.b_out, bt.label, o.prob, dz, dA[L],
-                                                          loss_part);
-    loss_final_kernel<<<1, 256, 0, st>>>(loss_part, c.ws.loss_blocks, B, o.loss);
+                                                          loss_part); }
+    { KernelScope ks(&c.prof, "loss_final", st);
+    loss_final_kernel<<<1, 256, 0, st>>>(loss_part, c.ws.loss_blocks, B, o.loss); }
     // backward
     const int rows = 128;
-    colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, HT, H[L], dz, p.gw_out, rows);
-    sum_vec_kernel<<<1, 1024, 0, st>>>(B, dz, p.gb_out);
+    { KernelScope ks(&c.prof, "colsum", st);
+    colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, HT, H[L], dz, p.gw_out, rows); }
+    { KernelScope ks(&c.prof, "sum_vec", st);
+    sum_vec_kernel<<<1, 1024, 0, st>>>(B, dz, p.gb_out); }
     for (int l = L - 1; l >= 0; --l) {
         const int K = p.fan[l], N = p.fan[l + 1];
         // dW_l = H_l^T dA_{l+1}
         launch_gemm<TX, TX, float, TX, EPI_ATOMIC>(K, N, B, H[l], 1, K, dA[l + 1], N, 1, p.gW[l], N, nullptr,
-                                                   (const TX*)nullptr, 0, splits_for(K, N, B), st);
-        colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, N, dA[l + 1], nullptr, p.gb[l], rows);
+                                                   (const TX*)nullptr, 0, splits_for(K, N, B), st, &c.prof, "simt_gemm_dw");
+        { KernelScope ks(&c.prof, "colsum", st);
+        colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, N, dA[l + 1], nullptr, p.gb[l], rows); }
         if (l > 0) {
             launch_gemm<TX, TX, TX, TX, EPI_MASK>(B, K, N, dA[l + 1], N, 1, static_cast<const TX*>(Wop[l]), 1, N,
-                                                  dA[l], K, nullptr, H[l], K, 1, st);
+                                                  dA[l], K, nullptr, H[l], K, 1, st, &c.prof, "simt_gemm_dh");
         } else {
             launch_gemm<TX, TX, float, TX, EPI_NONE>(B, K, N, dA[l + 1], N, 1, static_cast<const TX*>(Wop[l]), 1, N,
-                                                     o.dX, K, nullptr, (const TX*)nullptr, 0, 1, st);
+                                                     o.dX, K, nullptr, (const TX*)nullptr, 0, 1, st, &c.prof, "simt_gemm_dx");
         }
     }
     return cudaGetLastError();

@@ -49,6 +49,7 @@ struct gear_ctx_impl {
     cudaStream_t last_stream;
     bool alive;
     void* tc_state;     // tensor-core head state (tensor maps), owned by head_tc.cu; may be null
+    mutable Profiler prof;
 
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(static_cast<char*>(buf.workspace) + off); }
     DevState* state() const { return at<DevState>(ws.state); }

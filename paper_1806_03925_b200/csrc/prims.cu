@@ -116,7 +116,7 @@ radix_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restric
 }
 
 int radix_sort_pairs(const SortBufs& b, int64_t n_max, const int64_t* n_dev, int bits, bool identity_vals,
-                     cudaStream_t st) {
+                     cudaStream_t st, Profiler* prof) {
     if (n_max <= 0) return 0;
     const int n_tiles = (int)sort_tiles(n_max);
     const int passes = (bits + 7) / 8;
@@ -125,11 +125,14 @@ int radix_sort_pairs(const SortBufs& b, int64_t n_max, const int64_t* n_dev, int
     for (int p = 0; p < passes; ++p) {
         const int shift = p * width;
         const uint32_t mask = (1u << width) - 1u;
-        radix_hist_kernel<<<n_tiles, RS_THREADS, 0, st>>>(b.keys[cur], n_max, n_dev, shift, mask, b.hist, n_tiles);
-        radix_scan_rows_kernel<<<RS_BUCKETS, RS_THREADS, 0, st>>>(b.hist, b.tot, n_tiles);
+        { KernelScope k(prof, "radix_hist", st);
+        radix_hist_kernel<<<n_tiles, RS_THREADS, 0, st>>>(b.keys[cur], n_max, n_dev, shift, mask, b.hist, n_tiles); }
+        { KernelScope k(prof, "radix_scan_rows", st);
+        radix_scan_rows_kernel<<<RS_BUCKETS, RS_THREADS, 0, st>>>(b.hist, b.tot, n_tiles); }
         const uint32_t* vin = (p == 0 && identity_vals) ? nullptr : b.vals[cur];
+        { KernelScope k(prof, "radix_scatter", st);
         radix_scatter_kernel<<<n_tiles, RS_THREADS, 0, st>>>(b.keys[cur], vin, b.keys[cur ^ 1], b.vals[cur ^ 1],
-                                                             n_max, n_dev, shift, mask, b.hist, b.tot, n_tiles);
+                                                             n_max, n_dev, shift, mask, b.hist, b.tot, n_tiles); }
         cur ^= 1;
     }
     return cur;
@@ -153,7 +156,8 @@ scan_pairs_kernel(uint2* __restrict__ data, int64_t m, uint2* __restrict__ total
     if (threadIdx.x == 0) *total = make_uint2(ca, cb);
 }
 
-void scan_pairs(uint2* data, int64_t m, uint2* total, cudaStream_t st) {
+void scan_pairs(uint2* data, int64_t m, uint2* total, cudaStream_t st, Profiler* prof) {
+    KernelScope k(prof, "scan_pairs", st);
     scan_pairs_kernel<<<1, 1024, 0, st>>>(data, m, total);
 }
 
