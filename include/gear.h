@@ -75,7 +75,8 @@ enum {
     GEAR_DEV_BAD_ID = 1,         /* an ID outside [0, vocab) was skipped */
     GEAR_DEV_READY_OVERFLOW = 2, /* an accumulate call would have overflowed the ready queue and was dropped whole */
     GEAR_DEV_OUT_CAPACITY = 4,   /* a collect call found cap too small and left everything in place */
-    GEAR_DEV_BAD_CSR = 8         /* img_off not non-decreasing / not ending at nnz */
+    GEAR_DEV_BAD_CSR = 8,        /* img_off not non-decreasing / not ending at nnz */
+    GEAR_DEV_TIMEOUT = 16        /* a bounded wait inside a kernel gave up; the step's results are invalid */
 };
 
 /* tags of the procedural table fill (SplitMix64 streams, see gear_fill_uniform) */
@@ -176,6 +177,10 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
  * a call may complete several groups of one image.  grads rows must be 16-byte aligned (ld multiple of 4).
  * If the queue cannot take every group the call completes, the whole call is dropped and
  * GEAR_DEV_READY_OVERFLOW is raised.
+ * img_id == NULL means "the image occurrences of the batch of the most recent gear_forward_backward on
+ * this ctx" (n must equal that batch's nnz; the batch's img_id array must not have changed): their IDs
+ * were already key-sorted during that call, so the sort is not repeated.  GEAR_ERR_STATE if there is no
+ * such batch.
  */
 int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* grads, int64_t ld,
                              const int32_t* src_row, const float* scale, int64_t n, void* stream);

@@ -32,19 +32,6 @@ constexpr int AF_THREADS = 256;
 constexpr int AF_ITEMS = 4;
 constexpr int AF_TILE = AF_THREADS * AF_ITEMS;
 
-__global__ void __launch_bounds__(256)
-acc_keys_kernel(const int32_t* __restrict__ ids, int64_t n, int64_t vocab, uint32_t* __restrict__ keys,
-                DevState* __restrict__ state) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i == 0) { state->n_valid = 0; }
-    if (i < n) {
-        const int id = ids[i];
-        const bool ok = id >= 0 && id < vocab;
-        keys[i] = ok ? (uint32_t)id : (uint32_t)vocab;
-        if (!ok) atomicOr(&state->status, GEAR_DEV_BAD_ID);
-    }
-}
-
 __device__ __forceinline__ uint32_t warp_inclusive_max(uint32_t v) {
     const unsigned lane = lane_id();
 #pragma unroll
@@ -132,6 +119,7 @@ __device__ __forceinline__ void tile_flags(TileFlags& f, const uint32_t* __restr
         }
         if (i + 1 == n || ks[i + 1] >= vocab) state->n_valid = i + 1;   // exactly one thread sees this
     }
+    if (blockIdx.x == 0 && threadIdx.x == 0 && (n == 0 || ks[0] >= vocab)) state->n_valid = 0;   // no valid row at all
 }
 
 __global__ void __launch_bounds__(AF_THREADS)
@@ -320,11 +308,21 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     if (n <= 0) return cudaSuccess;
     const int64_t vocab = c.cfg.img_vocab;
     const int D = c.cfg.dfv_dim, M = c.cfg.M;
-    SortBufs sb = c.sort_bufs();
+    SortJob sb = c.sort_job(gear_ctx_impl::SORT_IMG);
     DevState* state = c.state();
-    { KernelScope ks(&c.prof, "acc_keys", st);
-    acc_keys_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(img_id, n, vocab, sb.keys[0], state); }
-    const int cur = radix_sort_pairs(sb, n, nullptr, bits_for(vocab), true, st, &c.prof);
+    int cur = c.img_sorted_buf;
+    if (img_id) {
+        SortBatch batch = c.sort_batch();
+        batch.n_jobs = 1;
+        batch.job[0] = sb;
+        batch.job[0].ids = img_id;
+        batch.job[0].sentinel = (uint32_t)vocab;
+        batch.job[0].n_max = n;
+        batch.job[0].bits = bits_for(vocab);
+        cudaError_t se;
+        cur = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
+        if (se != cudaSuccess) return se;
+    }
     const uint32_t* ks = sb.keys[cur];
     const int64_t n_tiles = ceil_div(n, AF_TILE);
     uint2* tile_cnt = c.at<uint2>(c.ws.tile_cnt);
@@ -400,7 +398,7 @@ __global__ void collect_end_kernel(DevState* __restrict__ state) {
 cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
                                  int64_t* d_n, cudaStream_t st) {
     DevState* state = c.state();
-    SortBufs sb = c.sort_bufs();
+    SortJob sb = c.sort_job(gear_ctx_impl::SORT_READY);
     const int64_t n_max = c.ws.ready_cap;
     { KernelScope k(&c.prof, "collect_begin", st);
     collect_begin_kernel<<<1, 1, 0, st>>>(state, cap, d_n); }
@@ -408,7 +406,15 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     { KernelScope k(&c.prof, "collect_keys", st);
     collect_keys_kernel<<<(unsigned)(blocks > 1184 ? 1184 : blocks), 256, 0, st>>>(c.at<int32_t>(c.ws.q_id), state,
                                                                                  sb.keys[0]); }
-    const int cur = radix_sort_pairs(sb, n_max, &state->collect_n, bits_for(c.cfg.img_vocab), true, st, &c.prof);
+    SortBatch batch = c.sort_batch();
+    batch.n_jobs = 1;
+    batch.job[0] = sb;
+    batch.job[0].n_max = n_max;
+    batch.job[0].n_dev = &state->collect_n;
+    batch.job[0].bits = bits_for(c.cfg.img_vocab);
+    cudaError_t se;
+    const int cur = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
+    if (se != cudaSuccess) return se;
     int64_t want = ceil_div(n_max, 8);
     { KernelScope k(&c.prof, "collect_move", st);
     collect_move_kernel<<<(unsigned)(want > 1184 ? 1184 : want), 256, 0, st>>>(sb.keys[cur], sb.vals[cur],

@@ -52,9 +52,6 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
     const int d_in = 2 * c.emb_dim + c.dfv_dim;
     const size_t B = (size_t)c.max_batch;
     p->ready_cap = c.ready_cap > 0 ? c.ready_cap : c.max_nnz;
-    p->sort_cap = c.max_nnz;
-    if (p->sort_cap < c.max_batch) p->sort_cap = c.max_batch;
-    if (p->sort_cap < p->ready_cap) p->sort_cap = p->ready_cap;
     p->loss_blocks = (int)ceil_div(c.max_batch, 8);
     if (p->loss_blocks > 592) p->loss_blocks = 592;
 
@@ -70,12 +67,17 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
     }
     p->dz = take(B * 4);
     p->loss_part = take((size_t)p->loss_blocks * 4);
-    for (int i = 0; i < 2; ++i) {
-        p->sort_keys[i] = take((size_t)p->sort_cap * 4);
-        p->sort_vals[i] = take((size_t)p->sort_cap * 4);
+    p->sort_n[0] = p->sort_n[1] = c.max_batch;
+    p->sort_n[2] = c.max_nnz;
+    p->sort_n[3] = p->ready_cap;
+    for (int s = 0; s < 4; ++s) {
+        for (int i = 0; i < 2; ++i) {
+            p->sort_keys[s][i] = take((size_t)p->sort_n[s] * 4);
+            p->sort_vals[s][i] = take((size_t)p->sort_n[s] * 4);
+        }
+        p->sort_hist[s] = take((size_t)RS_BUCKETS * sort_tiles(p->sort_n[s]) * 4);
+        p->sort_tot[s] = take(RS_BUCKETS * 4);
     }
-    p->sort_hist = take((size_t)RS_BUCKETS * sort_tiles(p->sort_cap) * 4);
-    p->sort_tot = take(RS_BUCKETS * 4);
     p->tile_cnt = take((size_t)(ceil_div(c.max_nnz, 1024) + 1) * sizeof(uint2));
     p->grp_start = take((size_t)c.max_nnz * 4);
     p->grp_slot = take((size_t)c.max_nnz * 4);
@@ -146,6 +148,11 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
     c.n_params = param_count(*cfg);
     c.alive = true;
     c.tc_state = nullptr;
+    c.gbs.device_counter = &c.state()->grid_barrier;
+    c.gbs.host_base = 0;
+    c.img_sorted = false;
+    c.img_sorted_n = 0;
+    c.img_sorted_buf = 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
 
@@ -180,12 +187,38 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     if (b.nnz > 0 && !b.img_id) return arg_fail("NULL img_id");
     if (!o.loss || !o.head_grad || !o.dX) return arg_fail("loss, head_grad and dX are required outputs");
     if ((o.user_grad == nullptr) != (o.url_grad == nullptr)) return arg_fail("user_grad and url_grad: both or neither");
+    if (c.cfg.head_dtype == GEAR_BF16 && (!aligned16(o.head_grad) || !aligned16(c.buf.head_params)))
+        return arg_fail("bf16 head: head_params and head_grad must be 16-byte aligned");
     if (!aligned16(o.dX) || (o.x_debug && !aligned16(o.x_debug)) || (o.user_grad && !aligned16(o.user_grad)) ||
         (o.url_grad && !aligned16(o.url_grad)))
         return arg_fail("dX, x_debug, user_grad, url_grad must be 16-byte aligned");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
 
+    // The three ID arrays of the batch are key-sorted in one launch: the user and URL orders drive the embedding
+    // scatter below, the image order is kept for gear_accumulate_dfv_grad (img_id == NULL).
+    c.img_sorted = false;
+    int sorted_buf = 0;
+    if (b.B > 0) {
+        SortBatch batch = c.sort_batch();
+        batch.job[0] = c.sort_job(gear_ctx_impl::SORT_USER);
+        batch.job[0].ids = b.user_id; batch.job[0].sentinel = (uint32_t)c.cfg.user_vocab;
+        batch.job[0].n_max = b.B; batch.job[0].bits = bits_for(c.cfg.user_vocab);
+        batch.job[1] = c.sort_job(gear_ctx_impl::SORT_URL);
+        batch.job[1].ids = b.url_id; batch.job[1].sentinel = (uint32_t)c.cfg.url_vocab;
+        batch.job[1].n_max = b.B; batch.job[1].bits = bits_for(c.cfg.url_vocab);
+        batch.n_jobs = 2;
+        if (b.nnz > 0) {
+            batch.job[2] = c.sort_job(gear_ctx_impl::SORT_IMG);
+            batch.job[2].ids = b.img_id; batch.job[2].sentinel = (uint32_t)c.cfg.img_vocab;
+            batch.job[2].n_max = b.nnz; batch.job[2].bits = bits_for(c.cfg.img_vocab);
+            batch.n_jobs = 3;
+        }
+        cudaError_t se;
+        sorted_buf = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
+        if (se != cudaSuccess) return cuda_fail(se, "id sort");
+        if (b.nnz > 0) { c.img_sorted = true; c.img_sorted_n = b.nnz; c.img_sorted_buf = sorted_buf; }
+    }
     cudaError_t e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
     if (e != cudaSuccess) return cuda_fail(e, "gather");
     e = launch_head_simt(c, b, o, st);
@@ -194,9 +227,9 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     float* ut = o.user_grad ? o.user_grad : c.buf.user_emb;
     float* ht = o.url_grad ? o.url_grad : c.buf.url_emb;
     const float alpha = o.user_grad ? 1.0f : -lr;
-    e = launch_emb_scatter(c, b.user_id, b.B, c.cfg.user_vocab, ut, o.dX, c.d_in, 0, alpha, st);
+    e = launch_emb_reduce(c, gear_ctx_impl::SORT_USER, sorted_buf, b.B, c.cfg.user_vocab, ut, o.dX, c.d_in, 0, alpha, st);
     if (e != cudaSuccess) return cuda_fail(e, "user embedding scatter");
-    e = launch_emb_scatter(c, b.url_id, b.B, c.cfg.url_vocab, ht, o.dX, c.d_in, E, alpha, st);
+    e = launch_emb_reduce(c, gear_ctx_impl::SORT_URL, sorted_buf, b.B, c.cfg.url_vocab, ht, o.dX, c.d_in, E, alpha, st);
     if (e != cudaSuccess) return cuda_fail(e, "url embedding scatter");
     return GEAR_OK;
 }
@@ -207,7 +240,12 @@ int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* 
     gear_ctx_impl& c = ctx->impl;
     if (n < 0 || n > c.cfg.max_nnz) return arg_fail("n outside [0, max_nnz]");
     if (n == 0) return GEAR_OK;
-    if (!img_id || !grads) return arg_fail("NULL pointer");
+    if (!grads) return arg_fail("NULL pointer");
+    if (!img_id && (!c.img_sorted || c.img_sorted_n != n)) {
+        snprintf(g_last_error, sizeof(g_last_error),
+                 "img_id == NULL needs a preceding gear_forward_backward whose nnz equals n");
+        return GEAR_ERR_STATE;
+    }
     if (ld < c.cfg.dfv_dim || ld % 4 || !aligned16(grads)) return arg_fail("grads rows must be 16-byte aligned, ld >= dfv_dim");
     if (c.cfg.accum_mode != GEAR_ACC_SORT) return arg_fail("accum_mode not available");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -263,10 +301,20 @@ int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready) {
     DevState h;
     cudaError_t e = cudaStreamSynchronize(c.last_stream);
     if (e == cudaSuccess) e = cudaMemcpy(&h, c.state(), sizeof(DevState), cudaMemcpyDeviceToHost);
-    if (e == cudaSuccess && h.status != 0) e = cudaMemset(&c.state()->status, 0, sizeof(int32_t));
+    if (h.tc_error != 0) h.status |= GEAR_DEV_TIMEOUT;
+    if (e == cudaSuccess && h.status != 0) e = cudaMemset(c.state(), 0, 2 * sizeof(int32_t));   // status, tc_error
+    if (e == cudaSuccess && h.tc_error != 0) {
+        // an abandoned grid barrier leaves its arrival counter short: start the count again
+        e = cudaMemset(&c.state()->grid_barrier, 0, sizeof(unsigned long long));
+        c.gbs.host_base = 0;
+    }
     if (e != cudaSuccess) return cuda_fail(e, "gear_status");
     if (device_status) *device_status = h.status;
     if (pending_ready) *pending_ready = h.q_count;
+    if (h.status & GEAR_DEV_TIMEOUT) {
+        snprintf(g_last_error, sizeof(g_last_error), "a bounded device wait gave up (code %d)", h.tc_error);
+        return GEAR_ERR_CUDA;
+    }
     if (h.status & GEAR_DEV_BAD_ID) return GEAR_ERR_BAD_ID;
     if (h.status & (GEAR_DEV_READY_OVERFLOW | GEAR_DEV_OUT_CAPACITY)) return GEAR_ERR_CAPACITY;
     if (h.status & GEAR_DEV_BAD_CSR) return GEAR_ERR_ARG;

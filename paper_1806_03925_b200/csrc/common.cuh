@@ -16,14 +16,15 @@ namespace gear {
 // call has to synchronise to learn a size produced by an earlier kernel.
 struct DevState {
     int32_t status;        // GEAR_DEV_* bits, sticky
-    int32_t drop_call;     // set by the accumulate planner when the ready queue would overflow
+    int32_t tc_error;      // non-zero: a bounded wait of the tensor-core head gave up (code of the wait)
     int64_t q_count;       // averages waiting in the ready queue
     int64_t n_valid;       // accumulate: rows with an in-range ID (sorted prefix length)
     int64_t n_groups;      // accumulate: groups found in this call
     int64_t n_complete;    // accumulate: groups of this call that reached M
     int64_t exp_total;     // expiry scan: entries found
     int64_t collect_n;     // collect_ready: entries moved by the running call
-    int64_t pad[9];
+    unsigned long long grid_barrier;   // arrival counter of the cooperative sort's grid barrier
+    int64_t pad[8];
 };
 static_assert(sizeof(DevState) == 128, "DevState layout");
 
@@ -143,12 +144,40 @@ struct SortBufs {
 
 inline int64_t sort_tiles(int64_t n_max) { return n_max > 0 ? ceil_div(n_max, RS_TILE) : 1; }
 
-// Stable LSD radix sort of (key, value) pairs on the low `bits` bits of the key.  Input pairs are in
-// bufs.keys[0] / bufs.vals[0]; with identity_vals the first pass uses the element index as value.
-// n_dev (optional, device) caps the element count at min(*n_dev, n_max).  Returns the index (0 or 1)
-// of the buffer pair that holds the sorted result.
-int radix_sort_pairs(const SortBufs& bufs, int64_t n_max, const int64_t* n_dev, int bits, bool identity_vals,
-                     cudaStream_t st, Profiler* prof);
+// One array to sort: (key, value) pairs ordered by the low `bits` bits of the key, equal keys in input order.
+struct SortJob {
+    const int32_t* ids;     // if set, pass 0 reads these: key = id if 0 <= id < sentinel, else sentinel
+    uint32_t sentinel;      // key of out-of-range IDs (sorts last when bits covers it)
+    int32_t* status;        // device status word that gets GEAR_DEV_BAD_ID when a sentinel key is met (may be null)
+    uint32_t* keys[2];      // without ids the input keys are keys[0]
+    uint32_t* vals[2];      // with identity_vals the value of element i is i, else vals[0][i]
+    uint32_t* hist;         // [256][n_tiles]
+    uint32_t* tot;          // [256]
+    int64_t n_max;          // element count (or its upper bound when n_dev is given)
+    const int64_t* n_dev;   // optional device-resident count, capped at n_max
+    int bits;
+    int identity_vals;
+    int width, n_tiles;     // filled in by sort_jobs
+};
+
+struct SortBatch {
+    SortJob job[3];
+    int n_jobs;
+    int passes;                       // filled in by sort_jobs
+    unsigned long long* barrier_ctr;  // filled in by sort_jobs
+    unsigned long long barrier_base;
+    int32_t* err;                     // device word that receives a non-zero code when a grid barrier gives up
+};
+
+// Arrival counter of the grid barrier (device) and what all launches so far will have added to it (host).
+struct GridBarrierState {
+    unsigned long long* device_counter;
+    unsigned long long host_base;
+};
+
+// Sorts every job of the batch in one cooperative launch.  Returns the index (0 or 1) of the keys/vals
+// buffer pair that holds the sorted result of every job.
+int sort_jobs(SortBatch& batch, GridBarrierState* gbs, cudaStream_t st, Profiler* prof, cudaError_t* err_out);
 
 // In-place exclusive scan of m (a, b) counter pairs by one block; the totals go to total[0..1].
 void scan_pairs(uint2* data, int64_t m, uint2* total, cudaStream_t st, Profiler* prof);

@@ -11,15 +11,6 @@
 
 namespace gear {
 
-__global__ void __launch_bounds__(256)
-emb_keys_kernel(const int32_t* __restrict__ ids, int n, int64_t vocab, uint32_t* __restrict__ keys) {
-    int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) {
-        int id = ids[i];
-        keys[i] = (id >= 0 && id < vocab) ? (uint32_t)id : (uint32_t)vocab;   // out-of-range IDs sort last
-    }
-}
-
 constexpr int ES_SEG = 8;    // sorted positions walked by one lane group
 
 // LPR lanes share a row: lane c of the group owns the float4 chunks c, c + LPR, ... (NQ of them)
@@ -75,13 +66,10 @@ emb_reduce_kernel(const uint32_t* __restrict__ ks, const uint32_t* __restrict__ 
     }
 }
 
-cudaError_t launch_emb_scatter(const gear_ctx_impl& c, const int32_t* ids, int32_t B, int64_t vocab, float* table,
-                               const float* dX, int ldx, int col0, float alpha, cudaStream_t st) {
+cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int which, int cur, int32_t B, int64_t vocab, float* table,
+                              const float* dX, int ldx, int col0, float alpha, cudaStream_t st) {
     if (B <= 0) return cudaSuccess;
-    SortBufs sb = c.sort_bufs();
-    { KernelScope ks(&c.prof, "emb_keys", st);
-    emb_keys_kernel<<<(unsigned)ceil_div(B, 256), 256, 0, st>>>(ids, B, vocab, sb.keys[0]); }
-    const int cur = radix_sort_pairs(sb, B, nullptr, bits_for(vocab), true, st, &c.prof);
+    SortJob sb = c.sort_job(which);
     const int E = c.cfg.emb_dim, n_chunks = E / 4;
     int lpr = 1;
     while (lpr < n_chunks && lpr < 32) lpr <<= 1;

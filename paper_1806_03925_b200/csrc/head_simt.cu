@@ -249,9 +249,16 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
             Wop[l] = p.W[l];
         }
     }
+    int32_t* tc_err = &c.state()->tc_error;
+    cudaError_t tce = cudaSuccess;
     // forward
     for (int l = 0; l < L; ++l) {
         const int K = p.fan[l], N = p.fan[l + 1];
+        if constexpr (BF) {
+            tce = tc_gemm_kmajor(&c.prof, "tc_gemm_fwd", B, N, K, H[l], K, c.at<__nv_bfloat16>(c.ws.wbt[l]), K, 0,
+                                 H[l + 1], N, p.b[l], nullptr, 0, tc_err, st);
+            if (tce != cudaSuccess) return tce;
+        } else
         launch_gemm<TX, TX, TX, TX, EPI_BIAS_RELU>(B, N, K, H[l], K, 1, static_cast<const TX*>(Wop[l]), N, 1,
                                                     H[l + 1], N, p.b[l], (const TX*)nullptr, 0, 1, st, &c.prof,
                                                     "simt_gemm_fwd");
@@ -271,11 +278,22 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
     for (int l = L - 1; l >= 0; --l) {
         const int K = p.fan[l], N = p.fan[l + 1];
         // dW_l = H_l^T dA_{l+1}
+        if constexpr (BF) {
+            tce = tc_gemm_mnmajor(&c.prof, "tc_gemm_dw", K, N, B, H[l], K, dA[l + 1], N, p.gW[l], N, tc_err, st);
+            if (tce != cudaSuccess) return tce;
+        } else
         launch_gemm<TX, TX, float, TX, EPI_ATOMIC>(K, N, B, H[l], 1, K, dA[l + 1], N, 1, p.gW[l], N, nullptr,
                                                    (const TX*)nullptr, 0, splits_for(K, N, B), st, &c.prof, "simt_gemm_dw");
         { KernelScope ks(&c.prof, "colsum", st);
         colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, N, dA[l + 1], nullptr, p.gb[l], rows); }
-        if (l > 0) {
+        if constexpr (BF) {
+            const __nv_bfloat16* wb = c.at<__nv_bfloat16>(c.ws.wb[l]);
+            if (l > 0) tce = tc_gemm_kmajor(&c.prof, "tc_gemm_dh", B, K, N, dA[l + 1], N, wb, N, 1, dA[l], K, nullptr,
+                                            H[l], K, tc_err, st);
+            else tce = tc_gemm_kmajor(&c.prof, "tc_gemm_dx", B, K, N, dA[l + 1], N, wb, N, 2, o.dX, K, nullptr, nullptr,
+                                      0, tc_err, st);
+            if (tce != cudaSuccess) return tce;
+        } else if (l > 0) {
             launch_gemm<TX, TX, TX, TX, EPI_MASK>(B, K, N, dA[l + 1], N, 1, static_cast<const TX*>(Wop[l]), 1, N,
                                                   dA[l], K, nullptr, H[l], K, 1, st, &c.prof, "simt_gemm_dh");
         } else {

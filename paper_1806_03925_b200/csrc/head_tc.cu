@@ -1,0 +1,422 @@
+// bf16 matrix products of the head on the 5th-generation tensor cores (sm_100a):
+// tcgen05.mma with fp32 accumulators in tensor memory, operands staged in shared memory by TMA.
+//
+// One persistent kernel, one CTA per SM, three roles:
+//   warp 0     TMA producer: streams 128 x 64 (A) and BN x 64 (B) bf16 tiles through a ring of
+//              shared-memory stages (128-byte swizzle), one mbarrier pair per stage;
+//   warp 1     MMA issuer: one elected lane issues tcgen05.mma (M 128, N BN, K 16) into one of two
+//              accumulator buffers in tensor memory and commits each stage back to the producer;
+//   warps 2-5  epilogue: tcgen05.ld the finished accumulator (32 lanes x 32 columns per instruction),
+//              apply bias+ReLU / ReLU mask / nothing, and store; meanwhile the MMA warp already fills
+//              the other accumulator buffer with the next tile.
+// Two operand layouts:
+//   K-major   C[M][N] = A[M][K] . W[N][K]^T     (activations x weights; K contiguous in both)
+//   MN-major  C[M][N] += A[K][M]^T . B[K][N]    (weight gradients: the reduction runs over the batch,
+//                                                split across CTAs, partial tiles added with red.global)
+// No cluster launch and no multicast.  Every wait is bounded: on a timeout the kernel records an error
+// code, leaves its loops, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace gear {
+
+constexpr int TC_BM = 128;
+constexpr int TC_BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
+constexpr int TC_THREADS = 192;
+constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
+
+enum { TC_EPI_BIAS_RELU = 0, TC_EPI_MASK = 1, TC_EPI_F32 = 2, TC_EPI_RED = 3 };
+
+template <int BN> struct TcCfg {
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
+    static constexpr int B_BYTES = BN * TC_BK * 2;               // 32 KB or 16 KB
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
+    static_assert(SMEM > 116 * 1024, "one CTA per SM: two CTAs would both ask for tensor memory");
+    static_assert(SMEM <= 227 * 1024, "shared memory budget");
+};
+
+struct TcArgs {
+    int M, N, K;              // output rows, output columns, reduction length
+    int m_tiles, n_tiles, k_splits, kb_per_split;   // kb = blocks of TC_BK along K
+    void* out; int64_t ldo;
+    const float* bias;
+    const __nv_bfloat16* mask; int64_t ldm;
+    int32_t* err;             // device word that receives a non-zero code on a timeout
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and records `code`) if the phase never completed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* err, int code) {
+    for (uint32_t i = 0; i < TC_SPIN_LIMIT; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if (i > 64) __nanosleep(32);
+        if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int32_t*>(err) != 0) return false;
+    }
+    atomicCAS(err, 0, code);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1).
+//   K-major operand : rows of 128 bytes, 8-row groups 1024 bytes apart (SBO); LBO unused.
+//   MN-major operand: 64-element (128-byte) slabs along M/N, `lbo` bytes apart; 8-deep K groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;            // descriptor version
+    d |= (uint64_t)2 << 61;            // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t instr_desc(int bn, bool mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((mn_major ? 1u : 0u) << 15) | ((mn_major ? 1u : 0u) << 16) |
+           ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+// ---------------------------------------------------------------- the kernel
+template <int BN, bool MN_MAJOR, int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs g) {
+    using Cfg = TcCfg<BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;                  // operand stages, 1024-byte aligned
+    const uint32_t bars = tiles + STAGES * Cfg::STAGE_BYTES;        // mbarriers, then the tmem address word
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto acc_full = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+    auto acc_empty = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+    const uint32_t tmem_word = bars + 8u * (2 * STAGES + 4);
+    volatile uint32_t* tmem_word_ptr =
+        reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_word - raw));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = g.m_tiles * g.n_tiles * g.k_splits;
+    const int total_kb = (g.K + TC_BK - 1) / TC_BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 128); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" :: "l"(&map_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" :: "l"(&map_b) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(tmem_word), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_word_ptr;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int mt = t % g.m_tiles, nt = (t / g.m_tiles) % g.n_tiles, ks = t / (g.m_tiles * g.n_tiles);
+                const int kb0 = ks * g.kb_per_split, kb1 = min(total_kb, kb0 + g.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!(ok = mbar_wait(empty_bar(s), ((it / STAGES) & 1u) ^ 1u, g.err, 1))) break;
+                    const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
+                    mbar_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
+                    if (!MN_MAJOR) {
+                        tma_load_2d(a_dst, &map_a, full_bar(s), kb * TC_BK, mt * TC_BM);     // 128 rows x 64 k
+                        tma_load_2d(b_dst, &map_b, full_bar(s), kb * TC_BK, nt * BN);        // BN rows x 64 k
+                    } else {
+                        // 64 k-rows x 64 columns per box; the slabs of one operand sit 8 KB apart
+#pragma unroll
+                        for (int j = 0; j < TC_BM / 64; ++j)
+                            tma_load_2d(a_dst + j * 8192, &map_a, full_bar(s), mt * TC_BM + j * 64, kb * TC_BK);
+#pragma unroll
+                        for (int j = 0; j < BN / 64; ++j)
+                            tma_load_2d(b_dst + j * 8192, &map_b, full_bar(s), nt * BN + j * 64, kb * TC_BK);
+                    }
+                }
+            }
+            if (*reinterpret_cast<volatile int32_t*>(g.err) != 0) {
+                // leaving early: let the copies already issued land before the CTA gives its shared memory back
+                const uint32_t first = it > (uint32_t)STAGES ? it - STAGES : 0u;
+                for (uint32_t j = first; j < it; ++j)
+                    for (uint32_t spin = 0; spin < (1u << 16) && !mbar_try(full_bar(j % STAGES), (j / STAGES) & 1u); ++spin)
+                        __nanosleep(64);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(BN, MN_MAJOR);
+            uint32_t it = 0, tile_it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
+                const int ks = t / (g.m_tiles * g.n_tiles);
+                const int kb0 = ks * g.kb_per_split, kb1 = min(total_kb, kb0 + g.kb_per_split);
+                const int a = tile_it & 1;
+                if (!(ok = mbar_wait(acc_empty(a), ((tile_it >> 1) & 1u) ^ 1u, g.err, 2))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * BN);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!(ok = mbar_wait(full_bar(s), (it / STAGES) & 1u, g.err, 3))) break;
+                    tc_fence_after();
+                    const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, b_src = a_src + Cfg::A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k) {
+                        uint64_t da, db;
+                        if (!MN_MAJOR) {
+                            da = smem_desc(a_src + k * 32, 16, 1024);
+                            db = smem_desc(b_src + k * 32, 16, 1024);
+                        } else {
+                            da = smem_desc(a_src + k * 2048, 8192, 1024);
+                            db = smem_desc(b_src + k * 2048, 8192, 1024);
+                        }
+                        tc_mma(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                    }
+                    tc_commit(empty_bar(s));            // the stage may be refilled once these MMAs have read it
+                }
+                if (ok) tc_commit(acc_full(a));          // accumulator complete
+            }
+        }
+    } else {
+        // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32 * (warp % 4) ..
+        const int quarter = warp & 3;
+        uint32_t tile_it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
+            const int mt = t % g.m_tiles, nt = (t / g.m_tiles) % g.n_tiles;
+            const int a = tile_it & 1;
+            if (!(ok = mbar_wait(acc_full(a), (tile_it >> 1) & 1u, g.err, 4))) break;
+            tc_fence_after();
+            const int m = mt * TC_BM + quarter * 32 + lane;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tc_ld32(t_row + c0, r);
+                tc_wait_ld();
+                const int n0 = nt * BN + c0;
+                if (m < g.M && n0 < g.N) {
+                    const int nv = min(32, g.N - n0);                 // N is a multiple of 8
+                    if (EPI == TC_EPI_BIAS_RELU || EPI == TC_EPI_MASK) {
+                        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(g.out) + (int64_t)m * g.ldo + n0;
+                        for (int j = 0; j < nv; j += 8) {
+                            float v[8];
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(r[j + q]);
+                            if (EPI == TC_EPI_BIAS_RELU) {
+                                const float4 b0 = ld_f4(g.bias + n0 + j), b1 = ld_f4(g.bias + n0 + j + 4);
+                                v[0] = fmaxf(v[0] + b0.x, 0.f); v[1] = fmaxf(v[1] + b0.y, 0.f);
+                                v[2] = fmaxf(v[2] + b0.z, 0.f); v[3] = fmaxf(v[3] + b0.w, 0.f);
+                                v[4] = fmaxf(v[4] + b1.x, 0.f); v[5] = fmaxf(v[5] + b1.y, 0.f);
+                                v[6] = fmaxf(v[6] + b1.z, 0.f); v[7] = fmaxf(v[7] + b1.w, 0.f);
+                            } else {
+                                const uint4 mk = *reinterpret_cast<const uint4*>(g.mask + (int64_t)m * g.ldm + n0 + j);
+                                const uint32_t w[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    // a post-ReLU activation is > 0 exactly when its bf16 pattern is non-zero and positive
+                                    const uint32_t lo = w[q] & 0xffffu, hi = w[q] >> 16;
+                                    if (!(lo != 0u && lo < 0x8000u)) v[2 * q] = 0.f;
+                                    if (!(hi != 0u && hi < 0x8000u)) v[2 * q + 1] = 0.f;
+                                }
+                            }
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+                                pk[q] = *reinterpret_cast<uint32_t*>(&h2);
+                            }
+                            *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    } else {
+                        float* dst = static_cast<float*>(g.out) + (int64_t)m * g.ldo + n0;
+                        for (int j = 0; j < nv; j += 4) {
+                            const float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                         __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                            if (EPI == TC_EPI_RED) red_add_f4(dst + j, v);
+                            else st_f4(dst + j, v);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty(a));                   // 128 arrivals hand the buffer back to the MMA warp
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     :: "r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][cols] with leading dimension ld (elements); box = box_rows x 64 columns, 128-byte swizzle.
+// Out-of-range parts of a box read as zero.
+static bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int BN, bool MN, int EPI>
+static cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& g, cudaStream_t st) {
+    using Cfg = TcCfg<BN>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, MN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             Cfg::SMEM);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const int tiles = g.m_tiles * g.n_tiles * g.k_splits;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    tc_gemm_kernel<BN, MN, EPI><<<grid, TC_THREADS, Cfg::SMEM, st>>>(ma, mb, g);
+    return cudaGetLastError();
+}
+
+template <bool MN, int EPI>
+static cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& g, cudaStream_t st) {
+    return bn == 256 ? launch_variant<256, MN, EPI>(ma, mb, g, st) : launch_variant<128, MN, EPI>(ma, mb, g, st);
+}
+
+cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
+                           const __nv_bfloat16* W, int64_t ldw, int epi, void* out, int64_t ldo, const float* bias,
+                           const __nv_bfloat16* mask, int64_t ldm, int32_t* err, cudaStream_t st) {
+    if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
+    const int bn = N > 128 ? 256 : 128;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, M, K, lda, TC_BM) || !make_map(&mb, W, N, K, ldw, bn)) return cudaErrorInvalidValue;
+    TcArgs g;
+    g.M = M; g.N = N; g.K = K;
+    g.m_tiles = (int)ceil_div(M, TC_BM); g.n_tiles = (int)ceil_div(N, bn); g.k_splits = 1;
+    g.kb_per_split = (int)ceil_div(K, TC_BK);
+    g.out = out; g.ldo = ldo; g.bias = bias; g.mask = mask; g.ldm = ldm; g.err = err;
+    KernelScope ks(prof, name, st);
+    switch (epi) {
+    case TC_EPI_BIAS_RELU: return launch_bn<false, TC_EPI_BIAS_RELU>(bn, ma, mb, g, st);
+    case TC_EPI_MASK: return launch_bn<false, TC_EPI_MASK>(bn, ma, mb, g, st);
+    default: return launch_bn<false, TC_EPI_F32>(bn, ma, mb, g, st);
+    }
+}
+
+cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
+                            const __nv_bfloat16* Bm, int64_t ldb, float* out, int64_t ldo, int32_t* err,
+                            cudaStream_t st) {
+    if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
+    const int bn = N > 128 ? 256 : 128;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, K, M, lda, 64) || !make_map(&mb, Bm, K, N, ldb, 64)) return cudaErrorInvalidValue;
+    TcArgs g;
+    g.M = M; g.N = N; g.K = K;
+    g.m_tiles = (int)ceil_div(M, TC_BM); g.n_tiles = (int)ceil_div(N, bn);
+    const int total_kb = (int)ceil_div(K, TC_BK);
+    int splits = (int)ceil_div(sm_count(), (int64_t)g.m_tiles * g.n_tiles);
+    if (splits > total_kb) splits = total_kb;
+    if (splits < 1) splits = 1;
+    g.kb_per_split = (int)ceil_div(total_kb, splits);
+    g.k_splits = (int)ceil_div(total_kb, g.kb_per_split);
+    g.out = out; g.ldo = ldo; g.bias = nullptr; g.mask = nullptr; g.ldm = 0; g.err = err;
+    KernelScope ks(prof, name, st);
+    return launch_bn<true, TC_EPI_RED>(bn, ma, mb, g, st);
+}
+
+}  // namespace gear

@@ -23,8 +23,10 @@ struct WsPlan {
     size_t loss_part;                   // [loss_blocks] fp32 per-block partial losses
     size_t wb[MAX_LAYERS];              // bf16 head: W_l as [in][out]
     size_t wbt[MAX_LAYERS];             // bf16 head: W_l as [out][in]
-    size_t sort_keys[2], sort_vals[2];  // [sort_cap] uint32
-    size_t sort_hist, sort_tot;
+    // four sets of sort buffers: user IDs, URL IDs (max_batch each), image IDs (max_nnz), ready queue (ready_cap)
+    size_t sort_keys[4][2], sort_vals[4][2];
+    size_t sort_hist[4], sort_tot[4];
+    int64_t sort_n[4];
     size_t tile_cnt;                    // [sort tiles + 1] uint2 per-tile (groups, complete) counts
     size_t grp_start;                   // [max_nnz] uint32 (top bit: first group of its image in this call)
     size_t grp_slot;                    // [max_nnz] int32 ready-queue slot or -1
@@ -33,7 +35,6 @@ struct WsPlan {
     size_t exp_bits;                    // [ceil(img_vocab / 32)] uint32 expired bitmap
     size_t exp_cnt;                     // [expiry tiles + 1] uint2
     size_t total;
-    int64_t sort_cap;
     int64_t ready_cap;
     int loss_blocks;
 };
@@ -50,14 +51,29 @@ struct gear_ctx_impl {
     bool alive;
     void* tc_state;     // tensor-core head state (tensor maps), owned by head_tc.cu; may be null
     mutable Profiler prof;
+    mutable GridBarrierState gbs;
+    // image IDs of the last gear_forward_backward batch, already sorted (reused by gear_accumulate_dfv_grad)
+    bool img_sorted;
+    int64_t img_sorted_n;
+    int img_sorted_buf;
 
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(static_cast<char*>(buf.workspace) + off); }
     DevState* state() const { return at<DevState>(ws.state); }
-    SortBufs sort_bufs() const {
-        SortBufs b;
-        b.keys[0] = at<uint32_t>(ws.sort_keys[0]); b.keys[1] = at<uint32_t>(ws.sort_keys[1]);
-        b.vals[0] = at<uint32_t>(ws.sort_vals[0]); b.vals[1] = at<uint32_t>(ws.sort_vals[1]);
-        b.hist = at<uint32_t>(ws.sort_hist); b.tot = at<uint32_t>(ws.sort_tot);
+    enum { SORT_USER = 0, SORT_URL = 1, SORT_IMG = 2, SORT_READY = 3 };
+    // a job over buffer set `which`; the caller fills ids / n / bits
+    SortJob sort_job(int which) const {
+        SortJob j{};
+        j.keys[0] = at<uint32_t>(ws.sort_keys[which][0]); j.keys[1] = at<uint32_t>(ws.sort_keys[which][1]);
+        j.vals[0] = at<uint32_t>(ws.sort_vals[which][0]); j.vals[1] = at<uint32_t>(ws.sort_vals[which][1]);
+        j.hist = at<uint32_t>(ws.sort_hist[which]); j.tot = at<uint32_t>(ws.sort_tot[which]);
+        j.sentinel = 0xffffffffu;
+        j.status = &state()->status;
+        j.identity_vals = 1;
+        return j;
+    }
+    SortBatch sort_batch() const {
+        SortBatch b{};
+        b.err = &state()->tc_error;
         return b;
     }
 };
@@ -74,11 +90,22 @@ cudaError_t launch_gather(const gear_ctx_impl& c, const gear_batch& b, int32_t* 
 // head_simt.cu: forward + backward of the head with fp32 FMA products (operands fp32 or bf16)
 cudaError_t launch_head_simt(const gear_ctx_impl& c, const gear_batch& b, const gear_step_out& o, cudaStream_t st);
 
+// head_tc.cu: bf16 products on tcgen05 tensor cores.  epi: 0 bias+ReLU -> bf16, 1 ReLU mask -> bf16, 2 plain fp32.
+cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
+                           const __nv_bfloat16* W, int64_t ldw, int epi, void* out, int64_t ldo, const float* bias,
+                           const __nv_bfloat16* mask, int64_t ldm, int32_t* err, cudaStream_t st);
+// out[M][N] (fp32) += A[K][M]^T . Bm[K][N]
+cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
+                            const __nv_bfloat16* Bm, int64_t ldb, float* out, int64_t ldo, int32_t* err,
+                            cudaStream_t st);
+
 // emb_scatter.cu
-cudaError_t launch_emb_scatter(const gear_ctx_impl& c, const int32_t* ids, int32_t B, int64_t vocab, float* table,
-                               const float* dX, int ldx, int col0, float alpha, cudaStream_t st);
+// table[id] += alpha * (sum of the dX rows of the views with that id), given the sorted (id, view) pairs of buffer set `which`
+cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int which, int buf, int32_t B, int64_t vocab, float* table,
+                              const float* dX, int ldx, int col0, float alpha, cudaStream_t st);
 
 // accumulate.cu
+// img_id == nullptr: use the image IDs sorted by the last gear_forward_backward (buffer set SORT_IMG)
 cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
                               const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st);
 cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* seq, float* avg, int64_t cap,

@@ -1,141 +1,228 @@
 // Stable LSD radix sort of (key, value) pairs and small scan helpers.
 //
-// Every pass is three kernels -- per-tile digit histogram, per-digit scan over tiles, stable scatter --
-// so no kernel ever waits on another block.  A tile is RS_TILE consecutive elements; a warp owns
-// 32 * RS_ITEMS consecutive elements of it and ranks equal digits with match_any, which keeps equal keys
-// in index order.
+// One cooperative, persistent kernel sorts up to three independent arrays ("jobs") in one launch.  Every
+// pass has three phases over tiles of RS_TILE consecutive elements -- per-tile digit histogram, per-digit
+// scan over tiles, stable scatter -- separated by a grid-wide barrier.  A warp owns 32 * RS_ITEMS
+// consecutive elements of a tile and ranks equal digits with match_any, which keeps equal keys in index
+// order.  The first pass can read raw int32 IDs and map out-of-range ones to a sentinel key that sorts
+// last, so no separate key-building launch is needed.
+//
+// The grid barrier is a monotonically increasing 64-bit arrival counter: barrier k of a launch completes
+// when the counter reaches base + grid * (k + 1), where the host knows `base` (it adds up what every
+// earlier launch contributes).  The kernel is launched cooperatively, so all blocks are resident; the
+// spin is bounded all the same, and a block that gives up records an error and makes every later barrier
+// of the launch fall through.
 #include "common.cuh"
 
 namespace gear {
 
+constexpr uint32_t GRID_SPIN_LIMIT = 1u << 21;
+
 __device__ __forceinline__ int64_t effective_n(int64_t n_max, const int64_t* n_dev) {
     if (!n_dev) return n_max;
-    int64_t n = *n_dev;
+    int64_t n = __ldcg(n_dev);
     return n < n_max ? (n < 0 ? 0 : n) : n_max;
 }
 
-__global__ void __launch_bounds__(RS_THREADS)
-radix_hist_kernel(const uint32_t* __restrict__ keys, int64_t n_max, const int64_t* __restrict__ n_dev,
-                  int shift, uint32_t mask, uint32_t* __restrict__ hist, int n_tiles) {
-    __shared__ uint32_t h[RS_BUCKETS];
-    const int64_t n = effective_n(n_max, n_dev);
-    h[threadIdx.x] = 0;
+// All threads of every block call this.  Returns false once the launch has been abandoned.
+__device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned long long target, int32_t* err) {
+    __shared__ int ok_flag;
     __syncthreads();
-    const int64_t base = (int64_t)blockIdx.x * RS_TILE;
-#pragma unroll 4
-    for (int it = 0; it < RS_ITEMS; ++it) {
-        int64_t i = base + it * RS_THREADS + threadIdx.x;
-        if (i < n) atomicAdd(&h[(keys[i] >> shift) & mask], 1u);
+    if (threadIdx.x == 0) {
+        int ok = 1;
+        __threadfence();
+        atomicAdd(ctr, 1ull);
+        uint32_t spin = 0;
+        while (*reinterpret_cast<volatile unsigned long long*>(ctr) < target) {
+            if (++spin > GRID_SPIN_LIMIT) { atomicCAS(err, 0, 100); ok = 0; break; }
+            if ((spin & 255u) == 255u && *reinterpret_cast<volatile int32_t*>(err) != 0) { ok = 0; break; }
+            __nanosleep(20);
+        }
+        __threadfence();
+        ok_flag = ok;
     }
     __syncthreads();
-    hist[(int64_t)threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
+    return ok_flag != 0;
 }
 
-// One block per digit: exclusive scan of that digit's per-tile counts; the digit total goes to tot[d].
-__global__ void __launch_bounds__(RS_THREADS)
-radix_scan_rows_kernel(uint32_t* __restrict__ hist, uint32_t* __restrict__ tot, int n_tiles) {
-    __shared__ uint32_t scratch[33];
-    uint32_t* row = hist + (int64_t)blockIdx.x * n_tiles;
-    uint32_t carry = 0;
-    for (int base = 0; base < n_tiles; base += RS_THREADS) {
-        int i = base + threadIdx.x;
-        uint32_t v = i < n_tiles ? row[i] : 0u;
-        uint32_t total;
-        uint32_t ex = block_exclusive_scan(v, scratch, &total);
-        if (i < n_tiles) row[i] = carry + ex;
-        carry += total;
+__device__ __forceinline__ uint32_t load_key(const SortJob& j, int pass, int64_t i, int src) {
+    if (pass == 0 && j.ids) {
+        const int32_t id = __ldcg(j.ids + i);
+        return (id >= 0 && (uint32_t)id < j.sentinel) ? (uint32_t)id : j.sentinel;
     }
-    if (threadIdx.x == 0) tot[blockIdx.x] = carry;
+    return __ldcg(j.keys[src] + i);
 }
 
 __global__ void __launch_bounds__(RS_THREADS)
-radix_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ vin,
-                     uint32_t* __restrict__ kout, uint32_t* __restrict__ vout,
-                     int64_t n_max, const int64_t* __restrict__ n_dev, int shift, uint32_t mask,
-                     const uint32_t* __restrict__ hist, const uint32_t* __restrict__ tot, int n_tiles) {
+coop_sort_kernel(const SortBatch batch) {
     __shared__ uint32_t scratch[33];
     __shared__ uint32_t base[RS_BUCKETS];
     __shared__ uint32_t wcnt[RS_THREADS / 32][RS_BUCKETS];
-    const int64_t n = effective_n(n_max, n_dev);
-    const int64_t tile0 = (int64_t)blockIdx.x * RS_TILE;
-    if (tile0 >= n) return;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
+    int total_tiles = 0;
+    for (int j = 0; j < batch.n_jobs; ++j) total_tiles += batch.job[j].n_tiles;
+    unsigned long long target = batch.barrier_base;
 
-    {   // global start of every digit, plus what earlier tiles put into it
-        uint32_t t = tot[threadIdx.x];
-        uint32_t ex = block_exclusive_scan(t, scratch, nullptr);
-        base[threadIdx.x] = ex + hist[(int64_t)threadIdx.x * n_tiles + blockIdx.x];
-    }
-    for (int w = 0; w < RS_THREADS / 32; ++w) wcnt[w][threadIdx.x] = 0;
-    __syncthreads();
+    for (int pass = 0; pass < batch.passes; ++pass) {
+        const int src = pass & 1, dst = src ^ 1;
 
-    uint32_t key[RS_ITEMS], rank[RS_ITEMS];
-    const int64_t seg0 = tile0 + (int64_t)warp * (32 * RS_ITEMS);
-#pragma unroll
-    for (int it = 0; it < RS_ITEMS; ++it) {
-        int64_t i = seg0 + it * 32 + lane;
-        key[it] = i < n ? kin[i] : 0u;
-    }
-#pragma unroll
-    for (int it = 0; it < RS_ITEMS; ++it) {
-        int64_t i = seg0 + it * 32 + lane;
-        const bool valid = i < n;
-        const uint32_t d = valid ? ((key[it] >> shift) & mask) : 0xffffu;
-        const uint32_t peers = __match_any_sync(0xffffffffu, d);
-        const int leader = __ffs(peers) - 1;
-        uint32_t old = 0;
-        if (valid && (int)lane == leader) {
-            old = wcnt[warp][d];
-            wcnt[warp][d] = old + __popc(peers);
+        // ---- phase A: digit histogram of every tile
+        for (int w = blockIdx.x; w < total_tiles; w += gridDim.x) {
+            int jj = 0, t = w;
+            while (t >= batch.job[jj].n_tiles) { t -= batch.job[jj].n_tiles; ++jj; }
+            const SortJob& j = batch.job[jj];
+            const int64_t n = effective_n(j.n_max, j.n_dev);
+            const int shift = pass * j.width;
+            const uint32_t mask = (1u << j.width) - 1u;
+            base[threadIdx.x] = 0;
+            __syncthreads();
+            const int64_t tile0 = (int64_t)t * RS_TILE;
+            bool bad = false;
+#pragma unroll 4
+            for (int it = 0; it < RS_ITEMS; ++it) {
+                const int64_t i = tile0 + it * RS_THREADS + threadIdx.x;
+                if (i < n) {
+                    const uint32_t k = load_key(j, pass, i, src);
+                    bad |= (k == j.sentinel);
+                    atomicAdd(&base[(k >> shift) & mask], 1u);
+                }
+            }
+            if (bad && pass == 0 && j.ids && j.status) atomicOr(j.status, GEAR_DEV_BAD_ID);
+            __syncthreads();
+            __stcg(j.hist + (int64_t)threadIdx.x * j.n_tiles + t, base[threadIdx.x]);
+            __syncthreads();
         }
-        old = __shfl_sync(0xffffffffu, old, leader);
-        rank[it] = old + __popc(peers & ((1u << lane) - 1u));
-        __syncwarp();
-    }
-    __syncthreads();
-    {   // turn the per-warp digit counts into exclusive offsets across the warps of this tile
-        uint32_t run = 0;
-#pragma unroll
-        for (int w = 0; w < RS_THREADS / 32; ++w) {
-            uint32_t c = wcnt[w][threadIdx.x];
-            wcnt[w][threadIdx.x] = run;
-            run += c;
+        target += gridDim.x;
+        if (!grid_barrier(batch.barrier_ctr, target, batch.err)) return;
+
+        // ---- phase B: per digit, exclusive scan of the per-tile counts; digit totals
+        for (int r = blockIdx.x; r < batch.n_jobs * RS_BUCKETS; r += gridDim.x) {
+            const SortJob& j = batch.job[r / RS_BUCKETS];
+            const int d = r % RS_BUCKETS;
+            uint32_t* row = j.hist + (int64_t)d * j.n_tiles;
+            uint32_t carry = 0;
+            for (int b0 = 0; b0 < j.n_tiles; b0 += RS_THREADS) {
+                const int i = b0 + threadIdx.x;
+                const uint32_t v = i < j.n_tiles ? __ldcg(row + i) : 0u;
+                uint32_t total;
+                const uint32_t ex = block_exclusive_scan(v, scratch, &total);
+                if (i < j.n_tiles) __stcg(row + i, carry + ex);
+                carry += total;
+            }
+            if (threadIdx.x == 0) __stcg(j.tot + d, carry);
         }
-    }
-    __syncthreads();
+        target += gridDim.x;
+        if (!grid_barrier(batch.barrier_ctr, target, batch.err)) return;
+
+        // ---- phase C: stable scatter
+        for (int w = blockIdx.x; w < total_tiles; w += gridDim.x) {
+            int jj = 0, t = w;
+            while (t >= batch.job[jj].n_tiles) { t -= batch.job[jj].n_tiles; ++jj; }
+            const SortJob& j = batch.job[jj];
+            const int64_t n = effective_n(j.n_max, j.n_dev);
+            const int64_t tile0 = (int64_t)t * RS_TILE;
+            if (tile0 >= n) continue;                       // uniform over the block
+            const int shift = pass * j.width;
+            const uint32_t mask = (1u << j.width) - 1u;
+            {
+                const uint32_t tt = __ldcg(j.tot + threadIdx.x);
+                const uint32_t ex = block_exclusive_scan(tt, scratch, nullptr);
+                base[threadIdx.x] = ex + __ldcg(j.hist + (int64_t)threadIdx.x * j.n_tiles + t);
+            }
+            for (int w2 = 0; w2 < RS_THREADS / 32; ++w2) wcnt[w2][threadIdx.x] = 0;
+            __syncthreads();
+            uint32_t key[RS_ITEMS], rank[RS_ITEMS];
+            const int64_t seg0 = tile0 + (int64_t)warp * (32 * RS_ITEMS);
 #pragma unroll
-    for (int it = 0; it < RS_ITEMS; ++it) {
-        int64_t i = seg0 + it * 32 + lane;
-        if (i < n) {
-            const uint32_t d = (key[it] >> shift) & mask;
-            const uint32_t pos = base[d] + wcnt[warp][d] + rank[it];
-            kout[pos] = key[it];
-            vout[pos] = vin ? vin[i] : (uint32_t)i;
+            for (int it = 0; it < RS_ITEMS; ++it) {
+                const int64_t i = seg0 + it * 32 + lane;
+                key[it] = i < n ? load_key(j, pass, i, src) : 0u;
+            }
+#pragma unroll
+            for (int it = 0; it < RS_ITEMS; ++it) {
+                const int64_t i = seg0 + it * 32 + lane;
+                const bool valid = i < n;
+                const uint32_t d = valid ? ((key[it] >> shift) & mask) : 0xffffu;
+                const uint32_t peers = __match_any_sync(0xffffffffu, d);
+                const int leader = __ffs(peers) - 1;
+                uint32_t old = 0;
+                if (valid && (int)lane == leader) {
+                    old = wcnt[warp][d];
+                    wcnt[warp][d] = old + __popc(peers);
+                }
+                old = __shfl_sync(0xffffffffu, old, leader);
+                rank[it] = old + __popc(peers & ((1u << lane) - 1u));
+                __syncwarp();
+            }
+            __syncthreads();
+            {
+                uint32_t run = 0;
+#pragma unroll
+                for (int w2 = 0; w2 < RS_THREADS / 32; ++w2) {
+                    const uint32_t c = wcnt[w2][threadIdx.x];
+                    wcnt[w2][threadIdx.x] = run;
+                    run += c;
+                }
+            }
+            __syncthreads();
+            const bool identity = (pass == 0 && j.identity_vals);
+#pragma unroll
+            for (int it = 0; it < RS_ITEMS; ++it) {
+                const int64_t i = seg0 + it * 32 + lane;
+                if (i < n) {
+                    const uint32_t d = (key[it] >> shift) & mask;
+                    const uint32_t pos = base[d] + wcnt[warp][d] + rank[it];
+                    __stcg(j.keys[dst] + pos, key[it]);
+                    __stcg(j.vals[dst] + pos, identity ? (uint32_t)i : __ldcg(j.vals[src] + i));
+                }
+            }
+            __syncthreads();
+        }
+        if (pass + 1 < batch.passes) {
+            target += gridDim.x;
+            if (!grid_barrier(batch.barrier_ctr, target, batch.err)) return;
         }
     }
 }
 
-int radix_sort_pairs(const SortBufs& b, int64_t n_max, const int64_t* n_dev, int bits, bool identity_vals,
-                     cudaStream_t st, Profiler* prof) {
-    if (n_max <= 0) return 0;
-    const int n_tiles = (int)sort_tiles(n_max);
-    const int passes = (bits + 7) / 8;
-    const int width = (bits + passes - 1) / passes;
-    int cur = 0;
-    for (int p = 0; p < passes; ++p) {
-        const int shift = p * width;
-        const uint32_t mask = (1u << width) - 1u;
-        { KernelScope k(prof, "radix_hist", st);
-        radix_hist_kernel<<<n_tiles, RS_THREADS, 0, st>>>(b.keys[cur], n_max, n_dev, shift, mask, b.hist, n_tiles); }
-        { KernelScope k(prof, "radix_scan_rows", st);
-        radix_scan_rows_kernel<<<RS_BUCKETS, RS_THREADS, 0, st>>>(b.hist, b.tot, n_tiles); }
-        const uint32_t* vin = (p == 0 && identity_vals) ? nullptr : b.vals[cur];
-        { KernelScope k(prof, "radix_scatter", st);
-        radix_scatter_kernel<<<n_tiles, RS_THREADS, 0, st>>>(b.keys[cur], vin, b.keys[cur ^ 1], b.vals[cur ^ 1],
-                                                             n_max, n_dev, shift, mask, b.hist, b.tot, n_tiles); }
-        cur ^= 1;
+static int coop_grid_limit() {
+    static int limit = 0;
+    if (!limit) {
+        int dev = 0, sms = 0, per_sm = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, coop_sort_kernel, RS_THREADS, 0);
+        if (sms <= 0) sms = 148;
+        if (per_sm <= 0) per_sm = 1;
+        if (per_sm > 2) per_sm = 2;
+        limit = sms * per_sm;
     }
-    return cur;
+    return limit;
+}
+
+int sort_jobs(SortBatch& batch, GridBarrierState* gbs, cudaStream_t st, Profiler* prof, cudaError_t* err_out) {
+    *err_out = cudaSuccess;
+    int passes = 1, total_tiles = 0;
+    for (int j = 0; j < batch.n_jobs; ++j) {
+        const int p = (batch.job[j].bits + 7) / 8;
+        if (p > passes) passes = p;
+    }
+    for (int j = 0; j < batch.n_jobs; ++j) {
+        SortJob& job = batch.job[j];
+        job.width = (job.bits + passes - 1) / passes;
+        job.n_tiles = (int)sort_tiles(job.n_max);
+        total_tiles += job.n_tiles;
+    }
+    batch.passes = passes;
+    int grid = total_tiles < coop_grid_limit() ? total_tiles : coop_grid_limit();
+    if (grid < 1) grid = 1;
+    batch.barrier_ctr = gbs->device_counter;
+    batch.barrier_base = gbs->host_base;
+    gbs->host_base += (unsigned long long)grid * (unsigned long long)(3 * passes - 1);
+    KernelScope k(prof, "coop_sort", st);
+    void* args[] = {&batch};
+    *err_out = cudaLaunchCooperativeKernel((const void*)coop_sort_kernel, dim3(grid), dim3(RS_THREADS), args, 0, st);
+    return passes & 1;
 }
 
 // ---------------------------------------------------------------- scan of counter pairs

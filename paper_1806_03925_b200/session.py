@@ -99,10 +99,14 @@ class GearSession:
                                         x_debug=self.x_debug, user_grad=self.user_grad, url_grad=self.url_grad,
                                         B=b.B, nnz=b.nnz)
 
-    def accumulate_from_step(self, b: DeviceBatch):
-        """Event 5 in its indirect form: row r of the batch is dX[row_view[r], 2E:] * inv_n[row_view[r]]."""
+    def accumulate_from_step(self, b: DeviceBatch, reuse_sorted_ids: bool = True):
+        """Event 5 in its indirect form: row r of the batch is dX[row_view[r], 2E:] * inv_n[row_view[r]].
+        With reuse_sorted_ids the image IDs sorted during forward_backward are used (img_id = NULL)."""
+        if b.nnz == 0:
+            return 0
         ptr = self.dX.data_ptr() + 4 * 2 * self.p.emb_dim
-        return gb.gear_accumulate_dfv_grad(self.ctx, b.img_id, ptr, self.d_in, self.row_view, self.inv_n, b.nnz)
+        return gb.gear_accumulate_dfv_grad(self.ctx, None if reuse_sorted_ids else b.img_id, ptr, self.d_in,
+                                           self.row_view, self.inv_n, b.nnz)
 
     def accumulate_rows(self, img_id: torch.Tensor, grads: torch.Tensor):
         assert grads.dtype == torch.float32 and grads.shape[1] == self.p.dfv_dim
