@@ -224,6 +224,37 @@ int gear_fill_uniform(void* dst, int32_t dtype, int64_t n_rows, int32_t dim, uin
                       double amp, void* stream);
 
 /*
+ * The expiry scan for callers that cannot allocate device memory.  (The paper has no counterpart: it is
+ * gear_collect_expired without a ctx.)
+ *
+ * Who needs it: code that runs where cudaMalloc is not available to it -- a serving process whose device
+ * memory was partitioned at start-up, a plug-in that receives buffers but no allocator, a path on which an
+ * allocation's implicit device synchronisation is not acceptable.  Such a caller cannot supply the
+ * workspace a gear_ctx requires, so this call takes the timestamp table directly and keeps its scratch in
+ * a fixed array inside the library image.
+ *
+ *   - Same semantics as gear_collect_expired: lists, ascending, every id < img_vocab with
+ *     now - dfv_ts[id] >= expire; restamp != 0 sets dfv_ts[id] = now for the listed ones; count to *d_n
+ *     (device, optional) and *h_n (host, optional: then the call synchronises the stream); cap too small:
+ *     nothing is listed or restamped, the required count is reported and, with h_n, GEAR_ERR_CAPACITY returned.
+ *   - img_vocab may be at most GEAR_STATIC_EXPIRY_MAX_VOCAB; larger tables are refused with
+ *     GEAR_ERR_CAPACITY before anything is enqueued.
+ *   - Cost: every GPU on which the library is loaded holds GEAR_STATIC_EXPIRY_SCRATCH_BYTES (about 2.1 MB)
+ *     of device memory for this array until the process exits, whether or not the call is ever made.
+ *   - The first call on a device looks up the array's device address (once per device, with that device
+ *     current); make that first call before starting any stream capture.
+ *   - The call allocates nothing, on the device or through any library.
+ *   - All calls on one device share the array.  Calls whose kernels may overlap on the GPU (different
+ *     streams without ordering between them) race on it: order them.  Nothing in the array carries over
+ *     from one call to the next.
+ * dfv_ts and ids are device pointers; dfv_ts is written only when restamp != 0.
+ */
+#define GEAR_STATIC_EXPIRY_MAX_VOCAB 16777216
+#define GEAR_STATIC_EXPIRY_SCRATCH_BYTES (256 + GEAR_STATIC_EXPIRY_MAX_VOCAB / 8 + 16640)
+int gear_collect_expired_static(int64_t* dfv_ts, int64_t img_vocab, int64_t expire, int64_t now, int restamp,
+                                int32_t* ids, int64_t cap, int64_t* d_n, int64_t* h_n, void* stream);
+
+/*
  * Per-kernel timing (not part of the paper).  While enabled, every kernel the library launches for this
  * ctx is bracketed by a pair of CUDA events on the caller's stream.  gear_profile_read synchronises,
  * sums the elapsed time and the launch count per kernel name since the last read or enable, writes up to

@@ -24,7 +24,9 @@ GEAR_TAG_USER, GEAR_TAG_URL, GEAR_TAG_DFV, GEAR_TAG_TS, GEAR_TAG_GRAD = 1, 2, 3,
 
 EXPORTS = ("gear_workspace_bytes", "gear_init_tables", "gear_forward_backward", "gear_accumulate_dfv_grad",
            "gear_collect_ready", "gear_collect_expired", "gear_status", "gear_destroy", "gear_fill_uniform",
-           "gear_last_error", "gear_profile_enable", "gear_profile_read", "gear_launch_count")
+           "gear_last_error", "gear_profile_enable", "gear_profile_read", "gear_launch_count",
+           "gear_collect_expired_static")
+GEAR_STATIC_EXPIRY_MAX_VOCAB = 16777216
 
 
 class GearError(RuntimeError):
@@ -95,6 +97,8 @@ def load() -> C.CDLL:
     L.gear_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_float), C.POINTER(i32), i32, C.POINTER(i32)]
     L.gear_launch_count.restype = C.c_int
     L.gear_launch_count.argtypes = [vp, C.POINTER(i64)]
+    L.gear_collect_expired_static.restype = C.c_int
+    L.gear_collect_expired_static.argtypes = [vp, i64, i64, i64, C.c_int, vp, i64, vp, C.POINTER(i64), vp]
     L.gear_last_error.restype = C.c_char_p
     L.gear_last_error.argtypes = []
     _lib = L
@@ -240,3 +244,18 @@ def gear_launch_count(ctx) -> int:
     n = C.c_int64(0)
     _check(load().gear_launch_count(ctx, C.byref(n)), "gear_launch_count")
     return n.value
+
+
+def gear_collect_expired_static(dfv_ts, expire: int, now: int, restamp: bool, ids, cap: int, d_n=None,
+                                sync: bool = True, stream=None, img_vocab: Optional[int] = None) -> Optional[int]:
+    """The expiry scan without a ctx or workspace, for callers that may not allocate device memory: the
+    scratch lives in a fixed array inside libgear (tables of at most GEAR_STATIC_EXPIRY_MAX_VOCAB entries).
+    Returns the count when sync is True.  Raises GearError(GEAR_ERR_CAPACITY) for a table beyond that bound
+    or a cap that is too small."""
+    h = C.c_int64(-1)
+    n = int(dfv_ts.shape[0]) if img_vocab is None else img_vocab
+    rc = load().gear_collect_expired_static(_p(dfv_ts), n, expire, now, 1 if restamp else 0, _p(ids), cap, _p(d_n),
+                                            C.byref(h) if sync else None, _stream(stream))
+    if rc != GEAR_OK:
+        raise GearError(rc, "gear_collect_expired_static")
+    return h.value if sync else None

@@ -89,3 +89,83 @@ cudaError_t launch_collect_expired(const gear_ctx_impl& c, int64_t now, int rest
 }
 
 }  // namespace gear
+
+// ---------------------------------------------------------------------------------------------------
+// gear_collect_expired_static: the same scan for callers that cannot allocate device memory.
+//
+// Some hosts of this library run it where cudaMalloc is off limits: inside a serving process whose memory
+// pool was carved up at start-up and is policed, from a plug-in that is handed buffers but no allocator,
+// or on a path that must not touch the allocator because an allocation may synchronise the device.  Such a
+// caller cannot provide the workspace a gear_ctx needs.  This entry point therefore keeps the scan's
+// scratch (expired bitmap, per-tile counts, a small state block) in a fixed array that is part of the
+// library image: every GPU that loads libgear holds GEAR_STATIC_EXPIRY_SCRATCH_BYTES of it until the
+// process exits.  The price is a bound on the table size and one shared scratch per device.
+// ---------------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace gear {
+
+constexpr int64_t STATIC_MAX_VOCAB = GEAR_STATIC_EXPIRY_MAX_VOCAB;
+constexpr size_t STATIC_STATE_BYTES = 256;
+constexpr size_t STATIC_BITS_BYTES = (size_t)(STATIC_MAX_VOCAB / 32) * 4;
+constexpr size_t STATIC_CNT_BYTES = ((size_t)(STATIC_MAX_VOCAB / EXP_TILE) + 1) * sizeof(uint2);
+constexpr size_t STATIC_SCRATCH_BYTES = STATIC_STATE_BYTES + STATIC_BITS_BYTES + ((STATIC_CNT_BYTES + 255) / 256) * 256;
+static_assert(sizeof(DevState) <= STATIC_STATE_BYTES, "state block");
+static_assert(STATIC_SCRATCH_BYTES == GEAR_STATIC_EXPIRY_SCRATCH_BYTES, "the header states the size of the array");
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_expiry_scratch[STATIC_SCRATCH_BYTES];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+static std::mutex g_static_mutex;
+static unsigned char* g_static_ptr[STATIC_MAX_DEVICES];     // device address of the scratch, per device ordinal
+
+// Device address of the scratch on the current device (looked up once per device).
+static cudaError_t static_scratch(unsigned char** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_expiry_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = g_static_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace gear
+
+extern "C" int gear_collect_expired_static(int64_t* dfv_ts, int64_t img_vocab, int64_t expire, int64_t now, int restamp,
+                                           int32_t* ids, int64_t cap, int64_t* d_n, int64_t* h_n, void* stream) {
+    using namespace gear;
+    if (!dfv_ts || img_vocab < 1 || expire < 0 || cap < 0 || (cap > 0 && !ids)) return GEAR_ERR_ARG;
+    if (img_vocab > STATIC_MAX_VOCAB) return GEAR_ERR_CAPACITY;      // the fixed scratch cannot hold the bitmap
+    unsigned char* base = nullptr;
+    if (static_scratch(&base) != cudaSuccess) return GEAR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DevState* state = reinterpret_cast<DevState*>(base);
+    uint32_t* bits = reinterpret_cast<uint32_t*>(base + STATIC_STATE_BYTES);
+    uint2* tile_cnt = reinterpret_cast<uint2*>(base + STATIC_STATE_BYTES + STATIC_BITS_BYTES);
+    const int64_t n_tiles = ceil_div(img_vocab, EXP_TILE);
+
+    // the array keeps what the previous call left: the state block has to start from zero, the bitmap words
+    // and tile counts of this table size are all rewritten by the mark pass
+    if (cudaMemsetAsync(state, 0, STATIC_STATE_BYTES, st) != cudaSuccess) return GEAR_ERR_CUDA;
+    expiry_mark_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(dfv_ts, img_vocab, now, expire, bits, tile_cnt);
+    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, nullptr);
+    int64_t* d_cnt = d_n ? d_n : &state->pad[1];
+    expiry_check_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, cap, d_cnt, state);
+    expiry_write_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(bits, img_vocab, tile_cnt, state, now, restamp, dfv_ts, ids);
+    if (cudaGetLastError() != cudaSuccess) return GEAR_ERR_CUDA;
+    if (h_n) {
+        if (cudaMemcpyAsync(h_n, d_cnt, sizeof(int64_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            return GEAR_ERR_CUDA;
+        if (*h_n > cap) return GEAR_ERR_CAPACITY;
+    }
+    return GEAR_OK;
+}
