@@ -48,6 +48,7 @@ struct TileFlags {
     bool head[AF_ITEMS];       // starts a group
     bool first[AF_ITEMS];      // ... and is the first row of its image in this call
     bool complete[AF_ITEMS];   // ... and the group reaches M
+    int c0[AF_ITEMS];          // rows the image already holds in the table
     int64_t i0;                // first position owned by this thread
 };
 
@@ -105,11 +106,13 @@ __device__ __forceinline__ void tile_flags(TileFlags& f, const uint32_t* __restr
     for (int t = 0; t < AF_ITEMS; ++t) {
         const int64_t i = f.i0 + t;
         f.head[t] = f.first[t] = f.complete[t] = false;
+        f.c0[t] = 0;
         if (i >= n || f.key[t] >= vocab) continue;
         uint32_t rs = max(run_start[t], before_thread);
         const int64_t start = rs ? (int64_t)rs - 1 : (int64_t)carry;
         const int64_t j = i - start;                 // rank of this row among the call's rows of its image
         const int c0 = cnt[f.key[t]];
+        f.c0[t] = c0;
         const int rem = (int)((c0 + j) % M);
         if (j == 0 || rem == 0) {
             f.head[t] = true;
@@ -121,6 +124,10 @@ __device__ __forceinline__ void tile_flags(TileFlags& f, const uint32_t* __restr
     }
     if (blockIdx.x == 0 && threadIdx.x == 0 && (n == 0 || ks[0] >= vocab)) state->n_valid = 0;   // no valid row at all
 }
+
+struct RowSource {
+    const uint32_t* perm; const float* grads; int64_t ld; const int32_t* src_row; const float* scale;
+};
 
 __global__ void __launch_bounds__(AF_THREADS)
 acc_flag_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int M, const int32_t* __restrict__ cnt,
@@ -139,8 +146,8 @@ acc_flag_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int 
 
 __global__ void __launch_bounds__(AF_THREADS)
 acc_plan_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int M, const int32_t* __restrict__ cnt,
-                const uint2* __restrict__ tile_cnt, uint32_t* __restrict__ grp_start, int32_t* __restrict__ grp_slot,
-                DevState* __restrict__ state) {
+                const uint2* __restrict__ tile_cnt, uint4* __restrict__ grp_rec, RowSource rs,
+                int32_t* __restrict__ psrc, float* __restrict__ pscale, DevState* __restrict__ state) {
     __shared__ uint32_t smem[34];
     TileFlags f;
     tile_flags(f, ks, n, vocab, M, cnt, smem, state);
@@ -154,30 +161,39 @@ acc_plan_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int 
 #pragma unroll
     for (int t = 0; t < AF_ITEMS; ++t) {
         if (!f.head[t]) continue;
-        grp_start[gi] = (uint32_t)(f.i0 + t) | (f.first[t] ? 0x80000000u : 0u);
-        grp_slot[gi] = f.complete[t] ? (int32_t)(q_base + ci) : -1;
+        // one 16-byte record per group: start position (top bit: first group of its image in this call), image ID,
+        // ready-queue slot (-1: the group stays open), rows the image already held
+        grp_rec[gi] = make_uint4((uint32_t)(f.i0 + t) | (f.first[t] ? 0x80000000u : 0u), f.key[t],
+                                 (uint32_t)(f.complete[t] ? (int32_t)(q_base + ci) : -1), (uint32_t)f.c0[t]);
         ++gi;
         ci += f.complete[t];
     }
+    // where the gradient row of every sorted position lives and what it is scaled by, resolved through the sort
+    // permutation once, so that the reduce pass reads both with coalesced loads
+#pragma unroll
+    for (int t = 0; t < AF_ITEMS; ++t) {
+        const int64_t i = f.i0 + t;
+        if (i >= n || f.key[t] >= vocab) continue;
+        const uint32_t r = rs.perm[i];
+        const int32_t src = rs.src_row ? rs.src_row[r] : (int32_t)r;
+        psrc[i] = src;
+        pscale[i] = rs.scale ? rs.scale[src] : 1.f;
+    }
 }
 
-struct RowSource {
-    const uint32_t* perm; const float* grads; int64_t ld; const int32_t* src_row; const float* scale;
+struct RowGather {
+    const float* grads; int64_t ld; const int32_t* psrc; const float* pscale;
 };
 
 // Sum of the gradient rows at sorted positions [a, b), in order.  All 32 lanes call this together.
 template <int NQ>
-__device__ __forceinline__ void sum_rows(float4 (&acc)[NQ], const RowSource& rs, int64_t a, int64_t b, int n_chunks) {
+__device__ __forceinline__ void sum_rows(float4 (&acc)[NQ], const RowGather& rg, int64_t a, int64_t b, int n_chunks) {
     const unsigned lane = lane_id();
     for (int64_t p0 = a; p0 < b; p0 += 32) {
         const int m = (int)min((int64_t)32, b - p0);
-        int64_t my_s = 0;
+        int my_s = 0;
         float my_scale = 1.f;
-        if ((int)lane < m) {
-            const uint32_t r = rs.perm[p0 + lane];
-            my_s = rs.src_row ? (int64_t)rs.src_row[r] : (int64_t)r;
-            if (rs.scale) my_scale = rs.scale[my_s];
-        }
+        if ((int)lane < m) { my_s = rg.psrc[p0 + lane]; my_scale = rg.pscale[p0 + lane]; }
         for (int t0 = 0; t0 < m; t0 += 4) {
             float4 v[4][NQ];
             float sc[4];
@@ -189,7 +205,7 @@ __device__ __forceinline__ void sum_rows(float4 (&acc)[NQ], const RowSource& rs,
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
                     const int ch = lane + 32 * q;
-                    v[t][q] = (on && ch < n_chunks) ? ld_stream_f4(rs.grads + s * rs.ld + ch * 4)
+                    v[t][q] = (on && ch < n_chunks) ? ld_stream_f4(rg.grads + s * rg.ld + ch * 4)
                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
@@ -207,10 +223,10 @@ __device__ __forceinline__ void sum_rows(float4 (&acc)[NQ], const RowSource& rs,
 }
 
 template <int NQ>
-__global__ void __launch_bounds__(256)
-acc_reduce_kernel(const uint32_t* __restrict__ ks, RowSource rs, int D, int M, int64_t n_tiles, int64_t ready_cap,
-                  const uint2* __restrict__ tile_cnt, const uint32_t* __restrict__ grp_start,
-                  const int32_t* __restrict__ grp_slot, float* __restrict__ gsum, int32_t* __restrict__ gcnt,
+__global__ void __launch_bounds__(256, NQ <= 2 ? 4 : 2)
+acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, int64_t n_tiles, int64_t ready_cap,
+                  const uint2* __restrict__ tile_cnt, const uint4* __restrict__ grp_rec,
+                  float* __restrict__ gsum, int32_t* __restrict__ gcnt,
                   int32_t* __restrict__ q_id, float* __restrict__ q_avg, const DevState* __restrict__ state) {
     const uint2 totals = tile_cnt[n_tiles];
     const int64_t n_groups = totals.x;
@@ -218,39 +234,49 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowSource rs, int D, int M, i
     const int64_t n_valid = state->n_valid;
     const unsigned lane = lane_id();
     const int n_chunks = D / 4;
+    const float m_f = (float)M;
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    for (int64_t g = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); g < n_groups; g += warps) {
-        const uint32_t rec = grp_start[g];
-        const bool first = rec >> 31;
-        const int slot = grp_slot[g];
+    int64_t g = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    // records of this group and the next one (its start is this group's end), fetched one iteration ahead
+    uint4 rec = make_uint4(0u, 0u, 0u, 0u);
+    uint32_t next_start = 0;
+    if (g < n_groups) {
+        rec = grp_rec[g];
+        next_start = (g + 1 < n_groups) ? (grp_rec[g + 1].x & 0x7fffffffu) : (uint32_t)n_valid;
+    }
+    for (; g < n_groups; g += warps) {
+        const uint4 cur = rec;
+        const int64_t end = next_start;
+        const int64_t gn = g + warps;
+        if (gn < n_groups) {
+            rec = grp_rec[gn];
+            next_start = (gn + 1 < n_groups) ? (grp_rec[gn + 1].x & 0x7fffffffu) : (uint32_t)n_valid;
+        }
+        const bool first = cur.x >> 31;
+        const int slot = (int)cur.z;
         if (!first && slot < 0) continue;      // an image's trailing open group: settled by its first group's warp
-        const int64_t start = rec & 0x7fffffffu;
-        const int64_t end = (g + 1 < n_groups) ? (int64_t)(grp_start[g + 1] & 0x7fffffffu) : n_valid;
-        const uint32_t key = ks[start];
+        const int64_t start = cur.x & 0x7fffffffu;
+        const uint32_t key = cur.y;
+        const int c0 = first ? (int)cur.w : 0;
         float4 acc[NQ];
 #pragma unroll
         for (int q = 0; q < NQ; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        int c0 = 0;
         float* srow = gsum + (int64_t)key * D;
-        if (first) {
-            c0 = gcnt[key];
-            if (c0 > 0) {
+        if (c0 > 0) {
 #pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    const int ch = lane + 32 * q;
-                    if (ch < n_chunks) acc[q] = ld_f4(srow + ch * 4);
-                }
+            for (int q = 0; q < NQ; ++q) {
+                const int ch = lane + 32 * q;
+                if (ch < n_chunks) acc[q] = ld_f4(srow + ch * 4);
             }
         }
-        sum_rows<NQ>(acc, rs, start, end, n_chunks);
+        sum_rows<NQ>(acc, rg, start, end, n_chunks);
         if (slot >= 0) {
             float* qrow = q_avg + (int64_t)slot * D;
 #pragma unroll
             for (int q = 0; q < NQ; ++q) {
                 const int ch = lane + 32 * q;
                 if (ch < n_chunks)
-                    st_f4(qrow + ch * 4, make_float4(acc[q].x / (float)M, acc[q].y / (float)M, acc[q].z / (float)M,
-                                                     acc[q].w / (float)M));
+                    st_f4(qrow + ch * 4, make_float4(acc[q].x / m_f, acc[q].y / m_f, acc[q].z / m_f, acc[q].w / m_f));
             }
             if (lane == 0) q_id[slot] = (int32_t)key;
             if (!first) continue;
@@ -269,7 +295,7 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowSource rs, int D, int M, i
                 if (rest > 0) {
 #pragma unroll
                     for (int q = 0; q < NQ; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    sum_rows<NQ>(acc, rs, l - rest, l, n_chunks);
+                    sum_rows<NQ>(acc, rg, l - rest, l, n_chunks);
                 }
             }
             if (rest > 0 || c0 > 0) {
@@ -298,7 +324,7 @@ __global__ void acc_commit_kernel(const uint2* __restrict__ tile_cnt, int64_t n_
     state->n_groups = totals.x;
     state->n_complete = totals.y;
     if (state->q_count + (int64_t)totals.y > ready_cap) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
-    else state->q_count += totals.y;
+    else if (totals.y > 0) { state->q_count += totals.y; state->q_calls += 1; }
 }
 
 static int reduce_grid() { return 148 * 8; }
@@ -320,6 +346,7 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
         batch.job[0].n_max = n;
         batch.job[0].bits = bits_for(vocab);
         cudaError_t se;
+        batch.name = "sort_img";
         cur = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
         if (se != cudaSuccess) return se;
     }
@@ -329,17 +356,19 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     { KernelScope k(&c.prof, "acc_flag", st);
     acc_flag_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt, state); }
     scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, &c.prof);
-    uint32_t* grp_start = c.at<uint32_t>(c.ws.grp_start);
-    int32_t* grp_slot = c.at<int32_t>(c.ws.grp_slot);
+    uint4* grp_rec = c.at<uint4>(c.ws.grp_rec);
+    int32_t* psrc = c.at<int32_t>(c.ws.psrc);
+    float* pscale = c.at<float>(c.ws.pscale);
+    RowSource rs{sb.vals[cur], grads, ld, src_row, scale};
+    RowGather rg{grads, ld, psrc, pscale};
     { KernelScope k(&c.prof, "acc_plan", st);
     acc_plan_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt,
-                                                            grp_start, grp_slot, state); }
-    RowSource rs{sb.vals[cur], grads, ld, src_row, scale};
+                                                            grp_rec, rs, psrc, pscale, state); }
     const int nq = (int)ceil_div(D / 4, 32);
     int64_t want = ceil_div(n, 8);
     const int grid = (int)(want < reduce_grid() ? (want < 1 ? 1 : want) : reduce_grid());
-#define GEAR_ACC_LAUNCH(NQ) acc_reduce_kernel<NQ><<<grid, 256, 0, st>>>(ks, rs, D, M, n_tiles, c.ws.ready_cap, tile_cnt, \
-        grp_start, grp_slot, c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id), c.at<float>(c.ws.q_avg), state)
+#define GEAR_ACC_LAUNCH(NQ) acc_reduce_kernel<NQ><<<grid, 256, 0, st>>>(ks, rg, D, M, n_tiles, c.ws.ready_cap, tile_cnt, \
+        grp_rec, c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id), c.at<float>(c.ws.q_avg), state)
     { KernelScope k(&c.prof, "acc_reduce", st);
     if (nq <= 1) GEAR_ACC_LAUNCH(1);
     else if (nq <= 2) GEAR_ACC_LAUNCH(2);
@@ -348,6 +377,7 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
 #undef GEAR_ACC_LAUNCH
     { KernelScope k(&c.prof, "acc_commit", st);
     acc_commit_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, c.ws.ready_cap, state); }
+    ++c.acc_calls_pending;
     return cudaGetLastError();
 }
 
@@ -355,23 +385,31 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
 __global__ void collect_begin_kernel(DevState* __restrict__ state, int64_t cap, int64_t* __restrict__ d_n) {
     const int64_t n = state->q_count;
     if (d_n) *d_n = n;
-    if (n > cap) { atomicOr(&state->status, GEAR_DEV_OUT_CAPACITY); state->collect_n = -1; }
-    else state->collect_n = n;
+    if (n > cap) { atomicOr(&state->status, GEAR_DEV_OUT_CAPACITY); state->collect_n = -1; state->sort_n = 0; }
+    else {
+        state->collect_n = n;
+        // One accumulate call fills its slots in (id, group) order already; only a queue fed by several calls
+        // has to be re-ordered.
+        state->sort_n = state->q_calls <= 1 ? 0 : n;
+    }
 }
 
 __global__ void __launch_bounds__(256)
 collect_keys_kernel(const int32_t* __restrict__ q_id, const DevState* __restrict__ state, uint32_t* __restrict__ keys) {
-    const int64_t n = state->collect_n;
+    const int64_t n = state->sort_n;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         keys[i] = (uint32_t)q_id[i];
 }
 
 // One warp per output entry k: queue slot perm[k]; its emission number is its rank among equal IDs.
 __global__ void __launch_bounds__(256)
-collect_move_kernel(const uint32_t* __restrict__ ks, const uint32_t* __restrict__ perm, const float* __restrict__ q_avg,
+collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __restrict__ sorted_perm,
+                    const int32_t* __restrict__ q_id, const float* __restrict__ q_avg,
                     int D, const DevState* __restrict__ state, int32_t* __restrict__ ids, int32_t* __restrict__ seq,
                     float* __restrict__ avg) {
     const int64_t n = state->collect_n;
+    const bool in_order = state->sort_n == 0;          // the queue itself is sorted: no permutation
+    const uint32_t* ks = in_order ? reinterpret_cast<const uint32_t*>(q_id) : sorted_keys;
     const unsigned lane = lane_id();
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     for (int64_t k = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); k < n; k += warps) {
@@ -384,7 +422,7 @@ collect_move_kernel(const uint32_t* __restrict__ ks, const uint32_t* __restrict_
             const int64_t mid = (l + h) >> 1;
             if (ks[mid] == id) h = mid; else l = mid + 1;
         }
-        const float* src = q_avg + (int64_t)perm[k] * D;
+        const float* src = q_avg + (in_order ? k : (int64_t)sorted_perm[k]) * D;
         float* dst = avg + k * D;
         for (int ch = lane; ch < D / 4; ch += 32) st_f4(dst + ch * 4, ld_f4(src + ch * 4));
         if (lane == 0) { ids[k] = (int32_t)id; seq[k] = (int32_t)(k - l); }
@@ -392,7 +430,7 @@ collect_move_kernel(const uint32_t* __restrict__ ks, const uint32_t* __restrict_
 }
 
 __global__ void collect_end_kernel(DevState* __restrict__ state) {
-    if (state->collect_n >= 0) state->q_count = 0;
+    if (state->collect_n >= 0) { state->q_count = 0; state->q_calls = 0; }
 }
 
 cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
@@ -402,22 +440,31 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     const int64_t n_max = c.ws.ready_cap;
     { KernelScope k(&c.prof, "collect_begin", st);
     collect_begin_kernel<<<1, 1, 0, st>>>(state, cap, d_n); }
-    int64_t blocks = ceil_div(n_max, 256);
-    { KernelScope k(&c.prof, "collect_keys", st);
-    collect_keys_kernel<<<(unsigned)(blocks > 1184 ? 1184 : blocks), 256, 0, st>>>(c.at<int32_t>(c.ws.q_id), state,
-                                                                                 sb.keys[0]); }
-    SortBatch batch = c.sort_batch();
-    batch.n_jobs = 1;
-    batch.job[0] = sb;
-    batch.job[0].n_max = n_max;
-    batch.job[0].n_dev = &state->collect_n;
-    batch.job[0].bits = bits_for(c.cfg.img_vocab);
-    cudaError_t se;
-    const int cur = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
-    if (se != cudaSuccess) return se;
+    int cur = 0;
+    // A queue fed by at most one accumulate call is in (id, group) order already.  The host knows an upper bound
+    // of the number of feeding calls; only when that exceeds one are the sort kernels enqueued at all (the device
+    // then still decides from the exact count whether there is anything to re-order).
+    if (c.acc_calls_pending > 1) {
+        int64_t blocks = ceil_div(n_max, 256);
+        { KernelScope k(&c.prof, "collect_keys", st);
+        collect_keys_kernel<<<(unsigned)(blocks > 1184 ? 1184 : blocks), 256, 0, st>>>(c.at<int32_t>(c.ws.q_id), state,
+                                                                                     sb.keys[0]); }
+        SortBatch batch = c.sort_batch();
+        batch.n_jobs = 1;
+        batch.job[0] = sb;
+        batch.job[0].n_max = n_max;
+        batch.job[0].n_dev = &state->sort_n;
+        batch.job[0].bits = bits_for(c.cfg.img_vocab);
+        cudaError_t se;
+        batch.name = "sort_ready";
+        cur = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
+        if (se != cudaSuccess) return se;
+    }
+    if (cap >= c.ws.ready_cap) c.acc_calls_pending = 0;      // this collect cannot be refused: the queue will be empty
     int64_t want = ceil_div(n_max, 8);
     { KernelScope k(&c.prof, "collect_move", st);
     collect_move_kernel<<<(unsigned)(want > 1184 ? 1184 : want), 256, 0, st>>>(sb.keys[cur], sb.vals[cur],
+                                                                            c.at<int32_t>(c.ws.q_id),
                                                                             c.at<float>(c.ws.q_avg), c.cfg.dfv_dim,
                                                                             state, ids, seq, avg); }
     { KernelScope k(&c.prof, "collect_end", st);

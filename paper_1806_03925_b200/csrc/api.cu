@@ -67,6 +67,7 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
     }
     p->dz = take(B * 4);
     p->loss_part = take((size_t)p->loss_blocks * 4);
+    p->colsum_part = take((size_t)CS_BLOCKS * 1024 * 4);
     p->sort_n[0] = p->sort_n[1] = c.max_batch;
     p->sort_n[2] = c.max_nnz;
     p->sort_n[3] = p->ready_cap;
@@ -79,8 +80,9 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
         p->sort_tot[s] = take(RS_BUCKETS * 4);
     }
     p->tile_cnt = take((size_t)(ceil_div(c.max_nnz, 1024) + 1) * sizeof(uint2));
-    p->grp_start = take((size_t)c.max_nnz * 4);
-    p->grp_slot = take((size_t)c.max_nnz * 4);
+    p->grp_rec = take((size_t)c.max_nnz * 16);
+    p->psrc = take((size_t)c.max_nnz * 4);
+    p->pscale = take((size_t)c.max_nnz * 4);
     p->q_id = take((size_t)p->ready_cap * 4);
     p->q_avg = take((size_t)p->ready_cap * c.dfv_dim * 4);
     p->exp_bits = take((size_t)ceil_div(c.img_vocab, 32) * 4);
@@ -96,6 +98,15 @@ static int64_t param_count(const gear_config& c) {
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// the ctx's side stream and fork/join events (host-side driver objects, no device memory)
+static void release_host_objects(gear_ctx_impl& c) {
+    if (c.ev_fork) cudaEventDestroy(c.ev_fork);
+    if (c.ev_join) cudaEventDestroy(c.ev_join);
+    if (c.side_stream) cudaStreamDestroy(c.side_stream);
+    c.ev_fork = c.ev_join = nullptr;
+    c.side_stream = nullptr;
+}
 
 }  // namespace gear
 
@@ -153,10 +164,16 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
     c.img_sorted = false;
     c.img_sorted_n = 0;
     c.img_sorted_buf = 0;
+    c.acc_calls_pending = 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
+    c.side_stream = nullptr;
+    c.ev_fork = c.ev_join = nullptr;
 
-    cudaError_t e = cudaMemsetAsync(c.state(), 0, sizeof(DevState), st);
+    cudaError_t e = cudaStreamCreateWithFlags(&c.side_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_join, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c.state(), 0, sizeof(DevState), st);
     if (e == cudaSuccess && fill) {
         const double amp = 0.17320508075688773;   // uniform half-width for standard deviation 0.1
         e = launch_fill_uniform(buf->user_emb, GEAR_F32, cfg->user_vocab * cfg->emb_dim, seed, GEAR_TAG_USER, amp, st);
@@ -170,7 +187,7 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
         if (e == cudaSuccess) e = launch_fill_ts(buf->dfv_ts, cfg->img_vocab, seed, cfg->expire, now, st);
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    if (e != cudaSuccess) { delete ctx; return cuda_fail(e, "gear_init_tables"); }
+    if (e != cudaSuccess) { release_host_objects(c); delete ctx; return cuda_fail(e, "gear_init_tables"); }
     *out_ctx = ctx;
     return GEAR_OK;
 }
@@ -214,15 +231,26 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
             batch.job[2].n_max = b.nnz; batch.job[2].bits = bits_for(c.cfg.img_vocab);
             batch.n_jobs = 3;
         }
-        cudaError_t se;
-        sorted_buf = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
+        // The sort depends only on the ID arrays, so it runs on the ctx's side stream beside the gather and
+        // the head (fork here, join before the first consumer of a sorted order).
+        cudaError_t se = cudaEventRecord(c.ev_fork, st);
+        if (se == cudaSuccess) se = cudaStreamWaitEvent(c.side_stream, c.ev_fork, 0);
+        if (se != cudaSuccess) return cuda_fail(se, "fork");
+        batch.name = "sort_ids";
+        sorted_buf = sort_jobs(batch, &c.gbs, c.side_stream, &c.prof, &se);
         if (se != cudaSuccess) return cuda_fail(se, "id sort");
+        se = cudaEventRecord(c.ev_join, c.side_stream);
+        if (se != cudaSuccess) return cuda_fail(se, "join");
         if (b.nnz > 0) { c.img_sorted = true; c.img_sorted_n = b.nnz; c.img_sorted_buf = sorted_buf; }
     }
     cudaError_t e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
     if (e != cudaSuccess) return cuda_fail(e, "gather");
     e = launch_head_simt(c, b, o, st);
     if (e != cudaSuccess) return cuda_fail(e, "head");
+    if (b.B > 0) {
+        e = cudaStreamWaitEvent(st, c.ev_join, 0);
+        if (e != cudaSuccess) return cuda_fail(e, "join");
+    }
     const int E = c.cfg.emb_dim;
     float* ut = o.user_grad ? o.user_grad : c.buf.user_emb;
     float* ht = o.url_grad ? o.url_grad : c.buf.url_emb;
@@ -369,6 +397,8 @@ int gear_destroy(gear_ctx* ctx) {
     if (!ctx) return GEAR_OK;
     if (!ctx->impl.alive) return GEAR_ERR_STATE;
     cudaStreamSynchronize(ctx->impl.last_stream);
+    cudaStreamSynchronize(ctx->impl.side_stream);
+    release_host_objects(ctx->impl);
     ctx->impl.alive = false;
     delete ctx;
     return GEAR_OK;

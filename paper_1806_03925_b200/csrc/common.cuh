@@ -24,7 +24,11 @@ struct DevState {
     int64_t exp_total;     // expiry scan: entries found
     int64_t collect_n;     // collect_ready: entries moved by the running call
     unsigned long long grid_barrier;   // arrival counter of the cooperative sort's grid barrier
-    int64_t pad[8];
+    unsigned int colsum_ticket;        // blocks of the column-sum kernel that have delivered their partials
+    unsigned int pad32;
+    int64_t q_calls;       // accumulate calls that added to the ready queue since the last collect
+    int64_t sort_n;        // collect_ready: entries the queue sort has to order (0: the queue is already in order)
+    int64_t pad[5];
 };
 static_assert(sizeof(DevState) == 128, "DevState layout");
 
@@ -133,14 +137,8 @@ struct KernelScope {
 constexpr int RS_THREADS = 256;
 constexpr int RS_ITEMS = 16;
 constexpr int RS_TILE = RS_THREADS * RS_ITEMS;
-constexpr int RS_BUCKETS = 256;
-
-struct SortBufs {
-    uint32_t* keys[2];
-    uint32_t* vals[2];
-    uint32_t* hist;     // [256][n_tiles(n_max)]
-    uint32_t* tot;      // [256]
-};
+constexpr int RS_RADIX_BITS = 9;
+constexpr int RS_BUCKETS = 1 << RS_RADIX_BITS;
 
 inline int64_t sort_tiles(int64_t n_max) { return n_max > 0 ? ceil_div(n_max, RS_TILE) : 1; }
 
@@ -151,8 +149,8 @@ struct SortJob {
     int32_t* status;        // device status word that gets GEAR_DEV_BAD_ID when a sentinel key is met (may be null)
     uint32_t* keys[2];      // without ids the input keys are keys[0]
     uint32_t* vals[2];      // with identity_vals the value of element i is i, else vals[0][i]
-    uint32_t* hist;         // [256][n_tiles]
-    uint32_t* tot;          // [256]
+    uint32_t* hist;         // [RS_BUCKETS][n_tiles]
+    uint32_t* tot;          // [RS_BUCKETS]
     int64_t n_max;          // element count (or its upper bound when n_dev is given)
     const int64_t* n_dev;   // optional device-resident count, capped at n_max
     int bits;
@@ -163,7 +161,8 @@ struct SortJob {
 struct SortBatch {
     SortJob job[3];
     int n_jobs;
-    int passes;                       // filled in by sort_jobs
+    const char* name;                 // host only: the name the launch is timed under
+    int passes, n_barriers;           // filled in by sort_jobs
     unsigned long long* barrier_ctr;  // filled in by sort_jobs
     unsigned long long barrier_base;
     int32_t* err;                     // device word that receives a non-zero code when a grid barrier gives up

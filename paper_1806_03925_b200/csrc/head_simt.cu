@@ -99,39 +99,116 @@ static void launch_gemm(int M, int N, int K, const TA* A, int64_t sam, int64_t s
                                                           ldm, k_chunk);
 }
 
-// Output unit, loss and the gradient at the top hidden layer.  One warp per view.
+// 8 consecutive activations as floats (one 16-byte load for bf16, two for fp32)
+__device__ __forceinline__ void load8(const float* p, float* v) {
+    const float4 a = ld_f4(p), b = ld_f4(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float* v) {
+    const uint4 t = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { v[2 * k] = __uint_as_float(w[k] << 16); v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u); }
+}
+// stores 8 values in the head dtype and returns them as stored (rounded for bf16)
+__device__ __forceinline__ void store8(float* p, float* v) {
+    st_f4(p, make_float4(v[0], v[1], v[2], v[3]));
+    st_f4(p + 4, make_float4(v[4], v[5], v[6], v[7]));
+}
+__device__ __forceinline__ void store8(__nv_bfloat16* p, float* v) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+        w[k] = *reinterpret_cast<uint32_t*>(&h2);
+        v[2 * k] = __uint_as_float(w[k] << 16);
+        v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Output unit, loss and everything that hangs off the top hidden layer.  One warp per view, a lane owns
+// 8-column chunks (128-bit loads and stores), so the top activations are read once:
 //   z = h . w_out + b_out;  p = sigmoid(z);  BCE in its overflow-safe form;  dz = (p - y) / B
-//   dA_top[b][j] = dz * w_out[j] where h[b][j] > 0, else 0
-template <typename TX>
+//   dA_top[b][j] = dz * w_out[j] where h[b][j] > 0, else 0            (stored in the head dtype)
+//   gw_out[j] += sum_b h[b][j] dz[b];  gb_top[j] += sum_b dA_top[b][j];  gb_out += sum_b dz[b]
+// NQ = chunks per lane = ceil(H / 256).
+template <typename TX, int NQ>
 __global__ void __launch_bounds__(256)
 head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict__ w_out,
                 const float* __restrict__ b_out, const float* __restrict__ label, float* __restrict__ prob,
-                float* __restrict__ dz, TX* __restrict__ dA, float* __restrict__ loss_part) {
-    __shared__ float part[8];
+                float* __restrict__ dz, TX* __restrict__ dA, float* __restrict__ loss_part,
+                float* __restrict__ gw_out, float* __restrict__ gb_top, float* __restrict__ gb_out) {
+    __shared__ float part[8], gpart[8];
+    __shared__ float s_gw[1024], s_gb[1024];
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
-    float local = 0.f;
+    for (int j = threadIdx.x; j < H; j += 256) { s_gw[j] = 0.f; s_gb[j] = 0.f; }
+    float w[NQ][8], gw[NQ][8], gb[NQ][8];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        const int c0 = (lane + 32 * q) * 8;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { w[q][k] = c0 < H ? w_out[c0 + k] : 0.f; gw[q][k] = 0.f; gb[q][k] = 0.f; }
+    }
+    float local = 0.f, gsum = 0.f;
+    const float bias = b_out[0];
+    __syncthreads();
     for (int b = blockIdx.x * 8 + warp; b < B; b += gridDim.x * 8) {
         const TX* row = h + (int64_t)b * H;
+        float v[NQ][8];
         float z = 0.f;
-        for (int j = lane; j < H; j += 32) z = fmaf(to_f(row[j]), w_out[j], z);
-        z = warp_sum(z) + b_out[0];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const int c0 = (lane + 32 * q) * 8;
+            if (c0 < H) load8(row + c0, v[q]);
+            else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[q][k] = 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) z = fmaf(v[q][k], w[q][k], z);
+        }
+        z = warp_sum(z) + bias;
         const float y = label[b];
         const float p = 1.0f / (1.0f + expf(-z));
         const float g = (p - y) / (float)B;
         if (lane == 0) {
             local += fmaxf(z, 0.f) - z * y + log1pf(expf(-fabsf(z)));
+            gsum += g;
             if (prob) prob[b] = p;
             dz[b] = g;
         }
         TX* drow = dA + (int64_t)b * H;
-        for (int j = lane; j < H; j += 32) drow[j] = from_f<TX>(to_f(row[j]) > 0.f ? g * w_out[j] : 0.f);
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const int c0 = (lane + 32 * q) * 8;
+            if (c0 >= H) continue;
+            float d[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                gw[q][k] = fmaf(v[q][k], g, gw[q][k]);
+                d[k] = v[q][k] > 0.f ? g * w[q][k] : 0.f;
+            }
+            store8(drow + c0, d);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) gb[q][k] += d[k];
+        }
     }
-    if (lane == 0) part[warp] = local;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        const int c0 = (lane + 32 * q) * 8;
+        if (c0 >= H) continue;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { atomicAdd(&s_gw[c0 + k], gw[q][k]); atomicAdd(&s_gb[c0 + k], gb[q][k]); }
+    }
+    if (lane == 0) { part[warp] = local; gpart[warp] = gsum; }
     __syncthreads();
+    for (int j = threadIdx.x; j < H; j += 256) { atomicAdd(gw_out + j, s_gw[j]); atomicAdd(gb_top + j, s_gb[j]); }
     if (threadIdx.x == 0) {
-        float s = 0.f;
-        for (int w = 0; w < 8; ++w) s += part[w];
+        float s = 0.f, t = 0.f;
+        for (int k = 0; k < 8; ++k) { s += part[k]; t += gpart[k]; }
         loss_part[blockIdx.x] = s;
+        atomicAdd(gb_out, t);
     }
 }
 
@@ -149,42 +226,62 @@ __global__ void loss_final_kernel(const float* __restrict__ part, int n, int B, 
     }
 }
 
-// out[n] += sum_b A[b][n] * (w ? w[b] : 1): bias gradients and the output-weight gradient.
+// out[n] += sum_b A[b][n]: bias gradient of a lower hidden layer.  A block of 256 threads sums its own range of
+// rows: thread t owns the 8 columns of chunk t % (N/8) (128-bit loads) and every (256 / (N/8))-th row, four loads
+// in flight.  Each block adds its partial sums to the output with one atomic per column.
 template <typename TA>
 __global__ void __launch_bounds__(256)
-colsum_kernel(int B, int N, const TA* __restrict__ A, const float* __restrict__ w, float* __restrict__ out,
-              int rows_per_block) {
+colsum_kernel(int B, int N, const TA* __restrict__ A, float* __restrict__ out) {
+    __shared__ float s[1024];
+    const int tpr = N / 8, rpp = 256 / tpr;
+    const int chunk = threadIdx.x % tpr, rsub = threadIdx.x / tpr;
+    const int rows_per_block = (int)ceil_div(B, gridDim.x);
     const int b0 = blockIdx.x * rows_per_block, b1 = min(B, b0 + rows_per_block);
-    for (int n = threadIdx.x; n < N; n += blockDim.x) {
-        float s = 0.f;
-        for (int b = b0; b < b1; ++b) s = fmaf(to_f(A[(int64_t)b * N + n]), w ? w[b] : 1.f, s);
-        atomicAdd(out + n, s);
-    }
-}
-
-__global__ void sum_vec_kernel(int n, const float* __restrict__ v, float* __restrict__ out) {
-    __shared__ float sm[32];
-    float s = 0.f;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) s += v[i];
-    s = warp_sum(s);
-    if (lane_id() == 0) sm[threadIdx.x >> 5] = s;
+    for (int j = threadIdx.x; j < N; j += 256) s[j] = 0.f;
     __syncthreads();
-    if (threadIdx.x < 32) {
-        float t = threadIdx.x < (blockDim.x >> 5) ? sm[threadIdx.x] : 0.f;
-        t = warp_sum(t);
-        if (threadIdx.x == 0) out[0] = t;
+    if (rsub < rpp) {
+        float acc[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+        for (int b = b0 + rsub; b < b1; b += 4 * rpp) {
+            float v[4][8];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                if (b + r * rpp < b1) load8(A + (int64_t)(b + r * rpp) * N + chunk * 8, v[r]);
+                else {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) v[r][k] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int k = 0; k < 8; ++k) acc[k] += v[r][k];
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) atomicAdd(&s[chunk * 8 + k], acc[k]);
     }
+    __syncthreads();
+    for (int j = threadIdx.x; j < N; j += 256) atomicAdd(out + j, s[j]);
 }
 
+// fp32 master weights -> bf16 in both orientations, all hidden layers in one launch (blockIdx.y = layer)
+struct RoundArgs {
+    int fan_in[MAX_LAYERS], fan_out[MAX_LAYERS];
+    const float* W[MAX_LAYERS];
+    __nv_bfloat16* wb[MAX_LAYERS];
+    __nv_bfloat16* wbt[MAX_LAYERS];
+};
 __global__ void __launch_bounds__(256)
-round_weights_kernel(int fan_in, int fan_out, const float* __restrict__ W, __nv_bfloat16* __restrict__ wb,
-                     __nv_bfloat16* __restrict__ wbt) {
+round_weights_kernel(const RoundArgs a) {
+    const int l = blockIdx.y;
+    const int fan_in = a.fan_in[l], fan_out = a.fan_out[l];
     const int64_t n = (int64_t)fan_in * fan_out;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-        const __nv_bfloat16 v = __float2bfloat16_rn(W[i]);
-        wb[i] = v;
+        const __nv_bfloat16 v = __float2bfloat16_rn(a.W[l][i]);
+        a.wb[l][i] = v;
         const int r = (int)(i / fan_out), c = (int)(i % fan_out);
-        wbt[(int64_t)c * fan_in + r] = v;
+        a.wbt[l][(int64_t)c * fan_in + r] = v;
     }
 }
 
@@ -238,16 +335,19 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
 
     // weights as the products see them
     const void* Wop[MAX_LAYERS];
-    for (int l = 0; l < L; ++l) {
-        if (BF) {
-            __nv_bfloat16* wb = c.at<__nv_bfloat16>(c.ws.wb[l]);
-            KernelScope ks(&c.prof, "round_weights", st);
-            round_weights_kernel<<<64, 256, 0, st>>>(p.fan[l], p.fan[l + 1], p.W[l], wb,
-                                                     c.at<__nv_bfloat16>(c.ws.wbt[l]));
-            Wop[l] = wb;
-        } else {
-            Wop[l] = p.W[l];
+    if (BF) {
+        RoundArgs ra;
+        int64_t biggest = 0;
+        for (int l = 0; l < L; ++l) {
+            ra.fan_in[l] = p.fan[l]; ra.fan_out[l] = p.fan[l + 1]; ra.W[l] = p.W[l];
+            ra.wb[l] = c.at<__nv_bfloat16>(c.ws.wb[l]); ra.wbt[l] = c.at<__nv_bfloat16>(c.ws.wbt[l]);
+            Wop[l] = ra.wb[l];
+            if ((int64_t)p.fan[l] * p.fan[l + 1] > biggest) biggest = (int64_t)p.fan[l] * p.fan[l + 1];
         }
+        KernelScope ks(&c.prof, "round_weights", st);
+        round_weights_kernel<<<dim3((unsigned)ceil_div(biggest, 256), (unsigned)L), 256, 0, st>>>(ra);
+    } else {
+        for (int l = 0; l < L; ++l) Wop[l] = p.W[l];
     }
     int32_t* tc_err = &c.state()->tc_error;
     cudaError_t tce = cudaSuccess;
@@ -264,17 +364,19 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
                                                     "simt_gemm_fwd");
     }
     const int HT = p.fan[L];
-    { KernelScope ks(&c.prof, "head_out", st);
-    head_out_kernel<TX><<<c.ws.loss_blocks, 256, 0, st>>>(B, HT, H[L], p.w_out, p.b_out, bt.label, o.prob, dz, dA[L],
-                                                          loss_part); }
+    {
+        KernelScope ks(&c.prof, "head_out", st);
+        const int nq = (int)ceil_div(HT, 256);
+#define GEAR_HEAD_OUT(NQ) head_out_kernel<TX, NQ><<<c.ws.loss_blocks, 256, 0, st>>>(B, HT, H[L], p.w_out, p.b_out, bt.label, \
+        o.prob, dz, dA[L], loss_part, p.gw_out, p.gb[L - 1], p.gb_out)
+        if (nq <= 1) GEAR_HEAD_OUT(1);
+        else if (nq == 2) GEAR_HEAD_OUT(2);
+        else GEAR_HEAD_OUT(4);
+#undef GEAR_HEAD_OUT
+    }
     { KernelScope ks(&c.prof, "loss_final", st);
     loss_final_kernel<<<1, 256, 0, st>>>(loss_part, c.ws.loss_blocks, B, o.loss); }
     // backward
-    const int rows = 128;
-    { KernelScope ks(&c.prof, "colsum", st);
-    colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, HT, H[L], dz, p.gw_out, rows); }
-    { KernelScope ks(&c.prof, "sum_vec", st);
-    sum_vec_kernel<<<1, 1024, 0, st>>>(B, dz, p.gb_out); }
     for (int l = L - 1; l >= 0; --l) {
         const int K = p.fan[l], N = p.fan[l + 1];
         // dW_l = H_l^T dA_{l+1}
@@ -284,8 +386,11 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
         } else
         launch_gemm<TX, TX, float, TX, EPI_ATOMIC>(K, N, B, H[l], 1, K, dA[l + 1], N, 1, p.gW[l], N, nullptr,
                                                    (const TX*)nullptr, 0, splits_for(K, N, B), st, &c.prof, "simt_gemm_dw");
-        { KernelScope ks(&c.prof, "colsum", st);
-        colsum_kernel<TX><<<(unsigned)ceil_div(B, rows), 256, 0, st>>>(B, N, dA[l + 1], nullptr, p.gb[l], rows); }
+        if (l < L - 1) {     // the top layer's bias gradient came out of head_out_kernel
+            KernelScope ks(&c.prof, "colsum", st);
+            const int blocks = B < CS_BLOCKS * 8 ? (int)ceil_div(B, 8) : CS_BLOCKS;
+            colsum_kernel<TX><<<blocks, 256, 0, st>>>(B, N, dA[l + 1], p.gb[l]);
+        }
         if constexpr (BF) {
             const __nv_bfloat16* wb = c.at<__nv_bfloat16>(c.ws.wb[l]);
             if (l > 0) tce = tc_gemm_kmajor(&c.prof, "tc_gemm_dh", B, K, N, dA[l + 1], N, wb, N, 1, dA[l], K, nullptr,

@@ -12,6 +12,7 @@ namespace gear {
 
 constexpr int EXP_TILE = 8192;     // entries of the timestamp table per block of the expiry scan
 constexpr int MAX_LAYERS = 2;
+constexpr int CS_BLOCKS = 296;      // blocks of the column-sum kernel (two per SM)
 
 // Byte offsets into the caller's workspace.  Everything is 256-byte aligned.
 struct WsPlan {
@@ -21,6 +22,7 @@ struct WsPlan {
     size_t da[MAX_LAYERS];              // [max_batch][hidden[l]] head dtype: gradient at the pre-activation
     size_t dz;                          // [max_batch] fp32
     size_t loss_part;                   // [loss_blocks] fp32 per-block partial losses
+    size_t colsum_part;                 // [CS_BLOCKS][1024] fp32 per-block partial column sums
     size_t wb[MAX_LAYERS];              // bf16 head: W_l as [in][out]
     size_t wbt[MAX_LAYERS];             // bf16 head: W_l as [out][in]
     // four sets of sort buffers: user IDs, URL IDs (max_batch each), image IDs (max_nnz), ready queue (ready_cap)
@@ -28,8 +30,8 @@ struct WsPlan {
     size_t sort_hist[4], sort_tot[4];
     int64_t sort_n[4];
     size_t tile_cnt;                    // [sort tiles + 1] uint2 per-tile (groups, complete) counts
-    size_t grp_start;                   // [max_nnz] uint32 (top bit: first group of its image in this call)
-    size_t grp_slot;                    // [max_nnz] int32 ready-queue slot or -1
+    size_t grp_rec;                     // [max_nnz] uint4 group records (start | first flag, image ID, queue slot, held rows)
+    size_t psrc, pscale;                // [max_nnz] int32 / fp32: source row and scale of every sorted position
     size_t q_id;                        // [ready_cap] int32
     size_t q_avg;                       // [ready_cap][dfv_dim] fp32
     size_t exp_bits;                    // [ceil(img_vocab / 32)] uint32 expired bitmap
@@ -50,12 +52,15 @@ struct gear_ctx_impl {
     cudaStream_t last_stream;
     bool alive;
     void* tc_state;     // tensor-core head state (tensor maps), owned by head_tc.cu; may be null
+    cudaStream_t side_stream;          // runs the ID sort of a step beside the gather and the head
+    cudaEvent_t ev_fork, ev_join;
     mutable Profiler prof;
     mutable GridBarrierState gbs;
     // image IDs of the last gear_forward_backward batch, already sorted (reused by gear_accumulate_dfv_grad)
     bool img_sorted;
     int64_t img_sorted_n;
     int img_sorted_buf;
+    mutable int acc_calls_pending;      // accumulate calls enqueued since a collect that was sure to drain the queue
 
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(static_cast<char*>(buf.workspace) + off); }
     DevState* state() const { return at<DevState>(ws.state); }

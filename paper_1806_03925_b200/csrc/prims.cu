@@ -1,11 +1,16 @@
 // Stable LSD radix sort of (key, value) pairs and small scan helpers.
 //
-// One cooperative, persistent kernel sorts up to three independent arrays ("jobs") in one launch.  Every
-// pass has three phases over tiles of RS_TILE consecutive elements -- per-tile digit histogram, per-digit
-// scan over tiles, stable scatter -- separated by a grid-wide barrier.  A warp owns 32 * RS_ITEMS
-// consecutive elements of a tile and ranks equal digits with match_any, which keeps equal keys in index
-// order.  The first pass can read raw int32 IDs and map out-of-range ones to a sentinel key that sorts
-// last, so no separate key-building launch is needed.
+// One cooperative, persistent kernel sorts up to three independent arrays ("jobs") in one launch.  A pass
+// (digits of up to 9 bits) has three phases over tiles of RS_TILE consecutive elements, separated by
+// grid-wide barriers:
+//   count    per-tile digit histogram -> hist[digit][tile]
+//   scan     one warp per digit: exclusive scan of that digit's per-tile counts, digit total
+//   scatter  each tile looks up where its digits start, ranks its elements and writes them out.  A warp owns
+//            32 * RS_ITEMS consecutive elements of a tile and ranks equal digits with match_any, which
+//            keeps equal keys in index order.
+// The first pass can read raw int32 IDs and map out-of-range ones to a sentinel key that sorts last, so no
+// separate key-building launch is needed.  Arrays whose live size (known only on the device) fits a few
+// tiles are sorted by block 0 alone, with block-level barriers only.
 //
 // The grid barrier is a monotonically increasing 64-bit arrival counter: barrier k of a launch completes
 // when the counter reaches base + grid * (k + 1), where the host knows `base` (it adds up what every
@@ -16,7 +21,8 @@
 
 namespace gear {
 
-constexpr uint32_t GRID_SPIN_LIMIT = 1u << 21;
+constexpr uint32_t GRID_SPIN_LIMIT = 1u << 22;
+constexpr int RS_SOLO_TILES = 3;        // live tiles (all jobs) up to which block 0 sorts alone
 
 __device__ __forceinline__ int64_t effective_n(int64_t n_max, const int64_t* n_dev) {
     if (!n_dev) return n_max;
@@ -24,7 +30,7 @@ __device__ __forceinline__ int64_t effective_n(int64_t n_max, const int64_t* n_d
     return n < n_max ? (n < 0 ? 0 : n) : n_max;
 }
 
-// All threads of every block call this.  Returns false once the launch has been abandoned.
+// All threads of every participating block call this.  Returns false once the launch has been abandoned.
 __device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned long long target, int32_t* err) {
     __shared__ int ok_flag;
     __syncthreads();
@@ -35,8 +41,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* ctr, unsigned l
         uint32_t spin = 0;
         while (*reinterpret_cast<volatile unsigned long long*>(ctr) < target) {
             if (++spin > GRID_SPIN_LIMIT) { atomicCAS(err, 0, 100); ok = 0; break; }
-            if ((spin & 255u) == 255u && *reinterpret_cast<volatile int32_t*>(err) != 0) { ok = 0; break; }
-            __nanosleep(20);
+            if ((spin & 1023u) == 1023u && *reinterpret_cast<volatile int32_t*>(err) != 0) { ok = 0; break; }
         }
         __threadfence();
         ok_flag = ok;
@@ -58,23 +63,43 @@ coop_sort_kernel(const SortBatch batch) {
     __shared__ uint32_t scratch[33];
     __shared__ uint32_t base[RS_BUCKETS];
     __shared__ uint32_t wcnt[RS_THREADS / 32][RS_BUCKETS];
+    __shared__ int live_tiles[3];
+    __shared__ int64_t live_n[3];
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
-    int total_tiles = 0;
-    for (int j = 0; j < batch.n_jobs; ++j) total_tiles += batch.job[j].n_tiles;
-    unsigned long long target = batch.barrier_base;
 
-    for (int pass = 0; pass < batch.passes; ++pass) {
+    if (threadIdx.x == 0) {
+        for (int j = 0; j < batch.n_jobs; ++j) {
+            live_n[j] = effective_n(batch.job[j].n_max, batch.job[j].n_dev);
+            live_tiles[j] = (int)ceil_div(live_n[j], RS_TILE);
+        }
+    }
+    __syncthreads();
+    int total_tiles = 0;
+    for (int j = 0; j < batch.n_jobs; ++j) total_tiles += live_tiles[j];
+    // small problems: block 0 alone, no grid barrier (it still advances the arrival counter on behalf of all)
+    const bool solo = total_tiles <= RS_SOLO_TILES;
+    if (solo && blockIdx.x != 0) return;
+    const int nblk = solo ? 1 : gridDim.x;
+    unsigned long long target = batch.barrier_base;
+    auto sync_all = [&]() -> bool {
+        if (solo) { __syncthreads(); return true; }
+        target += gridDim.x;
+        return grid_barrier(batch.barrier_ctr, target, batch.err);
+    };
+    bool ok = true;
+
+    for (int pass = 0; pass < batch.passes && ok; ++pass) {
         const int src = pass & 1, dst = src ^ 1;
 
-        // ---- phase A: digit histogram of every tile
-        for (int w = blockIdx.x; w < total_tiles; w += gridDim.x) {
+        // ---- count: digit histogram of every live tile
+        for (int w = blockIdx.x; w < total_tiles; w += nblk) {
             int jj = 0, t = w;
-            while (t >= batch.job[jj].n_tiles) { t -= batch.job[jj].n_tiles; ++jj; }
+            while (t >= live_tiles[jj]) { t -= live_tiles[jj]; ++jj; }
             const SortJob& j = batch.job[jj];
-            const int64_t n = effective_n(j.n_max, j.n_dev);
+            const int64_t n = live_n[jj];
             const int shift = pass * j.width;
             const uint32_t mask = (1u << j.width) - 1u;
-            base[threadIdx.x] = 0;
+            for (int d = threadIdx.x; d < RS_BUCKETS; d += RS_THREADS) base[d] = 0;
             __syncthreads();
             const int64_t tile0 = (int64_t)t * RS_TILE;
             bool bad = false;
@@ -89,47 +114,63 @@ coop_sort_kernel(const SortBatch batch) {
             }
             if (bad && pass == 0 && j.ids && j.status) atomicOr(j.status, GEAR_DEV_BAD_ID);
             __syncthreads();
-            __stcg(j.hist + (int64_t)threadIdx.x * j.n_tiles + t, base[threadIdx.x]);
+            for (int d = threadIdx.x; d <= (int)mask; d += RS_THREADS)
+                __stcg(j.hist + (int64_t)d * j.n_tiles + t, base[d]);
             __syncthreads();
         }
-        target += gridDim.x;
-        if (!grid_barrier(batch.barrier_ctr, target, batch.err)) return;
+        if (!(ok = sync_all())) break;
 
-        // ---- phase B: per digit, exclusive scan of the per-tile counts; digit totals
-        for (int r = blockIdx.x; r < batch.n_jobs * RS_BUCKETS; r += gridDim.x) {
-            const SortJob& j = batch.job[r / RS_BUCKETS];
-            const int d = r % RS_BUCKETS;
+        // ---- scan: per digit (one warp per row), exclusive scan of the per-tile counts; digit totals
+        for (int r = blockIdx.x * (RS_THREADS / 32) + warp; r < batch.n_jobs * RS_BUCKETS; r += nblk * (RS_THREADS / 32)) {
+            const int jj = r / RS_BUCKETS, d = r % RS_BUCKETS;
+            const SortJob& j = batch.job[jj];
+            if (d >= (1 << j.width)) continue;
             uint32_t* row = j.hist + (int64_t)d * j.n_tiles;
             uint32_t carry = 0;
-            for (int b0 = 0; b0 < j.n_tiles; b0 += RS_THREADS) {
-                const int i = b0 + threadIdx.x;
-                const uint32_t v = i < j.n_tiles ? __ldcg(row + i) : 0u;
-                uint32_t total;
-                const uint32_t ex = block_exclusive_scan(v, scratch, &total);
-                if (i < j.n_tiles) __stcg(row + i, carry + ex);
-                carry += total;
+            for (int b0 = 0; b0 < live_tiles[jj]; b0 += 32) {
+                const int i = b0 + lane;
+                const uint32_t v = i < live_tiles[jj] ? __ldcg(row + i) : 0u;
+                const uint32_t inc = warp_inclusive_scan(v);
+                if (i < live_tiles[jj]) __stcg(row + i, carry + inc - v);
+                carry += __shfl_sync(0xffffffffu, inc, 31);
             }
-            if (threadIdx.x == 0) __stcg(j.tot + d, carry);
+            if (lane == 0) __stcg(j.tot + d, carry);
         }
-        target += gridDim.x;
-        if (!grid_barrier(batch.barrier_ctr, target, batch.err)) return;
+        if (!(ok = sync_all())) break;
 
-        // ---- phase C: stable scatter
-        for (int w = blockIdx.x; w < total_tiles; w += gridDim.x) {
+        // ---- scatter
+        for (int w = blockIdx.x; w < total_tiles; w += nblk) {
             int jj = 0, t = w;
-            while (t >= batch.job[jj].n_tiles) { t -= batch.job[jj].n_tiles; ++jj; }
+            while (t >= live_tiles[jj]) { t -= live_tiles[jj]; ++jj; }
             const SortJob& j = batch.job[jj];
-            const int64_t n = effective_n(j.n_max, j.n_dev);
+            const int64_t n = live_n[jj];
             const int64_t tile0 = (int64_t)t * RS_TILE;
-            if (tile0 >= n) continue;                       // uniform over the block
             const int shift = pass * j.width;
             const uint32_t mask = (1u << j.width) - 1u;
-            {
-                const uint32_t tt = __ldcg(j.tot + threadIdx.x);
-                const uint32_t ex = block_exclusive_scan(tt, scratch, nullptr);
-                base[threadIdx.x] = ex + __ldcg(j.hist + (int64_t)threadIdx.x * j.n_tiles + t);
+            {   // where each digit of this tile starts in the output
+                uint32_t tot[RS_BUCKETS / RS_THREADS], before[RS_BUCKETS / RS_THREADS];
+#pragma unroll
+                for (int q = 0; q < RS_BUCKETS / RS_THREADS; ++q) {
+                    const int d = threadIdx.x * (RS_BUCKETS / RS_THREADS) + q;     // a thread owns adjacent digits
+                    tot[q] = before[q] = 0;
+                    if (d <= (int)mask) {
+                        tot[q] = __ldcg(j.tot + d);
+                        before[q] = __ldcg(j.hist + (int64_t)d * j.n_tiles + t);
+                    }
+                }
+                uint32_t mine = 0;
+#pragma unroll
+                for (int q = 0; q < RS_BUCKETS / RS_THREADS; ++q) mine += tot[q];
+                uint32_t ex = block_exclusive_scan(mine, scratch, nullptr);
+#pragma unroll
+                for (int q = 0; q < RS_BUCKETS / RS_THREADS; ++q) {
+                    base[threadIdx.x * (RS_BUCKETS / RS_THREADS) + q] = ex + before[q];
+                    ex += tot[q];
+                }
             }
-            for (int w2 = 0; w2 < RS_THREADS / 32; ++w2) wcnt[w2][threadIdx.x] = 0;
+            for (int d = threadIdx.x; d < RS_BUCKETS; d += RS_THREADS)
+#pragma unroll
+                for (int w2 = 0; w2 < RS_THREADS / 32; ++w2) wcnt[w2][d] = 0;
             __syncthreads();
             uint32_t key[RS_ITEMS], rank[RS_ITEMS];
             const int64_t seg0 = tile0 + (int64_t)warp * (32 * RS_ITEMS);
@@ -155,12 +196,12 @@ coop_sort_kernel(const SortBatch batch) {
                 __syncwarp();
             }
             __syncthreads();
-            {
+            for (int d = threadIdx.x; d < RS_BUCKETS; d += RS_THREADS) {
                 uint32_t run = 0;
 #pragma unroll
                 for (int w2 = 0; w2 < RS_THREADS / 32; ++w2) {
-                    const uint32_t c = wcnt[w2][threadIdx.x];
-                    wcnt[w2][threadIdx.x] = run;
+                    const uint32_t c = wcnt[w2][d];
+                    wcnt[w2][d] = run;
                     run += c;
                 }
             }
@@ -178,10 +219,12 @@ coop_sort_kernel(const SortBatch batch) {
             }
             __syncthreads();
         }
-        if (pass + 1 < batch.passes) {
-            target += gridDim.x;
-            if (!grid_barrier(batch.barrier_ctr, target, batch.err)) return;
-        }
+        if (pass + 1 < batch.passes && !(ok = sync_all())) break;
+    }
+    if (solo && threadIdx.x == 0) {
+        // the host has already booked this launch's arrivals: deliver them
+        __threadfence();
+        atomicAdd(batch.barrier_ctr, (unsigned long long)gridDim.x * (unsigned long long)batch.n_barriers);
     }
 }
 
@@ -204,7 +247,7 @@ int sort_jobs(SortBatch& batch, GridBarrierState* gbs, cudaStream_t st, Profiler
     *err_out = cudaSuccess;
     int passes = 1, total_tiles = 0;
     for (int j = 0; j < batch.n_jobs; ++j) {
-        const int p = (batch.job[j].bits + 7) / 8;
+        const int p = (batch.job[j].bits + RS_RADIX_BITS - 1) / RS_RADIX_BITS;
         if (p > passes) passes = p;
     }
     for (int j = 0; j < batch.n_jobs; ++j) {
@@ -216,10 +259,11 @@ int sort_jobs(SortBatch& batch, GridBarrierState* gbs, cudaStream_t st, Profiler
     batch.passes = passes;
     int grid = total_tiles < coop_grid_limit() ? total_tiles : coop_grid_limit();
     if (grid < 1) grid = 1;
+    batch.n_barriers = 3 * passes - 1;
     batch.barrier_ctr = gbs->device_counter;
     batch.barrier_base = gbs->host_base;
-    gbs->host_base += (unsigned long long)grid * (unsigned long long)(3 * passes - 1);
-    KernelScope k(prof, "coop_sort", st);
+    gbs->host_base += (unsigned long long)grid * (unsigned long long)batch.n_barriers;
+    KernelScope k(prof, batch.name ? batch.name : "coop_sort", st);
     void* args[] = {&batch};
     *err_out = cudaLaunchCooperativeKernel((const void*)coop_sort_kernel, dim3(grid), dim3(RS_THREADS), args, 0, st);
     return passes & 1;

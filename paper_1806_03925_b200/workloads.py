@@ -90,6 +90,13 @@ PRESETS: Dict[str, GearPreset] = {
         hidden=(512, 256), M=32, expire=100,
         zipf_user=1.05, zipf_url=1.05, zipf_img=1.05, img_dist="poisson", img_lo=1, img_hi=16,
         img_lambda=4.0),
+    # the large-table shapes on tables of a few GB: the case profiler captures run on
+    "large_2m": GearPreset(
+        name="large_2m", batch=65536, steps=30, user_vocab=4_000_000, url_vocab=2_000_000,
+        img_vocab=2_000_000, emb_dim=64, dfv_dim=256, dfv_dtype=BF16, head_dtype=BF16,
+        hidden=(512, 256), M=32, expire=100,
+        zipf_user=1.05, zipf_url=1.05, zipf_img=1.05, img_dist="poisson", img_lo=1, img_hi=16,
+        img_lambda=4.0),
     "skew": GearPreset(
         name="skew", batch=32768, steps=30, user_vocab=1_000_000, url_vocab=1_000_000,
         img_vocab=4_000_000, emb_dim=32, dfv_dim=128, dfv_dtype=F32, head_dtype=F32,
