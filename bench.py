@@ -58,6 +58,7 @@ class ClockSampler:
 
     def __init__(self, gpu_index: int):
         self.gpu, self.proc, self.lines = gpu_index, None, []
+        self.t_open = self.t_close = None
 
     def start(self):
         try:
@@ -71,7 +72,15 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
+
+    def open_window(self):
+        """Samples count from here (the start of the first timed region) ..."""
+        self.t_open = time.monotonic()
+
+    def close_window(self):
+        """... to here (the end of the last one)."""
+        self.t_close = time.monotonic()
 
     def stop(self):
         if self.proc is None:
@@ -83,7 +92,10 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.lines:
+        t0 = self.t_open if self.t_open is not None else 0.0
+        t1 = self.t_close if self.t_close is not None else float("inf")
+        inside = [ln for (t, ln) in self.lines if t0 <= t <= t1 + 0.05]
+        for line in inside:
             f = [x.strip() for x in line.split(",")]
             if len(f) < 8:
                 continue
@@ -251,6 +263,8 @@ def run_ours(args):
     gb.load()
     p = preset_for(args.workload)
     K, W = args.steps, args.warmup
+    sampler = ClockSampler(local)          # started early: nvidia-smi needs a moment before its first line
+    sampler.start()
     seed = rank                                   # every replica draws its own tables and batches
     src = BatchSource(p, seed)
     host_batches = [src.batch(s) for s in range(N_BATCHES)]
@@ -293,10 +307,9 @@ def run_ours(args):
             ms = float(t.item())
         return ms
 
-    # ---- device-resident throughput (clocks are sampled from here to the end of the end-to-end pass:
+    # ---- device-resident throughput (clock samples count from here to the end of the end-to-end pass:
     #      every region in between runs the same step under load)
-    sampler = ClockSampler(local)
-    sampler.start()
+    sampler.open_window()
     for s in range(W):
         one_step(dev_batches[s % N_BATCHES])
     launches0 = gb.gear_launch_count(sess.ctx)
@@ -328,20 +341,22 @@ def run_ours(args):
     for s in range(min(W, 3)):
         e2e_step(s)
     ms_e2e = timed(e2e_step, K)
+    sampler.close_window()
     clocks = sampler.stop()
     d2h_bytes = 4 + 16
 
     # ---- per-kernel timing pass (profiling on; not part of the throughput numbers)
     ready_counts = []
+    KP = min(K, 50)
     gb.gear_profile_enable(sess.ctx, True)
-    for s in range(K):
+    for s in range(KP):
         one_step(dev_batches[s % N_BATCHES])
         ready_counts.append(int(sess.d_counts[0].item()))
     prof = gb.gear_profile_read(sess.ctx, 64)
     gb.gear_profile_enable(sess.ctx, False)
     stats["n_ready"] = float(np.mean(ready_counts)) if ready_counts else 0.0
     total_ms = sum(v[0] for v in prof.values()) or 1.0
-    kernels = sorted(({"name": k, "launches_per_step": v[1] / K, "ms_per_step": v[0] / K, "share": v[0] / total_ms,
+    kernels = sorted(({"name": k, "launches_per_step": v[1] / KP, "ms_per_step": v[0] / KP, "share": v[0] / total_ms,
                        "ms_per_launch": v[0] / v[1]} for k, v in prof.items()), key=lambda d: -d["ms_per_step"])
     peaks = measured_peaks()
     top = kernels[0]
@@ -375,7 +390,8 @@ def run_ours(args):
             "device_status": status}
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            sample = {"large": 4096, "medium": 4096, "tiny": 256}.get(args.workload, 1024)
+            # sized for roughly 10-30 s of single-thread CPU time
+            sample = {"large": 32768, "large_2m": 32768, "medium": 4096, "tiny": 256}.get(args.workload, 8192)
             line["cpu_baseline"] = cpu_baseline(p, BatchSource(p, 0), sample)
         else:
             line["cpu_baseline"] = None
@@ -388,12 +404,18 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=["large", "large_2m", "medium", "tiny", "skew"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    # defaults: a few hundred milliseconds of device time per timed region for the CUDA path (so that the
+    # clock sampler sees it), a couple of minutes of host time for the CPU oracle
+    if args.steps is None:
+        args.steps = 400 if args.impl == "ours" else 20
+    if args.warmup is None:
+        args.warmup = 20 if args.impl == "ours" else 2
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
