@@ -239,7 +239,7 @@ int gear_fill_uniform(void* dst, int32_t dtype, int64_t n_rows, int32_t dim, uin
  *     nothing is listed or restamped, the required count is reported and, with h_n, GEAR_ERR_CAPACITY returned.
  *   - img_vocab may be at most GEAR_STATIC_EXPIRY_MAX_VOCAB; larger tables are refused with
  *     GEAR_ERR_CAPACITY before anything is enqueued.
- *   - Cost: every GPU on which the library is loaded holds GEAR_STATIC_EXPIRY_SCRATCH_BYTES (about 2.1 MB)
+ *   - Cost: every GPU on which the library is loaded holds GEAR_STATIC_EXPIRY_SCRATCH_BYTES (about 2.2 MB)
  *     of device memory for this array until the process exits, whether or not the call is ever made.
  *   - The first call on a device looks up the array's device address (once per device, with that device
  *     current); make that first call before starting any stream capture.
@@ -250,7 +250,7 @@ int gear_fill_uniform(void* dst, int32_t dtype, int64_t n_rows, int32_t dim, uin
  * dfv_ts and ids are device pointers; dfv_ts is written only when restamp != 0.
  */
 #define GEAR_STATIC_EXPIRY_MAX_VOCAB 16777216
-#define GEAR_STATIC_EXPIRY_SCRATCH_BYTES (256 + GEAR_STATIC_EXPIRY_MAX_VOCAB / 8 + 16640)
+#define GEAR_STATIC_EXPIRY_SCRATCH_BYTES (256 + GEAR_STATIC_EXPIRY_MAX_VOCAB / 8 + 65792)
 int gear_collect_expired_static(int64_t* dfv_ts, int64_t img_vocab, int64_t expire, int64_t now, int restamp,
                                 int32_t* ids, int64_t cap, int64_t* d_n, int64_t* h_n, void* stream);
 
@@ -259,7 +259,9 @@ int gear_collect_expired_static(int64_t* dfv_ts, int64_t img_vocab, int64_t expi
  * ctx is bracketed by a pair of CUDA events on the caller's stream.  gear_profile_read synchronises,
  * sums the elapsed time and the launch count per kernel name since the last read or enable, writes up to
  * cap entries (names: cap rows of 64 chars, NUL-terminated; total_ms, launches: cap entries) and clears
- * the records.  Event records cost a few microseconds each: do not time throughput with profiling on.
+ * the records.  Event records cost a few microseconds each, and while profiling is on the library keeps all
+ * its work on the caller's stream (no side stream), so that every kernel is timed alone: do not time
+ * throughput with profiling on.
  * gear_launch_count returns the number of kernels this ctx has launched since it was created.
  */
 int gear_profile_enable(gear_ctx* ctx, int on);

@@ -86,7 +86,7 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
     p->q_id = take((size_t)p->ready_cap * 4);
     p->q_avg = take((size_t)p->ready_cap * c.dfv_dim * 4);
     p->exp_bits = take((size_t)ceil_div(c.img_vocab, 32) * 4);
-    p->exp_cnt = take((size_t)(ceil_div(c.img_vocab, EXP_TILE) + 1) * sizeof(uint2));
+    p->exp_cnt = take((size_t)(ceil_div(c.img_vocab, EXP_MARK_TILE) + 1) * sizeof(uint2));
     p->total = off;
     return GEAR_OK;
 }
@@ -216,6 +216,7 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     // scatter below, the image order is kept for gear_accumulate_dfv_grad (img_id == NULL).
     c.img_sorted = false;
     int sorted_buf = 0;
+    bool joined_needed = false;
     if (b.B > 0) {
         SortBatch batch = c.sort_batch();
         batch.job[0] = c.sort_job(gear_ctx_impl::SORT_USER);
@@ -232,22 +233,30 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
             batch.n_jobs = 3;
         }
         // The sort depends only on the ID arrays, so it runs on the ctx's side stream beside the gather and
-        // the head (fork here, join before the first consumer of a sorted order).
-        cudaError_t se = cudaEventRecord(c.ev_fork, st);
-        if (se == cudaSuccess) se = cudaStreamWaitEvent(c.side_stream, c.ev_fork, 0);
-        if (se != cudaSuccess) return cuda_fail(se, "fork");
+        // the head (fork here, join before the first consumer of a sorted order).  With per-kernel timing on,
+        // everything stays on the caller's stream so that each kernel is timed alone.
+        const bool forked = !c.prof.on;
+        cudaError_t se = cudaSuccess;
+        if (forked) {
+            se = cudaEventRecord(c.ev_fork, st);
+            if (se == cudaSuccess) se = cudaStreamWaitEvent(c.side_stream, c.ev_fork, 0);
+            if (se != cudaSuccess) return cuda_fail(se, "fork");
+        }
         batch.name = "sort_ids";
-        sorted_buf = sort_jobs(batch, &c.gbs, c.side_stream, &c.prof, &se);
+        sorted_buf = sort_jobs(batch, &c.gbs, forked ? c.side_stream : st, &c.prof, &se);
         if (se != cudaSuccess) return cuda_fail(se, "id sort");
-        se = cudaEventRecord(c.ev_join, c.side_stream);
-        if (se != cudaSuccess) return cuda_fail(se, "join");
+        if (forked) {
+            se = cudaEventRecord(c.ev_join, c.side_stream);
+            if (se != cudaSuccess) return cuda_fail(se, "join");
+        }
+        joined_needed = forked;
         if (b.nnz > 0) { c.img_sorted = true; c.img_sorted_n = b.nnz; c.img_sorted_buf = sorted_buf; }
     }
     cudaError_t e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
     if (e != cudaSuccess) return cuda_fail(e, "gather");
     e = launch_head_simt(c, b, o, st);
     if (e != cudaSuccess) return cuda_fail(e, "head");
-    if (b.B > 0) {
+    if (joined_needed) {
         e = cudaStreamWaitEvent(st, c.ev_join, 0);
         if (e != cudaSuccess) return cuda_fail(e, "join");
     }

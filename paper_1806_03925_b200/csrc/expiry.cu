@@ -4,34 +4,39 @@
 // Three launches, none waits on another block:
 //   mark   streams the int64 timestamp table once (the only HBM-sized traffic: 8 bytes per image),
 //          evaluates now - ts >= expire, packs the predicate 32 entries to a word with a warp ballot and
-//          counts per tile;
-//   scan   one block scans the tile counts and checks the caller's capacity;
-//   write  re-reads only the bitmap (1 bit per image), ranks the set bits with popc + block scan
-//          and writes the ascending ID list; listed entries are restamped on request.
+//          counts per 2048-entry tile;
+//   scan   one block scans the tile counts;
+//   write  checks the caller's capacity, re-reads only the bitmap (1 bit per image), ranks the set bits
+//          with popc + block scan and writes the ascending ID list; listed entries are restamped on request.
 #include "common.cuh"
 #include "internal.h"
 
 namespace gear {
 
 constexpr int EXP_THREADS = 256;
+constexpr int EXP_MARK_ITEMS = EXP_MARK_TILE / EXP_THREADS;
 static_assert(EXP_TILE == EXP_THREADS * 32, "one bitmap word per thread in the write pass");
+static_assert(EXP_MARK_TILE % (EXP_THREADS * 1) == 0 && EXP_TILE % EXP_MARK_TILE == 0, "mark tiles nest in write tiles");
 
+// One block per EXP_MARK_TILE timestamps.  All of a thread's loads are issued before the first ballot, so a
+// block keeps its whole 16 KB tile in flight; the small tiles leave the balancing to the block scheduler.
 __global__ void __launch_bounds__(EXP_THREADS)
 expiry_mark_kernel(const int64_t* __restrict__ ts, int64_t vocab, int64_t now, int64_t expire,
                    uint32_t* __restrict__ bits, uint2* __restrict__ tile_cnt) {
-    __shared__ uint32_t scratch[33];
-    const int64_t tile0 = (int64_t)blockIdx.x * EXP_TILE;
+    __shared__ uint32_t warp_cnt[EXP_THREADS / 32];
+    const int64_t tile0 = (int64_t)blockIdx.x * EXP_MARK_TILE;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
-    uint32_t count = 0;
-#pragma unroll 8
-    for (int it = 0; it < EXP_TILE / EXP_THREADS; ++it) {
+    int64_t t[EXP_MARK_ITEMS];
+#pragma unroll
+    for (int it = 0; it < EXP_MARK_ITEMS; ++it) {
         const int64_t i = tile0 + (int64_t)it * EXP_THREADS + threadIdx.x;
-        bool expired = false;
-        if (i < vocab) {
-            int64_t t;
-            asm volatile("ld.global.nc.L1::no_allocate.s64 %0, [%1];" : "=l"(t) : "l"(ts + i));
-            expired = now - t >= expire;
-        }
+        t[it] = i < vocab ? __ldcs(reinterpret_cast<const long long*>(ts) + i) : 0;
+    }
+    uint32_t count = 0;
+#pragma unroll
+    for (int it = 0; it < EXP_MARK_ITEMS; ++it) {
+        const int64_t i = tile0 + (int64_t)it * EXP_THREADS + threadIdx.x;
+        const bool expired = i < vocab && now - t[it] >= expire;
         const uint32_t word = __ballot_sync(0xffffffffu, expired);
         if (lane == 0) {
             const int64_t w = (tile0 + (int64_t)it * EXP_THREADS) / 32 + warp;
@@ -39,29 +44,34 @@ expiry_mark_kernel(const int64_t* __restrict__ ts, int64_t vocab, int64_t now, i
             count += __popc(word);
         }
     }
-    uint32_t total;
-    block_exclusive_scan(count, scratch, &total);
-    if (threadIdx.x == 0) tile_cnt[blockIdx.x] = make_uint2(total, 0u);
+    if (lane == 0) warp_cnt[warp] = count;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t total = 0;
+#pragma unroll
+        for (int w = 0; w < EXP_THREADS / 32; ++w) total += warp_cnt[w];
+        tile_cnt[blockIdx.x] = make_uint2(total, 0u);
+    }
 }
 
-__global__ void expiry_check_kernel(const uint2* __restrict__ tile_cnt, int64_t n_tiles, int64_t cap,
-                                    int64_t* __restrict__ d_n, DevState* __restrict__ state) {
-    const int64_t total = tile_cnt[n_tiles].x;
-    if (d_n) *d_n = total;
-    if (total > cap) { atomicOr(&state->status, GEAR_DEV_OUT_CAPACITY); state->exp_total = -1; }
-    else state->exp_total = total;
-}
-
+// One block per EXP_TILE entries: re-reads the bitmap only.  Every block compares the total with the
+// caller's capacity itself; block 0 reports the count and raises the status bit.
 __global__ void __launch_bounds__(EXP_THREADS)
 expiry_write_kernel(const uint32_t* __restrict__ bits, int64_t vocab, const uint2* __restrict__ tile_cnt,
-                    const DevState* __restrict__ state, int64_t now, int restamp, int64_t* __restrict__ ts,
-                    int32_t* __restrict__ ids) {
+                    int64_t n_mark_tiles, int64_t cap, int64_t* __restrict__ d_n, DevState* __restrict__ state,
+                    int64_t now, int restamp, int64_t* __restrict__ ts, int32_t* __restrict__ ids) {
     __shared__ uint32_t scratch[33];
-    if (state->exp_total < 0) return;                       // capacity too small: nothing listed, nothing restamped
+    const int64_t total = tile_cnt[n_mark_tiles].x;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (d_n) *d_n = total;
+        state->exp_total = total > cap ? -1 : total;
+        if (total > cap) atomicOr(&state->status, GEAR_DEV_OUT_CAPACITY);
+    }
+    if (total > cap) return;                                // capacity too small: nothing listed, nothing restamped
     const int64_t w = (int64_t)blockIdx.x * EXP_THREADS + threadIdx.x;
     uint32_t word = (w * 32 < vocab) ? bits[w] : 0u;
     const uint32_t ex = block_exclusive_scan(__popc(word), scratch, nullptr);
-    int64_t out = (int64_t)tile_cnt[blockIdx.x].x + ex;
+    int64_t out = (int64_t)tile_cnt[(int64_t)blockIdx.x * (EXP_TILE / EXP_MARK_TILE)].x + ex;
     while (word) {
         const int bit = __ffs(word) - 1;
         word &= word - 1;
@@ -71,21 +81,24 @@ expiry_write_kernel(const uint32_t* __restrict__ bits, int64_t vocab, const uint
     }
 }
 
+// The three launches of one scan over scratch (bits, tile_cnt, state).  prof may be null.
+static cudaError_t enqueue_expiry_scan(int64_t* ts, int64_t vocab, int64_t expire, int64_t now, int restamp,
+                                       int32_t* ids, int64_t cap, int64_t* d_n, uint32_t* bits, uint2* tile_cnt,
+                                       DevState* state, Profiler* prof, cudaStream_t st) {
+    const int64_t n_mark = ceil_div(vocab, EXP_MARK_TILE), n_write = ceil_div(vocab, EXP_TILE);
+    { KernelScope k(prof, "expiry_mark", st);
+    expiry_mark_kernel<<<(unsigned)n_mark, EXP_THREADS, 0, st>>>(ts, vocab, now, expire, bits, tile_cnt); }
+    scan_pairs(tile_cnt, n_mark, tile_cnt + n_mark, st, prof);
+    { KernelScope k(prof, "expiry_write", st);
+    expiry_write_kernel<<<(unsigned)n_write, EXP_THREADS, 0, st>>>(bits, vocab, tile_cnt, n_mark, cap, d_n, state, now,
+                                                                  restamp, ts, ids); }
+    return cudaGetLastError();
+}
+
 cudaError_t launch_collect_expired(const gear_ctx_impl& c, int64_t now, int restamp, int32_t* ids, int64_t cap,
                                    int64_t* d_n, cudaStream_t st) {
-    const int64_t vocab = c.cfg.img_vocab;
-    const int64_t n_tiles = ceil_div(vocab, EXP_TILE);
-    uint32_t* bits = c.at<uint32_t>(c.ws.exp_bits);
-    uint2* tile_cnt = c.at<uint2>(c.ws.exp_cnt);
-    { KernelScope k(&c.prof, "expiry_mark", st);
-    expiry_mark_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(c.buf.dfv_ts, vocab, now, c.cfg.expire, bits, tile_cnt); }
-    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, &c.prof);
-    { KernelScope k(&c.prof, "expiry_check", st);
-    expiry_check_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, cap, d_n, c.state()); }
-    { KernelScope k(&c.prof, "expiry_write", st);
-    expiry_write_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(bits, vocab, tile_cnt, c.state(), now, restamp,
-                                                                  c.buf.dfv_ts, ids); }
-    return cudaGetLastError();
+    return enqueue_expiry_scan(c.buf.dfv_ts, c.cfg.img_vocab, c.cfg.expire, now, restamp, ids, cap, d_n,
+                               c.at<uint32_t>(c.ws.exp_bits), c.at<uint2>(c.ws.exp_cnt), c.state(), &c.prof, st);
 }
 
 }  // namespace gear
@@ -108,7 +121,7 @@ namespace gear {
 constexpr int64_t STATIC_MAX_VOCAB = GEAR_STATIC_EXPIRY_MAX_VOCAB;
 constexpr size_t STATIC_STATE_BYTES = 256;
 constexpr size_t STATIC_BITS_BYTES = (size_t)(STATIC_MAX_VOCAB / 32) * 4;
-constexpr size_t STATIC_CNT_BYTES = ((size_t)(STATIC_MAX_VOCAB / EXP_TILE) + 1) * sizeof(uint2);
+constexpr size_t STATIC_CNT_BYTES = ((size_t)(STATIC_MAX_VOCAB / EXP_MARK_TILE) + 1) * sizeof(uint2);
 constexpr size_t STATIC_SCRATCH_BYTES = STATIC_STATE_BYTES + STATIC_BITS_BYTES + ((STATIC_CNT_BYTES + 255) / 256) * 256;
 static_assert(sizeof(DevState) <= STATIC_STATE_BYTES, "state block");
 static_assert(STATIC_SCRATCH_BYTES == GEAR_STATIC_EXPIRY_SCRATCH_BYTES, "the header states the size of the array");
@@ -150,17 +163,14 @@ extern "C" int gear_collect_expired_static(int64_t* dfv_ts, int64_t img_vocab, i
     DevState* state = reinterpret_cast<DevState*>(base);
     uint32_t* bits = reinterpret_cast<uint32_t*>(base + STATIC_STATE_BYTES);
     uint2* tile_cnt = reinterpret_cast<uint2*>(base + STATIC_STATE_BYTES + STATIC_BITS_BYTES);
-    const int64_t n_tiles = ceil_div(img_vocab, EXP_TILE);
 
     // the array keeps what the previous call left: the state block has to start from zero, the bitmap words
     // and tile counts of this table size are all rewritten by the mark pass
     if (cudaMemsetAsync(state, 0, STATIC_STATE_BYTES, st) != cudaSuccess) return GEAR_ERR_CUDA;
-    expiry_mark_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(dfv_ts, img_vocab, now, expire, bits, tile_cnt);
-    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, nullptr);
     int64_t* d_cnt = d_n ? d_n : &state->pad[1];
-    expiry_check_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, cap, d_cnt, state);
-    expiry_write_kernel<<<(unsigned)n_tiles, EXP_THREADS, 0, st>>>(bits, img_vocab, tile_cnt, state, now, restamp, dfv_ts, ids);
-    if (cudaGetLastError() != cudaSuccess) return GEAR_ERR_CUDA;
+    if (enqueue_expiry_scan(dfv_ts, img_vocab, expire, now, restamp, ids, cap, d_cnt, bits, tile_cnt, state, nullptr, st) !=
+        cudaSuccess)
+        return GEAR_ERR_CUDA;
     if (h_n) {
         if (cudaMemcpyAsync(h_n, d_cnt, sizeof(int64_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
             cudaStreamSynchronize(st) != cudaSuccess)

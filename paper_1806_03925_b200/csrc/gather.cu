@@ -1,31 +1,38 @@
 // Events 1-3 of the step: build the head input X[b] = [user row | url row | mean of the view's DFVs].
 //
-// One warp per page view.  Every lane owns 16-byte chunks of the rows (128-bit loads, a full row is read
-// by consecutive lanes), so each table row is fetched with fully used 32-byte sectors.  The pooled sum is
-// fp32, taken in slot order, divided once by n_b.  HBM bound: the kernel moves
-// B*(2E*4) + nnz*D*sizeof(dfv) bytes of table rows and writes B*Din*sizeof(x).
+// One warp per page view at a time.  Every lane owns 16-byte chunks of a row (128-bit loads; consecutive lanes read
+// a row end to end, so each fetch uses full 32-byte sectors).  The loads of up to eight DFV rows of the
+// view, and of its two embedding rows, are issued back to back before the first one is used; the code for
+// each row count is straight-line (one dispatch per view on the number of rows), which keeps the
+// instruction count per byte low enough for the memory system to be the limit.  The pooled sum is fp32,
+// taken in slot order, divided once by n_b.  HBM bound: the kernel moves B*(2E*4) + nnz*D*sizeof(dfv)
+// bytes of table rows and writes B*Din*sizeof(x).
+#include <algorithm>
+#include <cfloat>
+
 #include "common.cuh"
 #include "internal.h"
 
 namespace gear {
 
-template <typename T> struct Chunk;                         // 16 bytes of a table row as floats
+constexpr int GP_WARPS = 8;      // warps (views) per block
+
+template <typename T> struct Chunk;                         // 16 bytes of a table row
 template <> struct Chunk<float> {
     static constexpr int PER = 4;
-    __device__ static void load(const float* row, int ch, float* v) {
-        float4 t = ld_f4(row + ch * 4);
-        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    __device__ static __forceinline__ void add(float* acc, const uint4& t) {
+        acc[0] += __uint_as_float(t.x); acc[1] += __uint_as_float(t.y);
+        acc[2] += __uint_as_float(t.z); acc[3] += __uint_as_float(t.w);
     }
 };
 template <> struct Chunk<__nv_bfloat16> {
     static constexpr int PER = 8;
-    __device__ static void load(const __nv_bfloat16* row, int ch, float* v) {
-        uint4 t = *reinterpret_cast<const uint4*>(row + ch * 8);
+    __device__ static __forceinline__ void add(float* acc, const uint4& t) {
         const uint32_t w[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            v[2 * k] = __uint_as_float(w[k] << 16);
-            v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+            acc[2 * k] += __uint_as_float(w[k] << 16);
+            acc[2 * k + 1] += __uint_as_float(w[k] & 0xffff0000u);
         }
     }
 };
@@ -45,6 +52,14 @@ template <int N> __device__ __forceinline__ void store_x(__nv_bfloat16* dst, con
     else *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
 }
 
+// x / n for a small positive integer n held as nf, with rinv = 1 / nf: the product x * rinv corrected by one
+// exact residual step, which yields the correctly rounded quotient (infinities and NaNs pass through).
+__device__ __forceinline__ float div_by_count(float x, float nf, float rinv) {
+    const float q = x * rinv;
+    const float q2 = fmaf(fmaf(-q, nf, x), rinv, q);
+    return fabsf(q) <= FLT_MAX ? q2 : q;
+}
+
 struct GatherArgs {
     const float* user_emb; const float* url_emb; const void* dfv;
     int64_t user_vocab, url_vocab, img_vocab;
@@ -56,90 +71,161 @@ struct GatherArgs {
     DevState* state;
 };
 
-// NQ = 16-byte chunks of a DFV row per lane
+// Adds rows j .. j + K - 1 of the view to acc, in order; their IDs sit in lanes (j + t) % 32 of my_id
+// (-1: the row counts as zeros).  All K loads are issued before the first addition.
+template <typename TD, int NQ, int K>
+__device__ __forceinline__ void add_rows(float (&acc)[NQ][Chunk<TD>::PER], const TD* __restrict__ dfv, int D,
+                                         int n_chunks, int my_id, int j, int lane) {
+    uint4 v[K][NQ];
+#pragma unroll
+    for (int t = 0; t < K; ++t) {
+        const int id = __shfl_sync(0xffffffffu, my_id, (j + t) & 31);
+        const uint4* __restrict__ row = reinterpret_cast<const uint4*>(dfv + (int64_t)(id < 0 ? 0 : id) * D);
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const int ch = lane + 32 * q;
+            v[t][q] = (id >= 0 && ch < n_chunks) ? __ldg(row + ch) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < K; ++t)
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) Chunk<TD>::add(acc[q], v[t][q]);
+}
+
+struct ViewRec { int uid, hid, s, n; };
+
+// The record of view b as every lane of the warp reads it (same words: one transaction each).
+// Out-of-range views read as empty.
+__device__ __forceinline__ ViewRec load_view(const GatherArgs& a, int b) {
+    ViewRec r{-1, -1, 0, 0};
+    if (b < a.B) {
+        r.uid = __ldg(a.user_id + b); r.hid = __ldg(a.url_id + b);
+        r.s = __ldg(a.img_off + b);
+        r.n = __ldg(a.img_off + b + 1) - r.s;                 // validated when the view is processed
+    }
+    return r;
+}
+
+// NQ = 16-byte chunks of a DFV row per lane.  A warp walks views b, b + W, b + 2W, ... (W = warps of the grid)
+// and keeps two stages of look-ahead in registers: the record of the view after next and the image IDs of
+// the next view are requested before the current view's rows are summed, so that per view only one memory
+// round trip (the rows themselves) is exposed.
 template <typename TD, typename TX, int NQ>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(GP_WARPS * 32, NQ <= 2 ? 3 : 2)
 gather_pool_kernel(const GatherArgs a) {
     constexpr int PER = Chunk<TD>::PER;
-    const unsigned lane = lane_id();
-    const int warps_per_block = blockDim.x >> 5;
+    constexpr int KMAX = NQ >= 8 ? 1 : 8 / NQ;               // rows in flight per warp
+    const int lane = (int)lane_id();
+    const int W = gridDim.x * GP_WARPS;
     const int Din = 2 * a.E + a.D;
     const int n_chunks = a.D / PER;
-    const TD* dfv = static_cast<const TD*>(a.dfv);
+    const int ce = a.E / 4;                                    // 16-byte chunks per embedding row
+    const TD* __restrict__ dfv = static_cast<const TD*>(a.dfv);
     int flags = 0;
 
-    for (int b = blockIdx.x * warps_per_block + (threadIdx.x >> 5); b < a.B; b += gridDim.x * warps_per_block) {
-        TX* x = static_cast<TX*>(a.X) + (int64_t)b * Din;
-        TX* xd = a.x_debug ? static_cast<TX*>(a.x_debug) + (int64_t)b * Din : nullptr;
+    auto load_ids = [&](const ViewRec& r, int j0) -> int {     // IDs j0 + lane of the view (unchecked), -1 past its end
+        const bool ok = r.s >= 0 && r.n >= 0 && (int64_t)r.s + r.n <= a.nnz;
+        return (ok && j0 + lane < r.n) ? __ldg(a.img_id + r.s + j0 + lane) : -1;
+    };
 
-        // user and URL-hash embedding rows: plain copies
-        const int u = a.user_id[b], h = a.url_id[b];
-        const bool u_ok = u >= 0 && u < a.user_vocab, h_ok = h >= 0 && h < a.url_vocab;
-        if (!u_ok || !h_ok) flags |= GEAR_DEV_BAD_ID;
-        for (int ch = lane; ch < a.E / 4; ch += 32) {
-            float v[4] = {0.f, 0.f, 0.f, 0.f}, w[4] = {0.f, 0.f, 0.f, 0.f};
-            if (u_ok) Chunk<float>::load(a.user_emb + (int64_t)u * a.E, ch, v);
-            if (h_ok) Chunk<float>::load(a.url_emb + (int64_t)h * a.E, ch, w);
-            store_x<4>(x + ch * 4, v);
-            store_x<4>(x + a.E + ch * 4, w);
-            if (xd) { store_x<4>(xd + ch * 4, v); store_x<4>(xd + a.E + ch * 4, w); }
+    int b = blockIdx.x * GP_WARPS + (int)(threadIdx.x >> 5);
+    ViewRec cur = load_view(a, b), nxt = load_view(a, b + W);
+    int ids_cur = load_ids(cur, 0);
+
+    for (; b < a.B; b += W) {
+        // ---- look-ahead: IDs of the next view, record of the one after it
+        const int ids_nxt = load_ids(nxt, 0);
+        const ViewRec nxt2 = load_view(a, b + 2 * W);
+
+        TX* __restrict__ x = static_cast<TX*>(a.X) + (int64_t)b * Din;
+        TX* __restrict__ xd = a.x_debug ? static_cast<TX*>(a.x_debug) + (int64_t)b * Din : nullptr;
+        int uid = cur.uid, hid = cur.hid, s = cur.s, n = cur.n;
+        if (uid < 0 || uid >= a.user_vocab) { uid = -1; flags |= GEAR_DEV_BAD_ID; }
+        if (hid < 0 || hid >= a.url_vocab) { hid = -1; flags |= GEAR_DEV_BAD_ID; }
+        if (s < 0 || n < 0 || (int64_t)s + n > a.nnz) { flags |= GEAR_DEV_BAD_CSR; s = 0; n = 0; }
+        int my_id = ids_cur;
+        if (lane < n) {
+            if (my_id < 0 || my_id >= a.img_vocab) { my_id = -1; flags |= GEAR_DEV_BAD_ID; }
+            if (a.row_view) a.row_view[s + lane] = b;
+        } else my_id = -1;
+
+        // ---- user and URL-hash rows: the first 2E columns of X are the two rows end to end.  The common case
+        //      (at most 32 chunks) is loaded here and stored after the DFV loads have been issued.
+        float4 emb = make_float4(0.f, 0.f, 0.f, 0.f);
+        {
+            const bool is_url = lane >= ce;
+            const int id = is_url ? hid : uid;
+            const float* __restrict__ table = is_url ? a.url_emb : a.user_emb;
+            if (lane < 2 * ce && id >= 0)
+                emb = __ldg(reinterpret_cast<const float4*>(table + (int64_t)id * a.E + (is_url ? lane - ce : lane) * 4));
         }
 
-        // DFV rows of the view, summed in slot order
-        int s = a.img_off[b], e = a.img_off[b + 1];
-        if (s < 0 || e < s || e > a.nnz) { flags |= GEAR_DEV_BAD_CSR; e = s = 0; }
-        const int n = e - s;
+        // ---- DFV rows, summed in slot order
         float acc[NQ][PER];
 #pragma unroll
         for (int q = 0; q < NQ; ++q)
 #pragma unroll
             for (int k = 0; k < PER; ++k) acc[q][k] = 0.f;
-
-        for (int j0 = 0; j0 < n; j0 += 32) {
-            const int m = min(32, n - j0);
-            int my_id = -1;
-            if ((int)lane < m) {
-                my_id = a.img_id[s + j0 + lane];
-                if (a.row_view) a.row_view[s + j0 + lane] = b;
-                if (my_id < 0 || my_id >= a.img_vocab) { flags |= GEAR_DEV_BAD_ID; my_id = -1; }
+        int j = 0;
+        auto next_ids = [&]() {                                    // IDs 32.. of a long view
+            if (j >= 32 && (j & 31) == 0) {
+                my_id = load_ids(cur, j);
+                if (j + lane < n) {
+                    if (my_id < 0 || my_id >= a.img_vocab) { my_id = -1; flags |= GEAR_DEV_BAD_ID; }
+                    if (a.row_view) a.row_view[s + j + lane] = b;
+                } else my_id = -1;
             }
-            for (int j = 0; j < m; j += 4) {
-                float v[4][NQ][PER];
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const int id = __shfl_sync(0xffffffffu, my_id, (j + t) & 31);
-                    const bool on = (j + t) < m && id >= 0;
-#pragma unroll
-                    for (int q = 0; q < NQ; ++q) {
-                        const int ch = lane + 32 * q;
-                        if (on && ch < n_chunks) Chunk<TD>::load(dfv + (int64_t)id * a.D, ch, v[t][q]);
-                        else {
-#pragma unroll
-                            for (int k = 0; k < PER; ++k) v[t][q][k] = 0.f;
-                        }
-                    }
-                }
-#pragma unroll
-                for (int t = 0; t < 4; ++t)
-#pragma unroll
-                    for (int q = 0; q < NQ; ++q)
-#pragma unroll
-                        for (int k = 0; k < PER; ++k) acc[q][k] += v[t][q][k];
+        };
+        while (n - j >= KMAX) {
+            next_ids();
+            add_rows<TD, NQ, KMAX>(acc, dfv, a.D, n_chunks, my_id, j, lane);
+            j += KMAX;
+        }
+        if (KMAX > 1 && j < n) {
+            next_ids();
+            switch (n - j) {                                       // 1 .. KMAX - 1 rows left: straight-line code for each count
+            case 1: add_rows<TD, NQ, 1>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 2: if constexpr (KMAX > 2) add_rows<TD, NQ, 2>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 3: if constexpr (KMAX > 3) add_rows<TD, NQ, 3>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 4: if constexpr (KMAX > 4) add_rows<TD, NQ, 4>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 5: if constexpr (KMAX > 5) add_rows<TD, NQ, 5>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 6: if constexpr (KMAX > 6) add_rows<TD, NQ, 6>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            default: if constexpr (KMAX > 7) add_rows<TD, NQ, 7>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
             }
         }
-        const float nf = (float)n;
+
+        // ---- write the row of X
+        if (lane < 2 * ce) {
+            const float f[4] = {emb.x, emb.y, emb.z, emb.w};
+            store_x<4>(x + lane * 4, f);
+            if (xd) store_x<4>(xd + lane * 4, f);
+        }
+        for (int c = 32 + lane; c < 2 * ce; c += 32) {             // embedding rows wider than 32 chunks in total
+            const bool is_url = c >= ce;
+            const int id = is_url ? hid : uid;
+            const float* __restrict__ table = is_url ? a.url_emb : a.user_emb;
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (id >= 0) t = __ldg(reinterpret_cast<const float4*>(table + (int64_t)id * a.E + (is_url ? c - ce : c) * 4));
+            const float f[4] = {t.x, t.y, t.z, t.w};
+            store_x<4>(x + c * 4, f);
+            if (xd) store_x<4>(xd + c * 4, f);
+        }
+        const float nf = (float)n, rinv = n > 0 ? 1.0f / nf : 0.f;
 #pragma unroll
         for (int q = 0; q < NQ; ++q) {
             const int ch = lane + 32 * q;
             if (ch < n_chunks) {
                 float o[PER];
 #pragma unroll
-                for (int k = 0; k < PER; ++k) o[k] = n > 0 ? acc[q][k] / nf : 0.f;
+                for (int k = 0; k < PER; ++k) o[k] = n > 0 ? div_by_count(acc[q][k], nf, rinv) : 0.f;
                 store_x<PER>(x + 2 * a.E + ch * PER, o);
                 if (xd) store_x<PER>(xd + 2 * a.E + ch * PER, o);
             }
         }
-        if (a.inv_n && lane == 0) a.inv_n[b] = n > 0 ? 1.0f / nf : 0.f;
+        if (a.inv_n && lane == 0) a.inv_n[b] = rinv;
+
+        cur = nxt; nxt = nxt2; ids_cur = ids_nxt;
     }
     if (flags) atomicOr(&a.state->status, flags);
 }
@@ -149,14 +235,14 @@ static cudaError_t dispatch_nq(const GatherArgs& a, cudaStream_t st, Profiler* p
     constexpr int PER = Chunk<TD>::PER;
     const int n_chunks = a.D / PER;
     const int nq = (n_chunks + 31) / 32;
-    const int warps = 8;
-    int grid = (int)ceil_div(a.B, warps);
-    if (grid < 1) grid = 1;
+    // every block stays resident: three (two for wide rows) per SM
+    const int64_t resident = (int64_t)sm_count() * (nq <= 2 ? 3 : 2);
+    const int grid = (int)std::min<int64_t>(ceil_div(a.B, GP_WARPS), resident);
     KernelScope ks(prof, "gather_pool", st);
-    if (nq <= 1) gather_pool_kernel<TD, TX, 1><<<grid, warps * 32, 0, st>>>(a);
-    else if (nq <= 2) gather_pool_kernel<TD, TX, 2><<<grid, warps * 32, 0, st>>>(a);
-    else if (nq <= 4) gather_pool_kernel<TD, TX, 4><<<grid, warps * 32, 0, st>>>(a);
-    else gather_pool_kernel<TD, TX, 8><<<grid, warps * 32, 0, st>>>(a);
+    if (nq <= 1) gather_pool_kernel<TD, TX, 1><<<grid, GP_WARPS * 32, 0, st>>>(a);
+    else if (nq <= 2) gather_pool_kernel<TD, TX, 2><<<grid, GP_WARPS * 32, 0, st>>>(a);
+    else if (nq <= 4) gather_pool_kernel<TD, TX, 4><<<grid, GP_WARPS * 32, 0, st>>>(a);
+    else gather_pool_kernel<TD, TX, 8><<<grid, GP_WARPS * 32, 0, st>>>(a);
     return cudaGetLastError();
 }
 

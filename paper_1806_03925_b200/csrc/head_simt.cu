@@ -356,7 +356,7 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
         const int K = p.fan[l], N = p.fan[l + 1];
         if constexpr (BF) {
             tce = tc_gemm_kmajor(&c.prof, "tc_gemm_fwd", B, N, K, H[l], K, c.at<__nv_bfloat16>(c.ws.wbt[l]), K, 0,
-                                 H[l + 1], N, p.b[l], nullptr, 0, tc_err, st);
+                                 H[l + 1], N, p.b[l], nullptr, 0, nullptr, tc_err, st);
             if (tce != cudaSuccess) return tce;
         } else
         launch_gemm<TX, TX, TX, TX, EPI_BIAS_RELU>(B, N, K, H[l], K, 1, static_cast<const TX*>(Wop[l]), N, 1,
@@ -386,7 +386,9 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
         } else
         launch_gemm<TX, TX, float, TX, EPI_ATOMIC>(K, N, B, H[l], 1, K, dA[l + 1], N, 1, p.gW[l], N, nullptr,
                                                    (const TX*)nullptr, 0, splits_for(K, N, B), st, &c.prof, "simt_gemm_dw");
-        if (l < L - 1) {     // the top layer's bias gradient came out of head_out_kernel
+        // bias gradient of a lower layer (the top layer's came out of head_out_kernel); the tensor-core path
+        // sums the columns of dA inside the epilogue of the product that makes dA
+        if (!BF && l < L - 1) {
             KernelScope ks(&c.prof, "colsum", st);
             const int blocks = B < CS_BLOCKS * 8 ? (int)ceil_div(B, 8) : CS_BLOCKS;
             colsum_kernel<TX><<<blocks, 256, 0, st>>>(B, N, dA[l + 1], p.gb[l]);
@@ -394,9 +396,9 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
         if constexpr (BF) {
             const __nv_bfloat16* wb = c.at<__nv_bfloat16>(c.ws.wb[l]);
             if (l > 0) tce = tc_gemm_kmajor(&c.prof, "tc_gemm_dh", B, K, N, dA[l + 1], N, wb, N, 1, dA[l], K, nullptr,
-                                            H[l], K, tc_err, st);
+                                            H[l], K, p.gb[l - 1], tc_err, st);
             else tce = tc_gemm_kmajor(&c.prof, "tc_gemm_dx", B, K, N, dA[l + 1], N, wb, N, 2, o.dX, K, nullptr, nullptr,
-                                      0, tc_err, st);
+                                      0, nullptr, tc_err, st);
             if (tce != cudaSuccess) return tce;
         } else if (l > 0) {
             launch_gemm<TX, TX, TX, TX, EPI_MASK>(B, K, N, dA[l + 1], N, 1, static_cast<const TX*>(Wop[l]), 1, N,

@@ -6,9 +6,13 @@
 //              shared-memory stages (128-byte swizzle), one mbarrier pair per stage;
 //   warp 1     MMA issuer: one elected lane issues tcgen05.mma (M 128, N BN, K 16) into one of two
 //              accumulator buffers in tensor memory and commits each stage back to the producer;
-//   warps 2-5  epilogue: tcgen05.ld the finished accumulator (32 lanes x 32 columns per instruction),
+//   warps 2-9  epilogue: tcgen05.ld the finished accumulator (32 lanes x 32 columns per instruction),
 //              apply bias+ReLU / ReLU mask / nothing, and store; meanwhile the MMA warp already fills
-//              the other accumulator buffer with the next tile.
+//              the other accumulator buffer with the next tile.  Two warps share each quarter of the
+//              tensor-memory lanes and split the tile's columns; the read of the next 32 columns and
+//              the loads of the bias / mask are in flight while the current 32 columns are processed.
+//              The ReLU-mask epilogue also sums its output columns (the bias gradient of the layer
+//              below): a shuffle transpose-reduction per 32 x 32 block, shared-memory partials per CTA.
 // Two operand layouts:
 //   K-major   C[M][N] = A[M][K] . W[N][K]^T     (activations x weights; K contiguous in both)
 //   MN-major  C[M][N] += A[K][M]^T . B[K][N]    (weight gradients: the reduction runs over the batch,
@@ -24,7 +28,9 @@ namespace gear {
 
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
-constexpr int TC_THREADS = 192;
+constexpr int TC_EPI_WARPS = 8;
+constexpr int TC_THREADS = 64 + 32 * TC_EPI_WARPS;
+constexpr int TC_MAX_N = 1024;            // widest output the column-sum partials cover
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
 enum { TC_EPI_BIAS_RELU = 0, TC_EPI_MASK = 1, TC_EPI_F32 = 2, TC_EPI_RED = 3 };
@@ -34,7 +40,8 @@ template <int BN> struct TcCfg {
     static constexpr int A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
     static constexpr int B_BYTES = BN * TC_BK * 2;               // 32 KB or 16 KB
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                                TC_MAX_N * 4 /*column sums*/;
     static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
     static_assert(SMEM > 116 * 1024, "one CTA per SM: two CTAs would both ask for tensor memory");
     static_assert(SMEM <= 227 * 1024, "shared memory budget");
@@ -46,6 +53,7 @@ struct TcArgs {
     void* out; int64_t ldo;
     const float* bias;
     const __nv_bfloat16* mask; int64_t ldm;
+    float* colsum;            // ReLU-mask epilogue: colsum[n] += sum over rows of the stored output (may be null)
     int32_t* err;             // device word that receives a non-zero code on a timeout
 };
 
@@ -107,7 +115,34 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Waits for the tensor-memory reads issued so far.  The registers are passed through so that no use of
+// them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
+
+__device__ __forceinline__ float4 ldg_f4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ uint4 ldg_u4(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+
+// v[i] of lane l is element (row l, column i) of a 32 x 32 block.  Returns, on lane l, the sum of column l.
+__device__ __forceinline__ float column_sums_32x32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        const bool upper = (lane & s) != 0;       // this lane keeps the upper half of the columns still held
+#pragma unroll
+        for (int i = 0; i < s; ++i) {
+            const float send = upper ? v[i] : v[i + s];
+            const float keep = upper ? v[i + s] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
+    }
+    return v[0];
+}
 
 // Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1).
 //   K-major operand : rows of 128 bytes, 8-row groups 1024 bytes apart (SBO); LBO unused.
@@ -145,6 +180,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t tmem_word = bars + 8u * (2 * STAGES + 4);
     volatile uint32_t* tmem_word_ptr =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_word - raw));
+    float* s_colsum = reinterpret_cast<float*>(smem_raw + (bars + 256u - raw));     // [TC_MAX_N] per-CTA column sums
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles * g.k_splits;
@@ -152,11 +188,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 128); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 32 * TC_EPI_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" :: "l"(&map_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" :: "l"(&map_b) : "memory");
     }
+    if (EPI == TC_EPI_MASK && g.colsum != nullptr)
+        for (int n = threadIdx.x; n < TC_MAX_N; n += TC_THREADS) s_colsum[n] = 0.f;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      :: "r"(tmem_word), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
@@ -238,8 +276,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     } else {
-        // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32 * (warp % 4) ..
+        // ---------------- epilogue: warp w reads tensor-memory lanes 32 * (w % 4) .. + 31 (its rows of the tile);
+        // warps 2..5 take the first half of the tile's columns, warps 6..9 the second half
         const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
+        constexpr int CHUNKS = BN / 64;                       // 32-column chunks per warp and tile
         uint32_t tile_it = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
@@ -248,64 +289,105 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (!(ok = mbar_wait(acc_full(a), (tile_it >> 1) & 1u, g.err, 4))) break;
             tc_fence_after();
             const int m = mt * TC_BM + quarter * 32 + lane;
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN);
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                tc_ld32(t_row + c0, r);
-                tc_wait_ld();
-                const int n0 = nt * BN + c0;
-                if (m < g.M && n0 < g.N) {
-                    const int nv = min(32, g.N - n0);                 // N is a multiple of 8
-                    if (EPI == TC_EPI_BIAS_RELU || EPI == TC_EPI_MASK) {
-                        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(g.out) + (int64_t)m * g.ldo + n0;
-                        for (int j = 0; j < nv; j += 8) {
-                            float v[8];
+            const bool row_ok = m < g.M;
+            const int col0 = nt * BN + half * (BN / 2);
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN + half * (BN / 2));
+            uint32_t r[2][32];
+            tc_ld32(t_row, r[0]);
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(r[j + q]);
-                            if (EPI == TC_EPI_BIAS_RELU) {
-                                const float4 b0 = ld_f4(g.bias + n0 + j), b1 = ld_f4(g.bias + n0 + j + 4);
-                                v[0] = fmaxf(v[0] + b0.x, 0.f); v[1] = fmaxf(v[1] + b0.y, 0.f);
-                                v[2] = fmaxf(v[2] + b0.z, 0.f); v[3] = fmaxf(v[3] + b0.w, 0.f);
-                                v[4] = fmaxf(v[4] + b1.x, 0.f); v[5] = fmaxf(v[5] + b1.y, 0.f);
-                                v[6] = fmaxf(v[6] + b1.z, 0.f); v[7] = fmaxf(v[7] + b1.w, 0.f);
-                            } else {
-                                const uint4 mk = *reinterpret_cast<const uint4*>(g.mask + (int64_t)m * g.ldm + n0 + j);
-                                const uint32_t w[4] = {mk.x, mk.y, mk.z, mk.w};
+            for (int c = 0; c < CHUNKS; ++c) {
+                const int n0 = col0 + c * 32;
+                const bool chunk_ok = n0 < g.N;               // warp-uniform; N is a multiple of 8
+                // what this chunk's epilogue reads from memory, requested while the tensor-memory read is in flight
+                float4 bias4[EPI == TC_EPI_BIAS_RELU ? 8 : 1];
+                uint4 mask4[EPI == TC_EPI_MASK ? 4 : 1];
+                if (EPI == TC_EPI_BIAS_RELU) {
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    // a post-ReLU activation is > 0 exactly when its bf16 pattern is non-zero and positive
-                                    const uint32_t lo = w[q] & 0xffffu, hi = w[q] >> 16;
-                                    if (!(lo != 0u && lo < 0x8000u)) v[2 * q] = 0.f;
-                                    if (!(hi != 0u && hi < 0x8000u)) v[2 * q + 1] = 0.f;
-                                }
-                            }
-                            uint32_t pk[4];
+                    for (int j = 0; j < 8; ++j)
+                        bias4[j] = (n0 + 4 * j < g.N) ? ldg_f4(g.bias + n0 + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                if (EPI == TC_EPI_MASK) {
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
-                                pk[q] = *reinterpret_cast<uint32_t*>(&h2);
-                            }
-                            *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    for (int j = 0; j < 4; ++j)
+                        mask4[j] = (row_ok && n0 + 8 * j < g.N) ? ldg_u4(g.mask + (int64_t)m * g.ldm + n0 + 8 * j)
+                                                                : make_uint4(0u, 0u, 0u, 0u);
+                }
+                tc_wait_ld(r[c & 1]);
+                if (c + 1 < CHUNKS) tc_ld32(t_row + (uint32_t)((c + 1) * 32), r[(c + 1) & 1]);
+                if (!chunk_ok) continue;
+                uint32_t (&acc)[32] = r[c & 1];
+                if (EPI == TC_EPI_BIAS_RELU || EPI == TC_EPI_MASK) {
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
+                    if (EPI == TC_EPI_BIAS_RELU) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            v[4 * j + 0] = fmaxf(v[4 * j + 0] + bias4[j].x, 0.f);
+                            v[4 * j + 1] = fmaxf(v[4 * j + 1] + bias4[j].y, 0.f);
+                            v[4 * j + 2] = fmaxf(v[4 * j + 2] + bias4[j].z, 0.f);
+                            v[4 * j + 3] = fmaxf(v[4 * j + 3] + bias4[j].w, 0.f);
                         }
                     } else {
-                        float* dst = static_cast<float*>(g.out) + (int64_t)m * g.ldo + n0;
-                        for (int j = 0; j < nv; j += 4) {
-                            const float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                                         __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-                            if (EPI == TC_EPI_RED) red_add_f4(dst + j, v);
-                            else st_f4(dst + j, v);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t w[4] = {mask4[j].x, mask4[j].y, mask4[j].z, mask4[j].w};
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                // a post-ReLU activation is > 0 exactly when its bf16 pattern is non-zero and positive
+                                const uint32_t lo = w[q] & 0xffffu, hi = w[q] >> 16;
+                                if (!(lo != 0u && lo < 0x8000u)) v[8 * j + 2 * q] = 0.f;
+                                if (!(hi != 0u && hi < 0x8000u)) v[8 * j + 2 * q + 1] = 0.f;
+                            }
                         }
+                    }
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) {
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+                        pk[q] = *reinterpret_cast<uint32_t*>(&h2);
+                    }
+                    if (row_ok) {
+                        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(g.out) + (int64_t)m * g.ldo + n0;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (n0 + 8 * j < g.N)
+                                *reinterpret_cast<uint4*>(dst + 8 * j) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                    }
+                    if (EPI == TC_EPI_MASK && g.colsum != nullptr) {
+                        // column sums of what was stored (the rounded values); rows past M and columns past N are zero
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) {
+                            v[2 * q] = row_ok ? __uint_as_float(pk[q] << 16) : 0.f;
+                            v[2 * q + 1] = row_ok ? __uint_as_float(pk[q] & 0xffff0000u) : 0.f;
+                        }
+                        const float cs = column_sums_32x32(v, lane);
+                        if (n0 + lane < g.N) atomicAdd(&s_colsum[n0 + lane], cs);
+                    }
+                } else if (row_ok) {
+                    float* dst = static_cast<float*>(g.out) + (int64_t)m * g.ldo + n0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (n0 + 4 * j >= g.N) continue;
+                        const float4 v4 = make_float4(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1]),
+                                                      __uint_as_float(acc[4 * j + 2]), __uint_as_float(acc[4 * j + 3]));
+                        if (EPI == TC_EPI_RED) red_add_f4(dst + 4 * j, v4);
+                        else st_f4(dst + 4 * j, v4);
                     }
                 }
             }
             tc_fence_before();
-            mbar_arrive(acc_empty(a));                   // 128 arrivals hand the buffer back to the MMA warp
+            mbar_arrive(acc_empty(a));                   // all epilogue threads arrive: the buffer returns to the MMA warp
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (EPI == TC_EPI_MASK && g.colsum != nullptr)
+        for (int n = threadIdx.x; n < g.N && n < TC_MAX_N; n += TC_THREADS) {
+            const float v = s_colsum[n];
+            if (v != 0.f) atomicAdd(g.colsum + n, v);
+        }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
@@ -346,17 +428,6 @@ static bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
-
 template <int BN, bool MN, int EPI>
 static cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& g, cudaStream_t st) {
     using Cfg = TcCfg<BN>;
@@ -380,7 +451,7 @@ static cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& m
 
 cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
                            const __nv_bfloat16* W, int64_t ldw, int epi, void* out, int64_t ldo, const float* bias,
-                           const __nv_bfloat16* mask, int64_t ldm, int32_t* err, cudaStream_t st) {
+                           const __nv_bfloat16* mask, int64_t ldm, float* colsum, int32_t* err, cudaStream_t st) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     const int bn = N > 128 ? 256 : 128;
     CUtensorMap ma, mb;
@@ -390,6 +461,8 @@ cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K
     g.m_tiles = (int)ceil_div(M, TC_BM); g.n_tiles = (int)ceil_div(N, bn); g.k_splits = 1;
     g.kb_per_split = (int)ceil_div(K, TC_BK);
     g.out = out; g.ldo = ldo; g.bias = bias; g.mask = mask; g.ldm = ldm; g.err = err;
+    g.colsum = (epi == TC_EPI_MASK && N <= TC_MAX_N) ? colsum : nullptr;
+    if (epi == TC_EPI_MASK && colsum != nullptr && g.colsum == nullptr) return cudaErrorInvalidValue;
     KernelScope ks(prof, name, st);
     switch (epi) {
     case TC_EPI_BIAS_RELU: return launch_bn<false, TC_EPI_BIAS_RELU>(bn, ma, mb, g, st);
@@ -414,7 +487,7 @@ cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int 
     if (splits < 1) splits = 1;
     g.kb_per_split = (int)ceil_div(total_kb, splits);
     g.k_splits = (int)ceil_div(total_kb, g.kb_per_split);
-    g.out = out; g.ldo = ldo; g.bias = nullptr; g.mask = nullptr; g.ldm = 0; g.err = err;
+    g.out = out; g.ldo = ldo; g.bias = nullptr; g.mask = nullptr; g.ldm = 0; g.colsum = nullptr; g.err = err;
     KernelScope ks(prof, name, st);
     return launch_bn<true, TC_EPI_RED>(bn, ma, mb, g, st);
 }

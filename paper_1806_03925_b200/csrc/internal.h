@@ -10,7 +10,8 @@
 
 namespace gear {
 
-constexpr int EXP_TILE = 8192;     // entries of the timestamp table per block of the expiry scan
+constexpr int EXP_TILE = 8192;     // entries of the timestamp table per block of the expiry scan's write pass
+constexpr int EXP_MARK_TILE = 2048; // ... and per block (and per count) of its mark pass
 constexpr int MAX_LAYERS = 2;
 constexpr int CS_BLOCKS = 296;      // blocks of the column-sum kernel (two per SM)
 
@@ -35,7 +36,7 @@ struct WsPlan {
     size_t q_id;                        // [ready_cap] int32
     size_t q_avg;                       // [ready_cap][dfv_dim] fp32
     size_t exp_bits;                    // [ceil(img_vocab / 32)] uint32 expired bitmap
-    size_t exp_cnt;                     // [expiry tiles + 1] uint2
+    size_t exp_cnt;                     // [expiry mark tiles + 1] uint2
     size_t total;
     int64_t ready_cap;
     int loss_blocks;
@@ -96,9 +97,10 @@ cudaError_t launch_gather(const gear_ctx_impl& c, const gear_batch& b, int32_t* 
 cudaError_t launch_head_simt(const gear_ctx_impl& c, const gear_batch& b, const gear_step_out& o, cudaStream_t st);
 
 // head_tc.cu: bf16 products on tcgen05 tensor cores.  epi: 0 bias+ReLU -> bf16, 1 ReLU mask -> bf16, 2 plain fp32.
+// colsum (epi 1 only, may be null): colsum[n] += sum over the rows of the stored (rounded) output.
 cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
                            const __nv_bfloat16* W, int64_t ldw, int epi, void* out, int64_t ldo, const float* bias,
-                           const __nv_bfloat16* mask, int64_t ldm, int32_t* err, cudaStream_t st);
+                           const __nv_bfloat16* mask, int64_t ldm, float* colsum, int32_t* err, cudaStream_t st);
 // out[M][N] (fp32) += A[K][M]^T . Bm[K][N]
 cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
                             const __nv_bfloat16* Bm, int64_t ldb, float* out, int64_t ldo, int32_t* err,

@@ -58,7 +58,9 @@ __device__ __forceinline__ uint32_t load_key(const SortJob& j, int pass, int64_t
     return __ldcg(j.keys[src] + i);
 }
 
-__global__ void __launch_bounds__(RS_THREADS)
+// At most 80 registers per thread (three blocks' worth per SM): a sort block then leaves room for a CTA of the
+// tensor-core head beside it, which matters because the ID sort of a step runs next to the gather and the head.
+__global__ void __launch_bounds__(RS_THREADS, 3)
 coop_sort_kernel(const SortBatch batch) {
     __shared__ uint32_t scratch[33];
     __shared__ uint32_t base[RS_BUCKETS];
