@@ -15,10 +15,11 @@
 //   4. plan pass: the flags again, now with their global prefix: group g starts at grp_start[g]; complete
 //      groups get consecutive ready-queue slots (a counter-threshold stream compaction: ballot-free block
 //      scan of the "count reaches M" predicate).
-//   5. reduce pass: one warp per group sums its rows (fp32, arrival order, 128-bit loads through the sort
-//      permutation) and either writes the average to its queue slot or, for the open group, the running
-//      sum and count back to the table.  The warp that owns the first group of an image also settles
-//      what the image's last, still open group leaves in the table, so no two warps touch one table row.
+//   5. reduce pass: a warp sums the rows of each of its groups (fp32, arrival order, whole rows staged through
+//      shared memory by asynchronous copies, addressed through the sort permutation) and either writes the
+//      average to its queue slot or, for the open group, the running sum and count back to the table.  The
+//      warp that owns the first group of an image also settles what the image's last, still open group
+//      leaves in the table, so no two warps touch one table row.
 //   6. commit: the queue length grows by the number of complete groups (or the call is dropped whole if
 //      the queue would overflow).
 // HBM bound: the reduce pass reads every gradient row once and reads/writes one accumulator row per
@@ -31,6 +32,7 @@ namespace gear {
 constexpr int AF_THREADS = 256;
 constexpr int AF_ITEMS = 4;
 constexpr int AF_TILE = AF_THREADS * AF_ITEMS;
+constexpr int ACC_SPAN = 16;         // sorted positions per unit of work of the reduce pass (at most 32)
 
 __device__ __forceinline__ uint32_t warp_inclusive_max(uint32_t v) {
     const unsigned lane = lane_id();
@@ -53,9 +55,10 @@ struct TileFlags {
 };
 
 // smem: 34 words.  Every thread of the block must call this.
+// run_end (optional): run_end[first position of an image's run] = one past its last position.
 __device__ __forceinline__ void tile_flags(TileFlags& f, const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab,
                                            int M, const int32_t* __restrict__ cnt, uint32_t* smem,
-                                           DevState* __restrict__ state) {
+                                           DevState* __restrict__ state, uint32_t* __restrict__ run_end = nullptr) {
     const int64_t tile0 = (int64_t)blockIdx.x * AF_TILE;
     f.i0 = tile0 + (int64_t)threadIdx.x * AF_ITEMS;
     uint32_t prev = vocab;   // key just before this thread's first position
@@ -120,7 +123,9 @@ __device__ __forceinline__ void tile_flags(TileFlags& f, const uint32_t* __restr
             const int64_t last = i + (M - rem) - 1;  // the row that brings the count to M
             f.complete[t] = last < n && ks[last] == f.key[t];
         }
-        if (i + 1 == n || ks[i + 1] >= vocab) state->n_valid = i + 1;   // exactly one thread sees this
+        const uint32_t after = i + 1 < n ? ks[i + 1] : vocab;
+        if (after >= vocab) state->n_valid = i + 1;                     // exactly one thread sees this
+        if (run_end && after != f.key[t]) run_end[start] = (uint32_t)(i + 1);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0 && (n == 0 || ks[0] >= vocab)) state->n_valid = 0;   // no valid row at all
 }
@@ -147,10 +152,11 @@ acc_flag_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int 
 __global__ void __launch_bounds__(AF_THREADS)
 acc_plan_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int M, const int32_t* __restrict__ cnt,
                 const uint2* __restrict__ tile_cnt, uint4* __restrict__ grp_rec, RowSource rs,
-                int32_t* __restrict__ psrc, float* __restrict__ pscale, DevState* __restrict__ state) {
+                int2* __restrict__ pmeta, uint32_t* __restrict__ blk_first, uint32_t* __restrict__ run_end,
+                DevState* __restrict__ state) {
     __shared__ uint32_t smem[34];
     TileFlags f;
-    tile_flags(f, ks, n, vocab, M, cnt, smem, state);
+    tile_flags(f, ks, n, vocab, M, cnt, smem, state, run_end);
     uint32_t g = 0, c = 0;
 #pragma unroll
     for (int t = 0; t < AF_ITEMS; ++t) { g += f.head[t]; c += f.complete[t]; }
@@ -160,6 +166,8 @@ acc_plan_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int 
     const int64_t q_base = state->q_count;
 #pragma unroll
     for (int t = 0; t < AF_ITEMS; ++t) {
+        // the reduce pass hands out spans of ACC_SPAN sorted positions: index of the first group that starts in each
+        if (((f.i0 + t) % ACC_SPAN) == 0 && f.i0 + t < n && f.key[t] < vocab) blk_first[(f.i0 + t) / ACC_SPAN] = gi;
         if (!f.head[t]) continue;
         // one 16-byte record per group: start position (top bit: first group of its image in this call), image ID,
         // ready-queue slot (-1: the group stays open), rows the image already held
@@ -168,153 +176,236 @@ acc_plan_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int 
         ++gi;
         ci += f.complete[t];
     }
-    // where the gradient row of every sorted position lives and what it is scaled by, resolved through the sort
-    // permutation once, so that the reduce pass reads both with coalesced loads
+    // where the gradient row of every sorted position lives and what it is scaled by (one 8-byte record), resolved
+    // through the sort permutation once, so that the reduce pass reads both with one coalesced load
 #pragma unroll
     for (int t = 0; t < AF_ITEMS; ++t) {
         const int64_t i = f.i0 + t;
         if (i >= n || f.key[t] >= vocab) continue;
         const uint32_t r = rs.perm[i];
         const int32_t src = rs.src_row ? rs.src_row[r] : (int32_t)r;
-        psrc[i] = src;
-        pscale[i] = rs.scale ? rs.scale[src] : 1.f;
+        pmeta[i] = make_int2(src, __float_as_int(rs.scale ? rs.scale[src] : 1.f));
     }
 }
 
 struct RowGather {
-    const float* grads; int64_t ld; const int32_t* psrc; const float* pscale;
+    const float* grads; int64_t ld; const int2* pmeta;      // pmeta[p] = (source row, scale bits) of sorted position p
 };
 
-// Sum of the gradient rows at sorted positions [a, b), in order.  All 32 lanes call this together.
-template <int NQ>
-__device__ __forceinline__ void sum_rows(float4 (&acc)[NQ], const RowGather& rg, int64_t a, int64_t b, int n_chunks) {
-    const unsigned lane = lane_id();
-    for (int64_t p0 = a; p0 < b; p0 += 32) {
-        const int m = (int)min((int64_t)32, b - p0);
-        int my_s = 0;
-        float my_scale = 1.f;
-        if ((int)lane < m) { my_s = rg.psrc[p0 + lane]; my_scale = rg.pscale[p0 + lane]; }
-        for (int t0 = 0; t0 < m; t0 += 4) {
-            float4 v[4][NQ];
-            float sc[4];
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                const int64_t s = __shfl_sync(0xffffffffu, my_s, (t0 + t) & 31);
-                sc[t] = __shfl_sync(0xffffffffu, my_scale, (t0 + t) & 31);
-                const bool on = t0 + t < m;
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    const int ch = lane + 32 * q;
-                    v[t][q] = (on && ch < n_chunks) ? ld_stream_f4(rg.grads + s * rg.ld + ch * 4)
-                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            }
-#pragma unroll
-            for (int t = 0; t < 4; ++t)
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    acc[q].x = fmaf(sc[t], v[t][q].x, acc[q].x);
-                    acc[q].y = fmaf(sc[t], v[t][q].y, acc[q].y);
-                    acc[q].z = fmaf(sc[t], v[t][q].z, acc[q].z);
-                    acc[q].w = fmaf(sc[t], v[t][q].w, acc[q].w);
-                }
-        }
-    }
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 reads nothing and fills the 16 bytes with zeros
+__device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void* gsrc, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(smem_dst), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory");
 }
 
-template <int NQ>
-__global__ void __launch_bounds__(256, NQ <= 2 ? 4 : 2)
+// What a lane knows about "its" group of a span: own rows [start, start + len), then zlen rows from zstart.
+struct LaneGroup {
+    uint32_t start, key, zstart;
+    int slot, c0, len, zlen, items;      // items = rows the warp stages for the group (0: nothing to do)
+    bool first;
+};
+
+// One row to stage: accumulator row `idx` of the table, or gradient row `idx` scaled by `scale`.
+// meta = group lane << 3 | accumulator row << 2 | last item of the group << 1 | last of the group's own rows.
+struct ItemDesc { int idx; float scale; int meta; };
+
+// The reduce pass.  A warp takes spans of ACC_SPAN sorted positions, span w, w + W, w + 2W, ... (W = warps of
+// the grid); the groups that start inside a span (at most ACC_SPAN, one per lane) are walked as one flat
+// sequence of items -- for every group first the image's accumulator row if it holds anything, then its
+// gradient rows in arrival order; the first group of an image, if it completes, is followed by the rows of
+// the image's trailing open group, so that one warp alone reads and writes the image's accumulator row.
+// Items are staged through a per-warp ring of S row-sized shared-memory slots with asynchronous copies
+// (cp.async, 16 bytes per lane, whole rows): the copy of item i + S - 1 is issued before item i is added,
+// across group boundaries, so a warp keeps S - 1 rows in flight whatever the group sizes are -- most
+// groups hold a single row, and registers alone cannot keep enough of those in flight.  What to copy is
+// worked out 32 items at a time, one item per lane (a search over the groups' item counts, the position
+// record fetched by the lane), one batch ahead of the copies; the inner loop only broadcasts a lane's
+// descriptor, copies and adds.  The group records of the next span are requested while the current span
+// streams.  Sums are fp32, in arrival order, starting from the stored partial sum.
+// FULL: a row is exactly NQ * 512 bytes, so no lane is ever idle.
+template <int NQ, int S, bool FULL>
+__global__ void __launch_bounds__(256, 2)
 acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, int64_t n_tiles, int64_t ready_cap,
                   const uint2* __restrict__ tile_cnt, const uint4* __restrict__ grp_rec,
+                  const uint32_t* __restrict__ blk_first, const uint32_t* __restrict__ run_end,
                   float* __restrict__ gsum, int32_t* __restrict__ gcnt,
                   int32_t* __restrict__ q_id, float* __restrict__ q_avg, const DevState* __restrict__ state) {
+    extern __shared__ float4 ring_mem[];                          // [warps][S][NQ * 32] float4
     const uint2 totals = tile_cnt[n_tiles];
     const int64_t n_groups = totals.x;
     if (state->q_count + (int64_t)totals.y > ready_cap) return;      // the whole call is dropped
     const int64_t n_valid = state->n_valid;
-    const unsigned lane = lane_id();
+    const int lane = (int)lane_id(), warp = (int)(threadIdx.x >> 5);
     const int n_chunks = D / 4;
     const float m_f = (float)M;
-    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    int64_t g = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    // records of this group and the next one (its start is this group's end), fetched one iteration ahead
-    uint4 rec = make_uint4(0u, 0u, 0u, 0u);
-    uint32_t next_start = 0;
-    if (g < n_groups) {
-        rec = grp_rec[g];
-        next_start = (g + 1 < n_groups) ? (grp_rec[g + 1].x & 0x7fffffffu) : (uint32_t)n_valid;
-    }
-    for (; g < n_groups; g += warps) {
-        const uint4 cur = rec;
-        const int64_t end = next_start;
-        const int64_t gn = g + warps;
-        if (gn < n_groups) {
-            rec = grp_rec[gn];
-            next_start = (gn + 1 < n_groups) ? (grp_rec[gn + 1].x & 0x7fffffffu) : (uint32_t)n_valid;
+    const int64_t W = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t n_spans = ceil_div(n_valid, ACC_SPAN);
+    float4* my_ring = ring_mem + (size_t)warp * S * (NQ * 32);
+    const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
+    constexpr uint32_t SLOT_BYTES = NQ * 32 * 16;
+
+    // group range of a span: lane 0 holds the first group, lane 1 one past the last
+    auto load_range = [&](int64_t span) -> uint32_t {
+        uint32_t v = 0;
+        if (span < n_spans && lane < 2) {
+            const int64_t w = span + lane;
+            v = w < n_spans ? __ldg(blk_first + w) : (uint32_t)n_groups;
         }
-        const bool first = cur.x >> 31;
-        const int slot = (int)cur.z;
-        if (!first && slot < 0) continue;      // an image's trailing open group: settled by its first group's warp
-        const int64_t start = cur.x & 0x7fffffffu;
-        const uint32_t key = cur.y;
-        const int c0 = first ? (int)cur.w : 0;
-        float4 acc[NQ];
-#pragma unroll
-        for (int q = 0; q < NQ; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        float* srow = gsum + (int64_t)key * D;
-        if (c0 > 0) {
-#pragma unroll
-            for (int q = 0; q < NQ; ++q) {
-                const int ch = lane + 32 * q;
-                if (ch < n_chunks) acc[q] = ld_f4(srow + ch * 4);
-            }
+        return v;
+    };
+    auto load_group = [&](int64_t g_lo, int64_t g_hi) -> LaneGroup {
+        LaneGroup r{0u, 0u, 0u, -1, 0, 0, 0, 0, false};
+        const int64_t g = g_lo + lane;
+        if (g < g_hi) {
+            const uint4 rec = __ldg(grp_rec + g);
+            const uint32_t end = (g + 1 < n_groups) ? (__ldg(&grp_rec[g + 1].x) & 0x7fffffffu) : (uint32_t)n_valid;
+            r.start = rec.x & 0x7fffffffu; r.first = rec.x >> 31; r.key = rec.y; r.slot = (int)rec.z;
+            r.c0 = r.first ? (int)rec.w : 0;
+            r.len = (int)(end - r.start);
         }
-        sum_rows<NQ>(acc, rg, start, end, n_chunks);
-        if (slot >= 0) {
-            float* qrow = q_avg + (int64_t)slot * D;
+        return r;
+    };
+
+    int64_t span = (int64_t)blockIdx.x * (blockDim.x >> 5) + warp;
+    uint32_t range_cur = load_range(span), range_nxt = load_range(span + W);
+    LaneGroup G = load_group(__shfl_sync(0xffffffffu, range_cur, 0), __shfl_sync(0xffffffffu, range_cur, 1));
+
+    for (; span < n_spans; span += W) {
+        // ---- look-ahead: group records of the next span, group range of the one after it
+        const LaneGroup G_nxt = load_group(__shfl_sync(0xffffffffu, range_nxt, 0), __shfl_sync(0xffffffffu, range_nxt, 1));
+        const uint32_t range_nxt2 = load_range(span + 2 * W);
+
+        // ---- complete this lane's group
+        if (G.first && G.slot >= 0) {
+            // what the image's remaining rows leave in the table: the rows of its trailing open group
+            const uint32_t run_stop = __ldg(run_end + G.start);
+            G.zlen = (int)(((int64_t)G.c0 + (int64_t)(run_stop - G.start)) % M);
+            G.zstart = run_stop - (uint32_t)G.zlen;
+        }
+        // an image's trailing open group itself (not first, no queue slot) is skipped here
+        if (G.len > 0 && (G.first || G.slot >= 0)) G.items = (G.c0 > 0 ? 1 : 0) + G.len + G.zlen;
+        const int incl = (int)warp_inclusive_scan((uint32_t)G.items);      // items of the groups in lanes 0 .. lane
+        const int total_items = __shfl_sync(0xffffffffu, incl, 31);
+        if (total_items > 0) {
+            // descriptor of item base + lane
+            auto make_desc = [&](int base) -> ItemDesc {
+                const int i = base + lane;
+                int l = 0;                                      // group lane: the first one with incl > i
 #pragma unroll
-            for (int q = 0; q < NQ; ++q) {
-                const int ch = lane + 32 * q;
-                if (ch < n_chunks)
-                    st_f4(qrow + ch * 4, make_float4(acc[q].x / m_f, acc[q].y / m_f, acc[q].z / m_f, acc[q].w / m_f));
-            }
-            if (lane == 0) q_id[slot] = (int32_t)key;
-            if (!first) continue;
-            // what the image's remaining rows leave in the table
-            int64_t rest = 0;
-            if (end < n_valid && ks[end] == key) {
-                int64_t lo = end, step = 1, hi = end + 1;          // ks[lo] == key
-                while (hi < n_valid && ks[hi] == key) { lo = hi; step <<= 1; hi = min(lo + step, n_valid); }
-                // first index in (lo, hi] whose key differs (hi == n_valid counts as differing)
-                int64_t l = lo + 1, h = hi;
-                while (l < h) {
-                    const int64_t mid = (l + h) >> 1;
-                    if (ks[mid] == key) l = mid + 1; else h = mid;
+                for (int step = ACC_SPAN / 2; step >= 1; step >>= 1) {
+                    const int v = __shfl_sync(0xffffffffu, incl, l + step - 1);
+                    if (v <= i) l += step;
                 }
-                rest = (l - end) % M;
-                if (rest > 0) {
+                const int incl_l = __shfl_sync(0xffffffffu, incl, l), items_l = __shfl_sync(0xffffffffu, G.items, l);
+                const int c0_l = __shfl_sync(0xffffffffu, G.c0, l), len_l = __shfl_sync(0xffffffffu, G.len, l);
+                const uint32_t start_l = __shfl_sync(0xffffffffu, G.start, l);
+                const uint32_t zstart_l = __shfl_sync(0xffffffffu, G.zstart, l);
+                const uint32_t key_l = __shfl_sync(0xffffffffu, G.key, l);
+                const int k = i - (incl_l - items_l);           // item number within the group
+                const int tab = c0_l > 0 ? 1 : 0, own_end = tab + len_l;
+                const bool ok = i < total_items, is_tab = k < tab;
+                const int64_t p = k < own_end ? (int64_t)start_l + (k - tab) : (int64_t)zstart_l + (k - own_end);
+                int2 pm = make_int2(0, __float_as_int(1.f));
+                if (ok && !is_tab) pm = __ldg(rg.pmeta + p);
+                ItemDesc d;
+                d.idx = (ok && is_tab) ? (int)key_l : pm.x;
+                d.scale = __int_as_float(pm.y);
+                d.meta = (l << 3) | (is_tab ? 4 : 0) | (k + 1 == items_l ? 2 : 0) | (k + 1 == own_end ? 1 : 0);
+                return d;
+            };
+
+            float4 acc[NQ];
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+            // acc holds the group's own rows (own_done) and/or everything the warp adds for it (all_done)
+            auto settle = [&](int l, bool own_done, bool all_done) {
+                const uint32_t key = __shfl_sync(0xffffffffu, G.key, l);
+                const int slot = __shfl_sync(0xffffffffu, G.slot, l);
+                float* srow = gsum + (int64_t)key * D;
+                if (own_done && slot >= 0) {                    // the group reached M: its average joins the queue
+                    float* qrow = q_avg + (int64_t)slot * D;
+#pragma unroll
+                    for (int q = 0; q < NQ; ++q) {
+                        const int ch = lane + 32 * q;
+                        if (FULL || ch < n_chunks)
+                            st_f4(qrow + ch * 4, make_float4(acc[q].x / m_f, acc[q].y / m_f, acc[q].z / m_f, acc[q].w / m_f));
+                        acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    if (lane == 0) q_id[slot] = (int32_t)key;
+                }
+                if (all_done) {
+                    const int c0 = __shfl_sync(0xffffffffu, G.c0, l), len = __shfl_sync(0xffffffffu, G.len, l);
+                    const int zlen = __shfl_sync(0xffffffffu, G.zlen, l);
+                    const bool first = __shfl_sync(0xffffffffu, (int)G.first, l) != 0;
+                    // the table row: the open group (this one if it did not complete, else the image's trailing one)
+                    const bool write_row = first && (slot < 0 || zlen > 0 || c0 > 0);
+                    if (write_row) {
+#pragma unroll
+                        for (int q = 0; q < NQ; ++q) {
+                            const int ch = lane + 32 * q;
+                            if (FULL || ch < n_chunks) st_f4(srow + ch * 4, acc[q]);
+                        }
+                        if (lane == 0) gcnt[key] = slot < 0 ? c0 + len : zlen;
+                    }
 #pragma unroll
                     for (int q = 0; q < NQ; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    sum_rows<NQ>(acc, rg, l - rest, l, n_chunks);
                 }
-            }
-            if (rest > 0 || c0 > 0) {
+            };
+
+            ItemDesc cur = make_desc(0), nxt = make_desc(32);
+            int islot = 0, cslot = 0;
+            // copy of item `item` (lane `ji` of cur, or lane ji - 32 of nxt); past the end: an empty copy
+            auto issue = [&](int item, int ji) {
+                const bool in_cur = ji < 32;
+                const int idx = __shfl_sync(0xffffffffu, in_cur ? cur.idx : nxt.idx, ji & 31);
+                const int meta = __shfl_sync(0xffffffffu, in_cur ? cur.meta : nxt.meta, ji & 31);
+                const bool is_tab = (meta & 4) != 0;
+                const float* src = (is_tab ? gsum : rg.grads) + (int64_t)idx * (is_tab ? (int64_t)D : rg.ld);
+                const uint32_t dst = ring_addr + (uint32_t)islot * SLOT_BYTES;
+                const int bytes = item < total_items ? 16 : 0;
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
                     const int ch = lane + 32 * q;
-                    if (ch < n_chunks) st_f4(srow + ch * 4, rest > 0 ? acc[q] : make_float4(0.f, 0.f, 0.f, 0.f));
+                    const bool on = FULL || ch < n_chunks;          // lanes past the end of a narrow row copy nothing
+                    cp_async_16(dst + (uint32_t)ch * 16u, src + (on ? ch * 4 : 0), on ? bytes : 0);
                 }
-                if (lane == 0) gcnt[key] = (int32_t)rest;
-            }
-        } else {
-            // the image's only group in this call, still open
+                cp_async_commit();
+                islot = islot + 1 == S ? 0 : islot + 1;
+            };
+
+            // ---- the pipeline: S - 1 items ahead
+            __syncwarp();
 #pragma unroll
-            for (int q = 0; q < NQ; ++q) {
-                const int ch = lane + 32 * q;
-                if (ch < n_chunks) st_f4(srow + ch * 4, acc[q]);
+            for (int i = 0; i < S - 1; ++i) issue(i, i);
+            for (int base = 0; base < total_items; base += 32) {
+                const int n_in = min(32, total_items - base);
+                for (int j = 0; j < n_in; ++j) {
+                    __syncwarp();                                 // every lane is done with the slot refilled next
+                    issue(base + j + S - 1, j + S - 1);
+                    cp_async_wait<S - 1>();
+                    __syncwarp();                                 // ... and sees the other lanes' copies of item base + j
+                    const float scale = __shfl_sync(0xffffffffu, cur.scale, j);
+                    const int meta = __shfl_sync(0xffffffffu, cur.meta, j);
+                    const float4* row = my_ring + (size_t)cslot * (NQ * 32);
+#pragma unroll
+                    for (int q = 0; q < NQ; ++q) {
+                        const float4 v = row[lane + 32 * q];
+                        acc[q].x = fmaf(scale, v.x, acc[q].x); acc[q].y = fmaf(scale, v.y, acc[q].y);
+                        acc[q].z = fmaf(scale, v.z, acc[q].z); acc[q].w = fmaf(scale, v.w, acc[q].w);
+                    }
+                    if (meta & 3) settle(meta >> 3, (meta & 1) != 0, (meta & 2) != 0);
+                    cslot = cslot + 1 == S ? 0 : cslot + 1;
+                }
+                cur = nxt;
+                nxt = make_desc(base + 64);
             }
-            if (lane == 0) gcnt[key] = c0 + (int32_t)(end - start);
+            cp_async_wait<0>();
         }
+        G = G_nxt; range_nxt = range_nxt2;
     }
 }
 
@@ -326,8 +417,6 @@ __global__ void acc_commit_kernel(const uint2* __restrict__ tile_cnt, int64_t n_
     if (state->q_count + (int64_t)totals.y > ready_cap) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
     else if (totals.y > 0) { state->q_count += totals.y; state->q_calls += 1; }
 }
-
-static int reduce_grid() { return 148 * 8; }
 
 cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
                               const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st) {
@@ -357,24 +446,39 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     acc_flag_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt, state); }
     scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, &c.prof);
     uint4* grp_rec = c.at<uint4>(c.ws.grp_rec);
-    int32_t* psrc = c.at<int32_t>(c.ws.psrc);
-    float* pscale = c.at<float>(c.ws.pscale);
+    int2* pmeta = c.at<int2>(c.ws.pmeta);
     RowSource rs{sb.vals[cur], grads, ld, src_row, scale};
-    RowGather rg{grads, ld, psrc, pscale};
+    RowGather rg{grads, ld, pmeta};
+    uint32_t* blk_first = c.at<uint32_t>(c.ws.blk_first);
+    uint32_t* run_end = c.at<uint32_t>(c.ws.run_end);
     { KernelScope k(&c.prof, "acc_plan", st);
     acc_plan_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt,
-                                                            grp_rec, rs, psrc, pscale, state); }
+                                                            grp_rec, rs, pmeta, blk_first, run_end, state); }
     const int nq = (int)ceil_div(D / 4, 32);
-    int64_t want = ceil_div(n, 8);
-    const int grid = (int)(want < reduce_grid() ? (want < 1 ? 1 : want) : reduce_grid());
-#define GEAR_ACC_LAUNCH(NQ) acc_reduce_kernel<NQ><<<grid, 256, 0, st>>>(ks, rg, D, M, n_tiles, c.ws.ready_cap, tile_cnt, \
-        grp_rec, c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id), c.at<float>(c.ws.q_avg), state)
+    const int64_t want = ceil_div(ceil_div(n, ACC_SPAN), 8);
+    const int resident = sm_count() * 2;                          // every block stays resident
+    const int grid = (int)(want < resident ? (want < 1 ? 1 : want) : resident);
+    cudaError_t le = cudaSuccess;
     { KernelScope k(&c.prof, "acc_reduce", st);
-    if (nq <= 1) GEAR_ACC_LAUNCH(1);
-    else if (nq <= 2) GEAR_ACC_LAUNCH(2);
-    else if (nq <= 4) GEAR_ACC_LAUNCH(4);
-    else GEAR_ACC_LAUNCH(8); }
+    auto launch = [&](auto kernel, int slot_bytes, int slots) {
+        const int smem = 8 * slots * slot_bytes;
+        le = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (le != cudaSuccess) return;
+        kernel<<<grid, 256, smem, st>>>(ks, rg, D, M, n_tiles, c.ws.ready_cap, tile_cnt, grp_rec, blk_first, run_end,
+                                        c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id),
+                                        c.at<float>(c.ws.q_avg), state);
+    };
+    // ring depth: as many row slots as about 96 KB per block (two blocks per SM) allow, at most 8
+    const bool full = D == nq * 128;                              // every lane owns a chunk of every row
+#define GEAR_ACC_LAUNCH(NQ, S) \
+    do { if (full) launch(acc_reduce_kernel<NQ, S, true>, NQ * 512, S); else launch(acc_reduce_kernel<NQ, S, false>, NQ * 512, S); } while (0)
+    if (nq <= 1) GEAR_ACC_LAUNCH(1, 8);
+    else if (nq <= 2) GEAR_ACC_LAUNCH(2, 8);
+    else if (nq <= 4) GEAR_ACC_LAUNCH(4, 5);
+    else GEAR_ACC_LAUNCH(8, 3);
 #undef GEAR_ACC_LAUNCH
+    }
+    if (le != cudaSuccess) return le;
     { KernelScope k(&c.prof, "acc_commit", st);
     acc_commit_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, c.ws.ready_cap, state); }
     ++c.acc_calls_pending;

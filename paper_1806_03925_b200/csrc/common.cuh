@@ -105,6 +105,23 @@ __device__ __forceinline__ void red_add_f4(float* p, float4 v) {
                  :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
+// L2 eviction priorities: data that is read again soon is kept (evict_last), data touched once is let go first
+// (evict_first), so that a streamed table does not push a reused matrix out of the L2.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void st_f4_hint(float* p, float4 v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1,%2,%3,%4}, %5;"
+                 :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy) : "memory");
+}
+
 // ---------------------------------------------------------------- launch accounting / per-kernel timing
 // Every kernel launch of the library goes through a KernelScope: it counts the launch and, when profiling
 // is on, brackets it with a pair of CUDA events on the caller's stream (read back by gear_profile_read).

@@ -280,6 +280,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // warps 2..5 take the first half of the tile's columns, warps 6..9 the second half
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;
+        const uint64_t keep_policy = l2_policy_evict_last();
         constexpr int CHUNKS = BN / 64;                       // 32-column chunks per warp and tile
         uint32_t tile_it = 0;
         bool ok = true;
@@ -372,7 +373,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const float4 v4 = make_float4(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1]),
                                                       __uint_as_float(acc[4 * j + 2]), __uint_as_float(acc[4 * j + 3]));
                         if (EPI == TC_EPI_RED) red_add_f4(dst + 4 * j, v4);
-                        else st_f4(dst + 4 * j, v4);
+                        else st_f4_hint(dst + 4 * j, v4, keep_policy);      // dX is read again right after: keep it in the L2
                     }
                 }
             }

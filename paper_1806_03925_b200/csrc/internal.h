@@ -32,7 +32,9 @@ struct WsPlan {
     int64_t sort_n[4];
     size_t tile_cnt;                    // [sort tiles + 1] uint2 per-tile (groups, complete) counts
     size_t grp_rec;                     // [max_nnz] uint4 group records (start | first flag, image ID, queue slot, held rows)
-    size_t psrc, pscale;                // [max_nnz] int32 / fp32: source row and scale of every sorted position
+    size_t blk_first;                   // [ceil(max_nnz / 16) + 2] uint32: first group that starts in each span of sorted positions
+    size_t run_end;                     // [max_nnz] uint32: at the first position of an image's run, one past its last
+    size_t pmeta;                       // [max_nnz] int2: source row and scale (fp32 bits) of every sorted position
     size_t q_id;                        // [ready_cap] int32
     size_t q_avg;                       // [ready_cap][dfv_dim] fp32
     size_t exp_bits;                    // [ceil(img_vocab / 32)] uint32 expired bitmap
