@@ -65,9 +65,14 @@ enum { GEAR_F32 = 0, GEAR_BF16 = 1 };
 enum {
     GEAR_ACC_SORT = 0,       /* stable key sort + segmented reduction: groups split exactly at every
                                 M-th arrival in row order; deterministic */
-    GEAR_ACC_ATOMIC = 1      /* fp32 atomic adds on the accumulator rows: arrival order (hence group
-                                membership) is whatever the hardware makes it; counts and emission
-                                counts still match the sorted path */
+    GEAR_ACC_ATOMIC = 1      /* fp32 reductions on the accumulator rows in whatever order the hardware takes
+                                them: which arrivals share a group is not defined.  Counts and the number of
+                                emissions per image equal the sorted path's; after the rows of a call have been
+                                added, an image holding k >= M gradients emits floor(k / M) averages, each the mean
+                                of all k pooled gradients, and keeps (k mod M) / k of the pooled sum, so that
+                                M * (emitted averages) + kept sum = pooled sum.  A call is refused whole
+                                (GEAR_DEV_READY_OVERFLOW) unless the queue has room for n more entries.
+                                Needs M < 2^29.  Not bit-reproducible from run to run */
 };
 
 /* bits of the device status word (sticky until gear_status clears them) */

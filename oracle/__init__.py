@@ -74,6 +74,8 @@ def lib():
         L.orc_dfv_grad_rows.argtypes = [i32, i32, vp, vp, i32, i32, vp]
         L.orc_accumulate.restype = i64
         L.orc_accumulate.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, i64, vp, vp, vp, i64, vp, vp]
+        L.orc_accumulate_pooled.restype = i64
+        L.orc_accumulate_pooled.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, i64, vp, vp, vp, i64, vp]
         L.orc_collect_ready.restype = None
         L.orc_collect_ready.argtypes = [vp, vp, i64]
         L.orc_collect_expired.restype = i64
@@ -239,7 +241,9 @@ class GearOracle:
         return rows
 
     # -- event 6 --------------------------------------------------------------
-    def accumulate(self, img_id, grads: np.ndarray, want_members: bool = False):
+    def accumulate(self, img_id, grads: np.ndarray, want_members: bool = False, pooled: bool = False):
+        """pooled: the order-free store (orc_accumulate_pooled): emissions carry the mean of all
+        gradients pooled for the image."""
         ids = _c(img_id, np.int32)
         g = _c(grads, np.float64)
         n = len(ids)
@@ -251,9 +255,15 @@ class GearOracle:
         eavg = np.zeros((cap, self.D), dtype=np.float64); eavg[:n0] = self._emit_avg
         n_emit = C.c_int64(n0)
         members = np.zeros(n, dtype=np.int64) if want_members else None
-        bad = lib().orc_accumulate(_ptr(self.gsum), _ptr(self.gcnt), _ptr(self.seq), self.V, self.D, self.M,
-                                   _ptr(ids), _ptr(g), n, _ptr(eid), _ptr(eseq), _ptr(eavg), cap,
-                                   C.byref(n_emit), _ptr(members))
+        if pooled:
+            assert not want_members
+            bad = lib().orc_accumulate_pooled(_ptr(self.gsum), _ptr(self.gcnt), _ptr(self.seq), self.V, self.D,
+                                              self.M, _ptr(ids), _ptr(g), n, _ptr(eid), _ptr(eseq), _ptr(eavg), cap,
+                                              C.byref(n_emit))
+        else:
+            bad = lib().orc_accumulate(_ptr(self.gsum), _ptr(self.gcnt), _ptr(self.seq), self.V, self.D, self.M,
+                                       _ptr(ids), _ptr(g), n, _ptr(eid), _ptr(eseq), _ptr(eavg), cap,
+                                       C.byref(n_emit), _ptr(members))
         assert bad >= 0
         k = n_emit.value
         self._emit_id, self._emit_seq, self._emit_avg = eid[:k], eseq[:k], eavg[:k]

@@ -22,6 +22,9 @@
  *   orc_accumulate        Section 1 (third point) and event 6: keep the
  *                         gradients of an image until M have arrived, then
  *                         emit their average.
+ *   orc_accumulate_pooled the same store when arrival order is not recorded
+ *                         (asynchronous workers): emissions carry the mean of
+ *                         the pooled gradients.
  *   orc_collect_expired   Section 1 (second point) and Section 3: cached
  *                         inference results older than the inference-expired
  *                         time are dropped / refreshed.
@@ -434,6 +437,52 @@ int64_t orc_accumulate(double* sum, int32_t* cnt, int32_t* seq, int64_t vocab, i
         }
     }
     free(open_head); free(next_in_group);
+    return bad;
+}
+
+/*
+ * The same store when the order of arrival is not recorded (the paper's
+ * workers push gradients asynchronously, Section 3 events 5 and 6, so the
+ * store may only know how many gradients an image holds and their sum).
+ * All arrivals of the call are added first; then every image holding
+ * k >= M gradients emits floor(k / M) averages, each the mean of all k pooled
+ * gradients, and keeps k mod M gradients' worth of that mean:
+ *     avg = sum / k;   emit floor(k / M) times;   sum = avg * (k mod M);   cnt = k mod M.
+ * M * (sum of the emitted averages) + the kept sum equals the pooled sum, and
+ * counts and emission counts are those of orc_accumulate.  Emissions are
+ * listed image by image in order of first arrival.  Returns the number of
+ * out-of-range IDs, or -1 if the emit list overflowed.
+ */
+int64_t orc_accumulate_pooled(double* sum, int32_t* cnt, int32_t* seq, int64_t vocab, int32_t D, int32_t M,
+                              const int32_t* ids, const double* grads, int64_t n,
+                              int32_t* emit_id, int32_t* emit_seq, double* emit_avg,
+                              int64_t emit_cap, int64_t* n_emit) {
+    int64_t bad = 0;
+    for (int64_t r = 0; r < n; ++r) {
+        int32_t id = ids[r];
+        if (id < 0 || id >= vocab) { ++bad; continue; }
+        double* s = sum + (int64_t)id * D;
+        const double* g = grads + r * D;
+        for (int c = 0; c < D; ++c) s[c] += g[c];
+        cnt[id] += 1;
+    }
+    for (int64_t r = 0; r < n; ++r) {
+        int32_t id = ids[r];
+        if (id < 0 || id >= vocab) continue;
+        const int32_t k = cnt[id];
+        if (k < M) continue;                       /* also true once the image has been settled */
+        double* s = sum + (int64_t)id * D;
+        const int32_t e_count = k / M, rest = k % M;
+        for (int32_t j = 0; j < e_count; ++j) {
+            if (*n_emit >= emit_cap) return -1;
+            int64_t e = (*n_emit)++;
+            emit_id[e] = id;
+            emit_seq[e] = seq[id]++;
+            for (int c = 0; c < D; ++c) emit_avg[e * D + c] = s[c] / (double)k;
+        }
+        for (int c = 0; c < D; ++c) s[c] = s[c] / (double)k * (double)rest;
+        cnt[id] = rest;
+    }
     return bad;
 }
 

@@ -485,6 +485,104 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------- GEAR_ACC_ATOMIC: the store without arrival order
+// Rows are added to the accumulator rows with fp32 reductions in whatever order the hardware takes them, so
+// which arrivals share a group is not defined; what is defined (and equal to the ordered path) is every
+// image's count and its number of emissions.  After all rows of the call have been added, every image that
+// was touched and now holds k >= M gradients emits floor(k / M) averages, each the mean of all k pooled
+// gradients, and keeps k mod M gradients' worth of that mean, so that nothing is lost or counted twice.
+// Under heavy skew the reductions of a hot image serialise on its accumulator row; that is the cost the
+// sorted path avoids.
+constexpr int32_t ACC_TOUCHED = 0x40000000;      // bit of dfv_gcnt[id] while a call is in flight: id is on the touched list
+
+__global__ void __launch_bounds__(256)
+acc_atomic_add_kernel(const int32_t* __restrict__ img_id, int64_t n, int64_t vocab, const float* __restrict__ grads,
+                      int64_t ld, const int32_t* __restrict__ src_row, const float* __restrict__ scale, int D,
+                      float* __restrict__ gsum, int32_t* __restrict__ gcnt, int32_t* __restrict__ touched,
+                      int64_t ready_cap, DevState* __restrict__ state) {
+    // a call completes at most n groups: refuse it whole if the queue could not take them
+    const bool drop = state->q_count + n > ready_cap;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        state->pad[3] = drop ? 1 : 0;
+        if (drop) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
+    }
+    if (drop) return;
+    const unsigned lane = lane_id();
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    int flags = 0;
+    for (int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < n; r += warps) {
+        const int32_t id = img_id[r];
+        if (id < 0 || id >= vocab) { flags |= GEAR_DEV_BAD_ID; continue; }
+        const int64_t s = src_row ? src_row[r] : r;
+        const float sc = scale ? scale[s] : 1.f;
+        for (int ch = lane; ch < D / 4; ch += 32) {
+            const float4 v = ld_stream_f4(grads + s * ld + ch * 4);
+            red_add_f4(gsum + (int64_t)id * D + ch * 4, make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w));
+        }
+        if (lane == 0) {
+            const int32_t before = atomicOr(&gcnt[id], ACC_TOUCHED);
+            if (!(before & ACC_TOUCHED)) {
+                const unsigned long long pos = atomicAdd(reinterpret_cast<unsigned long long*>(&state->pad[2]), 1ull);
+                touched[pos] = id;
+            }
+            atomicAdd(&gcnt[id], 1);
+        }
+    }
+    if (flags) atomicOr(&state->status, flags);
+}
+
+__global__ void __launch_bounds__(256)
+acc_atomic_settle_kernel(const int32_t* __restrict__ touched, int D, int M, float* __restrict__ gsum,
+                         int32_t* __restrict__ gcnt, int32_t* __restrict__ q_id, float* __restrict__ q_avg,
+                         DevState* __restrict__ state) {
+    if (state->pad[3] != 0) return;                            // the call was dropped
+    const int64_t n_touched = state->pad[2];
+    const unsigned lane = lane_id();
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    if (blockIdx.x == 0 && threadIdx.x == 0)                   // emission order is not ID order: collect has to sort
+        atomicAdd(reinterpret_cast<unsigned long long*>(&state->q_calls), 2ull);
+    for (int64_t t = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); t < n_touched; t += warps) {
+        const int32_t id = touched[t];
+        const int32_t k = gcnt[id] & ~ACC_TOUCHED;
+        const int32_t e = k / M, rest = k % M;
+        float* row = gsum + (int64_t)id * D;
+        if (e > 0) {
+            unsigned long long slot0 = 0;
+            if (lane == 0) slot0 = atomicAdd(reinterpret_cast<unsigned long long*>(&state->q_count), (unsigned long long)e);
+            slot0 = __shfl_sync(0xffffffffu, slot0, 0);
+            const float kf = (float)k, rf = (float)rest;
+            for (int ch = lane; ch < D / 4; ch += 32) {
+                const float4 sum = ld_f4(row + ch * 4);
+                const float4 avg = make_float4(sum.x / kf, sum.y / kf, sum.z / kf, sum.w / kf);
+                for (int32_t j = 0; j < e; ++j) st_f4(q_avg + (int64_t)(slot0 + j) * D + ch * 4, avg);
+                st_f4(row + ch * 4, make_float4(avg.x * rf, avg.y * rf, avg.z * rf, avg.w * rf));
+            }
+            for (int32_t j = lane; j < e; j += 32) q_id[slot0 + j] = id;
+        }
+        if (lane == 0) gcnt[id] = rest;
+    }
+}
+
+cudaError_t launch_accumulate_atomic(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
+                                     const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    DevState* state = c.state();
+    int32_t* touched = c.at<int32_t>(c.ws.pmeta);               // the sorted path's scratch is free in this mode
+    cudaError_t e = cudaMemsetAsync(&state->pad[2], 0, sizeof(int64_t), st);
+    if (e != cudaSuccess) return e;
+    const int64_t want = ceil_div(n, 8);
+    const int resident = sm_count() * 8;
+    const int grid = (int)(want < resident ? (want < 1 ? 1 : want) : resident);
+    { KernelScope k(&c.prof, "acc_atomic_add", st);
+    acc_atomic_add_kernel<<<grid, 256, 0, st>>>(img_id, n, c.cfg.img_vocab, grads, ld, src_row, scale, c.cfg.dfv_dim,
+                                                c.buf.dfv_gsum, c.buf.dfv_gcnt, touched, c.ws.ready_cap, state); }
+    { KernelScope k(&c.prof, "acc_atomic_settle", st);
+    acc_atomic_settle_kernel<<<grid, 256, 0, st>>>(touched, c.cfg.dfv_dim, c.cfg.M, c.buf.dfv_gsum, c.buf.dfv_gcnt,
+                                                   c.at<int32_t>(c.ws.q_id), c.at<float>(c.ws.q_avg), state); }
+    c.acc_calls_pending += 2;
+    return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------- event 6b: hand the ready queue over
 __global__ void collect_begin_kernel(DevState* __restrict__ state, int64_t cap, int64_t* __restrict__ d_n) {
     const int64_t n = state->q_count;

@@ -41,6 +41,7 @@ static int validate_config(const gear_config& c) {
     if (c.max_nnz < 1 || c.max_nnz > vmax) return arg_fail("max_nnz in [1, 2^31 - 2]");
     if (c.ready_cap < 0 || c.ready_cap > vmax) return arg_fail("ready_cap in [0, 2^31 - 2]");
     if (c.accum_mode != GEAR_ACC_SORT && c.accum_mode != GEAR_ACC_ATOMIC) return arg_fail("accum_mode");
+    if (c.accum_mode == GEAR_ACC_ATOMIC && c.M >= (1 << 29)) return arg_fail("GEAR_ACC_ATOMIC needs M < 2^29");
     return GEAR_OK;
 }
 
@@ -165,6 +166,7 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
     c.img_sorted = false;
     c.img_sorted_n = 0;
     c.img_sorted_buf = 0;
+    c.last_img_id = nullptr;
     c.acc_calls_pending = 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
@@ -227,7 +229,7 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
         batch.job[1].ids = b.url_id; batch.job[1].sentinel = (uint32_t)c.cfg.url_vocab;
         batch.job[1].n_max = b.B; batch.job[1].bits = bits_for(c.cfg.url_vocab);
         batch.n_jobs = 2;
-        if (b.nnz > 0) {
+        if (b.nnz > 0 && c.cfg.accum_mode == GEAR_ACC_SORT) {      // the atomic mode takes the image IDs as they come
             batch.job[2] = c.sort_job(gear_ctx_impl::SORT_IMG);
             batch.job[2].ids = b.img_id; batch.job[2].sentinel = (uint32_t)c.cfg.img_vocab;
             batch.job[2].n_max = b.nnz; batch.job[2].bits = bits_for(c.cfg.img_vocab);
@@ -251,7 +253,7 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
             if (se != cudaSuccess) return cuda_fail(se, "join");
         }
         joined_needed = forked;
-        if (b.nnz > 0) { c.img_sorted = true; c.img_sorted_n = b.nnz; c.img_sorted_buf = sorted_buf; }
+        if (b.nnz > 0) { c.img_sorted = true; c.img_sorted_n = b.nnz; c.img_sorted_buf = sorted_buf; c.last_img_id = b.img_id; }
     }
     cudaError_t e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
     if (e != cudaSuccess) return cuda_fail(e, "gather");
@@ -285,10 +287,11 @@ int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* 
         return GEAR_ERR_STATE;
     }
     if (ld < c.cfg.dfv_dim || ld % 4 || !aligned16(grads)) return arg_fail("grads rows must be 16-byte aligned, ld >= dfv_dim");
-    if (c.cfg.accum_mode != GEAR_ACC_SORT) return arg_fail("accum_mode not available");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
-    cudaError_t e = launch_accumulate(c, img_id, grads, ld, src_row, scale, n, st);
+    cudaError_t e = c.cfg.accum_mode == GEAR_ACC_ATOMIC
+                        ? launch_accumulate_atomic(c, img_id ? img_id : c.last_img_id, grads, ld, src_row, scale, n, st)
+                        : launch_accumulate(c, img_id, grads, ld, src_row, scale, n, st);
     return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "accumulate");
 }
 

@@ -60,6 +60,7 @@ struct gear_ctx_impl {
     mutable Profiler prof;
     mutable GridBarrierState gbs;
     // image IDs of the last gear_forward_backward batch, already sorted (reused by gear_accumulate_dfv_grad)
+    const int32_t* last_img_id;         // img_id array of that batch (the atomic mode reads it unsorted)
     bool img_sorted;
     int64_t img_sorted_n;
     int img_sorted_buf;
@@ -117,6 +118,9 @@ cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int which, int buf, int32_
 // img_id == nullptr: use the image IDs sorted by the last gear_forward_backward (buffer set SORT_IMG)
 cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
                               const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st);
+// GEAR_ACC_ATOMIC: reductions on the accumulator rows, then one settle pass over the touched images
+cudaError_t launch_accumulate_atomic(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
+                                     const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st);
 cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
                                  int64_t* d_n, cudaStream_t st);
 

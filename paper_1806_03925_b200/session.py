@@ -36,7 +36,8 @@ class GearSession:
     def __init__(self, p: GearPreset, head_params: np.ndarray, max_batch: Optional[int] = None,
                  max_nnz: Optional[int] = None, seed: int = 0, fill: bool = True, now: int = 0,
                  tables: Optional[Dict[str, np.ndarray]] = None, ready_cap: int = 0, device: str = "cuda",
-                 want_emb_grad: bool = False, want_debug: bool = False, expired_cap: Optional[int] = None):
+                 want_emb_grad: bool = False, want_debug: bool = False, expired_cap: Optional[int] = None,
+                 accum_mode: int = gb.GEAR_ACC_SORT):
         gb.load()
         self.p = p
         self.dev = torch.device(device)
@@ -47,7 +48,7 @@ class GearSession:
         self.cfg = gb.make_config(p.user_vocab, p.url_vocab, p.img_vocab, p.emb_dim, p.dfv_dim,
                                   gb.GEAR_BF16 if p.dfv_dtype == BF16 else gb.GEAR_F32,
                                   gb.GEAR_BF16 if p.head_dtype == BF16 else gb.GEAR_F32,
-                                  list(p.hidden), p.M, p.expire, self.max_batch, self.max_nnz, ready_cap)
+                                  list(p.hidden), p.M, p.expire, self.max_batch, self.max_nnz, ready_cap, accum_mode)
         dev = self.dev
         if tables is None:
             self.user_emb = torch.empty((p.user_vocab, p.emb_dim), dtype=torch.float32, device=dev)

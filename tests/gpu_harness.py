@@ -82,8 +82,10 @@ class Pair:
     """A GearSession on the GPU and a GearOracle on the CPU over the same problem."""
 
     def __init__(self, p: GearPreset, batches: List[Batch], seed: int = 0, dense: Optional[bool] = None,
-                 now0: int = 0, ready_cap: int = 0, want_emb_grad: bool = False, extra_img_ids=None):
-        self.p, self.seed = p, seed
+                 now0: int = 0, ready_cap: int = 0, want_emb_grad: bool = False, extra_img_ids=None,
+                 atomic: bool = False):
+        # atomic: GEAR_ACC_ATOMIC on the device against the oracle's order-free (pooled) store
+        self.p, self.seed, self.atomic = p, seed, atomic
         if dense is None:
             dense = max(p.user_vocab, p.url_vocab, p.img_vocab) <= 200_000
         cat = lambda k: np.concatenate([getattr(b, k) for b in batches]) if batches else np.zeros(0, np.int32)
@@ -99,7 +101,8 @@ class Pair:
         if extra_img_ids is not None:
             max_nnz = max(max_nnz, len(extra_img_ids))
         self.gpu = GearSession(p, self.params, max_batch=max_b, max_nnz=max_nnz, seed=seed, fill=True, now=now0,
-                               ready_cap=ready_cap, want_emb_grad=want_emb_grad, want_debug=True)
+                               ready_cap=ready_cap, want_emb_grad=want_emb_grad, want_debug=True,
+                               accum_mode=1 if atomic else 0)
         dfv_np = np.uint16 if p.dfv_dtype == BF16 else np.float32
         self.cpu = GearOracle(
             oracle.fill_rows(seed, oracle.TAG_USER, p.emb_dim, self.ru.rows, self.ru.n, np.float32),
@@ -177,7 +180,7 @@ class Pair:
 
         # event 5 + 6
         gpu.accumulate_from_step(db)
-        cpu.accumulate(img, cpu.dfv_grad_rows(b.img_off, r.dX))
+        cpu.accumulate(img, cpu.dfv_grad_rows(b.img_off, r.dX), pooled=self.atomic)
         self.compare_store(check_tables)
         n_ready = self.collect_and_compare()
         n_exp = self.expire_and_compare(now)

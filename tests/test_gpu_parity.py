@@ -87,6 +87,21 @@ def test_skew_config_reduced(gb, M):
         assert out[0]["n_ready"] > 4096
 
 
+@pytest.mark.parametrize("M", [1, 64])
+def test_skew_config_reduced_atomic_mode(gb, M):
+    # GEAR_ACC_ATOMIC under the same contention: counts, emission (id, seq) pairs exact; averages and kept sums
+    # against the oracle's order-free store (the order of the fp32 reductions is the hardware's)
+    p = PRESETS["skew"].scaled(M=M, img_vocab=100_000, user_vocab=100_000, url_vocab=100_000)
+    src = BatchSource(p, 0)
+    batches = [src.batch(s, 4096) for s in range(3)]
+    pair = _pair(p, batches, seed=0, atomic=True)
+    try:
+        out = [pair.step_and_compare(b, now=s + 1) for s, b in enumerate(batches)]
+    finally:
+        pair.close()
+    assert sum(o["n_ready"] for o in out) > 0
+
+
 def test_large_shapes_reduced(gb):
     # large-table head (384-512-256-1, bf16 DFV dim 256, E 64, M 32) on small tables and 1536 views
     p = PRESETS["large"].scaled(user_vocab=80_000, url_vocab=60_000, img_vocab=40_000)
@@ -94,14 +109,14 @@ def test_large_shapes_reduced(gb):
 
 
 # ------------------------------------------------------------------ accumulate-only (micro-benchmark shapes, reduced)
-@pytest.mark.parametrize("zipf_s,M", [(0.0, 8), (1.1, 8), (1.1, 64)])
-def test_accumulate_only_reduced(gb, zipf_s, M):
+@pytest.mark.parametrize("zipf_s,M,atomic", [(0.0, 8, False), (1.1, 8, False), (1.1, 64, False), (1.1, 8, True)])
+def test_accumulate_only_reduced(gb, zipf_s, M, atomic):
     from gpu_harness import assert_close, _np
     V, D, n = 50_000, 128, 200_003
     p = PRESETS["skew"].scaled(img_vocab=V, dfv_dim=D, M=M, user_vocab=16, url_vocab=16, expire=1 << 40)
     mp = workloads.MicroPreset("t", n, V, D, M, zipf_s)
     ids = workloads.micro_ids(mp, seed=3)
-    pair = _pair(p, [], seed=3, dense=True, extra_img_ids=ids, ready_cap=n)
+    pair = _pair(p, [], seed=3, dense=True, extra_img_ids=ids, ready_cap=2 * n, atomic=atomic)
     try:
         g = torch.empty((n, D), dtype=torch.float32, device="cuda")
         gb.gear_fill_uniform(g, seed=3, tag=gb.GEAR_TAG_GRAD, amp=1.0)
@@ -110,7 +125,7 @@ def test_accumulate_only_reduced(gb, zipf_s, M):
         half = n // 2 + 1
         for lo, hi in ((0, half), (half, n)):       # two calls before one collect: emission numbers continue
             pair.gpu.accumulate_rows(ids_t[lo:hi], g[lo:hi])
-            pair.cpu.accumulate(ids[lo:hi], g_cpu[lo:hi])
+            pair.cpu.accumulate(ids[lo:hi], g_cpu[lo:hi], pooled=atomic)
             pair.compare_store()
         n_ready = pair.collect_and_compare()
         k = np.bincount(ids, minlength=V)

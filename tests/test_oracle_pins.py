@@ -434,6 +434,53 @@ def test_M1_emits_every_row_in_order_and_keeps_the_table_empty():
     assert list(orc.collect_ready()[1]) == [0] * 3 or len(set(ids[:3])) < 3
 
 
+def test_pooled_store_conserves_sums_and_matches_the_ordered_store_where_order_cannot_matter():
+    """The order-free store (asynchronous arrivals): same counts and emission counts as the ordered one,
+    M * (sum of averages) + kept sum == pooled sum, every emission of an image is the pooled mean; where an
+    image receives exactly M gradients into an empty store, or identical gradients, both stores agree."""
+    from paper_1806_03925_b200 import workloads
+    M, V, D, n = 4, 200, 6, 3000
+    rng = np.random.default_rng(21)
+    ids = workloads.ZipfIds(V, 1.1).sample(rng, n)
+    g = rng.normal(size=(n, D))
+    mk = lambda: GearOracle(np.zeros((1, 1)), np.zeros((1, 1)), np.zeros((V, D)), (1,), M, 0)
+    a, b = mk(), mk()
+    tot = np.zeros((V, D)); cnt = np.zeros(V, dtype=np.int64)
+    for lo, hi in ((0, 1200), (1200, n)):
+        before_sum, before_cnt = b.gsum.copy(), b.gcnt.copy()
+        a.accumulate(ids[lo:hi], g[lo:hi])
+        b.accumulate(ids[lo:hi], g[lo:hi], pooled=True)
+        assert np.array_equal(a.gcnt, b.gcnt)                       # counts are order-free
+        np.add.at(tot, ids[lo:hi], g[lo:hi]); np.add.at(cnt, ids[lo:hi], 1)
+        # every emission of this call is the mean of what the image held plus what arrived
+        k_call = np.bincount(ids[lo:hi], minlength=V) + before_cnt
+        pooled = before_sum.copy(); np.add.at(pooled, ids[lo:hi], g[lo:hi])
+        new = slice(len(b._emit_id) - int((k_call // M).sum()), len(b._emit_id))
+        for i, avg in zip(b._emit_id[new], b._emit_avg[new]):
+            np.testing.assert_allclose(avg, pooled[i] / k_call[i], atol=1e-12)
+    ea, eb = a.collect_ready(), b.collect_ready()
+    assert np.array_equal(np.bincount(ea[0], minlength=V), np.bincount(eb[0], minlength=V))
+    assert np.array_equal(np.bincount(eb[0], minlength=V), cnt // M)
+    sa, sb = oracle.sort_emissions(*ea), oracle.sort_emissions(*eb)
+    assert np.array_equal(sa[0], sb[0]) and np.array_equal(sa[1], sb[1])    # same (id, seq) pairs
+    emitted = np.zeros((V, D)); np.add.at(emitted, eb[0], M * eb[2])
+    np.testing.assert_allclose(emitted + b.gsum, tot, atol=1e-10)           # nothing lost, nothing counted twice
+    # exactly M gradients into an empty store: one group either way
+    c, d = mk(), mk()
+    ids2 = np.repeat(np.arange(5, dtype=np.int32), M); g2 = rng.normal(size=(5 * M, D))
+    perm = rng.permutation(5 * M)
+    c.accumulate(ids2[perm], g2[perm]); d.accumulate(ids2[perm], g2[perm], pooled=True)
+    sc, sd = oracle.sort_emissions(*c.collect_ready()), oracle.sort_emissions(*d.collect_ready())
+    np.testing.assert_allclose(sc[2], sd[2], atol=1e-12)
+    assert not d.gcnt.any() and np.abs(d.gsum).max() == 0.0
+    # identical gradients: any grouping gives the same averages and residual
+    e, f = mk(), mk()
+    ids3 = np.zeros(11, dtype=np.int32); g3 = np.tile(rng.normal(size=(1, D)), (11, 1))
+    e.accumulate(ids3, g3); f.accumulate(ids3, g3, pooled=True)
+    np.testing.assert_allclose(e.gsum, f.gsum, atol=1e-12)
+    np.testing.assert_allclose(e.collect_ready()[2], f.collect_ready()[2], atol=1e-12)
+
+
 def test_bad_image_ids_are_ignored_by_accumulate():
     orc = GearOracle(np.zeros((1, 1)), np.zeros((1, 1)), np.zeros((3, 2)), (1,), 2, 0)
     bad = orc.accumulate(np.array([0, 7, -1, 0], dtype=np.int32), np.ones((4, 2)))
