@@ -603,7 +603,9 @@ collect_keys_kernel(const int32_t* __restrict__ q_id, const DevState* __restrict
         keys[i] = (uint32_t)q_id[i];
 }
 
-// One warp per output entry k: queue slot perm[k]; its emission number is its rank among equal IDs.
+// Output entry k comes from queue slot perm[k] (or k itself when the queue is already in order); its emission
+// number is its rank among equal IDs.  IDs and emission numbers: one thread per entry.  Rows: a warp copies
+// eight rows at a time, 16 bytes per lane, all loads issued before the first store.
 __global__ void __launch_bounds__(256)
 collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __restrict__ sorted_perm,
                     const int32_t* __restrict__ q_id, const float* __restrict__ q_avg,
@@ -612,9 +614,8 @@ collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __
     const int64_t n = state->collect_n;
     const bool in_order = state->sort_n == 0;          // the queue itself is sorted: no permutation
     const uint32_t* ks = in_order ? reinterpret_cast<const uint32_t*>(q_id) : sorted_keys;
-    const unsigned lane = lane_id();
-    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    for (int64_t k = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); k < n; k += warps) {
+    const int64_t threads = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n; k += threads) {
         const uint32_t id = ks[k];
         // first index of this ID's run: gallop backwards, then bisect
         int64_t hi = k, step = 1, lo = k - 1;                  // ks[hi] == id
@@ -624,10 +625,29 @@ collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __
             const int64_t mid = (l + h) >> 1;
             if (ks[mid] == id) h = mid; else l = mid + 1;
         }
-        const float* src = q_avg + (in_order ? k : (int64_t)sorted_perm[k]) * D;
-        float* dst = avg + k * D;
-        for (int ch = lane; ch < D / 4; ch += 32) st_f4(dst + ch * 4, ld_f4(src + ch * 4));
-        if (lane == 0) { ids[k] = (int32_t)id; seq[k] = (int32_t)(k - l); }
+        ids[k] = (int32_t)id;
+        seq[k] = (int32_t)(k - l);
+    }
+    const unsigned lane = lane_id();
+    const int64_t warps = threads >> 5;
+    const int chunks = D / 4;
+    constexpr int R = 8;
+    for (int64_t k0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; k0 < n; k0 += R * warps) {
+        int64_t src[R];
+#pragma unroll
+        for (int t = 0; t < R; ++t) {
+            const int64_t k = k0 + t * warps;
+            src[t] = k < n ? (in_order ? k : (int64_t)sorted_perm[k]) : -1;
+        }
+        for (int ch = lane; ch < chunks; ch += 32) {
+            float4 v[R];
+#pragma unroll
+            for (int t = 0; t < R; ++t)
+                v[t] = src[t] >= 0 ? ld_stream_f4(q_avg + src[t] * D + ch * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int t = 0; t < R; ++t)
+                if (src[t] >= 0) st_f4(avg + (k0 + t * warps) * D + ch * 4, v[t]);
+        }
     }
 }
 

@@ -239,7 +239,7 @@ static int coop_grid_limit() {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, coop_sort_kernel, RS_THREADS, 0);
         if (sms <= 0) sms = 148;
         if (per_sm <= 0) per_sm = 1;
-        if (per_sm > 2) per_sm = 2;
+        if (per_sm > 3) per_sm = 3;
         limit = sms * per_sm;
     }
     return limit;
