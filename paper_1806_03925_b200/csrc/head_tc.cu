@@ -31,6 +31,8 @@ constexpr int TC_BK = 64;                 // 64 bf16 = 128 bytes = one swizzle r
 constexpr int TC_EPI_WARPS = 8;
 constexpr int TC_THREADS = 64 + 32 * TC_EPI_WARPS;
 constexpr int TC_MAX_N = 1024;            // widest output the column-sum partials cover
+constexpr int TC_STAGE_PITCH = 80;        // bytes between rows of a warp's store-staging block (64 of data + 16 of padding)
+constexpr int TC_STAGE_BYTES = 32 * TC_STAGE_PITCH;
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
 enum { TC_EPI_BIAS_RELU = 0, TC_EPI_MASK = 1, TC_EPI_F32 = 2, TC_EPI_RED = 3 };
@@ -41,7 +43,7 @@ template <int BN> struct TcCfg {
     static constexpr int B_BYTES = BN * TC_BK * 2;               // 32 KB or 16 KB
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
-                                TC_MAX_N * 4 /*column sums*/;
+                                TC_MAX_N * 4 /*column sums*/ + TC_EPI_WARPS * TC_STAGE_BYTES /*store staging*/;
     static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
     static_assert(SMEM > 116 * 1024, "one CTA per SM: two CTAs would both ask for tensor memory");
     static_assert(SMEM <= 227 * 1024, "shared memory budget");
@@ -129,6 +131,33 @@ __device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[32]) {
 __device__ __forceinline__ float4 ldg_f4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ uint4 ldg_u4(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
+// Coalesced store of a 32-row x 64-byte block of which lane l holds row l.  A thread of the epilogue owns a row of
+// the accumulator, so storing straight from registers would touch 32 rows per instruction, 16 bytes each; the
+// block goes through a padded shared-memory buffer instead (conflict-free 128-bit writes) and leaves as 64-byte
+// row segments, eight rows per instruction.  rows / pieces: how many rows and 16-byte pieces of the block exist.
+template <bool KEEP_IN_L2>
+__device__ __forceinline__ void store_block_64B(uint4* stage, const uint4 (&v)[4], char* gdst, int64_t row_pitch, int rows,
+                                                int pieces, int lane, uint64_t policy) {
+    constexpr int P = TC_STAGE_PITCH / 16;
+    __syncwarp();                                           // the previous block has left the buffer
+#pragma unroll
+    for (int j = 0; j < 4; ++j) stage[lane * P + j] = v[j];
+    __syncwarp();
+    const int piece = lane & 3;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int row = it * 8 + (lane >> 2);
+        const uint4 x = stage[row * P + piece];
+        if (row < rows && piece < pieces) {
+            char* dst = gdst + (int64_t)row * row_pitch + piece * 16;
+            if (KEEP_IN_L2)
+                asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1,%2,%3,%4}, %5;"
+                             :: "l"(dst), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w), "l"(policy) : "memory");
+            else *reinterpret_cast<uint4*>(dst) = x;
+        }
+    }
+}
+
 // v[i] of lane l is element (row l, column i) of a 32 x 32 block.  Returns, on lane l, the sum of column l.
 __device__ __forceinline__ float column_sums_32x32(float (&v)[32], int lane) {
 #pragma unroll
@@ -164,8 +193,10 @@ __host__ __device__ constexpr uint32_t instr_desc(int bn, bool mn_major) {
 }
 
 // ---------------------------------------------------------------- the kernel
+// At most 128 registers per thread: a CTA (320 threads) then fits on an SM beside a block of the ID sort, which
+// runs on a side stream while the head starts.  One CTA per SM follows from the shared-memory footprint.
 template <int BN, bool MN_MAJOR, int EPI>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __maxnreg__(128)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs g) {
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
@@ -181,6 +212,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     volatile uint32_t* tmem_word_ptr =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_word - raw));
     float* s_colsum = reinterpret_cast<float*>(smem_raw + (bars + 256u - raw));     // [TC_MAX_N] per-CTA column sums
+    uint4* s_stage = reinterpret_cast<uint4*>(smem_raw + (bars + 256u + TC_MAX_N * 4u - raw));   // [TC_EPI_WARPS] store staging
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles * g.k_splits;
@@ -289,8 +321,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int a = tile_it & 1;
             if (!(ok = mbar_wait(acc_full(a), (tile_it >> 1) & 1u, g.err, 4))) break;
             tc_fence_after();
-            const int m = mt * TC_BM + quarter * 32 + lane;
+            const int m0 = mt * TC_BM + quarter * 32;         // first row of this warp's block
+            const int m = m0 + lane;
             const bool row_ok = m < g.M;
+            const int rows = min(32, max(0, g.M - m0));
+            uint4* stage = s_stage + (warp - 2) * (TC_STAGE_BYTES / 16);
             const int col0 = nt * BN + half * (BN / 2);
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN + half * (BN / 2));
             uint32_t r[2][32];
@@ -348,12 +383,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
                         pk[q] = *reinterpret_cast<uint32_t*>(&h2);
                     }
-                    if (row_ok) {
-                        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(g.out) + (int64_t)m * g.ldo + n0;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            if (n0 + 8 * j < g.N)
-                                *reinterpret_cast<uint4*>(dst + 8 * j) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                    {
+                        const uint4 blk[4] = {make_uint4(pk[0], pk[1], pk[2], pk[3]), make_uint4(pk[4], pk[5], pk[6], pk[7]),
+                                              make_uint4(pk[8], pk[9], pk[10], pk[11]), make_uint4(pk[12], pk[13], pk[14], pk[15])};
+                        char* dst = reinterpret_cast<char*>(static_cast<__nv_bfloat16*>(g.out) + (int64_t)m0 * g.ldo + n0);
+                        store_block_64B<false>(stage, blk, dst, g.ldo * 2, rows, min(4, (g.N - n0) / 8), lane, 0ull);
                     }
                     if (EPI == TC_EPI_MASK && g.colsum != nullptr) {
                         // column sums of what was stored (the rounded values); rows past M and columns past N are zero
@@ -365,15 +399,27 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const float cs = column_sums_32x32(v, lane);
                         if (n0 + lane < g.N) atomicAdd(&s_colsum[n0 + lane], cs);
                     }
-                } else if (row_ok) {
-                    float* dst = static_cast<float*>(g.out) + (int64_t)m * g.ldo + n0;
+                } else if (EPI == TC_EPI_RED) {
+                    if (row_ok) {
+                        float* dst = static_cast<float*>(g.out) + (int64_t)m * g.ldo + n0;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (n0 + 4 * j >= g.N) continue;
-                        const float4 v4 = make_float4(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1]),
-                                                      __uint_as_float(acc[4 * j + 2]), __uint_as_float(acc[4 * j + 3]));
-                        if (EPI == TC_EPI_RED) red_add_f4(dst + 4 * j, v4);
-                        else st_f4_hint(dst + 4 * j, v4, keep_policy);      // dX is read again right after: keep it in the L2
+                        for (int j = 0; j < 8; ++j) {
+                            if (n0 + 4 * j >= g.N) continue;
+                            red_add_f4(dst + 4 * j, make_float4(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1]),
+                                                                __uint_as_float(acc[4 * j + 2]), __uint_as_float(acc[4 * j + 3])));
+                        }
+                    }
+                } else {
+                    // fp32 output (dX), two 16-column halves; it is read again right after: keep it in the L2
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint4 blk[4] = {make_uint4(acc[16 * h + 0], acc[16 * h + 1], acc[16 * h + 2], acc[16 * h + 3]),
+                                              make_uint4(acc[16 * h + 4], acc[16 * h + 5], acc[16 * h + 6], acc[16 * h + 7]),
+                                              make_uint4(acc[16 * h + 8], acc[16 * h + 9], acc[16 * h + 10], acc[16 * h + 11]),
+                                              make_uint4(acc[16 * h + 12], acc[16 * h + 13], acc[16 * h + 14], acc[16 * h + 15])};
+                        char* dst = reinterpret_cast<char*>(static_cast<float*>(g.out) + (int64_t)m0 * g.ldo + n0 + 16 * h);
+                        store_block_64B<true>(stage, blk, dst, g.ldo * 4, rows, min(4, max(0, (g.N - n0 - 16 * h) / 4)), lane,
+                                              keep_policy);
                     }
                 }
             }
