@@ -71,6 +71,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
 }
+// Arrival that orders nothing but the barrier itself: the epilogue hands its accumulator buffer back with this one,
+// so that the hand-over does not wait for the tile's global stores to drain (tensor-memory reads are complete by
+// then: tcgen05.wait::ld, then tcgen05.fence::before_thread_sync).
+__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar) {
+    asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile("{\n\t.reg .pred p;\n\t"
@@ -192,6 +198,133 @@ __host__ __device__ constexpr uint32_t instr_desc(int bn, bool mn_major) {
            ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
+// Epilogue of one finished accumulator buffer `a`, as run by one of the eight epilogue warps: warp w reads
+// tensor-memory lanes 32 * (w % 4) .. + 31 (its rows of the tile); warps 2..5 take the first half of the tile's
+// columns, warps 6..9 the second half.
+template <int BN, int EPI>
+__device__ __forceinline__ void epilogue_tile(const TcArgs& g, uint32_t tmem_base, int a, int mt, int nt, int warp, int lane,
+                                              float* s_colsum, uint4* s_stage, uint64_t keep_policy) {
+    const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
+    constexpr int CHUNKS = BN / 64;                       // 32-column chunks per warp and tile
+    const int m0 = mt * TC_BM + quarter * 32;         // first row of this warp's block
+    const int m = m0 + lane;
+    const bool row_ok = m < g.M;
+    const int rows = min(32, max(0, g.M - m0));
+    uint4* stage = s_stage + (warp - 2) * (TC_STAGE_BYTES / 16);
+    const int col0 = nt * BN + half * (BN / 2);
+    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN + half * (BN / 2));
+    uint32_t r[2][32];
+    tc_ld32(t_row, r[0]);
+#pragma unroll
+    for (int c = 0; c < CHUNKS; ++c) {
+        const int n0 = col0 + c * 32;
+        const bool chunk_ok = n0 < g.N;               // warp-uniform; N is a multiple of 8
+        // what this chunk's epilogue reads from memory, requested while the tensor-memory read is in flight
+        float4 bias4[EPI == TC_EPI_BIAS_RELU ? 8 : 1];
+        uint4 mask4[EPI == TC_EPI_MASK ? 4 : 1];
+        if (EPI == TC_EPI_BIAS_RELU) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                bias4[j] = (n0 + 4 * j < g.N) ? ldg_f4(g.bias + n0 + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (EPI == TC_EPI_MASK) {
+            // the 32 x 64-byte block of the mask, fetched as 64-byte row segments (eight rows per instruction);
+            // each lane picks up its own row from the staging buffer once the loads have landed
+            const int piece = lane & 3;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int row = j * 8 + (lane >> 2);
+                mask4[j] = (row < rows && n0 + 8 * piece < g.N)
+                               ? ldg_u4(g.mask + (int64_t)(m0 + row) * g.ldm + n0 + 8 * piece) : make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        tc_wait_ld(r[c & 1]);
+        if (c + 1 < CHUNKS) tc_ld32(t_row + (uint32_t)((c + 1) * 32), r[(c + 1) & 1]);
+        if (!chunk_ok) continue;
+        if (EPI == TC_EPI_MASK) {
+            constexpr int P = TC_STAGE_PITCH / 16;
+            __syncwarp();                               // the previous block has left the buffer
+#pragma unroll
+            for (int j = 0; j < 4; ++j) stage[(j * 8 + (lane >> 2)) * P + (lane & 3)] = mask4[j];
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) mask4[j] = stage[lane * P + j];
+        }
+        uint32_t (&acc)[32] = r[c & 1];
+        if (EPI == TC_EPI_BIAS_RELU || EPI == TC_EPI_MASK) {
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
+            if (EPI == TC_EPI_BIAS_RELU) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    v[4 * j + 0] = fmaxf(v[4 * j + 0] + bias4[j].x, 0.f);
+                    v[4 * j + 1] = fmaxf(v[4 * j + 1] + bias4[j].y, 0.f);
+                    v[4 * j + 2] = fmaxf(v[4 * j + 2] + bias4[j].z, 0.f);
+                    v[4 * j + 3] = fmaxf(v[4 * j + 3] + bias4[j].w, 0.f);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t w[4] = {mask4[j].x, mask4[j].y, mask4[j].z, mask4[j].w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        // a post-ReLU activation is > 0 exactly when its bf16 pattern is non-zero and positive: with the
+                        // pattern in the top half of a word, that word is then at least 0x00010000 as a signed integer
+                        if ((int32_t)(w[q] << 16) < 0x10000) v[8 * j + 2 * q] = 0.f;
+                        if ((int32_t)w[q] < 0x10000) v[8 * j + 2 * q + 1] = 0.f;
+                    }
+                }
+            }
+            uint32_t pk[16];
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+                pk[q] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            {
+                const uint4 blk[4] = {make_uint4(pk[0], pk[1], pk[2], pk[3]), make_uint4(pk[4], pk[5], pk[6], pk[7]),
+                                      make_uint4(pk[8], pk[9], pk[10], pk[11]), make_uint4(pk[12], pk[13], pk[14], pk[15])};
+                char* dst = reinterpret_cast<char*>(static_cast<__nv_bfloat16*>(g.out) + (int64_t)m0 * g.ldo + n0);
+                store_block_64B<false>(stage, blk, dst, g.ldo * 2, rows, min(4, (g.N - n0) / 8), lane, 0ull);
+            }
+            if (EPI == TC_EPI_MASK && g.colsum != nullptr) {
+                // column sums of what was stored (the rounded values); rows past M and columns past N are zero
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    v[2 * q] = row_ok ? __uint_as_float(pk[q] << 16) : 0.f;
+                    v[2 * q + 1] = row_ok ? __uint_as_float(pk[q] & 0xffff0000u) : 0.f;
+                }
+                const float cs = column_sums_32x32(v, lane);
+                if (n0 + lane < g.N) atomicAdd(&s_colsum[n0 + lane], cs);
+            }
+        } else if (EPI == TC_EPI_RED) {
+            if (row_ok) {
+                float* dst = static_cast<float*>(g.out) + (int64_t)m * g.ldo + n0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (n0 + 4 * j >= g.N) continue;
+                    red_add_f4(dst + 4 * j, make_float4(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1]),
+                                                        __uint_as_float(acc[4 * j + 2]), __uint_as_float(acc[4 * j + 3])));
+                }
+            }
+        } else {
+            // fp32 output (dX), two 16-column halves; it is read again right after: keep it in the L2
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint4 blk[4] = {make_uint4(acc[16 * h + 0], acc[16 * h + 1], acc[16 * h + 2], acc[16 * h + 3]),
+                                      make_uint4(acc[16 * h + 4], acc[16 * h + 5], acc[16 * h + 6], acc[16 * h + 7]),
+                                      make_uint4(acc[16 * h + 8], acc[16 * h + 9], acc[16 * h + 10], acc[16 * h + 11]),
+                                      make_uint4(acc[16 * h + 12], acc[16 * h + 13], acc[16 * h + 14], acc[16 * h + 15])};
+                char* dst = reinterpret_cast<char*>(static_cast<float*>(g.out) + (int64_t)m0 * g.ldo + n0 + 16 * h);
+                store_block_64B<true>(stage, blk, dst, g.ldo * 4, rows, min(4, max(0, (g.N - n0 - 16 * h) / 4)), lane,
+                                      keep_policy);
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------- the kernel
 // At most 128 registers per thread: a CTA (320 threads) then fits on an SM beside a block of the ID sort, which
 // runs on a side stream while the head starts.  One CTA per SM follows from the shared-memory footprint.
@@ -308,123 +441,27 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     } else {
-        // ---------------- epilogue: warp w reads tensor-memory lanes 32 * (w % 4) .. + 31 (its rows of the tile);
-        // warps 2..5 take the first half of the tile's columns, warps 6..9 the second half
-        const int quarter = warp & 3;
-        const int half = (warp - 2) >> 2;
+        // ---------------- epilogue warps
         const uint64_t keep_policy = l2_policy_evict_last();
-        constexpr int CHUNKS = BN / 64;                       // 32-column chunks per warp and tile
         uint32_t tile_it = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
             const int mt = t % g.m_tiles, nt = (t / g.m_tiles) % g.n_tiles;
             const int a = tile_it & 1;
+            if (EPI == TC_EPI_MASK) {
+                // the rows of the ReLU mask this warp will need: ask the L2 for them now, the wait below covers the trip
+                const int m = mt * TC_BM + (warp & 3) * 32 + lane, c0 = nt * BN + ((warp - 2) >> 2) * (BN / 2);
+                if (m < g.M)
+#pragma unroll
+                    for (int c = 0; c < BN / 2; c += 64)           // one 128-byte line per 64 bf16 columns
+                        if (c0 + c < g.N)
+                            asm volatile("prefetch.global.L2 [%0];" :: "l"(g.mask + (int64_t)m * g.ldm + c0 + c));
+            }
             if (!(ok = mbar_wait(acc_full(a), (tile_it >> 1) & 1u, g.err, 4))) break;
             tc_fence_after();
-            const int m0 = mt * TC_BM + quarter * 32;         // first row of this warp's block
-            const int m = m0 + lane;
-            const bool row_ok = m < g.M;
-            const int rows = min(32, max(0, g.M - m0));
-            uint4* stage = s_stage + (warp - 2) * (TC_STAGE_BYTES / 16);
-            const int col0 = nt * BN + half * (BN / 2);
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN + half * (BN / 2));
-            uint32_t r[2][32];
-            tc_ld32(t_row, r[0]);
-#pragma unroll
-            for (int c = 0; c < CHUNKS; ++c) {
-                const int n0 = col0 + c * 32;
-                const bool chunk_ok = n0 < g.N;               // warp-uniform; N is a multiple of 8
-                // what this chunk's epilogue reads from memory, requested while the tensor-memory read is in flight
-                float4 bias4[EPI == TC_EPI_BIAS_RELU ? 8 : 1];
-                uint4 mask4[EPI == TC_EPI_MASK ? 4 : 1];
-                if (EPI == TC_EPI_BIAS_RELU) {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        bias4[j] = (n0 + 4 * j < g.N) ? ldg_f4(g.bias + n0 + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-                if (EPI == TC_EPI_MASK) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        mask4[j] = (row_ok && n0 + 8 * j < g.N) ? ldg_u4(g.mask + (int64_t)m * g.ldm + n0 + 8 * j)
-                                                                : make_uint4(0u, 0u, 0u, 0u);
-                }
-                tc_wait_ld(r[c & 1]);
-                if (c + 1 < CHUNKS) tc_ld32(t_row + (uint32_t)((c + 1) * 32), r[(c + 1) & 1]);
-                if (!chunk_ok) continue;
-                uint32_t (&acc)[32] = r[c & 1];
-                if (EPI == TC_EPI_BIAS_RELU || EPI == TC_EPI_MASK) {
-                    float v[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
-                    if (EPI == TC_EPI_BIAS_RELU) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            v[4 * j + 0] = fmaxf(v[4 * j + 0] + bias4[j].x, 0.f);
-                            v[4 * j + 1] = fmaxf(v[4 * j + 1] + bias4[j].y, 0.f);
-                            v[4 * j + 2] = fmaxf(v[4 * j + 2] + bias4[j].z, 0.f);
-                            v[4 * j + 3] = fmaxf(v[4 * j + 3] + bias4[j].w, 0.f);
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t w[4] = {mask4[j].x, mask4[j].y, mask4[j].z, mask4[j].w};
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                // a post-ReLU activation is > 0 exactly when its bf16 pattern is non-zero and positive
-                                const uint32_t lo = w[q] & 0xffffu, hi = w[q] >> 16;
-                                if (!(lo != 0u && lo < 0x8000u)) v[8 * j + 2 * q] = 0.f;
-                                if (!(hi != 0u && hi < 0x8000u)) v[8 * j + 2 * q + 1] = 0.f;
-                            }
-                        }
-                    }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int q = 0; q < 16; ++q) {
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
-                        pk[q] = *reinterpret_cast<uint32_t*>(&h2);
-                    }
-                    {
-                        const uint4 blk[4] = {make_uint4(pk[0], pk[1], pk[2], pk[3]), make_uint4(pk[4], pk[5], pk[6], pk[7]),
-                                              make_uint4(pk[8], pk[9], pk[10], pk[11]), make_uint4(pk[12], pk[13], pk[14], pk[15])};
-                        char* dst = reinterpret_cast<char*>(static_cast<__nv_bfloat16*>(g.out) + (int64_t)m0 * g.ldo + n0);
-                        store_block_64B<false>(stage, blk, dst, g.ldo * 2, rows, min(4, (g.N - n0) / 8), lane, 0ull);
-                    }
-                    if (EPI == TC_EPI_MASK && g.colsum != nullptr) {
-                        // column sums of what was stored (the rounded values); rows past M and columns past N are zero
-#pragma unroll
-                        for (int q = 0; q < 16; ++q) {
-                            v[2 * q] = row_ok ? __uint_as_float(pk[q] << 16) : 0.f;
-                            v[2 * q + 1] = row_ok ? __uint_as_float(pk[q] & 0xffff0000u) : 0.f;
-                        }
-                        const float cs = column_sums_32x32(v, lane);
-                        if (n0 + lane < g.N) atomicAdd(&s_colsum[n0 + lane], cs);
-                    }
-                } else if (EPI == TC_EPI_RED) {
-                    if (row_ok) {
-                        float* dst = static_cast<float*>(g.out) + (int64_t)m * g.ldo + n0;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            if (n0 + 4 * j >= g.N) continue;
-                            red_add_f4(dst + 4 * j, make_float4(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1]),
-                                                                __uint_as_float(acc[4 * j + 2]), __uint_as_float(acc[4 * j + 3])));
-                        }
-                    }
-                } else {
-                    // fp32 output (dX), two 16-column halves; it is read again right after: keep it in the L2
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint4 blk[4] = {make_uint4(acc[16 * h + 0], acc[16 * h + 1], acc[16 * h + 2], acc[16 * h + 3]),
-                                              make_uint4(acc[16 * h + 4], acc[16 * h + 5], acc[16 * h + 6], acc[16 * h + 7]),
-                                              make_uint4(acc[16 * h + 8], acc[16 * h + 9], acc[16 * h + 10], acc[16 * h + 11]),
-                                              make_uint4(acc[16 * h + 12], acc[16 * h + 13], acc[16 * h + 14], acc[16 * h + 15])};
-                        char* dst = reinterpret_cast<char*>(static_cast<float*>(g.out) + (int64_t)m0 * g.ldo + n0 + 16 * h);
-                        store_block_64B<true>(stage, blk, dst, g.ldo * 4, rows, min(4, max(0, (g.N - n0 - 16 * h) / 4)), lane,
-                                              keep_policy);
-                    }
-                }
-            }
+            epilogue_tile<BN, EPI>(g, tmem_base, a, mt, nt, warp, lane, s_colsum, s_stage, keep_policy);
             tc_fence_before();
-            mbar_arrive(acc_empty(a));                   // all epilogue threads arrive: the buffer returns to the MMA warp
+            mbar_arrive_relaxed(acc_empty(a));                   // all epilogue threads arrive: the buffer returns to the MMA warp
         }
     }
 
