@@ -138,6 +138,36 @@ def kernel_models(p, stats):
     return m
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu --set full captures summarised under
+# profiles/, taken on the large_2m workload (same batch and head, 4.6 GB of tables; a full-set capture of the 48.9 GB
+# workload would save and restore tens of GB per pass).  Second entry: what the figure scales with when the bench
+# runs another workload -- "work" = the kernel's algorithmic bytes (table-bound kernels: traffic grows with the rows
+# touched), "vocab" = image vocabulary, None = same shapes, taken as is.  ncu flushes the L2 before every pass, so
+# re-reads that hit the L2 in a real step count as DRAM traffic here.  A kernel that has changed since its capture
+# must be taken out of this table (traffic is then reported as null).
+NCU_TRAFFIC_LARGE_2M = {
+    "gather_pool": (64.7e6, "work"), "acc_reduce": (236.8e6, "work"), "expiry_mark": (16.0e6, "vocab"),
+    "emb_reduce": (23.6e6, "work"), "head_out": (34.4e6, None), "collect_move": (5.9e6, "work"),
+    "tc_gemm_fwd": (81.4e6, None), "tc_gemm_dw": (114.4e6, None), "tc_gemm_dh": (150.8e6, None), "tc_gemm_dx": (192.6e6, None),
+}
+# algorithmic bytes per launch of the table-bound kernels on large_2m (kernel_models on that workload's batches)
+NCU_WORK_LARGE_2M = {"gather_pool": 221.8e6, "acc_reduce": 226.4e6, "emb_reduce": 29.6e6, "collect_move": 18.0e6}
+
+
+def ncu_traffic(name, p, work):
+    """DRAM traffic per launch of kernel `name` on workload p, scaled from the large_2m capture; None if unknown."""
+    if name not in NCU_TRAFFIC_LARGE_2M or not p.name.startswith("large"):
+        return None
+    bytes_2m, scales_with = NCU_TRAFFIC_LARGE_2M[name]
+    if scales_with == "vocab":
+        return round(bytes_2m * p.img_vocab / 2_000_000)
+    if scales_with == "work":
+        if not work or name not in NCU_WORK_LARGE_2M:
+            return None
+        return round(bytes_2m * work / NCU_WORK_LARGE_2M[name])
+    return round(bytes_2m)
+
+
 def roofline_for(name, ms_per_launch, p, stats, peaks):
     """Roofline object of one kernel from its live per-launch time."""
     models = kernel_models(p, stats)
@@ -149,8 +179,8 @@ def roofline_for(name, ms_per_launch, p, stats, peaks):
         work = models[name][1]
         ach = work / sec / 1e9
         return {"kernel": name, "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": None, "peak_source": peaks["source"],
-                "work_per_launch": work}
+                "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": ncu_traffic(name, p, work),
+                "peak_source": peaks["source"], "work_per_launch": work}
     if name.startswith("simt_gemm") or name.startswith("tc_gemm"):
         # launches of one name share the step's products of that kind evenly
         per_launch = gemm_flops_fwd / max(len(p.hidden), 1)
@@ -162,7 +192,8 @@ def roofline_for(name, ms_per_launch, p, stats, peaks):
         else:
             peak, bound = ALU_F32_TFLOPS, "alu"
         return {"kernel": name, "bound": bound, "achieved": round(ach, 2), "peak": round(peak, 1), "unit": "TFLOP/s",
-                "frac": round(ach / peak, 4), "traffic": None, "peak_source": peaks["source"] if bound == "tensor"
+                "frac": round(ach / peak, 4), "traffic": ncu_traffic(name, p, None) if bound == "tensor" else None,
+                "peak_source": peaks["source"] if bound == "tensor"
                 else "148 SMs x 128 FMA lanes x 2 x 1.965 GHz", "work_per_launch": per_launch}
     return {"kernel": name, "bound": "latency", "achieved": None, "peak": None, "unit": None, "frac": None,
             "traffic": None}
@@ -246,26 +277,24 @@ def run_reference(args):
 # ---------------------------------------------------------------------------------------------
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     from paper_1806_03925_b200 import binding as gb
+    from paper_1806_03925_b200.replicas import Replicas
     from paper_1806_03925_b200 import workloads
     from paper_1806_03925_b200.session import DeviceBatch, GearSession
     from paper_1806_03925_b200.workloads import BatchSource
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    reps = Replicas.from_env()
+    rank, world, local = reps.rank, reps.world, reps.local_rank
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: libgear has no CPU path")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    reps.init("nccl", torch.device("cuda", local))
     gb.load()
     p = preset_for(args.workload)
     K, W = args.steps, args.warmup
     sampler = ClockSampler(local)          # started early: nvidia-smi needs a moment before its first line
     sampler.start()
-    seed = rank                                   # every replica draws its own tables and batches
+    seed = reps.seed                              # every replica draws its own tables and batches
     src = BatchSource(p, seed)
     host_batches = [src.batch(s) for s in range(N_BATCHES)]
     max_nnz = max(b.nnz for b in host_batches)
@@ -288,8 +317,7 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        reps.barrier()
         torch.cuda.synchronize()
 
     def timed(fn, steps):
@@ -300,12 +328,7 @@ def run_ours(args):
             fn(s)
         ev1.record(stream)
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return reps.max_over_ranks(ev0.elapsed_time(ev1), device="cuda")
 
     # ---- device-resident throughput (clock samples count from here to the end of the end-to-end pass:
     #      every region in between runs the same step under load)
@@ -377,8 +400,7 @@ def run_ours(args):
             hbm_kernels.append({"kernel": kd["name"], "GB/s": r["achieved"], "frac_of_measured": r["frac"],
                                 "frac_of_8TBs": round(r["achieved"] / 8000.0, 4), "ms": round(kd["ms_per_launch"], 4)})
 
-    views = p.batch * K * world
-    line = {"metric": METRIC, "value": round(views / (ms * 1e-3), 1), "unit": UNIT, "n_gpus": world, "steps": K,
+    line = {"metric": METRIC, "value": round(reps.whole_job_rate(p.batch * K, ms), 1), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if p.head_dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": "large tables" if p.name == "large" else p.name, "batch": p.batch,
@@ -389,7 +411,7 @@ def run_ours(args):
                              "no explicit flush" % N_BATCHES,
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks,
-            "e2e": {"value": round(views / (ms_e2e * 1e-3), 1), "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,
+            "e2e": {"value": round(reps.whole_job_rate(p.batch * K, ms_e2e), 1), "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,
                     "d2h_bytes_per_step": d2h_bytes, "ms_per_step": round(ms_e2e / K, 4)},
             "gpu_launches": int(launches),
             "roofline": roof,
@@ -406,8 +428,7 @@ def run_ours(args):
             line["cpu_baseline"] = None
         print(json.dumps(line), flush=True)
     sess.close()
-    if world > 1:
-        dist.destroy_process_group()
+    reps.close()
 
 
 def main():
