@@ -208,9 +208,10 @@ struct LaneGroup {
     bool first;
 };
 
-// One row to stage: accumulator row `idx` of the table, or gradient row `idx` scaled by `scale`.
-// meta = group lane << 3 | accumulator row << 2 | last item of the group << 1 | last of the group's own rows.
-struct ItemDesc { int idx; float scale; int meta; };
+// One row to stage, as the copy side sees it (where the row starts; bit 0 of the address word is set if the item
+// exists) and as the adding side sees it (what the row is scaled by and
+// meta = group lane << 2 | last item of the group << 1 | last of the group's own rows).
+struct ItemDesc { uint32_t addr_lo, addr_hi; float scale; int meta; };
 
 // The reduce pass.  A warp takes spans of ACC_SPAN sorted positions, span w, w + W, w + 2W, ... (W = warps of
 // the grid); the groups that start inside a span (at most ACC_SPAN, one per lane) are walked as one flat
@@ -227,7 +228,7 @@ struct ItemDesc { int idx; float scale; int meta; };
 // streams.  Sums are fp32, in arrival order, starting from the stored partial sum.
 // FULL: a row is exactly NQ * 512 bytes, so no lane is ever idle.
 template <int NQ, int S, bool FULL>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(256, NQ <= 2 ? 3 : 2)
 acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, int64_t n_tiles, int64_t ready_cap,
                   const uint2* __restrict__ tile_cnt, const uint4* __restrict__ grp_rec,
                   const uint32_t* __restrict__ blk_first, const uint32_t* __restrict__ run_end,
@@ -310,10 +311,12 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                 const int64_t p = k < own_end ? (int64_t)start_l + (k - tab) : (int64_t)zstart_l + (k - own_end);
                 int2 pm = make_int2(0, __float_as_int(1.f));
                 if (ok && !is_tab) pm = __ldg(rg.pmeta + p);
+                const float* row = (ok && is_tab) ? gsum + (int64_t)key_l * D : rg.grads + (int64_t)pm.x * rg.ld;
+                const uint64_t a = reinterpret_cast<uint64_t>(row) | (ok ? 1ull : 0ull);      // rows are 16-byte aligned
                 ItemDesc d;
-                d.idx = (ok && is_tab) ? (int)key_l : pm.x;
+                d.addr_lo = (uint32_t)a; d.addr_hi = (uint32_t)(a >> 32);
                 d.scale = __int_as_float(pm.y);
-                d.meta = (l << 3) | (is_tab ? 4 : 0) | (k + 1 == items_l ? 2 : 0) | (k + 1 == own_end ? 1 : 0);
+                d.meta = (l << 2) | (k + 1 == items_l ? 2 : 0) | (k + 1 == own_end ? 1 : 0);
                 return d;
             };
 
@@ -356,17 +359,17 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                 }
             };
 
-            ItemDesc cur = make_desc(0), nxt = make_desc(32);
+            // cur / nxt: the items being added (base .. base + 31) and the batch after them; icur / inxt: the same for the
+            // copies, which run S - 1 items ahead (lane j of icur is item base + j + S - 1)
+            ItemDesc cur = make_desc(0), nxt = make_desc(32), icur = make_desc(S - 1), inxt = make_desc(32 + S - 1);
             int islot = 0, cslot = 0;
-            // copy of item `item` (lane `ji` of cur, or lane ji - 32 of nxt); past the end: an empty copy
-            auto issue = [&](int item, int ji) {
-                const bool in_cur = ji < 32;
-                const int idx = __shfl_sync(0xffffffffu, in_cur ? cur.idx : nxt.idx, ji & 31);
-                const int meta = __shfl_sync(0xffffffffu, in_cur ? cur.meta : nxt.meta, ji & 31);
-                const bool is_tab = (meta & 4) != 0;
-                const float* src = (is_tab ? gsum : rg.grads) + (int64_t)idx * (is_tab ? (int64_t)D : rg.ld);
+            auto advance = [](int slot) { return (S & (S - 1)) == 0 ? ((slot + 1) & (S - 1)) : (slot + 1 == S ? 0 : slot + 1); };
+            // copy of the item in lane j of descriptor batch d (an empty copy if the item does not exist)
+            auto issue = [&](const ItemDesc& d, int j) {
+                const uint32_t lo = __shfl_sync(0xffffffffu, d.addr_lo, j), hi = __shfl_sync(0xffffffffu, d.addr_hi, j);
+                const float* src = reinterpret_cast<const float*>(((uint64_t)hi << 32) | (lo & ~15u));
+                const int bytes = (int)(lo & 1u) << 4;
                 const uint32_t dst = ring_addr + (uint32_t)islot * SLOT_BYTES;
-                const int bytes = item < total_items ? 16 : 0;
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
                     const int ch = lane + 32 * q;
@@ -374,18 +377,18 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                     cp_async_16(dst + (uint32_t)ch * 16u, src + (on ? ch * 4 : 0), on ? bytes : 0);
                 }
                 cp_async_commit();
-                islot = islot + 1 == S ? 0 : islot + 1;
+                islot = advance(islot);
             };
 
             // ---- the pipeline: S - 1 items ahead
             __syncwarp();
 #pragma unroll
-            for (int i = 0; i < S - 1; ++i) issue(i, i);
+            for (int i = 0; i < S - 1; ++i) issue(cur, i);
             for (int base = 0; base < total_items; base += 32) {
                 const int n_in = min(32, total_items - base);
                 for (int j = 0; j < n_in; ++j) {
                     __syncwarp();                                 // every lane is done with the slot refilled next
-                    issue(base + j + S - 1, j + S - 1);
+                    issue(icur, j);
                     cp_async_wait<S - 1>();
                     __syncwarp();                                 // ... and sees the other lanes' copies of item base + j
                     const float scale = __shfl_sync(0xffffffffu, cur.scale, j);
@@ -397,11 +400,12 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                         acc[q].x = fmaf(scale, v.x, acc[q].x); acc[q].y = fmaf(scale, v.y, acc[q].y);
                         acc[q].z = fmaf(scale, v.z, acc[q].z); acc[q].w = fmaf(scale, v.w, acc[q].w);
                     }
-                    if (meta & 3) settle(meta >> 3, (meta & 1) != 0, (meta & 2) != 0);
-                    cslot = cslot + 1 == S ? 0 : cslot + 1;
+                    if (meta & 3) settle(meta >> 2, (meta & 1) != 0, (meta & 2) != 0);
+                    cslot = advance(cslot);
                 }
-                cur = nxt;
+                cur = nxt; icur = inxt;
                 nxt = make_desc(base + 64);
+                inxt = make_desc(base + 64 + S - 1);
             }
             cp_async_wait<0>();
         }
@@ -456,7 +460,7 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
                                                             grp_rec, rs, pmeta, blk_first, run_end, state); }
     const int nq = (int)ceil_div(D / 4, 32);
     const int64_t want = ceil_div(ceil_div(n, ACC_SPAN), 8);
-    const int resident = sm_count() * 2;                          // every block stays resident
+    const int resident = sm_count() * (nq <= 2 ? 3 : 2);          // every block stays resident
     const int grid = (int)(want < resident ? (want < 1 ? 1 : want) : resident);
     cudaError_t le = cudaSuccess;
     { KernelScope k(&c.prof, "acc_reduce", st);
