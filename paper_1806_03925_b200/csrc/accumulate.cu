@@ -137,6 +137,7 @@ struct RowSource {
 __global__ void __launch_bounds__(AF_THREADS)
 acc_flag_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int M, const int32_t* __restrict__ cnt,
                 uint2* __restrict__ tile_cnt, DevState* __restrict__ state) {
+    wait_for_predecessor();
     __shared__ uint32_t smem[34];
     TileFlags f;
     tile_flags(f, ks, n, vocab, M, cnt, smem, state);
@@ -154,6 +155,7 @@ acc_plan_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int 
                 const uint2* __restrict__ tile_cnt, uint4* __restrict__ grp_rec, RowSource rs,
                 int2* __restrict__ pmeta, uint32_t* __restrict__ blk_first, uint32_t* __restrict__ run_end,
                 DevState* __restrict__ state) {
+    wait_for_predecessor();
     __shared__ uint32_t smem[34];
     TileFlags f;
     tile_flags(f, ks, n, vocab, M, cnt, smem, state, run_end);
@@ -234,6 +236,7 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                   const uint32_t* __restrict__ blk_first, const uint32_t* __restrict__ run_end,
                   float* __restrict__ gsum, int32_t* __restrict__ gcnt,
                   int32_t* __restrict__ q_id, float* __restrict__ q_avg, const DevState* __restrict__ state) {
+    wait_for_predecessor();
     extern __shared__ float4 ring_mem[];                          // [warps][S][NQ * 32] float4
     const uint2 totals = tile_cnt[n_tiles];
     const int64_t n_groups = totals.x;
@@ -415,6 +418,7 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
 
 __global__ void acc_commit_kernel(const uint2* __restrict__ tile_cnt, int64_t n_tiles, int64_t ready_cap,
                                   DevState* __restrict__ state) {
+    wait_for_predecessor();
     const uint2 totals = tile_cnt[n_tiles];
     state->n_groups = totals.x;
     state->n_complete = totals.y;
@@ -447,7 +451,7 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     const int64_t n_tiles = ceil_div(n, AF_TILE);
     uint2* tile_cnt = c.at<uint2>(c.ws.tile_cnt);
     { KernelScope k(&c.prof, "acc_flag", st);
-    acc_flag_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt, state); }
+    launch_dependent(acc_flag_kernel, dim3((unsigned)n_tiles), dim3(AF_THREADS), 0, st, ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt, state); }
     scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, &c.prof);
     uint4* grp_rec = c.at<uint4>(c.ws.grp_rec);
     int2* pmeta = c.at<int2>(c.ws.pmeta);
@@ -456,7 +460,7 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     uint32_t* blk_first = c.at<uint32_t>(c.ws.blk_first);
     uint32_t* run_end = c.at<uint32_t>(c.ws.run_end);
     { KernelScope k(&c.prof, "acc_plan", st);
-    acc_plan_kernel<<<(unsigned)n_tiles, AF_THREADS, 0, st>>>(ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt,
+    launch_dependent(acc_plan_kernel, dim3((unsigned)n_tiles), dim3(AF_THREADS), 0, st, ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt,
                                                             grp_rec, rs, pmeta, blk_first, run_end, state); }
     const int nq = (int)ceil_div(D / 4, 32);
     const int64_t want = ceil_div(ceil_div(n, ACC_SPAN), 8);
@@ -468,7 +472,7 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
         const int smem = 8 * slots * slot_bytes;
         le = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (le != cudaSuccess) return;
-        kernel<<<grid, 256, smem, st>>>(ks, rg, D, M, n_tiles, c.ws.ready_cap, tile_cnt, grp_rec, blk_first, run_end,
+        le = launch_dependent(kernel, dim3(grid), dim3(256), (size_t)smem, st, ks, rg, D, M, n_tiles, c.ws.ready_cap, tile_cnt, grp_rec, blk_first, run_end,
                                         c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id),
                                         c.at<float>(c.ws.q_avg), state);
     };
@@ -484,7 +488,7 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     }
     if (le != cudaSuccess) return le;
     { KernelScope k(&c.prof, "acc_commit", st);
-    acc_commit_kernel<<<1, 1, 0, st>>>(tile_cnt, n_tiles, c.ws.ready_cap, state); }
+    launch_dependent(acc_commit_kernel, dim3(1), dim3(1), 0, st, tile_cnt, n_tiles, c.ws.ready_cap, state); }
     ++c.acc_calls_pending;
     return cudaGetLastError();
 }
@@ -504,6 +508,7 @@ acc_atomic_add_kernel(const int32_t* __restrict__ img_id, int64_t n, int64_t voc
                       int64_t ld, const int32_t* __restrict__ src_row, const float* __restrict__ scale, int D,
                       float* __restrict__ gsum, int32_t* __restrict__ gcnt, int32_t* __restrict__ touched,
                       int64_t ready_cap, DevState* __restrict__ state) {
+    wait_for_predecessor();
     // a call completes at most n groups: refuse it whole if the queue could not take them
     const bool drop = state->q_count + n > ready_cap;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -539,6 +544,7 @@ __global__ void __launch_bounds__(256)
 acc_atomic_settle_kernel(const int32_t* __restrict__ touched, int D, int M, float* __restrict__ gsum,
                          int32_t* __restrict__ gcnt, int32_t* __restrict__ q_id, float* __restrict__ q_avg,
                          DevState* __restrict__ state) {
+    wait_for_predecessor();
     if (state->pad[3] != 0) return;                            // the call was dropped
     const int64_t n_touched = state->pad[2];
     const unsigned lane = lane_id();
@@ -578,10 +584,10 @@ cudaError_t launch_accumulate_atomic(const gear_ctx_impl& c, const int32_t* img_
     const int resident = sm_count() * 8;
     const int grid = (int)(want < resident ? (want < 1 ? 1 : want) : resident);
     { KernelScope k(&c.prof, "acc_atomic_add", st);
-    acc_atomic_add_kernel<<<grid, 256, 0, st>>>(img_id, n, c.cfg.img_vocab, grads, ld, src_row, scale, c.cfg.dfv_dim,
+    launch_dependent(acc_atomic_add_kernel, dim3(grid), dim3(256), 0, st, img_id, n, c.cfg.img_vocab, grads, ld, src_row, scale, c.cfg.dfv_dim,
                                                 c.buf.dfv_gsum, c.buf.dfv_gcnt, touched, c.ws.ready_cap, state); }
     { KernelScope k(&c.prof, "acc_atomic_settle", st);
-    acc_atomic_settle_kernel<<<grid, 256, 0, st>>>(touched, c.cfg.dfv_dim, c.cfg.M, c.buf.dfv_gsum, c.buf.dfv_gcnt,
+    launch_dependent(acc_atomic_settle_kernel, dim3(grid), dim3(256), 0, st, touched, c.cfg.dfv_dim, c.cfg.M, c.buf.dfv_gsum, c.buf.dfv_gcnt,
                                                    c.at<int32_t>(c.ws.q_id), c.at<float>(c.ws.q_avg), state); }
     c.acc_calls_pending += 2;
     return cudaGetLastError();
@@ -589,6 +595,7 @@ cudaError_t launch_accumulate_atomic(const gear_ctx_impl& c, const int32_t* img_
 
 // ---------------------------------------------------------------- event 6b: hand the ready queue over
 __global__ void collect_begin_kernel(DevState* __restrict__ state, int64_t cap, int64_t* __restrict__ d_n) {
+    wait_for_predecessor();
     const int64_t n = state->q_count;
     if (d_n) *d_n = n;
     if (n > cap) { atomicOr(&state->status, GEAR_DEV_OUT_CAPACITY); state->collect_n = -1; state->sort_n = 0; }
@@ -602,6 +609,7 @@ __global__ void collect_begin_kernel(DevState* __restrict__ state, int64_t cap, 
 
 __global__ void __launch_bounds__(256)
 collect_keys_kernel(const int32_t* __restrict__ q_id, const DevState* __restrict__ state, uint32_t* __restrict__ keys) {
+    wait_for_predecessor();
     const int64_t n = state->sort_n;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         keys[i] = (uint32_t)q_id[i];
@@ -615,6 +623,7 @@ collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __
                     const int32_t* __restrict__ q_id, const float* __restrict__ q_avg,
                     int D, const DevState* __restrict__ state, int32_t* __restrict__ ids, int32_t* __restrict__ seq,
                     float* __restrict__ avg) {
+    wait_for_predecessor();
     const int64_t n = state->collect_n;
     const bool in_order = state->sort_n == 0;          // the queue itself is sorted: no permutation
     const uint32_t* ks = in_order ? reinterpret_cast<const uint32_t*>(q_id) : sorted_keys;
@@ -656,6 +665,7 @@ collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __
 }
 
 __global__ void collect_end_kernel(DevState* __restrict__ state) {
+    wait_for_predecessor();
     if (state->collect_n >= 0) { state->q_count = 0; state->q_calls = 0; }
 }
 
@@ -665,7 +675,7 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     SortJob sb = c.sort_job(gear_ctx_impl::SORT_READY);
     const int64_t n_max = c.ws.ready_cap;
     { KernelScope k(&c.prof, "collect_begin", st);
-    collect_begin_kernel<<<1, 1, 0, st>>>(state, cap, d_n); }
+    launch_dependent(collect_begin_kernel, dim3(1), dim3(1), 0, st, state, cap, d_n); }
     int cur = 0;
     // A queue fed by at most one accumulate call is in (id, group) order already.  The host knows an upper bound
     // of the number of feeding calls; only when that exceeds one are the sort kernels enqueued at all (the device
@@ -673,7 +683,7 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     if (c.acc_calls_pending > 1) {
         int64_t blocks = ceil_div(n_max, 256);
         { KernelScope k(&c.prof, "collect_keys", st);
-        collect_keys_kernel<<<(unsigned)(blocks > 1184 ? 1184 : blocks), 256, 0, st>>>(c.at<int32_t>(c.ws.q_id), state,
+        launch_dependent(collect_keys_kernel, dim3((unsigned)(blocks > 1184 ? 1184 : blocks)), dim3(256), 0, st, c.at<int32_t>(c.ws.q_id), state,
                                                                                      sb.keys[0]); }
         SortBatch batch = c.sort_batch();
         batch.n_jobs = 1;
@@ -689,12 +699,12 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     if (cap >= c.ws.ready_cap) c.acc_calls_pending = 0;      // this collect cannot be refused: the queue will be empty
     int64_t want = ceil_div(n_max, 8);
     { KernelScope k(&c.prof, "collect_move", st);
-    collect_move_kernel<<<(unsigned)(want > 1184 ? 1184 : want), 256, 0, st>>>(sb.keys[cur], sb.vals[cur],
+    launch_dependent(collect_move_kernel, dim3((unsigned)(want > 1184 ? 1184 : want)), dim3(256), 0, st, sb.keys[cur], sb.vals[cur],
                                                                             c.at<int32_t>(c.ws.q_id),
                                                                             c.at<float>(c.ws.q_avg), c.cfg.dfv_dim,
                                                                             state, ids, seq, avg); }
     { KernelScope k(&c.prof, "collect_end", st);
-    collect_end_kernel<<<1, 1, 0, st>>>(state); }
+    launch_dependent(collect_end_kernel, dim3(1), dim3(1), 0, st, state); }
     return cudaGetLastError();
 }
 

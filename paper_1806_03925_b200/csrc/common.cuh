@@ -122,6 +122,26 @@ __device__ __forceinline__ void st_f4_hint(float* p, float4 v, uint64_t policy) 
                  :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy) : "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// The step is a chain of two dozen short kernels on one stream.  Launched this way, the blocks of a kernel may be
+// set up on SMs that the previous kernel in the stream has already left while its last blocks still run; every
+// such kernel calls wait_for_predecessor() before it touches memory, which returns once the previous kernel has
+// completed and its writes are visible.  That takes the launch latency out of the gaps between kernels.  Every
+// block of such a kernel must make the call, first thing, or the chain of completions would break.
+__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---------------------------------------------------------------- launch accounting / per-kernel timing
 // Every kernel launch of the library goes through a KernelScope: it counts the launch and, when profiling
 // is on, brackets it with a pair of CUDA events on the caller's stream (read back by gear_profile_read).

@@ -19,6 +19,7 @@ __global__ void __launch_bounds__(256)
 emb_reduce_kernel(const uint32_t* __restrict__ ks, const uint32_t* __restrict__ perm, int n, uint32_t vocab,
                   int E, int lpr, const float* __restrict__ dX, int64_t ldx, int col0,
                   float* __restrict__ table, float alpha) {
+    wait_for_predecessor();
     const int64_t gthread = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t group = gthread / lpr;
     const int c = (int)(gthread % lpr);
@@ -76,7 +77,7 @@ cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int which, int cur, int32_
     const int nq = (int)ceil_div(n_chunks, lpr);
     const int64_t groups = ceil_div(B, ES_SEG);
     const unsigned grid = (unsigned)ceil_div(groups * lpr, 256);
-#define GEAR_ES_LAUNCH(NQ) emb_reduce_kernel<NQ><<<grid, 256, 0, st>>>(sb.keys[cur], sb.vals[cur], B, (uint32_t)vocab, \
+#define GEAR_ES_LAUNCH(NQ) launch_dependent(emb_reduce_kernel<NQ>, dim3(grid), dim3(256), 0, st, sb.keys[cur], sb.vals[cur], B, (uint32_t)vocab, \
                                                                         E, lpr, dX, ldx, col0, table, alpha)
     KernelScope ks(&c.prof, "emb_reduce", st);
     if (nq <= 1) GEAR_ES_LAUNCH(1);

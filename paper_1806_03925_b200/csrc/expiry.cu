@@ -23,6 +23,7 @@ static_assert(EXP_MARK_TILE % (EXP_THREADS * 1) == 0 && EXP_TILE % EXP_MARK_TILE
 __global__ void __launch_bounds__(EXP_THREADS)
 expiry_mark_kernel(const int64_t* __restrict__ ts, int64_t vocab, int64_t now, int64_t expire,
                    uint32_t* __restrict__ bits, uint2* __restrict__ tile_cnt) {
+    wait_for_predecessor();
     __shared__ uint32_t warp_cnt[EXP_THREADS / 32];
     const int64_t tile0 = (int64_t)blockIdx.x * EXP_MARK_TILE;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
@@ -60,6 +61,7 @@ __global__ void __launch_bounds__(EXP_THREADS)
 expiry_write_kernel(const uint32_t* __restrict__ bits, int64_t vocab, const uint2* __restrict__ tile_cnt,
                     int64_t n_mark_tiles, int64_t cap, int64_t* __restrict__ d_n, DevState* __restrict__ state,
                     int64_t now, int restamp, int64_t* __restrict__ ts, int32_t* __restrict__ ids) {
+    wait_for_predecessor();
     __shared__ uint32_t scratch[33];
     const int64_t total = tile_cnt[n_mark_tiles].x;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -87,10 +89,10 @@ static cudaError_t enqueue_expiry_scan(int64_t* ts, int64_t vocab, int64_t expir
                                        DevState* state, Profiler* prof, cudaStream_t st) {
     const int64_t n_mark = ceil_div(vocab, EXP_MARK_TILE), n_write = ceil_div(vocab, EXP_TILE);
     { KernelScope k(prof, "expiry_mark", st);
-    expiry_mark_kernel<<<(unsigned)n_mark, EXP_THREADS, 0, st>>>(ts, vocab, now, expire, bits, tile_cnt); }
+    launch_dependent(expiry_mark_kernel, dim3((unsigned)n_mark), dim3(EXP_THREADS), 0, st, ts, vocab, now, expire, bits, tile_cnt); }
     scan_pairs(tile_cnt, n_mark, tile_cnt + n_mark, st, prof);
     { KernelScope k(prof, "expiry_write", st);
-    expiry_write_kernel<<<(unsigned)n_write, EXP_THREADS, 0, st>>>(bits, vocab, tile_cnt, n_mark, cap, d_n, state, now,
+    launch_dependent(expiry_write_kernel, dim3((unsigned)n_write), dim3(EXP_THREADS), 0, st, bits, vocab, tile_cnt, n_mark, cap, d_n, state, now,
                                                                   restamp, ts, ids); }
     return cudaGetLastError();
 }

@@ -114,6 +114,7 @@ __device__ __forceinline__ ViewRec load_view(const GatherArgs& a, int b) {
 template <typename TD, typename TX, int NQ>
 __global__ void __launch_bounds__(GP_WARPS * 32, NQ <= 2 ? 3 : 2)
 gather_pool_kernel(const GatherArgs a) {
+    wait_for_predecessor();
     constexpr int PER = Chunk<TD>::PER;
     constexpr int KMAX = NQ >= 8 ? 1 : 8 / NQ;               // rows in flight per warp
     const int lane = (int)lane_id();
@@ -239,10 +240,10 @@ static cudaError_t dispatch_nq(const GatherArgs& a, cudaStream_t st, Profiler* p
     const int64_t resident = (int64_t)sm_count() * (nq <= 2 ? 3 : 2);
     const int grid = (int)std::min<int64_t>(ceil_div(a.B, GP_WARPS), resident);
     KernelScope ks(prof, "gather_pool", st);
-    if (nq <= 1) gather_pool_kernel<TD, TX, 1><<<grid, GP_WARPS * 32, 0, st>>>(a);
-    else if (nq <= 2) gather_pool_kernel<TD, TX, 2><<<grid, GP_WARPS * 32, 0, st>>>(a);
-    else if (nq <= 4) gather_pool_kernel<TD, TX, 4><<<grid, GP_WARPS * 32, 0, st>>>(a);
-    else gather_pool_kernel<TD, TX, 8><<<grid, GP_WARPS * 32, 0, st>>>(a);
+    if (nq <= 1) launch_dependent(gather_pool_kernel<TD, TX, 1>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a);
+    else if (nq <= 2) launch_dependent(gather_pool_kernel<TD, TX, 2>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a);
+    else if (nq <= 4) launch_dependent(gather_pool_kernel<TD, TX, 4>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a);
+    else launch_dependent(gather_pool_kernel<TD, TX, 8>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a);
     return cudaGetLastError();
 }
 

@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(256)
 gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sam, int64_t sak,
             const TB* __restrict__ Bm, int64_t sbk, int64_t sbn, TC* __restrict__ C, int64_t ldc,
             const float* __restrict__ bias, const TM* __restrict__ mask, int64_t ldm, int k_chunk) {
+    wait_for_predecessor();
     __shared__ float As[GK][GT + 4];
     __shared__ float Bs[GK][GT + 4];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -95,7 +96,7 @@ static void launch_gemm(int M, int N, int K, const TA* A, int64_t sam, int64_t s
     int k_chunk = (int)ceil_div(ceil_div(K, splits), GK) * GK;
     splits = (int)ceil_div(K, k_chunk);
     dim3 grid((unsigned)ceil_div(N, GT), (unsigned)ceil_div(M, GT), (unsigned)splits);
-    gemm_kernel<TA, TB, TC, TM, EPI><<<grid, 256, 0, st>>>(M, N, K, A, sam, sak, B, sbk, sbn, C, ldc, bias, mask,
+    launch_dependent(gemm_kernel<TA, TB, TC, TM, EPI>, grid, dim3(256), 0, st, M, N, K, A, sam, sak, B, sbk, sbn, C, ldc, bias, mask,
                                                           ldm, k_chunk);
 }
 
@@ -139,6 +140,7 @@ head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict_
                 const float* __restrict__ b_out, const float* __restrict__ label, float* __restrict__ prob,
                 float* __restrict__ dz, TX* __restrict__ dA, float* __restrict__ loss_part,
                 float* __restrict__ gw_out, float* __restrict__ gb_top, float* __restrict__ gb_out) {
+    wait_for_predecessor();
     __shared__ float part[8], gpart[8];
     __shared__ float s_gw[1024], s_gb[1024];
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
@@ -213,6 +215,7 @@ head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict_
 }
 
 __global__ void loss_final_kernel(const float* __restrict__ part, int n, int B, float* __restrict__ loss) {
+    wait_for_predecessor();
     __shared__ float sm[32];
     float s = 0.f;
     for (int i = threadIdx.x; i < n; i += blockDim.x) s += part[i];
@@ -232,6 +235,7 @@ __global__ void loss_final_kernel(const float* __restrict__ part, int n, int B, 
 template <typename TA>
 __global__ void __launch_bounds__(256)
 colsum_kernel(int B, int N, const TA* __restrict__ A, float* __restrict__ out) {
+    wait_for_predecessor();
     __shared__ float s[1024];
     const int tpr = N / 8, rpp = 256 / tpr;
     const int chunk = threadIdx.x % tpr, rsub = threadIdx.x / tpr;
@@ -274,6 +278,7 @@ struct RoundArgs {
 };
 __global__ void __launch_bounds__(256)
 round_weights_kernel(const RoundArgs a) {
+    wait_for_predecessor();
     const int l = blockIdx.y;
     const int fan_in = a.fan_in[l], fan_out = a.fan_out[l];
     const int64_t n = (int64_t)fan_in * fan_out;
@@ -345,7 +350,7 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
             if ((int64_t)p.fan[l] * p.fan[l + 1] > biggest) biggest = (int64_t)p.fan[l] * p.fan[l + 1];
         }
         KernelScope ks(&c.prof, "round_weights", st);
-        round_weights_kernel<<<dim3((unsigned)ceil_div(biggest, 256), (unsigned)L), 256, 0, st>>>(ra);
+        launch_dependent(round_weights_kernel, dim3((unsigned)ceil_div(biggest, 256), (unsigned)L), dim3(256), 0, st, ra);
     } else {
         for (int l = 0; l < L; ++l) Wop[l] = p.W[l];
     }
@@ -367,7 +372,7 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
     {
         KernelScope ks(&c.prof, "head_out", st);
         const int nq = (int)ceil_div(HT, 256);
-#define GEAR_HEAD_OUT(NQ) head_out_kernel<TX, NQ><<<c.ws.loss_blocks, 256, 0, st>>>(B, HT, H[L], p.w_out, p.b_out, bt.label, \
+#define GEAR_HEAD_OUT(NQ) launch_dependent(head_out_kernel<TX, NQ>, dim3(c.ws.loss_blocks), dim3(256), 0, st, B, HT, H[L], p.w_out, p.b_out, bt.label, \
         o.prob, dz, dA[L], loss_part, p.gw_out, p.gb[L - 1], p.gb_out)
         if (nq <= 1) GEAR_HEAD_OUT(1);
         else if (nq == 2) GEAR_HEAD_OUT(2);
@@ -375,7 +380,7 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
 #undef GEAR_HEAD_OUT
     }
     { KernelScope ks(&c.prof, "loss_final", st);
-    loss_final_kernel<<<1, 256, 0, st>>>(loss_part, c.ws.loss_blocks, B, o.loss); }
+    launch_dependent(loss_final_kernel, dim3(1), dim3(256), 0, st, loss_part, c.ws.loss_blocks, B, o.loss); }
     // backward
     for (int l = L - 1; l >= 0; --l) {
         const int K = p.fan[l], N = p.fan[l + 1];
@@ -391,7 +396,7 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
         if (!BF && l < L - 1) {
             KernelScope ks(&c.prof, "colsum", st);
             const int blocks = B < CS_BLOCKS * 8 ? (int)ceil_div(B, 8) : CS_BLOCKS;
-            colsum_kernel<TX><<<blocks, 256, 0, st>>>(B, N, dA[l + 1], p.gb[l]);
+            launch_dependent(colsum_kernel<TX>, dim3(blocks), dim3(256), 0, st, B, N, dA[l + 1], p.gb[l]);
         }
         if constexpr (BF) {
             const __nv_bfloat16* wb = c.at<__nv_bfloat16>(c.ws.wb[l]);

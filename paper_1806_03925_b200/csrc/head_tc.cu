@@ -369,6 +369,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_word_ptr;
+    wait_for_predecessor();      // barriers, tensor memory and descriptors are set up while the previous kernel drains
 
     if (warp == 0) {
         // ---------------- TMA producer
@@ -524,8 +525,7 @@ static cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, 
     }
     const int tiles = g.m_tiles * g.n_tiles * g.k_splits;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    tc_gemm_kernel<BN, MN, EPI><<<grid, TC_THREADS, Cfg::SMEM, st>>>(ma, mb, g);
-    return cudaGetLastError();
+    return launch_dependent(tc_gemm_kernel<BN, MN, EPI>, dim3(grid), dim3(TC_THREADS), (size_t)Cfg::SMEM, st, ma, mb, g);
 }
 
 template <bool MN, int EPI>

@@ -274,6 +274,7 @@ int sort_jobs(SortBatch& batch, GridBarrierState* gbs, cudaStream_t st, Profiler
 // ---------------------------------------------------------------- scan of counter pairs
 __global__ void __launch_bounds__(1024)
 scan_pairs_kernel(uint2* __restrict__ data, int64_t m, uint2* __restrict__ total) {
+    wait_for_predecessor();
     __shared__ uint32_t scratch[33];
     uint32_t ca = 0, cb = 0;
     for (int64_t base = 0; base < m; base += blockDim.x) {
@@ -291,7 +292,7 @@ scan_pairs_kernel(uint2* __restrict__ data, int64_t m, uint2* __restrict__ total
 
 void scan_pairs(uint2* data, int64_t m, uint2* total, cudaStream_t st, Profiler* prof) {
     KernelScope k(prof, "scan_pairs", st);
-    scan_pairs_kernel<<<1, 1024, 0, st>>>(data, m, total);
+    launch_dependent(scan_pairs_kernel, dim3(1), dim3(1024), 0, st, data, m, total);
 }
 
 }  // namespace gear
