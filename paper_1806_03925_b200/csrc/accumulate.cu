@@ -20,8 +20,8 @@
 //      average to its queue slot or, for the open group, the running sum and count back to the table.  The
 //      warp that owns the first group of an image also settles what the image's last, still open group
 //      leaves in the table, so no two warps touch one table row.
-//   6. commit: the queue length grows by the number of complete groups (or the call is dropped whole if
-//      the queue would overflow).
+//   6. commit (by the block of the reduce pass that finishes last): the queue length grows by the number of
+//      complete groups (or the call is dropped whole if the queue would overflow).
 // HBM bound: the reduce pass reads every gradient row once and reads/writes one accumulator row per
 // distinct image; the sort and flag passes move 4-byte keys only.
 #include "common.cuh"
@@ -235,12 +235,28 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                   const uint2* __restrict__ tile_cnt, const uint4* __restrict__ grp_rec,
                   const uint32_t* __restrict__ blk_first, const uint32_t* __restrict__ run_end,
                   float* __restrict__ gsum, int32_t* __restrict__ gcnt,
-                  int32_t* __restrict__ q_id, float* __restrict__ q_avg, const DevState* __restrict__ state) {
+                  int32_t* __restrict__ q_id, float* __restrict__ q_avg, DevState* __restrict__ state) {
     wait_for_predecessor();
     extern __shared__ float4 ring_mem[];                          // [warps][S][NQ * 32] float4
     const uint2 totals = tile_cnt[n_tiles];
     const int64_t n_groups = totals.x;
-    if (state->q_count + (int64_t)totals.y > ready_cap) return;      // the whole call is dropped
+    // Step 6 of the plan (commit) is done by whichever block finishes last: by then every block has read the queue
+    // length it started from.  Every block, also one of a dropped call, leaves through this.
+    const bool dropped = state->q_count + (int64_t)totals.y > ready_cap;
+    auto leave = [&]() {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence();
+            unsigned int* ticket = reinterpret_cast<unsigned int*>(&state->pad[4]);
+            if (atomicInc(ticket, gridDim.x - 1) == gridDim.x - 1) {
+                state->n_groups = totals.x;
+                state->n_complete = totals.y;
+                if (dropped) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
+                else if (totals.y > 0) { state->q_count += totals.y; state->q_calls += 1; }
+            }
+        }
+    };
+    if (dropped) { leave(); return; }                                // the whole call is dropped
     const int64_t n_valid = state->n_valid;
     const int lane = (int)lane_id(), warp = (int)(threadIdx.x >> 5);
     const int n_chunks = D / 4;
@@ -414,16 +430,7 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
         }
         G = G_nxt; range_nxt = range_nxt2;
     }
-}
-
-__global__ void acc_commit_kernel(const uint2* __restrict__ tile_cnt, int64_t n_tiles, int64_t ready_cap,
-                                  DevState* __restrict__ state) {
-    wait_for_predecessor();
-    const uint2 totals = tile_cnt[n_tiles];
-    state->n_groups = totals.x;
-    state->n_complete = totals.y;
-    if (state->q_count + (int64_t)totals.y > ready_cap) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
-    else if (totals.y > 0) { state->q_count += totals.y; state->q_calls += 1; }
+    leave();
 }
 
 cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
@@ -487,8 +494,6 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
 #undef GEAR_ACC_LAUNCH
     }
     if (le != cudaSuccess) return le;
-    { KernelScope k(&c.prof, "acc_commit", st);
-    launch_dependent(acc_commit_kernel, dim3(1), dim3(1), 0, st, tile_cnt, n_tiles, c.ws.ready_cap, state); }
     ++c.acc_calls_pending;
     return cudaGetLastError();
 }
@@ -621,11 +626,20 @@ collect_keys_kernel(const int32_t* __restrict__ q_id, const DevState* __restrict
 __global__ void __launch_bounds__(256)
 collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __restrict__ sorted_perm,
                     const int32_t* __restrict__ q_id, const float* __restrict__ q_avg,
-                    int D, const DevState* __restrict__ state, int32_t* __restrict__ ids, int32_t* __restrict__ seq,
-                    float* __restrict__ avg) {
+                    int D, DevState* __restrict__ state, int32_t* __restrict__ ids, int32_t* __restrict__ seq,
+                    float* __restrict__ avg, int solo, int64_t cap, int64_t* __restrict__ d_n) {
     wait_for_predecessor();
-    const int64_t n = state->collect_n;
-    const bool in_order = state->sort_n == 0;          // the queue itself is sorted: no permutation
+    // solo: this launch is the whole hand-over (a queue fed by one accumulate call is in order already): it checks
+    // the caller's capacity itself and the last block to finish empties the queue
+    const int64_t n = solo ? state->q_count : state->collect_n;
+    if (solo) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            if (d_n) *d_n = n;
+            if (n > cap) atomicOr(&state->status, GEAR_DEV_OUT_CAPACITY);
+        }
+        if (n > cap) return;                            // nothing is consumed
+    }
+    const bool in_order = solo || state->sort_n == 0;  // the queue itself is sorted: no permutation
     const uint32_t* ks = in_order ? reinterpret_cast<const uint32_t*>(q_id) : sorted_keys;
     const int64_t threads = (int64_t)gridDim.x * blockDim.x;
     for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n; k += threads) {
@@ -662,6 +676,15 @@ collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __
                 if (src[t] >= 0) st_f4(avg + (k0 + t * warps) * D + ch * 4, v[t]);
         }
     }
+    if (solo) {
+        __shared__ int is_last;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence();
+            is_last = atomicInc(&state->pad32, gridDim.x - 1) == gridDim.x - 1;
+            if (is_last) { state->q_count = 0; state->q_calls = 0; }
+        }
+    }
 }
 
 __global__ void collect_end_kernel(DevState* __restrict__ state) {
@@ -674,7 +697,8 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     DevState* state = c.state();
     SortJob sb = c.sort_job(gear_ctx_impl::SORT_READY);
     const int64_t n_max = c.ws.ready_cap;
-    { KernelScope k(&c.prof, "collect_begin", st);
+    const bool solo = c.acc_calls_pending <= 1;
+    if (!solo) { KernelScope k(&c.prof, "collect_begin", st);
     launch_dependent(collect_begin_kernel, dim3(1), dim3(1), 0, st, state, cap, d_n); }
     int cur = 0;
     // A queue fed by at most one accumulate call is in (id, group) order already.  The host knows an upper bound
@@ -702,8 +726,8 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     launch_dependent(collect_move_kernel, dim3((unsigned)(want > 1184 ? 1184 : want)), dim3(256), 0, st, sb.keys[cur], sb.vals[cur],
                                                                             c.at<int32_t>(c.ws.q_id),
                                                                             c.at<float>(c.ws.q_avg), c.cfg.dfv_dim,
-                                                                            state, ids, seq, avg); }
-    { KernelScope k(&c.prof, "collect_end", st);
+                                                                            state, ids, seq, avg, solo ? 1 : 0, cap, d_n); }
+    if (!solo) { KernelScope k(&c.prof, "collect_end", st);
     launch_dependent(collect_end_kernel, dim3(1), dim3(1), 0, st, state); }
     return cudaGetLastError();
 }

@@ -24,8 +24,8 @@ struct DevState {
     int64_t exp_total;     // expiry scan: entries found
     int64_t collect_n;     // collect_ready: entries moved by the running call
     unsigned long long grid_barrier;   // arrival counter of the cooperative sort's grid barrier
-    unsigned int colsum_ticket;        // blocks of the column-sum kernel that have delivered their partials
-    unsigned int pad32;
+    unsigned int colsum_ticket;        // blocks of head_out_kernel that have delivered their partial loss (wraps to 0)
+    unsigned int pad32;                // blocks of a solo collect_move_kernel that have finished (wraps to 0)
     int64_t q_calls;       // accumulate calls that added to the ready queue since the last collect
     int64_t sort_n;        // collect_ready: entries the queue sort has to order (0: the queue is already in order)
     int64_t pad[5];

@@ -139,7 +139,8 @@ __global__ void __launch_bounds__(256)
 head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict__ w_out,
                 const float* __restrict__ b_out, const float* __restrict__ label, float* __restrict__ prob,
                 float* __restrict__ dz, TX* __restrict__ dA, float* __restrict__ loss_part,
-                float* __restrict__ gw_out, float* __restrict__ gb_top, float* __restrict__ gb_out) {
+                float* __restrict__ gw_out, float* __restrict__ gb_top, float* __restrict__ gb_out,
+                unsigned int* __restrict__ ticket, float* __restrict__ loss) {
     wait_for_predecessor();
     __shared__ float part[8], gpart[8];
     __shared__ float s_gw[1024], s_gb[1024];
@@ -212,20 +213,26 @@ head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict_
         loss_part[blockIdx.x] = s;
         atomicAdd(gb_out, t);
     }
-}
-
-__global__ void loss_final_kernel(const float* __restrict__ part, int n, int B, float* __restrict__ loss) {
-    wait_for_predecessor();
-    __shared__ float sm[32];
-    float s = 0.f;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) s += part[i];
-    s = warp_sum(s);
-    if (lane_id() == 0) sm[threadIdx.x >> 5] = s;
+    // The block that delivers its partial loss last adds them all up, always in block order (the ticket counts
+    // arrivals and wraps back to zero by itself, ready for the next launch).
+    __shared__ int is_last;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        is_last = atomicInc(ticket, gridDim.x - 1) == gridDim.x - 1;
+    }
     __syncthreads();
-    if (threadIdx.x < 32) {
-        float t = threadIdx.x < (blockDim.x >> 5) ? sm[threadIdx.x] : 0.f;
-        t = warp_sum(t);
-        if (threadIdx.x == 0) loss[0] = B > 0 ? t / (float)B : 0.f;
+    if (!is_last) return;
+    __threadfence();
+    float s = 0.f;
+    for (int i = threadIdx.x; i < (int)gridDim.x; i += 256) s += __ldcg(loss_part + i);
+    s = warp_sum(s);
+    __syncthreads();
+    if (lane == 0) part[warp] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int k = 0; k < 8; ++k) t += part[k];
+        loss[0] = B > 0 ? t / (float)B : 0.f;
     }
 }
 
@@ -276,17 +283,30 @@ struct RoundArgs {
     __nv_bfloat16* wb[MAX_LAYERS];
     __nv_bfloat16* wbt[MAX_LAYERS];
 };
+// 32 x 32 tiles through shared memory, so that both copies are written with coalesced rows
 __global__ void __launch_bounds__(256)
 round_weights_kernel(const RoundArgs a) {
     wait_for_predecessor();
-    const int l = blockIdx.y;
+    __shared__ __nv_bfloat16 tile[32][33];
+    const int l = blockIdx.z;
     const int fan_in = a.fan_in[l], fan_out = a.fan_out[l];
-    const int64_t n = (int64_t)fan_in * fan_out;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-        const __nv_bfloat16 v = __float2bfloat16_rn(a.W[l][i]);
-        a.wb[l][i] = v;
-        const int r = (int)(i / fan_out), c = (int)(i % fan_out);
-        a.wbt[l][(int64_t)c * fan_in + r] = v;
+    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    if (r0 >= fan_in || c0 >= fan_out) return;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int r = r0 + ty + 8 * k, c = c0 + tx;
+        if (r < fan_in && c < fan_out) {
+            const __nv_bfloat16 v = __float2bfloat16_rn(a.W[l][(int64_t)r * fan_out + c]);
+            a.wb[l][(int64_t)r * fan_out + c] = v;
+            tile[ty + 8 * k][tx] = v;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int c = c0 + ty + 8 * k, r = r0 + tx;
+        if (r < fan_in && c < fan_out) a.wbt[l][(int64_t)c * fan_in + r] = tile[tx][ty + 8 * k];
     }
 }
 
@@ -342,15 +362,17 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
     const void* Wop[MAX_LAYERS];
     if (BF) {
         RoundArgs ra;
-        int64_t biggest = 0;
+        int max_in = 0, max_out = 0;
         for (int l = 0; l < L; ++l) {
             ra.fan_in[l] = p.fan[l]; ra.fan_out[l] = p.fan[l + 1]; ra.W[l] = p.W[l];
             ra.wb[l] = c.at<__nv_bfloat16>(c.ws.wb[l]); ra.wbt[l] = c.at<__nv_bfloat16>(c.ws.wbt[l]);
             Wop[l] = ra.wb[l];
-            if ((int64_t)p.fan[l] * p.fan[l + 1] > biggest) biggest = (int64_t)p.fan[l] * p.fan[l + 1];
+            if (p.fan[l] > max_in) max_in = p.fan[l];
+            if (p.fan[l + 1] > max_out) max_out = p.fan[l + 1];
         }
         KernelScope ks(&c.prof, "round_weights", st);
-        launch_dependent(round_weights_kernel, dim3((unsigned)ceil_div(biggest, 256), (unsigned)L), dim3(256), 0, st, ra);
+        launch_dependent(round_weights_kernel, dim3((unsigned)ceil_div(max_out, 32), (unsigned)ceil_div(max_in, 32), (unsigned)L),
+                         dim3(256), 0, st, ra);
     } else {
         for (int l = 0; l < L; ++l) Wop[l] = p.W[l];
     }
@@ -373,14 +395,12 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
         KernelScope ks(&c.prof, "head_out", st);
         const int nq = (int)ceil_div(HT, 256);
 #define GEAR_HEAD_OUT(NQ) launch_dependent(head_out_kernel<TX, NQ>, dim3(c.ws.loss_blocks), dim3(256), 0, st, B, HT, H[L], p.w_out, p.b_out, bt.label, \
-        o.prob, dz, dA[L], loss_part, p.gw_out, p.gb[L - 1], p.gb_out)
+        o.prob, dz, dA[L], loss_part, p.gw_out, p.gb[L - 1], p.gb_out, &c.state()->colsum_ticket, o.loss)
         if (nq <= 1) GEAR_HEAD_OUT(1);
         else if (nq == 2) GEAR_HEAD_OUT(2);
         else GEAR_HEAD_OUT(4);
 #undef GEAR_HEAD_OUT
     }
-    { KernelScope ks(&c.prof, "loss_final", st);
-    launch_dependent(loss_final_kernel, dim3(1), dim3(256), 0, st, loss_part, c.ws.loss_blocks, B, o.loss); }
     // backward
     for (int l = L - 1; l >= 0; --l) {
         const int K = p.fan[l], N = p.fan[l + 1];
