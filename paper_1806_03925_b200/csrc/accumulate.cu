@@ -433,6 +433,40 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
     leave();
 }
 
+// Steps 2-4 of the plan over the sorted keys ks / permutation perm (flag pass, scan, plan pass).
+static cudaError_t enqueue_plan(const gear_ctx_impl& c, const uint32_t* ks, const uint32_t* perm, int64_t n,
+                                const int32_t* src_row, const float* scale, cudaStream_t st) {
+    const int64_t vocab = c.cfg.img_vocab;
+    const int M = c.cfg.M;
+    DevState* state = c.state();
+    const int64_t n_tiles = ceil_div(n, AF_TILE);
+    uint2* tile_cnt = c.at<uint2>(c.ws.tile_cnt);
+    { KernelScope k(&c.prof, "acc_flag", st);
+    launch_dependent(acc_flag_kernel, dim3((unsigned)n_tiles), dim3(AF_THREADS), 0, st, ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt, state); }
+    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, &c.prof);
+    RowSource rs{perm, nullptr, 0, src_row, scale};
+    { KernelScope k(&c.prof, "acc_plan", st);
+    launch_dependent(acc_plan_kernel, dim3((unsigned)n_tiles), dim3(AF_THREADS), 0, st, ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt,
+                     c.at<uint4>(c.ws.grp_rec), rs, c.at<int2>(c.ws.pmeta), c.at<uint32_t>(c.ws.blk_first),
+                     c.at<uint32_t>(c.ws.run_end), state); }
+    return cudaGetLastError();
+}
+
+// The plan for the image occurrences of the batch gear_forward_backward has just sorted, enqueued ahead of the
+// accumulate call that will use it (on the side stream, beside the head): it depends on the sorted IDs, the counts in
+// the table and the queue length only, none of which changes before that call unless another accumulate or collect
+// comes first -- those calls drop the plan.
+cudaError_t launch_accumulate_plan_ahead(const gear_ctx_impl& c, int64_t n, const int32_t* src_row, const float* scale,
+                                         cudaStream_t st) {
+    c.plan_ready = false;
+    if (n <= 0 || !c.img_sorted || !c.img_sort_valid || c.cfg.accum_mode != GEAR_ACC_SORT) return cudaSuccess;
+    SortJob sb = c.sort_job(gear_ctx_impl::SORT_IMG);
+    cudaError_t e = enqueue_plan(c, sb.keys[c.img_sorted_buf], sb.vals[c.img_sorted_buf], n, src_row, scale, st);
+    if (e != cudaSuccess) return e;
+    c.plan_ready = true; c.plan_n = n; c.plan_src_row = src_row; c.plan_scale = scale;
+    return cudaSuccess;
+}
+
 cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
                               const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st) {
     if (n <= 0) return cudaSuccess;
@@ -440,6 +474,11 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
     const int D = c.cfg.dfv_dim, M = c.cfg.M;
     SortJob sb = c.sort_job(gear_ctx_impl::SORT_IMG);
     DevState* state = c.state();
+    const bool planned = !img_id && c.plan_ready && c.plan_n == n && c.plan_src_row == src_row && c.plan_scale == scale;
+    c.plan_ready = false;
+    // "the batch of the last gear_forward_backward" after a call with explicit IDs has used the sort buffers: sort again
+    const bool resort_batch = !img_id && !c.img_sort_valid;
+    if (resort_batch) img_id = c.last_img_id;
     int cur = c.img_sorted_buf;
     if (img_id) {
         SortBatch batch = c.sort_batch();
@@ -453,22 +492,22 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
         batch.name = "sort_img";
         cur = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
         if (se != cudaSuccess) return se;
+        c.img_sort_valid = resort_batch;
+        if (resort_batch) c.img_sorted_buf = cur;
     }
     const uint32_t* ks = sb.keys[cur];
     const int64_t n_tiles = ceil_div(n, AF_TILE);
     uint2* tile_cnt = c.at<uint2>(c.ws.tile_cnt);
-    { KernelScope k(&c.prof, "acc_flag", st);
-    launch_dependent(acc_flag_kernel, dim3((unsigned)n_tiles), dim3(AF_THREADS), 0, st, ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt, state); }
-    scan_pairs(tile_cnt, n_tiles, tile_cnt + n_tiles, st, &c.prof);
+    if (!planned) {
+        cudaError_t pe = enqueue_plan(c, ks, sb.vals[cur], n, src_row, scale, st);
+        if (pe != cudaSuccess) return pe;
+    }
     uint4* grp_rec = c.at<uint4>(c.ws.grp_rec);
     int2* pmeta = c.at<int2>(c.ws.pmeta);
-    RowSource rs{sb.vals[cur], grads, ld, src_row, scale};
     RowGather rg{grads, ld, pmeta};
     uint32_t* blk_first = c.at<uint32_t>(c.ws.blk_first);
     uint32_t* run_end = c.at<uint32_t>(c.ws.run_end);
-    { KernelScope k(&c.prof, "acc_plan", st);
-    launch_dependent(acc_plan_kernel, dim3((unsigned)n_tiles), dim3(AF_THREADS), 0, st, ks, n, (uint32_t)vocab, M, c.buf.dfv_gcnt, tile_cnt,
-                                                            grp_rec, rs, pmeta, blk_first, run_end, state); }
+    (void)vocab; (void)state;
     const int nq = (int)ceil_div(D / 4, 32);
     const int64_t want = ceil_div(ceil_div(n, ACC_SPAN), 8);
     const int resident = sm_count() * (nq <= 2 ? 3 : 2);          // every block stays resident
@@ -580,6 +619,7 @@ acc_atomic_settle_kernel(const int32_t* __restrict__ touched, int D, int M, floa
 
 cudaError_t launch_accumulate_atomic(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
                                      const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st) {
+    c.plan_ready = false;
     if (n <= 0) return cudaSuccess;
     DevState* state = c.state();
     int32_t* touched = c.at<int32_t>(c.ws.pmeta);               // the sorted path's scratch is free in this mode
@@ -695,6 +735,7 @@ __global__ void collect_end_kernel(DevState* __restrict__ state) {
 cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
                                  int64_t* d_n, cudaStream_t st) {
     DevState* state = c.state();
+    c.plan_ready = false;                                    // a plan made ahead counted on the queue length of before
     SortJob sb = c.sort_job(gear_ctx_impl::SORT_READY);
     const int64_t n_max = c.ws.ready_cap;
     const bool solo = c.acc_calls_pending <= 1;

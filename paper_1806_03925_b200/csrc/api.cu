@@ -105,8 +105,9 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 static void release_host_objects(gear_ctx_impl& c) {
     if (c.ev_fork) cudaEventDestroy(c.ev_fork);
     if (c.ev_join) cudaEventDestroy(c.ev_join);
+    if (c.ev_gather) cudaEventDestroy(c.ev_gather);
     if (c.side_stream) cudaStreamDestroy(c.side_stream);
-    c.ev_fork = c.ev_join = nullptr;
+    c.ev_fork = c.ev_join = c.ev_gather = nullptr;
     c.side_stream = nullptr;
 }
 
@@ -164,6 +165,7 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
     c.gbs.device_counter = &c.state()->grid_barrier;
     c.gbs.host_base = 0;
     c.img_sorted = false;
+    c.img_sort_valid = false;
     c.img_sorted_n = 0;
     c.img_sorted_buf = 0;
     c.last_img_id = nullptr;
@@ -171,9 +173,11 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
     c.side_stream = nullptr;
-    c.ev_fork = c.ev_join = nullptr;
+    c.ev_fork = c.ev_join = c.ev_gather = nullptr;
+    c.plan_ready = false; c.plan_n = 0; c.plan_src_row = nullptr; c.plan_scale = nullptr;
 
     cudaError_t e = cudaStreamCreateWithFlags(&c.side_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_gather, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemsetAsync(c.state(), 0, sizeof(DevState), st);
@@ -218,6 +222,7 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     // The three ID arrays of the batch are key-sorted in one launch: the user and URL orders drive the embedding
     // scatter below, the image order is kept for gear_accumulate_dfv_grad (img_id == NULL).
     c.img_sorted = false;
+    c.img_sort_valid = false;
     int sorted_buf = 0;
     bool joined_needed = false;
     if (b.B > 0) {
@@ -248,15 +253,27 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
         batch.name = "sort_ids";
         sorted_buf = sort_jobs(batch, &c.gbs, forked ? c.side_stream : st, &c.prof, &se);
         if (se != cudaSuccess) return cuda_fail(se, "id sort");
-        if (forked) {
-            se = cudaEventRecord(c.ev_join, c.side_stream);
-            if (se != cudaSuccess) return cuda_fail(se, "join");
-        }
         joined_needed = forked;
-        if (b.nnz > 0) { c.img_sorted = true; c.img_sorted_n = b.nnz; c.img_sorted_buf = sorted_buf; c.last_img_id = b.img_id; }
+        if (b.nnz > 0) {
+            c.img_sorted = true; c.img_sorted_n = b.nnz; c.img_sorted_buf = sorted_buf; c.last_img_id = b.img_id;
+            c.img_sort_valid = c.cfg.accum_mode == GEAR_ACC_SORT;
+        }
     }
+    c.plan_ready = false;
     cudaError_t e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
     if (e != cudaSuccess) return cuda_fail(e, "gather");
+    if (joined_needed) {
+        // Still on the side stream, behind the sort: the plan of the accumulate call that usually follows (which rows
+        // form which group, where every group's rows and queue slot are).  It needs the gather's row_view / inv_n.
+        if (b.nnz > 0 && o.row_view && o.inv_n && c.cfg.accum_mode == GEAR_ACC_SORT) {
+            e = cudaEventRecord(c.ev_gather, st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(c.side_stream, c.ev_gather, 0);
+            if (e == cudaSuccess) e = launch_accumulate_plan_ahead(c, b.nnz, o.row_view, o.inv_n, c.side_stream);
+            if (e != cudaSuccess) return cuda_fail(e, "accumulate plan");
+        }
+        e = cudaEventRecord(c.ev_join, c.side_stream);
+        if (e != cudaSuccess) return cuda_fail(e, "join");
+    }
     e = launch_head_simt(c, b, o, st);
     if (e != cudaSuccess) return cuda_fail(e, "head");
     if (joined_needed) {

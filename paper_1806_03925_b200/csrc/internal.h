@@ -63,7 +63,15 @@ struct gear_ctx_impl {
     const int32_t* last_img_id;         // img_id array of that batch (the atomic mode reads it unsorted)
     bool img_sorted;
     int64_t img_sorted_n;
-    int img_sorted_buf;
+    mutable int img_sorted_buf;
+    mutable bool img_sort_valid;        // the sort buffers still hold that batch's order (an accumulate call with
+                                        // explicit IDs sorts into the same buffers)
+    // accumulate plan made ahead by gear_forward_backward (valid for exactly these arguments)
+    mutable bool plan_ready;
+    mutable int64_t plan_n;
+    mutable const int32_t* plan_src_row;
+    mutable const float* plan_scale;
+    cudaEvent_t ev_gather;              // the gather's outputs (row_view, inv_n) exist
     mutable int acc_calls_pending;      // accumulate calls enqueued since a collect that was sure to drain the queue
 
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(static_cast<char*>(buf.workspace) + off); }
@@ -121,6 +129,9 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
 // GEAR_ACC_ATOMIC: reductions on the accumulator rows, then one settle pass over the touched images
 cudaError_t launch_accumulate_atomic(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
                                      const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st);
+// steps 2-4 of the sorted accumulate for the batch just sorted by gear_forward_backward, ahead of the accumulate call
+cudaError_t launch_accumulate_plan_ahead(const gear_ctx_impl& c, int64_t n, const int32_t* src_row, const float* scale,
+                                         cudaStream_t st);
 cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
                                  int64_t* d_n, cudaStream_t st);
 

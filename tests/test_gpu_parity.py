@@ -173,6 +173,37 @@ def test_single_view_and_batch_of_one_image(gb):
         pair.close()
 
 
+def test_plan_made_ahead_is_dropped_when_other_calls_come_first(gb):
+    """gear_forward_backward prepares the plan of the accumulate call that usually follows.  Calls that change what the
+    plan was made from (another accumulate, a collect) in between must not be able to make that plan go stale."""
+    from paper_1806_03925_b200.session import DeviceBatch
+    p = PRESETS["tiny"].scaled(user_vocab=500, url_vocab=400, img_vocab=300, M=2)
+    src = BatchSource(p, 3)
+    b = src.batch(0, 200)
+    extra_ids = src.batch(1, 64).img_id
+    pair = _pair(p, [b], seed=3, dense=True, extra_img_ids=extra_ids)
+    try:
+        g, cpu = pair.gpu, pair.cpu
+        db = DeviceBatch.from_host(b)
+        g.forward_backward(db)
+        r = cpu.forward_backward(pair.params.astype(np.float64), pair.ru(b.user_id), pair.rh(b.url_id), b.img_off,
+                                 pair.ri(b.img_id), b.label)
+        # another accumulate call and a collect come between the step and its own accumulate
+        rows = torch.ones((len(extra_ids), p.dfv_dim), device="cuda") * 0.5
+        g.accumulate_rows(torch.from_numpy(extra_ids).cuda(), rows)
+        cpu.accumulate(pair.ri(extra_ids), np.full((len(extra_ids), p.dfv_dim), 0.5))
+        pair.compare_store()
+        pair.collect_and_compare()
+        g.accumulate_from_step(db)
+        cpu.accumulate(pair.ri(b.img_id), cpu.dfv_grad_rows(b.img_off, r.dX))
+        pair.compare_store()
+        assert pair.collect_and_compare() > 0
+        pair.status()
+        assert pair.status_bits == 0
+    finally:
+        pair.close()
+
+
 def test_zero_sized_calls_are_accepted(gb):
     b = _manual_batch([3], [4], [[8]], [1])
     p, pair = _tiny_pair([b])
