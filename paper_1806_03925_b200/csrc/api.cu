@@ -280,14 +280,11 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
         e = cudaStreamWaitEvent(st, c.ev_join, 0);
         if (e != cudaSuccess) return cuda_fail(e, "join");
     }
-    const int E = c.cfg.emb_dim;
     float* ut = o.user_grad ? o.user_grad : c.buf.user_emb;
     float* ht = o.url_grad ? o.url_grad : c.buf.url_emb;
     const float alpha = o.user_grad ? 1.0f : -lr;
-    e = launch_emb_reduce(c, gear_ctx_impl::SORT_USER, sorted_buf, b.B, c.cfg.user_vocab, ut, o.dX, c.d_in, 0, alpha, st);
-    if (e != cudaSuccess) return cuda_fail(e, "user embedding scatter");
-    e = launch_emb_reduce(c, gear_ctx_impl::SORT_URL, sorted_buf, b.B, c.cfg.url_vocab, ht, o.dX, c.d_in, E, alpha, st);
-    if (e != cudaSuccess) return cuda_fail(e, "url embedding scatter");
+    e = launch_emb_reduce(c, sorted_buf, b.B, ut, ht, o.dX, c.d_in, alpha, st);
+    if (e != cudaSuccess) return cuda_fail(e, "embedding scatter");
     return GEAR_OK;
 }
 

@@ -14,12 +14,20 @@ namespace gear {
 constexpr int ES_SEG = 8;    // sorted positions walked by one lane group
 
 // LPR lanes share a row: lane c of the group owns the float4 chunks c, c + LPR, ... (NQ of them)
+// One of the two tables of a launch (blockIdx.y picks it).
+struct EmbTable { const uint32_t* ks; const uint32_t* perm; uint32_t vocab; int col0; float* table; };
+
 template <int NQ>
 __global__ void __launch_bounds__(256)
-emb_reduce_kernel(const uint32_t* __restrict__ ks, const uint32_t* __restrict__ perm, int n, uint32_t vocab,
-                  int E, int lpr, const float* __restrict__ dX, int64_t ldx, int col0,
-                  float* __restrict__ table, float alpha) {
+emb_reduce_kernel(const EmbTable t0, const EmbTable t1, int n, int E, int lpr, const float* __restrict__ dX, int64_t ldx,
+                  float alpha) {
     wait_for_predecessor();
+    const EmbTable& t = blockIdx.y == 0 ? t0 : t1;
+    const uint32_t* __restrict__ ks = t.ks;
+    const uint32_t* __restrict__ perm = t.perm;
+    const uint32_t vocab = t.vocab;
+    const int col0 = t.col0;
+    float* __restrict__ table = t.table;
     const int64_t gthread = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t group = gthread / lpr;
     const int c = (int)(gthread % lpr);
@@ -67,18 +75,20 @@ emb_reduce_kernel(const uint32_t* __restrict__ ks, const uint32_t* __restrict__ 
     }
 }
 
-cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int which, int cur, int32_t B, int64_t vocab, float* table,
-                              const float* dX, int ldx, int col0, float alpha, cudaStream_t st) {
+// both tables of a step in one launch: user rows (columns 0 .. E) and URL-hash rows (columns E .. 2E) of dX
+cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int cur, int32_t B, float* user_table, float* url_table,
+                              const float* dX, int ldx, float alpha, cudaStream_t st) {
     if (B <= 0) return cudaSuccess;
-    SortJob sb = c.sort_job(which);
+    SortJob su = c.sort_job(gear_ctx_impl::SORT_USER), sh = c.sort_job(gear_ctx_impl::SORT_URL);
     const int E = c.cfg.emb_dim, n_chunks = E / 4;
     int lpr = 1;
     while (lpr < n_chunks && lpr < 32) lpr <<= 1;
     const int nq = (int)ceil_div(n_chunks, lpr);
     const int64_t groups = ceil_div(B, ES_SEG);
-    const unsigned grid = (unsigned)ceil_div(groups * lpr, 256);
-#define GEAR_ES_LAUNCH(NQ) launch_dependent(emb_reduce_kernel<NQ>, dim3(grid), dim3(256), 0, st, sb.keys[cur], sb.vals[cur], B, (uint32_t)vocab, \
-                                                                        E, lpr, dX, ldx, col0, table, alpha)
+    const dim3 grid((unsigned)ceil_div(groups * lpr, 256), 2);
+    const EmbTable t0{su.keys[cur], su.vals[cur], (uint32_t)c.cfg.user_vocab, 0, user_table};
+    const EmbTable t1{sh.keys[cur], sh.vals[cur], (uint32_t)c.cfg.url_vocab, E, url_table};
+#define GEAR_ES_LAUNCH(NQ) launch_dependent(emb_reduce_kernel<NQ>, grid, dim3(256), 0, st, t0, t1, B, E, lpr, dX, (int64_t)ldx, alpha)
     KernelScope ks(&c.prof, "emb_reduce", st);
     if (nq <= 1) GEAR_ES_LAUNCH(1);
     else if (nq <= 2) GEAR_ES_LAUNCH(2);

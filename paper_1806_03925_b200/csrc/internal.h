@@ -118,9 +118,10 @@ cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int 
                             cudaStream_t st);
 
 // emb_scatter.cu
-// table[id] += alpha * (sum of the dX rows of the views with that id), given the sorted (id, view) pairs of buffer set `which`
-cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int which, int buf, int32_t B, int64_t vocab, float* table,
-                              const float* dX, int ldx, int col0, float alpha, cudaStream_t st);
+// table[id] += alpha * (sum of the dX rows of the views with that id) for the user and the URL-hash table, given the
+// sorted (id, view) pairs of buffer sets SORT_USER / SORT_URL
+cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int buf, int32_t B, float* user_table, float* url_table,
+                              const float* dX, int ldx, float alpha, cudaStream_t st);
 
 // accumulate.cu
 // img_id == nullptr: use the image IDs sorted by the last gear_forward_backward (buffer set SORT_IMG)
