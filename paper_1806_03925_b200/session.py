@@ -74,7 +74,9 @@ class GearSession:
         self.ctx = gb.gear_init_tables(self.cfg, self.user_emb, self.url_emb, self.dfv, self.dfv_gsum, self.dfv_gcnt,
                                        self.dfv_ts, self.head_params, self.workspace, seed=seed, fill=fill, now=now)
         B, nnz = self.max_batch, self.max_nnz
-        self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
+        # loss and the two counts share one small buffer, so that a caller can read them back with a single copy
+        self.scalars = torch.zeros(3, dtype=torch.int64, device=dev)
+        self.loss = self.scalars[0:1].view(torch.float32)[0:1]
         self.prob = torch.zeros(B, dtype=torch.float32, device=dev)
         self.head_grad = torch.zeros(p.n_params, dtype=torch.float32, device=dev)
         self.dX = torch.zeros((B, self.d_in), dtype=torch.float32, device=dev)
@@ -90,7 +92,7 @@ class GearSession:
         self.ready_avg = torch.zeros((self.ready_cap, p.dfv_dim), dtype=torch.float32, device=dev)
         self.expired_cap = int(expired_cap if expired_cap is not None else p.img_vocab)
         self.expired_ids = torch.zeros(self.expired_cap, dtype=torch.int32, device=dev)
-        self.d_counts = torch.zeros(2, dtype=torch.int64, device=dev)
+        self.d_counts = self.scalars[1:3]
 
     # ---- the four calls of a step ---------------------------------------------------------------
     def forward_backward(self, b: DeviceBatch, lr: Optional[float] = None):
