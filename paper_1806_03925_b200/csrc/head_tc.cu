@@ -28,23 +28,31 @@ namespace gear {
 
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
-constexpr int TC_EPI_WARPS = 8;
-constexpr int TC_THREADS = 64 + 32 * TC_EPI_WARPS;
+// Epilogue warps per CTA (a multiple of four: each warp reaches one quarter of the tensor-memory lanes).
+constexpr int tc_threads(int ew) { return 64 + 32 * ew; }
 constexpr int TC_MAX_N = 1024;            // widest output the column-sum partials cover
-constexpr int TC_STAGE_PITCH = 80;        // bytes between rows of a warp's store-staging block (64 of data + 16 of padding)
+constexpr int TC_STAGE_PITCH = 80;        // bytes between rows of a warp's mask block in shared memory (64 of data + 16 of padding)
 constexpr int TC_STAGE_BYTES = 32 * TC_STAGE_PITCH;
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
 enum { TC_EPI_BIAS_RELU = 0, TC_EPI_MASK = 1, TC_EPI_F32 = 2, TC_EPI_RED = 3 };
 
-template <int BN> struct TcCfg {
-    static constexpr int STAGES = BN == 256 ? 4 : 6;
+constexpr int TC_OUT_BLOCK = 32 * 128;   // a warp's output block on its way to a TMA store: 32 rows of 128 bytes
+
+template <int BN, int EW, int EPI> struct TcCfg {
     static constexpr int A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
     static constexpr int B_BYTES = BN * TC_BK * 2;               // 32 KB or 16 KB
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
-                                TC_MAX_N * 4 /*column sums*/ + TC_EPI_WARPS * TC_STAGE_BYTES /*store staging*/;
+    // output blocks per epilogue warp: the fp32 store sends one per 32 columns and alternates between two
+    static constexpr int OUT_BUFS = EPI == TC_EPI_RED ? 0 : (EPI == TC_EPI_F32 && EW == 8 ? 2 : 1);
+    static constexpr int OUT_BYTES = EW * OUT_BUFS * TC_OUT_BLOCK;
+    static constexpr int MASK_BYTES = EPI == TC_EPI_MASK ? EW * TC_STAGE_BYTES : 0;
+    static constexpr int FIXED = 1024 /*alignment slack*/ + 256 /*barriers*/ + TC_MAX_N * 4 /*column sums*/ + OUT_BYTES + MASK_BYTES;
+    static constexpr int ROOM = (227 * 1024 - FIXED) / STAGE_BYTES;
+    static constexpr int STAGES = ROOM > (BN == 256 ? 4 : 6) ? (BN == 256 ? 4 : 6) : ROOM;
+    static constexpr int SMEM = STAGES * STAGE_BYTES + FIXED;
     static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
+    static_assert(STAGES >= 3, "operand ring too short");
     static_assert(SMEM > 116 * 1024, "one CTA per SM: two CTAs would both ask for tensor memory");
     static_assert(SMEM <= 227 * 1024, "shared memory budget");
 };
@@ -101,6 +109,29 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                  :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
 }
 
+// Store of a shared-memory box (128-byte swizzle) into the output matrix; parts of the box past the matrix edge are
+// dropped by the copy engine.  Bulk groups belong to the issuing thread: the same lane commits and waits.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 :: "l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// The same with an L2 eviction policy for the lines written.
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, uint32_t src, int x, int y, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+                 :: "l"(map), "r"(src), "r"(x), "r"(y), "l"(policy) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int PENDING>
+__device__ __forceinline__ void tma_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(PENDING) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void sts_u4(uint32_t addr, const uint4& v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" :: "r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -137,33 +168,6 @@ __device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[32]) {
 __device__ __forceinline__ float4 ldg_f4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ uint4 ldg_u4(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
-// Coalesced store of a 32-row x 64-byte block of which lane l holds row l.  A thread of the epilogue owns a row of
-// the accumulator, so storing straight from registers would touch 32 rows per instruction, 16 bytes each; the
-// block goes through a padded shared-memory buffer instead (conflict-free 128-bit writes) and leaves as 64-byte
-// row segments, eight rows per instruction.  rows / pieces: how many rows and 16-byte pieces of the block exist.
-template <bool KEEP_IN_L2>
-__device__ __forceinline__ void store_block_64B(uint4* stage, const uint4 (&v)[4], char* gdst, int64_t row_pitch, int rows,
-                                                int pieces, int lane, uint64_t policy) {
-    constexpr int P = TC_STAGE_PITCH / 16;
-    __syncwarp();                                           // the previous block has left the buffer
-#pragma unroll
-    for (int j = 0; j < 4; ++j) stage[lane * P + j] = v[j];
-    __syncwarp();
-    const int piece = lane & 3;
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int row = it * 8 + (lane >> 2);
-        const uint4 x = stage[row * P + piece];
-        if (row < rows && piece < pieces) {
-            char* dst = gdst + (int64_t)row * row_pitch + piece * 16;
-            if (KEEP_IN_L2)
-                asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1,%2,%3,%4}, %5;"
-                             :: "l"(dst), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w), "l"(policy) : "memory");
-            else *reinterpret_cast<uint4*>(dst) = x;
-        }
-    }
-}
-
 // v[i] of lane l is element (row l, column i) of a 32 x 32 block.  Returns, on lane l, the sum of column l.
 __device__ __forceinline__ float column_sums_32x32(float (&v)[32], int lane) {
 #pragma unroll
@@ -198,22 +202,33 @@ __host__ __device__ constexpr uint32_t instr_desc(int bn, bool mn_major) {
            ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
-// Epilogue of one finished accumulator buffer `a`, as run by one of the eight epilogue warps: warp w reads
-// tensor-memory lanes 32 * (w % 4) .. + 31 (its rows of the tile); warps 2..5 take the first half of the tile's
-// columns, warps 6..9 the second half.
-template <int BN, int EPI>
-__device__ __forceinline__ void epilogue_tile(const TcArgs& g, uint32_t tmem_base, int a, int mt, int nt, int warp, int lane,
-                                              float* s_colsum, uint4* s_stage, uint64_t keep_policy) {
+// Epilogue of one finished accumulator buffer `a`, as run by one of the epilogue warps: warp w reads
+// tensor-memory lanes 32 * (w % 4) .. + 31 (its rows of the tile); the EW / 4 warps of a lane quarter split the
+// tile's columns evenly (warps 2..5 take the first share, 6..9 the second, ...).
+//
+// Output leaves through the copy engine: a lane owns a row of the accumulator, so it writes its row's 128 bytes
+// (64 bf16 or 32 fp32 columns) into a 32-row block in shared memory, 16-byte pieces XOR-swizzled by the row number
+// (conflict-free 128-bit writes, and the layout a 128-byte-swizzle tensor map expects); one lane then hands the
+// block to a TMA store, which writes whole rows of it, drops what lies past the matrix edge and needs no register
+// or issue slot of the warp while it runs.  `out_buf` is the shared-memory address of this warp's block(s).
+template <int BN, int EPI, int EW>
+__device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap* map_out, uint32_t tmem_base, int a, int mt,
+                                              int nt, int warp, int lane, float* s_colsum, uint4* s_mask, uint32_t out_buf,
+                                              uint32_t& out_turn, uint64_t keep_policy) {
     const int quarter = warp & 3;
-    const int half = (warp - 2) >> 2;
-    constexpr int CHUNKS = BN / 64;                       // 32-column chunks per warp and tile
+    const int part = (warp - 2) >> 2;
+    constexpr int COLS = BN / (EW / 4);                   // columns per warp and tile
+    constexpr int CHUNKS = COLS / 32;                     // 32-column chunks per warp and tile
+    constexpr int OUT_BUFS = TcCfg<BN, EW, EPI>::OUT_BUFS;
+    static_assert(EPI == TC_EPI_F32 || EPI == TC_EPI_RED || CHUNKS % 2 == 0, "bf16 output leaves in blocks of 64 columns");
     const int m0 = mt * TC_BM + quarter * 32;         // first row of this warp's block
     const int m = m0 + lane;
     const bool row_ok = m < g.M;
     const int rows = min(32, max(0, g.M - m0));
-    uint4* stage = s_stage + (warp - 2) * (TC_STAGE_BYTES / 16);
-    const int col0 = nt * BN + half * (BN / 2);
-    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN + half * (BN / 2));
+    uint4* stage = s_mask + (warp - 2) * (TC_STAGE_BYTES / 16);
+    const int col0 = nt * BN + part * COLS;
+    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN + part * COLS);
+    const uint32_t swz = (uint32_t)(lane & 7);
     uint32_t r[2][32];
     tc_ld32(t_row, r[0]);
 #pragma unroll
@@ -230,7 +245,7 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, uint32_t tmem_bas
         }
         if (EPI == TC_EPI_MASK) {
             // the 32 x 64-byte block of the mask, fetched as 64-byte row segments (eight rows per instruction);
-            // each lane picks up its own row from the staging buffer once the loads have landed
+            // each lane picks up its own row from the shared-memory block once the loads have landed
             const int piece = lane & 3;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -241,7 +256,7 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, uint32_t tmem_bas
         }
         tc_wait_ld(r[c & 1]);
         if (c + 1 < CHUNKS) tc_ld32(t_row + (uint32_t)((c + 1) * 32), r[(c + 1) & 1]);
-        if (!chunk_ok) continue;
+        if (!chunk_ok || rows == 0) continue;
         if (EPI == TC_EPI_MASK) {
             constexpr int P = TC_STAGE_PITCH / 16;
             __syncwarp();                               // the previous block has left the buffer
@@ -284,10 +299,22 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, uint32_t tmem_bas
                 pk[q] = *reinterpret_cast<uint32_t*>(&h2);
             }
             {
-                const uint4 blk[4] = {make_uint4(pk[0], pk[1], pk[2], pk[3]), make_uint4(pk[4], pk[5], pk[6], pk[7]),
-                                      make_uint4(pk[8], pk[9], pk[10], pk[11]), make_uint4(pk[12], pk[13], pk[14], pk[15])};
-                char* dst = reinterpret_cast<char*>(static_cast<__nv_bfloat16*>(g.out) + (int64_t)m0 * g.ldo + n0);
-                store_block_64B<false>(stage, blk, dst, g.ldo * 2, rows, min(4, (g.N - n0) / 8), lane, 0ull);
+                // chunks 2k and 2k+1 fill the left and right half of one 64-column block
+                const int half = c & 1;
+                const uint32_t row_addr = out_buf + (uint32_t)lane * 128u;
+                if (half == 0) {
+                    if (lane == 0) tma_store_wait_read<0>();          // the block's previous contents have been read
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    sts_u4(row_addr + ((((uint32_t)(4 * half + j)) ^ swz) << 4),
+                           make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]));
+                if (half == 1 || n0 + 32 >= g.N) {
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) tma_store_2d(map_out, out_buf, n0 - 32 * half, m0);
+                }
             }
             if (EPI == TC_EPI_MASK && g.colsum != nullptr) {
                 // column sums of what was stored (the rounded values); rows past M and columns past N are zero
@@ -310,33 +337,34 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, uint32_t tmem_bas
                 }
             }
         } else {
-            // fp32 output (dX), two 16-column halves; it is read again right after: keep it in the L2
+            // fp32 output (dX): one block per 32 columns, alternating between the warp's blocks; it is read again right
+            // after (embedding and DFV gradients): ask the L2 to keep it
+            const uint32_t buf = out_buf + (OUT_BUFS == 2 ? (out_turn & 1u) * (uint32_t)TC_OUT_BLOCK : 0u);
+            ++out_turn;
+            if (lane == 0) tma_store_wait_read<OUT_BUFS - 1>();       // at most the other block is still being read
+            __syncwarp();
+            const uint32_t row_addr = buf + (uint32_t)lane * 128u;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint4 blk[4] = {make_uint4(acc[16 * h + 0], acc[16 * h + 1], acc[16 * h + 2], acc[16 * h + 3]),
-                                      make_uint4(acc[16 * h + 4], acc[16 * h + 5], acc[16 * h + 6], acc[16 * h + 7]),
-                                      make_uint4(acc[16 * h + 8], acc[16 * h + 9], acc[16 * h + 10], acc[16 * h + 11]),
-                                      make_uint4(acc[16 * h + 12], acc[16 * h + 13], acc[16 * h + 14], acc[16 * h + 15])};
-                char* dst = reinterpret_cast<char*>(static_cast<float*>(g.out) + (int64_t)m0 * g.ldo + n0 + 16 * h);
-                store_block_64B<true>(stage, blk, dst, g.ldo * 4, rows, min(4, max(0, (g.N - n0 - 16 * h) / 4)), lane,
-                                      keep_policy);
-            }
+            for (int j = 0; j < 8; ++j)
+                sts_u4(row_addr + (((uint32_t)j ^ swz) << 4), make_uint4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]));
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) tma_store_2d_hint(map_out, buf, n0, m0, keep_policy);
         }
     }
 }
 
 // ---------------------------------------------------------------- the kernel
-// At most 128 registers per thread: a CTA (320 threads) then fits on an SM beside a block of the ID sort, which
-// runs on a side stream while the head starts.  One CTA per SM follows from the shared-memory footprint.
-template <int BN, bool MN_MAJOR, int EPI>
-__global__ void __maxnreg__(128)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs g) {
-    using Cfg = TcCfg<BN>;
+template <int BN, bool MN_MAJOR, int EPI, int EW>
+__device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out,
+                                             const TcArgs& g) {
+    using Cfg = TcCfg<BN, EW, EPI>;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;                  // operand stages, 1024-byte aligned
-    const uint32_t bars = tiles + STAGES * Cfg::STAGE_BYTES;        // mbarriers, then the tmem address word
+    const uint32_t out_blocks = tiles + STAGES * Cfg::STAGE_BYTES;  // output blocks of the epilogue warps, 1024-byte aligned
+    const uint32_t bars = out_blocks + Cfg::OUT_BYTES;              // mbarriers, then the tmem address word
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     auto acc_full = [&](int a) { return bars + 8u * (2 * STAGES + a); };
@@ -345,7 +373,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     volatile uint32_t* tmem_word_ptr =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_word - raw));
     float* s_colsum = reinterpret_cast<float*>(smem_raw + (bars + 256u - raw));     // [TC_MAX_N] per-CTA column sums
-    uint4* s_stage = reinterpret_cast<uint4*>(smem_raw + (bars + 256u + TC_MAX_N * 4u - raw));   // [TC_EPI_WARPS] store staging
+    uint4* s_mask = reinterpret_cast<uint4*>(smem_raw + (bars + 256u + TC_MAX_N * 4u - raw));    // [EW] mask blocks
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles * g.k_splits;
@@ -353,13 +381,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 32 * TC_EPI_WARPS); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 32 * EW); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" :: "l"(&map_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" :: "l"(&map_b) : "memory");
+        if (EPI != TC_EPI_RED) asm volatile("prefetch.tensormap [%0];" :: "l"(&map_out) : "memory");
     }
     if (EPI == TC_EPI_MASK && g.colsum != nullptr)
-        for (int n = threadIdx.x; n < TC_MAX_N; n += TC_THREADS) s_colsum[n] = 0.f;
+        for (int n = threadIdx.x; n < TC_MAX_N; n += tc_threads(EW)) s_colsum[n] = 0.f;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      :: "r"(tmem_word), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
@@ -377,7 +406,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t it = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int mt = t % g.m_tiles, nt = (t / g.m_tiles) % g.n_tiles, ks = t / (g.m_tiles * g.n_tiles);
+                // column tiles of one row tile are neighbours in the order: CTAs that run side by side read the same rows of A,
+                // which then come from memory once
+                const int nt = t % g.n_tiles, mt = (t / g.n_tiles) % g.m_tiles, ks = t / (g.m_tiles * g.n_tiles);
                 const int kb0 = ks * g.kb_per_split, kb1 = min(total_kb, kb0 + g.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int s = it % STAGES;
@@ -443,33 +474,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ---------------- epilogue warps
+        const uint32_t out_buf = out_blocks + (uint32_t)((warp - 2) * Cfg::OUT_BUFS * TC_OUT_BLOCK);
         const uint64_t keep_policy = l2_policy_evict_last();
-        uint32_t tile_it = 0;
+        uint32_t tile_it = 0, out_turn = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
-            const int mt = t % g.m_tiles, nt = (t / g.m_tiles) % g.n_tiles;
+            const int nt = t % g.n_tiles, mt = (t / g.n_tiles) % g.m_tiles;
             const int a = tile_it & 1;
             if (EPI == TC_EPI_MASK) {
                 // the rows of the ReLU mask this warp will need: ask the L2 for them now, the wait below covers the trip
-                const int m = mt * TC_BM + (warp & 3) * 32 + lane, c0 = nt * BN + ((warp - 2) >> 2) * (BN / 2);
+                constexpr int COLS = BN / (EW / 4);
+                const int m = mt * TC_BM + (warp & 3) * 32 + lane, c0 = nt * BN + ((warp - 2) >> 2) * COLS;
                 if (m < g.M)
 #pragma unroll
-                    for (int c = 0; c < BN / 2; c += 64)           // one 128-byte line per 64 bf16 columns
+                    for (int c = 0; c < COLS; c += 64)             // one 128-byte line per 64 bf16 columns
                         if (c0 + c < g.N)
                             asm volatile("prefetch.global.L2 [%0];" :: "l"(g.mask + (int64_t)m * g.ldm + c0 + c));
             }
             if (!(ok = mbar_wait(acc_full(a), (tile_it >> 1) & 1u, g.err, 4))) break;
             tc_fence_after();
-            epilogue_tile<BN, EPI>(g, tmem_base, a, mt, nt, warp, lane, s_colsum, s_stage, keep_policy);
+            epilogue_tile<BN, EPI, EW>(g, &map_out, tmem_base, a, mt, nt, warp, lane, s_colsum, s_mask, out_buf, out_turn, keep_policy);
             tc_fence_before();
             mbar_arrive_relaxed(acc_empty(a));                   // all epilogue threads arrive: the buffer returns to the MMA warp
         }
+        if (EPI != TC_EPI_RED && lane == 0) tma_store_wait_all();   // this warp's stores have left shared memory and landed
     }
 
     tc_fence_before();
     __syncthreads();
     if (EPI == TC_EPI_MASK && g.colsum != nullptr)
-        for (int n = threadIdx.x; n < g.N && n < TC_MAX_N; n += TC_THREADS) {
+        for (int n = threadIdx.x; n < g.N && n < TC_MAX_N; n += tc_threads(EW)) {
             const float v = s_colsum[n];
             if (v != 0.f) atomicAdd(g.colsum + n, v);
         }
@@ -478,6 +512,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                      :: "r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
     }
+}
+
+// Eight epilogue warps, at most 128 registers per thread: a CTA (320 threads) then fits on an SM beside a block of
+// the ID sort.  One CTA per SM follows from the shared-memory footprint.
+template <int BN, bool MN_MAJOR, int EPI>
+__global__ void __maxnreg__(128)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_out, const TcArgs g) {
+    tc_gemm_body<BN, MN_MAJOR, EPI, 8>(map_a, map_b, map_out, g);
 }
 
 // ---------------------------------------------------------------- host side
@@ -513,24 +556,40 @@ static bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool MN, int EPI>
-static cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& g, cudaStream_t st) {
-    using Cfg = TcCfg<BN>;
+// fp32 matrix [rows][cols] with leading dimension ld (elements); box = box_rows x 32 columns, 128-byte swizzle.
+static bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, bool MN, int EPI, int EW>
+static cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const TcArgs& g,
+                                  cudaStream_t st) {
+    using Cfg = TcCfg<BN, EW, EPI>;
+    static_assert(EW == 8, "one kernel entry point: eight epilogue warps");
+    auto kernel = tc_gemm_kernel<BN, MN, EPI>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, MN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Cfg::SMEM);
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
         if (e != cudaSuccess) return e;
         configured = true;
     }
     const int tiles = g.m_tiles * g.n_tiles * g.k_splits;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    return launch_dependent(tc_gemm_kernel<BN, MN, EPI>, dim3(grid), dim3(TC_THREADS), (size_t)Cfg::SMEM, st, ma, mb, g);
+    return launch_dependent(kernel, dim3(grid), dim3(tc_threads(EW)), (size_t)Cfg::SMEM, st, ma, mb, mo, g);
 }
 
-template <bool MN, int EPI>
-static cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& g, cudaStream_t st) {
-    return bn == 256 ? launch_variant<256, MN, EPI>(ma, mb, g, st) : launch_variant<128, MN, EPI>(ma, mb, g, st);
+template <bool MN, int EPI, int EW = 8>
+static cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const TcArgs& g,
+                             cudaStream_t st) {
+    return bn == 256 ? launch_variant<256, MN, EPI, EW>(ma, mb, mo, g, st) : launch_variant<128, MN, EPI, EW>(ma, mb, mo, g, st);
 }
 
 cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
@@ -538,8 +597,10 @@ cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K
                            const __nv_bfloat16* mask, int64_t ldm, float* colsum, int32_t* err, cudaStream_t st) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     const int bn = N > 128 ? 256 : 128;
-    CUtensorMap ma, mb;
+    CUtensorMap ma, mb, mo;
     if (!make_map(&ma, A, M, K, lda, TC_BM) || !make_map(&mb, W, N, K, ldw, bn)) return cudaErrorInvalidValue;
+    // the output leaves in boxes of 32 rows x 128 bytes
+    if (!(epi == TC_EPI_F32 ? make_map_f32(&mo, out, M, N, ldo, 32) : make_map(&mo, out, M, N, ldo, 32))) return cudaErrorInvalidValue;
     TcArgs g;
     g.M = M; g.N = N; g.K = K;
     g.m_tiles = (int)ceil_div(M, TC_BM); g.n_tiles = (int)ceil_div(N, bn); g.k_splits = 1;
@@ -549,9 +610,9 @@ cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K
     if (epi == TC_EPI_MASK && colsum != nullptr && g.colsum == nullptr) return cudaErrorInvalidValue;
     KernelScope ks(prof, name, st);
     switch (epi) {
-    case TC_EPI_BIAS_RELU: return launch_bn<false, TC_EPI_BIAS_RELU>(bn, ma, mb, g, st);
-    case TC_EPI_MASK: return launch_bn<false, TC_EPI_MASK>(bn, ma, mb, g, st);
-    default: return launch_bn<false, TC_EPI_F32>(bn, ma, mb, g, st);
+    case TC_EPI_BIAS_RELU: return launch_bn<false, TC_EPI_BIAS_RELU>(bn, ma, mb, mo, g, st);
+    case TC_EPI_MASK: return launch_bn<false, TC_EPI_MASK>(bn, ma, mb, mo, g, st);
+    default: return launch_bn<false, TC_EPI_F32>(bn, ma, mb, mo, g, st);
     }
 }
 
@@ -573,7 +634,7 @@ cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int 
     g.k_splits = (int)ceil_div(total_kb, g.kb_per_split);
     g.out = out; g.ldo = ldo; g.bias = nullptr; g.mask = nullptr; g.ldm = 0; g.colsum = nullptr; g.err = err;
     KernelScope ks(prof, name, st);
-    return launch_bn<true, TC_EPI_RED>(bn, ma, mb, g, st);
+    return launch_bn<true, TC_EPI_RED>(bn, ma, mb, ma /*unused: partial tiles are added with red.global*/, g, st);
 }
 
 }  // namespace gear
