@@ -627,7 +627,8 @@ cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int 
     g.M = M; g.N = N; g.K = K;
     g.m_tiles = (int)ceil_div(M, TC_BM); g.n_tiles = (int)ceil_div(N, bn);
     const int total_kb = (int)ceil_div(K, TC_BK);
-    int splits = (int)ceil_div(sm_count(), (int64_t)g.m_tiles * g.n_tiles);
+    // as many slices of the reduction as fit in one wave of CTAs (one more would leave a second, nearly empty wave)
+    int splits = sm_count() / (g.m_tiles * g.n_tiles);
     if (splits > total_kb) splits = total_kb;
     if (splits < 1) splits = 1;
     g.kb_per_split = (int)ceil_div(total_kb, splits);
