@@ -54,7 +54,7 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
     const size_t B = (size_t)c.max_batch;
     p->ready_cap = c.ready_cap > 0 ? c.ready_cap : c.max_nnz;
     p->loss_blocks = (int)ceil_div(c.max_batch, 8);
-    if (p->loss_blocks > 592) p->loss_blocks = 592;
+    if (p->loss_blocks > 2 * sm_count()) p->loss_blocks = 2 * sm_count();   // two resident blocks of the output-unit kernel per SM
 
     p->state = take(sizeof(DevState));
     p->x = take(B * d_in * hsz);

@@ -128,20 +128,45 @@ __device__ __forceinline__ void store8(__nv_bfloat16* p, float* v) {
     *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// Output unit, loss and everything that hangs off the top hidden layer.  One warp per view, a lane owns
-// 8-column chunks (128-bit loads and stores), so the top activations are read once:
+// Eight consecutive activations as they sit in memory (kept in registers between the two passes over a row).
+template <typename TX> struct Raw8;
+template <> struct Raw8<float> {
+    float4 a, b;
+    __device__ __forceinline__ void load(const float* p) { a = ld_f4(p); b = ld_f4(p + 4); }
+    __device__ __forceinline__ void clear() { a = b = make_float4(0.f, 0.f, 0.f, 0.f); }
+    __device__ __forceinline__ void unpack(float* v) const {
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    }
+};
+template <> struct Raw8<__nv_bfloat16> {
+    uint4 t;
+    __device__ __forceinline__ void load(const __nv_bfloat16* p) { t = *reinterpret_cast<const uint4*>(p); }
+    __device__ __forceinline__ void clear() { t = make_uint4(0u, 0u, 0u, 0u); }
+    __device__ __forceinline__ void unpack(float* v) const {
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { v[2 * k] = __uint_as_float(w[k] << 16); v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u); }
+    }
+};
+
+// Output unit, loss and everything that hangs off the top hidden layer:
 //   z = h . w_out + b_out;  p = sigmoid(z);  BCE in its overflow-safe form;  dz = (p - y) / B
 //   dA_top[b][j] = dz * w_out[j] where h[b][j] > 0, else 0            (stored in the head dtype)
 //   gw_out[j] += sum_b h[b][j] dz[b];  gb_top[j] += sum_b dA_top[b][j];  gb_out += sum_b dz[b]
-// NQ = chunks per lane = ceil(H / 256).
-template <typename TX, int NQ>
-__global__ void __launch_bounds__(256)
+// A warp takes ROWS views at a time; a lane owns NQ = ceil(H / 256) chunks of 8 columns (128-bit loads and stores)
+// and keeps its part of the ROWS rows in registers, so the top activations are read once.  The ROWS dot products
+// are reduced together (a shuffle transpose-reduction: lane l ends up with the sum of row l >> (5 - log2 ROWS)),
+// and sigmoid, loss and dz of the ROWS views are then worked out side by side, one view per group of lanes.
+template <typename TX, int NQ, int ROWS>
+__global__ void __launch_bounds__(256, NQ == 4 ? 1 : 2)
 head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict__ w_out,
                 const float* __restrict__ b_out, const float* __restrict__ label, float* __restrict__ prob,
                 float* __restrict__ dz, TX* __restrict__ dA, float* __restrict__ loss_part,
                 float* __restrict__ gw_out, float* __restrict__ gb_top, float* __restrict__ gb_out,
                 unsigned int* __restrict__ ticket, float* __restrict__ loss) {
     wait_for_predecessor();
+    constexpr int LG = ROWS == 8 ? 3 : ROWS == 4 ? 2 : ROWS == 2 ? 1 : 0;
+    static_assert((1 << LG) == ROWS, "ROWS is 1, 2, 4 or 8");
     __shared__ float part[8], gpart[8];
     __shared__ float s_gw[1024], s_gb[1024];
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
@@ -155,46 +180,78 @@ head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict_
     }
     float local = 0.f, gsum = 0.f;
     const float bias = b_out[0];
+    const int my_row = (int)(lane >> (5 - LG));            // the row of a batch whose sum this lane ends up with
+    const bool my_first = (lane & ((32u >> LG) - 1u)) == 0u;   // one lane per row records the row's scalars
     __syncthreads();
-    for (int b = blockIdx.x * 8 + warp; b < B; b += gridDim.x * 8) {
-        const TX* row = h + (int64_t)b * H;
-        float v[NQ][8];
-        float z = 0.f;
+    for (int b0 = (blockIdx.x * 8 + warp) * ROWS; b0 < B; b0 += gridDim.x * 8 * ROWS) {
+        Raw8<TX> raw[ROWS][NQ];
 #pragma unroll
-        for (int q = 0; q < NQ; ++q) {
-            const int c0 = (lane + 32 * q) * 8;
-            if (c0 < H) load8(row + c0, v[q]);
-            else {
+        for (int j = 0; j < ROWS; ++j)
 #pragma unroll
-                for (int k = 0; k < 8; ++k) v[q][k] = 0.f;
+            for (int q = 0; q < NQ; ++q) {
+                const int c0 = (lane + 32 * q) * 8;
+                if (b0 + j < B && c0 < H) raw[j][q].load(h + (int64_t)(b0 + j) * H + c0);
+                else raw[j][q].clear();
             }
+        float z[ROWS];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) z = fmaf(v[q][k], w[q][k], z);
+        for (int j = 0; j < ROWS; ++j) {
+            z[j] = 0.f;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                float v[8];
+                raw[j][q].unpack(v);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) z[j] = fmaf(v[k], w[q][k], z[j]);
+            }
         }
-        z = warp_sum(z) + bias;
-        const float y = label[b];
-        const float p = 1.0f / (1.0f + expf(-z));
-        const float g = (p - y) / (float)B;
-        if (lane == 0) {
-            local += fmaxf(z, 0.f) - z * y + log1pf(expf(-fabsf(z)));
+        // rows still held: ROWS, ROWS / 2, ..., 1; each round hands half of them to the lane 16, 8, 4 away
+#pragma unroll
+        for (int r = 0; r < LG; ++r) {
+            const int s = 16 >> r, half = ROWS >> (r + 1);
+            const bool upper = (lane & s) != 0;
+#pragma unroll
+            for (int i = 0; i < half; ++i) {
+                const float send = upper ? z[i] : z[i + half];
+                const float keep = upper ? z[i + half] : z[i];
+                z[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+            }
+        }
+        float zz = z[0];
+#pragma unroll
+        for (int s = 16 >> LG; s >= 1; s >>= 1) zz += __shfl_xor_sync(0xffffffffu, zz, s);
+        zz += bias;
+        const int b = b0 + my_row;
+        const bool live = b < B;
+        const float y = live ? label[b] : 0.f;
+        const float p = 1.0f / (1.0f + expf(-zz));
+        const float g = live ? (p - y) / (float)B : 0.f;
+        if (live && my_first) {
+            local += fmaxf(zz, 0.f) - zz * y + log1pf(expf(-fabsf(zz)));
             gsum += g;
             if (prob) prob[b] = p;
             dz[b] = g;
         }
-        TX* drow = dA + (int64_t)b * H;
 #pragma unroll
-        for (int q = 0; q < NQ; ++q) {
-            const int c0 = (lane + 32 * q) * 8;
-            if (c0 >= H) continue;
-            float d[8];
+        for (int j = 0; j < ROWS; ++j) {
+            const float gj = __shfl_sync(0xffffffffu, g, j << (5 - LG));
+            if (b0 + j >= B) continue;                        // warp-uniform
+            TX* drow = dA + (int64_t)(b0 + j) * H;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                gw[q][k] = fmaf(v[q][k], g, gw[q][k]);
-                d[k] = v[q][k] > 0.f ? g * w[q][k] : 0.f;
+            for (int q = 0; q < NQ; ++q) {
+                const int c0 = (lane + 32 * q) * 8;
+                if (c0 >= H) continue;
+                float v[8], d[8];
+                raw[j][q].unpack(v);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    gw[q][k] = fmaf(v[k], gj, gw[q][k]);
+                    d[k] = v[k] > 0.f ? gj * w[q][k] : 0.f;
+                }
+                store8(drow + c0, d);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) gb[q][k] += d[k];
             }
-            store8(drow + c0, d);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) gb[q][k] += d[k];
         }
     }
 #pragma unroll
@@ -204,6 +261,8 @@ head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict_
 #pragma unroll
         for (int k = 0; k < 8; ++k) { atomicAdd(&s_gw[c0 + k], gw[q][k]); atomicAdd(&s_gb[c0 + k], gb[q][k]); }
     }
+    local = warp_sum(local);                 // one lane per row of a batch held that row's terms
+    gsum = warp_sum(gsum);
     if (lane == 0) { part[warp] = local; gpart[warp] = gsum; }
     __syncthreads();
     for (int j = threadIdx.x; j < H; j += 256) { atomicAdd(gw_out + j, s_gw[j]); atomicAdd(gb_top + j, s_gb[j]); }
@@ -394,11 +453,18 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
     {
         KernelScope ks(&c.prof, "head_out", st);
         const int nq = (int)ceil_div(HT, 256);
-#define GEAR_HEAD_OUT(NQ) launch_dependent(head_out_kernel<TX, NQ>, dim3(c.ws.loss_blocks), dim3(256), 0, st, B, HT, H[L], p.w_out, p.b_out, bt.label, \
+        // rows per warp and pass: as many as the registers hold (8 chunks of bf16, 4 of fp32)
+        constexpr int RMAX = BF ? 8 : 4;
+        const int rows = nq <= 1 ? RMAX : nq == 2 ? RMAX / 4 : 1;
+        // every warp gets the same number of passes where the batch allows it
+        const int64_t batches = ceil_div(B, rows);
+        const int64_t passes = ceil_div(batches, (int64_t)c.ws.loss_blocks * 8);
+        const int blocks = (int)ceil_div(batches, 8 * passes);
+#define GEAR_HEAD_OUT(NQ, ROWS) launch_dependent(head_out_kernel<TX, NQ, ROWS>, dim3(blocks), dim3(256), 0, st, B, HT, H[L], p.w_out, p.b_out, bt.label, \
         o.prob, dz, dA[L], loss_part, p.gw_out, p.gb[L - 1], p.gb_out, &c.state()->colsum_ticket, o.loss)
-        if (nq <= 1) GEAR_HEAD_OUT(1);
-        else if (nq == 2) GEAR_HEAD_OUT(2);
-        else GEAR_HEAD_OUT(4);
+        if (nq <= 1) GEAR_HEAD_OUT(1, RMAX);
+        else if (nq == 2) GEAR_HEAD_OUT(2, RMAX / 4);
+        else GEAR_HEAD_OUT(4, 1);
 #undef GEAR_HEAD_OUT
     }
     // backward
