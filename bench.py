@@ -8,8 +8,8 @@ gear_forward_backward (gather, head forward/backward, embedding scatter), gear_a
 gear_collect_ready and gear_collect_expired.  Prints ONE JSON line (rank 0).
 
 value      page views/s with the batches already resident in HBM (device-timed, max over ranks)
-e2e        the same with the batch arrays in pinned HOST memory, copied in inside the timed region, and
-           the loss and the two counts read back every step
+e2e        the same with the batch arrays in pinned HOST memory, every step's batch copied in inside the timed
+           region (one step ahead, on a copy stream) and every step's loss and two counts read back by the host
 roofline   the kernel with the largest share of the step, timed per launch with CUDA events inside the
            library (a second pass of K steps with profiling on), against the measured machine peaks
 cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload (rank 0, N=1)
@@ -308,9 +308,9 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
     now = [0]
 
-    def one_step(db):
+    def one_step(db, expiry_beside=True):
         now[0] += 1
-        sess.step(db, now[0], sync=False)
+        sess.step(db, now[0], sync=False, expiry_beside=expiry_beside)
 
     def barrier():
         torch.cuda.synchronize()
@@ -339,9 +339,11 @@ def run_ours(args):
     n_ready_mean = None
 
     # ---- end to end: host batches in, loss and counts out, every step
-    # One pinned host buffer per batch holding its five arrays back to back (16-byte aligned), and one device buffer
-    # of the same layout whose slices are the batch the step reads: one host->device copy per step.  The loss and
-    # the two counts come back with one device->host copy of the session's 24-byte scalar block.
+    # One pinned host buffer per batch holding its five arrays back to back (16-byte aligned), and two device buffers
+    # of the same layout whose slices are the batch a step reads: one host->device copy per step, issued on a copy
+    # stream one step ahead, so that batch s+1 travels while step s computes.  The loss and the two counts of a step
+    # come back with one device->host copy of the session's 24-byte scalar block; the host reads them one step
+    # late (while the next step runs) and the last step's before the timed region ends.
     def packed_layout(nnz_cap):
         sizes = [p.batch * 4, p.batch * 4, (p.batch + 1) * 4, nnz_cap * 4, p.batch * 4]
         offs, o = [], 0
@@ -350,13 +352,13 @@ def run_ours(args):
             o = (o + sz + 15) // 16 * 16
         return offs, o
     offs, total_bytes = packed_layout(max_nnz)
-    dev_pack = torch.empty(total_bytes, dtype=torch.uint8, device="cuda")
+    dev_packs = [torch.empty(total_bytes, dtype=torch.uint8, device="cuda") for _ in range(2)]
 
     def view(buf, off, n, dt):
         return buf[off:off + n * 4].view(dt)
-    stage = DeviceBatch(view(dev_pack, offs[0], p.batch, torch.int32), view(dev_pack, offs[1], p.batch, torch.int32),
-                        view(dev_pack, offs[2], p.batch + 1, torch.int32), view(dev_pack, offs[3], max_nnz, torch.int32),
-                        view(dev_pack, offs[4], p.batch, torch.float32), B=p.batch, nnz=0)
+    stages = [DeviceBatch(view(dp, offs[0], p.batch, torch.int32), view(dp, offs[1], p.batch, torch.int32),
+                          view(dp, offs[2], p.batch + 1, torch.int32), view(dp, offs[3], max_nnz, torch.int32),
+                          view(dp, offs[4], p.batch, torch.float32), B=p.batch, nnz=0) for dp in dev_packs]
     host_packs = []
     for hb in host_batches:
         hp = torch.zeros(total_bytes, dtype=torch.uint8).pin_memory()
@@ -365,19 +367,51 @@ def run_ours(args):
             hp[off:off + raw.numel()].copy_(raw)
         host_packs.append(hp)
     h2d_bytes = total_bytes
-    host_scalars = torch.zeros(3, dtype=torch.int64).pin_memory()
+    host_scalars = [torch.zeros(3, dtype=torch.int64).pin_memory() for _ in range(2)]
+    copy_stream = torch.cuda.Stream()
+    ev_arrived = [torch.cuda.Event() for _ in range(2)]      # batch in device buffer i has landed
+    ev_consumed = [torch.cuda.Event() for _ in range(2)]     # the step that read device buffer i is done
+    ev_result = [torch.cuda.Event() for _ in range(2)]       # the scalars of that step are in host buffer i
+    results = []
 
-    def e2e_step(s):
-        hb = host_batches[s % N_BATCHES]
-        dev_pack.copy_(host_packs[s % N_BATCHES], non_blocking=True)
-        stage.nnz = hb.nnz
-        one_step(stage)
-        host_scalars.copy_(sess.scalars, non_blocking=True)
-        stream.synchronize()                       # the caller reads the loss and the counts of this step
+    def send(s):
+        i = s % 2
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(ev_consumed[i])            # the buffer's previous batch has been used
+            dev_packs[i].copy_(host_packs[s % N_BATCHES], non_blocking=True)
+            ev_arrived[i].record(copy_stream)
 
-    for s in range(min(W, 3)):
-        e2e_step(s)
-    ms_e2e = timed(e2e_step, K)
+    def e2e_run(steps):
+        for i in range(2):
+            ev_consumed[i].record(stream)
+        send(0)
+        for s in range(steps):
+            i = s % 2
+            if s + 1 < steps:
+                send(s + 1)
+            stream.wait_event(ev_arrived[i])
+            stages[i].nnz = host_batches[s % N_BATCHES].nnz
+            one_step(stages[i])
+            ev_consumed[i].record(stream)
+            host_scalars[i].copy_(sess.scalars, non_blocking=True)
+            ev_result[i].record(stream)
+            if s > 0:
+                ev_result[1 - i].synchronize()                # the caller reads the loss and the counts of step s-1
+                results.append(int(host_scalars[1 - i][1]))
+        ev_result[(steps - 1) % 2].synchronize()
+        results.append(int(host_scalars[(steps - 1) % 2][1]))
+
+    def timed_run(fn, steps):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record(stream)
+        fn(steps)
+        ev1.record(stream)
+        barrier()
+        return reps.max_over_ranks(ev0.elapsed_time(ev1), device="cuda")
+
+    e2e_run(min(W, 3))
+    ms_e2e = timed_run(e2e_run, K)
     sampler.close_window()
     clocks = sampler.stop()
     d2h_bytes = 24
@@ -387,7 +421,7 @@ def run_ours(args):
     KP = min(K, 50)
     gb.gear_profile_enable(sess.ctx, True)
     for s in range(KP):
-        one_step(dev_batches[s % N_BATCHES])
+        one_step(dev_batches[s % N_BATCHES], expiry_beside=False)      # every kernel alone, on one stream
         ready_counts.append(int(sess.d_counts[0].item()))
     prof = gb.gear_profile_read(sess.ctx, 64)
     gb.gear_profile_enable(sess.ctx, False)
@@ -423,6 +457,8 @@ def run_ours(args):
                        "M": p.M, "expire": p.expire, "mean_nnz": round(stats["nnz"], 1),
                        "l2": "tables far exceed the 126 MB L2 and rows are Zipf-random; %d pre-generated batches cycle; "
                              "no explicit flush" % N_BATCHES,
+                       "streams": "training calls on one stream, the expiry scan of the same step on a second one, "
+                                  "forked at the step's start and joined at its end (inside the timed region)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks,
             "e2e": {"value": round(reps.whole_job_rate(p.batch * K, ms_e2e), 1), "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,

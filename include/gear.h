@@ -204,6 +204,10 @@ int gear_collect_ready(gear_ctx* ctx, int32_t* ids, int32_t* seq, float* avg, in
  * Expiry scan.  Lists, in ascending order, every image with now - dfv_ts[id] >= expire; with
  * restamp != 0 the listed entries get dfv_ts[id] = now (a refresh has been requested).  Count and
  * capacity behaviour as in gear_collect_ready (too small: nothing listed, nothing restamped).
+ * The scan reads and writes nothing the other calls use (only dfv_ts, its own part of the workspace and the
+ * device status word), so it may be enqueued on a stream of its own and run beside a training step on the
+ * same ctx; the caller orders it against its own readers and writers of dfv_ts, ids and d_n.  gear_status,
+ * gear_profile_* and gear_destroy wait for that stream as well.
  */
 int gear_collect_expired(gear_ctx* ctx, int64_t now, int restamp, int32_t* ids, int64_t cap,
                          int64_t* d_n, int64_t* h_n, void* stream);

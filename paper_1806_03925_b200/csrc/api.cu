@@ -309,6 +309,14 @@ int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* 
     return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "accumulate");
 }
 
+// Waits for everything the ctx has enqueued: the stream of the training calls and, if the expiry scan went to a
+// stream of its own, that one too.
+static cudaError_t sync_streams(const gear_ctx_impl& c) {
+    cudaError_t e = cudaStreamSynchronize(c.last_stream);
+    if (e == cudaSuccess && c.expiry_used && c.expiry_stream != c.last_stream) e = cudaStreamSynchronize(c.expiry_stream);
+    return e;
+}
+
 static int finish_count(gear_ctx_impl& c, const int64_t* d_src, int64_t cap, int64_t* h_n, cudaStream_t st) {
     if (!h_n) return GEAR_OK;
     cudaError_t e = cudaMemcpyAsync(h_n, d_src, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
@@ -343,7 +351,8 @@ int gear_collect_expired(gear_ctx* ctx, int64_t now, int restamp, int32_t* ids, 
     gear_ctx_impl& c = ctx->impl;
     if (cap < 0 || (cap > 0 && !ids)) return arg_fail("NULL output with cap > 0");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    c.last_stream = st;
+    c.expiry_stream = st;          // may differ from the stream of the training calls: the scan shares nothing with them
+    c.expiry_used = true;
     int64_t* d_cnt = d_n ? d_n : &c.state()->pad[1];
     cudaError_t e = launch_collect_expired(c, now, restamp, ids, cap, d_cnt, st);
     if (e != cudaSuccess) return cuda_fail(e, "collect_expired");
@@ -354,7 +363,7 @@ int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready) {
     if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
     gear_ctx_impl& c = ctx->impl;
     DevState h;
-    cudaError_t e = cudaStreamSynchronize(c.last_stream);
+    cudaError_t e = sync_streams(c);
     if (e == cudaSuccess) e = cudaMemcpy(&h, c.state(), sizeof(DevState), cudaMemcpyDeviceToHost);
     if (h.tc_error != 0) h.status |= GEAR_DEV_TIMEOUT;
     if (e == cudaSuccess && h.status != 0) e = cudaMemset(c.state(), 0, 2 * sizeof(int32_t));   // status, tc_error
@@ -378,7 +387,7 @@ int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready) {
 
 int gear_profile_enable(gear_ctx* ctx, int on) {
     if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
-    cudaStreamSynchronize(ctx->impl.last_stream);
+    sync_streams(ctx->impl);
     ctx->impl.prof.clear();
     ctx->impl.prof.on = on != 0;
     return GEAR_OK;
@@ -388,7 +397,7 @@ int gear_profile_read(gear_ctx* ctx, char* names, float* total_ms, int32_t* laun
     if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
     if (!n_out || cap < 0 || (cap > 0 && (!names || !total_ms || !launches))) return arg_fail("gear_profile_read");
     gear_ctx_impl& c = ctx->impl;
-    cudaError_t e = cudaStreamSynchronize(c.last_stream);
+    cudaError_t e = sync_streams(c);
     if (e != cudaSuccess) return cuda_fail(e, "gear_profile_read");
     int n = 0;
     for (const auto& r : c.prof.recs) {
@@ -423,7 +432,7 @@ int gear_launch_count(gear_ctx* ctx, int64_t* n_launches) {
 int gear_destroy(gear_ctx* ctx) {
     if (!ctx) return GEAR_OK;
     if (!ctx->impl.alive) return GEAR_ERR_STATE;
-    cudaStreamSynchronize(ctx->impl.last_stream);
+    sync_streams(ctx->impl);
     cudaStreamSynchronize(ctx->impl.side_stream);
     release_host_objects(ctx->impl);
     ctx->impl.alive = false;

@@ -53,6 +53,8 @@ struct gear_ctx_impl {
     int d_in;
     int64_t n_params;
     cudaStream_t last_stream;
+    cudaStream_t expiry_stream = nullptr;   // stream of the most recent gear_collect_expired
+    bool expiry_used = false;
     bool alive;
     void* tc_state;     // tensor-core head state (tensor maps), owned by head_tc.cu; may be null
     cudaStream_t side_stream;          // runs the ID sort of a step beside the gather and the head

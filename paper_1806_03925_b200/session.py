@@ -93,6 +93,7 @@ class GearSession:
         self.expired_cap = int(expired_cap if expired_cap is not None else p.img_vocab)
         self.expired_ids = torch.zeros(self.expired_cap, dtype=torch.int32, device=dev)
         self.d_counts = self.scalars[1:3]
+        self._expiry_stream = None
 
     # ---- the four calls of a step ---------------------------------------------------------------
     def forward_backward(self, b: DeviceBatch, lr: Optional[float] = None):
@@ -124,12 +125,29 @@ class GearSession:
         return gb.gear_collect_expired(self.ctx, now, restamp, self.expired_ids, self.expired_cap,
                                        d_n=self.d_counts[1:2], sync=sync)
 
-    def step(self, b: DeviceBatch, now: int, sync: bool = False):
-        """One pass of the whole hot path over one batch."""
+    def step(self, b: DeviceBatch, now: int, sync: bool = False, expiry_beside: bool = True):
+        """One pass of the whole hot path over one batch.  The expiry scan depends on nothing the training calls
+        produce: with expiry_beside it goes to a stream of its own, starts when the step starts and is joined
+        at the step's end, so that it runs beside the gather and the head."""
+        if not expiry_beside:
+            self.forward_backward(b)
+            self.accumulate_from_step(b)
+            n_ready = self.collect_ready(sync=sync)
+            n_exp = self.collect_expired(now, restamp=True, sync=sync)
+            return n_ready, n_exp
+        main = torch.cuda.current_stream()
+        if self._expiry_stream is None:
+            self._expiry_stream = torch.cuda.Stream()
+            self._ev_fork, self._ev_join = torch.cuda.Event(), torch.cuda.Event()
+        self._ev_fork.record(main)
+        self._expiry_stream.wait_event(self._ev_fork)      # earlier readers of expired_ids and the count are done
+        with torch.cuda.stream(self._expiry_stream):
+            n_exp = self.collect_expired(now, restamp=True, sync=sync)
+            self._ev_join.record(self._expiry_stream)
         self.forward_backward(b)
         self.accumulate_from_step(b)
         n_ready = self.collect_ready(sync=sync)
-        n_exp = self.collect_expired(now, restamp=True, sync=sync)
+        main.wait_event(self._ev_join)
         return n_ready, n_exp
 
     def status(self):

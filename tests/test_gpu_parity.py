@@ -374,3 +374,46 @@ def test_large_tables_full_size_sampled(gb):
         assert g.status()[1] == 0
     finally:
         g.close()
+
+
+# ------------------------------------------------------------------ the whole step, expiry scan on a second stream
+def test_step_with_expiry_on_its_own_stream_matches_step_on_one_stream(gb):
+    """GearSession.step forks the expiry scan onto a stream of its own and joins it at the step's end; the
+    results must be those of the same calls issued one after the other on one stream.  With every timestamp 0
+    and expire 3 the scan must list every image at now = 3 and, after the restamp, again at now = 6."""
+    from gpu_harness import assert_close, _np
+    from paper_1806_03925_b200.session import DeviceBatch, GearSession
+    p = PRESETS["medium"].scaled(batch=2048, user_vocab=50_000, url_vocab=50_000, img_vocab=300_001, expire=3, M=4)
+    src = BatchSource(p, 3)
+    batches = [src.batch(s) for s in range(7)]
+    max_nnz = max(b.nnz for b in batches)
+    sessions = [GearSession(p, workloads.head_params(p, 3), max_batch=p.batch, max_nnz=max_nnz, seed=3, fill=True, now=0,
+                            expired_cap=p.img_vocab) for _ in range(2)]
+    try:
+        for sess in sessions:
+            sess.dfv_ts.zero_()
+        torch.cuda.synchronize()
+        for s, b in enumerate(batches):
+            now = s + 1
+            out = []
+            for sess, beside in zip(sessions, (False, True)):
+                n_ready, n_exp = sess.step(DeviceBatch.from_host(b), now, sync=True, expiry_beside=beside)
+                torch.cuda.synchronize()
+                out.append((n_ready, n_exp, _np(sess.ready_ids[:n_ready]), _np(sess.ready_seq[:n_ready]),
+                            _np(sess.ready_avg[:n_ready]), _np(sess.expired_ids[:n_exp]), _np(sess.loss)))
+            a, c = out
+            assert a[0] == c[0] and a[1] == c[1], (now, a[:2], c[:2])
+            assert np.array_equal(a[2], c[2]) and np.array_equal(a[3], c[3]) and np.array_equal(a[5], c[5])
+            assert_close(c[4], a[4], 1e-5, "averaged gradients")
+            assert_close(c[6], a[6], 1e-5, "loss")
+            want_all = now in (3, 6)
+            assert c[1] == (p.img_vocab if want_all else 0), (now, c[1])
+            if want_all:
+                assert np.array_equal(c[5], np.arange(p.img_vocab, dtype=np.int32))
+        assert torch.equal(sessions[0].dfv_ts, sessions[1].dfv_ts)
+        assert int(sessions[1].dfv_ts.min().item()) == 6 and int(sessions[1].dfv_ts.max().item()) == 6
+        for sess in sessions:
+            assert sess.status()[1] == 0
+    finally:
+        for sess in sessions:
+            sess.close()
