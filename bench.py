@@ -133,8 +133,23 @@ def kernel_models(p, stats):
     m["emb_reduce"] = ("hbm", 2 * (B * E * 4 + B * 8 + stats["uniq_emb"] * E * 4 * 2))      # both tables, one launch
     m["collect_move"] = ("hbm", stats["n_ready"] * (D * 4 * 2 + 16))
     fan = [Din] + list(p.hidden)
-    for l in range(len(p.hidden)):
-        m.setdefault("gemm_flops", []).append(2 * B * fan[l] * fan[l + 1])
+    L = len(p.hidden)
+    m["head_out"] = ("hbm", B * fan[L] * xsz * 2 + B * 12)          # top activations in, their gradients out
+    # the head's products: (flops, bytes) per launch.  Launches of one name share the step's products of that kind
+    # evenly.  Bytes: every operand and the output once, in the dtype it has in memory (the weights' fp32 gradient,
+    # dX fp32, everything else in the head dtype); the ReLU mask of a hidden-layer gradient is one more operand.
+    def avg(xs):
+        return sum(xs) / max(len(xs), 1)
+    layers = range(L)
+    m["gemm"] = {
+        "fwd": (avg([2 * B * fan[l] * fan[l + 1] for l in layers]),
+                avg([(B * fan[l] + fan[l] * fan[l + 1] + B * fan[l + 1]) * xsz for l in layers])),
+        "dw": (avg([2 * B * fan[l] * fan[l + 1] for l in layers]),
+               avg([(B * fan[l] + B * fan[l + 1]) * xsz + fan[l] * fan[l + 1] * 4 for l in layers])),
+        "dh": (avg([2 * B * fan[l] * fan[l + 1] for l in layers if l > 0]),
+               avg([(B * fan[l + 1] + fan[l] * fan[l + 1] + 2 * B * fan[l]) * xsz for l in layers if l > 0])),
+        "dx": (2 * B * fan[0] * fan[1], (B * fan[1] + fan[0] * fan[1]) * xsz + B * fan[0] * 4),
+    }
     return m
 
 
@@ -173,7 +188,6 @@ def roofline_for(name, ms_per_launch, p, stats, peaks):
     models = kernel_models(p, stats)
     B = stats["B"]
     fan = [p.d_in] + list(p.hidden)
-    gemm_flops_fwd = sum(2 * B * fan[l] * fan[l + 1] for l in range(len(p.hidden)))
     sec = ms_per_launch * 1e-3
     if name in models and isinstance(models[name], tuple):
         work = models[name][1]
@@ -182,19 +196,24 @@ def roofline_for(name, ms_per_launch, p, stats, peaks):
                 "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": ncu_traffic(name, p, work),
                 "peak_source": peaks["source"], "work_per_launch": work}
     if name.startswith("simt_gemm") or name.startswith("tc_gemm"):
-        # launches of one name share the step's products of that kind evenly
-        per_launch = gemm_flops_fwd / max(len(p.hidden), 1)
-        if name.endswith("dx") or name.endswith("dh"):
-            per_launch = gemm_flops_fwd / max(len(p.hidden), 1)
-        ach = per_launch / sec / 1e12
+        flops, nbytes = models["gemm"][name.rsplit("_", 1)[1]]
         if name.startswith("tc_gemm"):
-            peak, bound = peaks["bf16_sustained"] or peaks["bf16_tflops"], "tensor"
+            peak, bound, src = peaks["bf16_sustained"] or peaks["bf16_tflops"], "tensor", peaks["source"]
         else:
-            peak, bound = ALU_F32_TFLOPS, "alu"
+            peak, bound, src = ALU_F32_TFLOPS, "alu", "148 SMs x 128 FMA lanes x 2 x 1.965 GHz"
+        # the roofline that binds: with reductions and outputs of a few hundred columns these products move a byte per
+        # ~100-200 flops, which is where a B200's tensor and memory rooflines cross
+        t_math, t_mem = flops / (peak * 1e12), nbytes / (peaks["hbm_gbs"] * 1e9)
+        if t_mem > t_math:
+            ach = nbytes / sec / 1e9
+            return {"kernel": name, "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": ncu_traffic(name, p, None),
+                    "peak_source": peaks["source"], "work_per_launch": nbytes,
+                    "math_frac": round(flops / sec / 1e12 / peak, 4)}
+        ach = flops / sec / 1e12
         return {"kernel": name, "bound": bound, "achieved": round(ach, 2), "peak": round(peak, 1), "unit": "TFLOP/s",
                 "frac": round(ach / peak, 4), "traffic": ncu_traffic(name, p, None) if bound == "tensor" else None,
-                "peak_source": peaks["source"] if bound == "tensor"
-                else "148 SMs x 128 FMA lanes x 2 x 1.965 GHz", "work_per_launch": per_launch}
+                "peak_source": src, "work_per_launch": flops, "memory_frac": round(nbytes / sec / 1e9 / peaks["hbm_gbs"], 4)}
     return {"kernel": name, "bound": "latency", "achieved": None, "peak": None, "unit": None, "frac": None,
             "traffic": None}
 
