@@ -12,7 +12,8 @@
 //              tensor-memory lanes and split the tile's columns; the read of the next 32 columns and
 //              the loads of the bias / mask are in flight while the current 32 columns are processed.
 //              The ReLU-mask epilogue also sums its output columns (the bias gradient of the layer
-//              below): a shuffle transpose-reduction per 32 x 32 block, shared-memory partials per CTA.
+//              below): each lane adds up two columns of the block staged for the store; per-CTA partials
+//              in shared memory.
 // Two operand layouts:
 //   K-major   C[M][N] = A[M][K] . W[N][K]^T     (activations x weights; K contiguous in both)
 //   MN-major  C[M][N] += A[K][M]^T . B[K][N]    (weight gradients: the reduction runs over the batch,
@@ -168,21 +169,6 @@ __device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[32]) {
 __device__ __forceinline__ float4 ldg_f4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ uint4 ldg_u4(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
-// v[i] of lane l is element (row l, column i) of a 32 x 32 block.  Returns, on lane l, the sum of column l.
-__device__ __forceinline__ float column_sums_32x32(float (&v)[32], int lane) {
-#pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) {
-        const bool upper = (lane & s) != 0;       // this lane keeps the upper half of the columns still held
-#pragma unroll
-        for (int i = 0; i < s; ++i) {
-            const float send = upper ? v[i] : v[i + s];
-            const float keep = upper ? v[i + s] : v[i];
-            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
-        }
-    }
-    return v[0];
-}
-
 // Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1).
 //   K-major operand : rows of 128 bytes, 8-row groups 1024 bytes apart (SBO); LBO unused.
 //   MN-major operand: 64-element (128-byte) slabs along M/N, `lbo` bytes apart; 8-deep K groups 1024 bytes apart.
@@ -268,10 +254,11 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
         }
         uint32_t (&acc)[32] = r[c & 1];
         if (EPI == TC_EPI_BIAS_RELU || EPI == TC_EPI_MASK) {
-            float v[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
+            uint32_t pk[16];
             if (EPI == TC_EPI_BIAS_RELU) {
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     v[4 * j + 0] = fmaxf(v[4 * j + 0] + bias4[j].x, 0.f);
@@ -279,24 +266,25 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
                     v[4 * j + 2] = fmaxf(v[4 * j + 2] + bias4[j].z, 0.f);
                     v[4 * j + 3] = fmaxf(v[4 * j + 3] + bias4[j].w, 0.f);
                 }
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+                    pk[q] = *reinterpret_cast<uint32_t*>(&h2);
+                }
             } else {
+                // two columns at a time: round the pair, then clear the halves whose activation was not positive (a
+                // packed compare of the two activations against zero gives all-ones per passing half)
+                const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const uint32_t w[4] = {mask4[j].x, mask4[j].y, mask4[j].z, mask4[j].w};
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        // a post-ReLU activation is > 0 exactly when its bf16 pattern is non-zero and positive: with the
-                        // pattern in the top half of a word, that word is then at least 0x00010000 as a signed integer
-                        if ((int32_t)(w[q] << 16) < 0x10000) v[8 * j + 2 * q] = 0.f;
-                        if ((int32_t)w[q] < 0x10000) v[8 * j + 2 * q + 1] = 0.f;
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(acc[8 * j + 2 * q]), __uint_as_float(acc[8 * j + 2 * q + 1]));
+                        const unsigned int keep = __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&w[q]), zero2);
+                        pk[4 * j + q] = *reinterpret_cast<uint32_t*>(&h2) & keep;
                     }
                 }
-            }
-            uint32_t pk[16];
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
-                pk[q] = *reinterpret_cast<uint32_t*>(&h2);
             }
             {
                 // chunks 2k and 2k+1 fill the left and right half of one 64-column block
@@ -314,17 +302,24 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) tma_store_2d(map_out, out_buf, n0 - 32 * half, m0);
-                }
-            }
-            if (EPI == TC_EPI_MASK && g.colsum != nullptr) {
-                // column sums of what was stored (the rounded values); rows past M and columns past N are zero
+                    if (EPI == TC_EPI_MASK && g.colsum != nullptr) {
+                        // column sums of what was stored (the rounded values), read back from the block: lane l owns
+                        // columns 2l and 2l + 1 of the 64, one word per row (rows past M hold zeros: their operand rows
+                        // and mask were read as zeros)
+                        const int nb = n0 - 32 * half + 2 * lane;
+                        float s_lo = 0.f, s_hi = 0.f;
 #pragma unroll
-                for (int q = 0; q < 16; ++q) {
-                    v[2 * q] = row_ok ? __uint_as_float(pk[q] << 16) : 0.f;
-                    v[2 * q + 1] = row_ok ? __uint_as_float(pk[q] & 0xffff0000u) : 0.f;
+                        for (int rr = 0; rr < 32; ++rr) {
+                            uint32_t wv;
+                            const uint32_t addr = out_buf + (uint32_t)rr * 128u + ((((uint32_t)lane >> 2) ^ (uint32_t)(rr & 7)) << 4) +
+                                                  (((uint32_t)lane & 3u) << 2);
+                            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(addr) : "memory");
+                            s_lo += __uint_as_float(wv << 16);
+                            s_hi += __uint_as_float(wv & 0xffff0000u);
+                        }
+                        if (nb < g.N) { atomicAdd(&s_colsum[nb], s_lo); atomicAdd(&s_colsum[nb + 1], s_hi); }
+                    }
                 }
-                const float cs = column_sums_32x32(v, lane);
-                if (n0 + lane < g.N) atomicAdd(&s_colsum[n0 + lane], cs);
             }
         } else if (EPI == TC_EPI_RED) {
             if (row_ok) {
