@@ -80,6 +80,8 @@ def lib():
         L.orc_collect_ready.argtypes = [vp, vp, i64]
         L.orc_collect_expired.restype = i64
         L.orc_collect_expired.argtypes = [vp, i64, i64, i64, C.c_int, vp]
+        L.orc_refresh_dfv.restype = i64
+        L.orc_refresh_dfv.argtypes = [vp, C.c_int, i64, i32, vp, i64, vp, vp, vp, i64, i64, i64]
         _lib = L
     return _lib
 
@@ -288,6 +290,19 @@ class GearOracle:
         n = lib().orc_collect_expired(_ptr(self.ts), len(self.ts), int(now), self.expire, 1 if restamp else 0,
                                       _ptr(out))
         return out[:n].copy()
+
+
+    # -- refresh of cached inference results ----------------------------------------
+    def refresh_dfv(self, ids, rows: np.ndarray, now: int, ts_ids=None) -> int:
+        """Stores rows[k] (fp32) as the cached DFV of image ids[k], rounded to the table's dtype, and stamps the
+        image with now.  ts_ids: index into the timestamp array where it differs from the table row (see __init__).
+        Returns the number of skipped (out-of-range) IDs."""
+        ids = _c(np.asarray(ids), np.int32)
+        rows = _c(np.asarray(rows), np.float32)
+        assert rows.ndim == 2 and rows.shape[0] == len(ids) and rows.shape[1] == self.D
+        tid = None if ts_ids is None else _c(np.asarray(ts_ids), np.int32)
+        return int(lib().orc_refresh_dfv(_ptr(self.dfv), _dtype_tag(self.dfv), self.V, self.D, _ptr(self.ts), len(self.ts),
+                                         _ptr(ids), _ptr(tid), _ptr(rows), rows.shape[1], len(ids), int(now)))
 
 
 def sort_emissions(ids: np.ndarray, seq: np.ndarray, avg: np.ndarray):

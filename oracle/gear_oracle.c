@@ -28,6 +28,9 @@
  *   orc_collect_expired   Section 1 (second point) and Section 3: cached
  *                         inference results older than the inference-expired
  *                         time are dropped / refreshed.
+ *   orc_refresh_dfv       Section 1 (second point) and Section 3: a refreshed
+ *                         Dense Feature Vector replaces the expired cached one
+ *                         and restarts its clock.
  *   orc_fill_*            not in the paper: counter-based table
  *                         initialisation (SplitMix64, Steele, Lea and Flood
  *                         2014) so that tables too large to ship can be
@@ -507,3 +510,29 @@ int64_t orc_collect_expired(int64_t* ts, int64_t vocab, int64_t now, int64_t exp
     }
     return n;
 }
+
+/*
+ * Refresh of cached inference results (Section 1, second point; Section 3: the
+ * Slowgear side recomputes a Dense Feature Vector once its cached copy has
+ * expired): row k of `rows` (fp32, leading dimension ld) replaces the cached
+ * DFV of image ids[k], rounded to the table's storage type, and that image's
+ * timestamp becomes now.  ts_ids[k] is the image's index into ts (a test that
+ * keeps only some rows of a large table passes compact row numbers in ids and
+ * the real IDs in ts_ids; NULL means ts_ids = ids).  Entries are taken in
+ * index order.  An ID outside [0, vocab) is skipped; the return value counts
+ * those.  The gradient store (sum, count) is not touched.
+ */
+int64_t orc_refresh_dfv(void* dfv, int dt, int64_t vocab, int32_t D, int64_t* ts, int64_t ts_len,
+                        const int32_t* ids, const int32_t* ts_ids, const float* rows, int64_t ld,
+                        int64_t n, int64_t now) {
+    int64_t bad = 0;
+    for (int64_t k = 0; k < n; ++k) {
+        const int64_t id = ids[k];
+        const int64_t t = ts_ids ? ts_ids[k] : id;
+        if (id < 0 || id >= vocab || t < 0 || t >= ts_len) { ++bad; continue; }
+        for (int32_t c = 0; c < D; ++c) store_elem(dfv, dt, id * (int64_t)D + c, (double)rows[k * ld + c]);
+        ts[t] = now;
+    }
+    return bad;
+}
+

@@ -566,6 +566,70 @@ def test_restamp_makes_an_id_reappear_exactly_T_later():
 
 
 # ----------------------------------------------------------------------------
+# refresh of cached inference results
+# ----------------------------------------------------------------------------
+def test_refresh_replaces_rows_rounds_to_the_table_dtype_and_restarts_the_clock():
+    rng = np.random.default_rng(3)
+    Vi, D = 9, 5
+    for dt in (np.float64, np.float32, np.uint16):
+        table = (rng.normal(size=(Vi, D)).astype(dt) if dt != np.uint16
+                 else (rng.integers(0, 2 ** 15, (Vi, D))).astype(np.uint16))
+        before = table.copy()
+        orc = GearOracle(np.zeros((1, 1)), np.zeros((1, 1)), table, (1,), 1, 3, ts=np.arange(Vi, dtype=np.int64))
+        ids = np.array([7, 2, -1, 4, Vi], dtype=np.int32)          # two of them out of range
+        rows = rng.normal(size=(len(ids), D)).astype(np.float32)
+        rows[1, 0] = 1.0 + 2.0 ** -8                               # a tie between two bfloat16 values: goes to even (1.0)
+        rows[1, 1] = 1.0 + 3 * 2.0 ** -8                           # ... and this one up (1.015625)
+        assert orc.refresh_dfv(ids, rows, now=40) == 2
+        for k, i in enumerate(ids):
+            if not 0 <= i < Vi:
+                continue
+            if dt == np.uint16:                                    # bit patterns, against torch's own rounding
+                want = torch.from_numpy(rows[k]).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+                assert np.array_equal(orc.dfv[i], want)
+            else:
+                assert np.array_equal(orc.dfv[i], rows[k].astype(dt))
+        if dt == np.uint16:
+            assert orc.dfv[2, 0] == 0x3f80 and orc.dfv[2, 1] == 0x3f82
+        untouched = [i for i in range(Vi) if i not in (7, 2, 4)]
+        assert np.array_equal(orc.dfv[untouched], before[untouched])
+        assert list(orc.ts) == [0, 1, 40, 3, 40, 5, 6, 40, 8]
+        assert not orc.gsum.any() and not orc.gcnt.any()           # the gradient store is left alone
+        # a refreshed image is not listed again before now + T, the others are
+        assert list(orc.collect_expired(now=42, restamp=False)) == [0, 1, 3, 5, 6, 8]
+        assert list(orc.collect_expired(now=43, restamp=False)) == list(range(Vi))
+
+
+def test_refresh_in_index_order_last_row_wins_and_ts_ids_may_differ():
+    table = np.zeros((3, 2), dtype=np.float32)
+    orc = GearOracle(np.zeros((1, 1)), np.zeros((1, 1)), table, (1,), 1, 1, ts=np.zeros(10, dtype=np.int64))
+    rows = np.array([[1, 1], [2, 2], [3, 3]], dtype=np.float32)
+    assert orc.refresh_dfv([1, 0, 1], rows, now=7, ts_ids=[9, 4, 9]) == 0
+    assert np.array_equal(orc.dfv, [[2, 2], [3, 3], [0, 0]])
+    assert list(np.nonzero(orc.ts)[0]) == [4, 9] and orc.ts[9] == 7
+
+
+def test_gear_loop_with_refresh_every_step_is_ordinary_training_of_the_dense_part():
+    """M = 1, expiry 0, linear Dense Part: every step the expired list is everything, the refreshed DFVs are
+    raw @ Wd for the current Wd, and the emitted averages give dLoss/dWd exactly (Eq. 1).  Two SGD steps on Wd
+    through the loop must equal two SGD steps with the gradient taken by finite differences."""
+    orc, params, batch, raw, Wd = _linear_dense_setup(15, M=1)
+    Wd_loop, Wd_ref, lr = Wd.copy(), Wd.copy(), 0.3
+    for step in range(2):
+        expired = orc.collect_expired(now=step, restamp=True)
+        assert len(expired) == orc.V
+        orc.refresh_dfv(expired, (raw[expired] @ Wd_loop).astype(np.float32), now=step)
+        orc.dfv[:] = raw @ Wd_loop                                 # keep the fp64 table exact (refresh rows are fp32)
+        r = orc.forward_backward(params, **batch)
+        orc.accumulate(batch["img_id"], orc.dfv_grad_rows(batch["img_off"], r.dX))
+        eid, _, eavg = orc.collect_ready()
+        Wd_loop = Wd_loop - lr * sum(np.outer(raw[i], a) for i, a in zip(eid, eavg))
+        Wd_ref = Wd_ref - lr * _dense_grad_by_finite_differences(orc, params, batch, raw, Wd_ref)
+        orc.dfv[:] = raw @ Wd_loop
+    np.testing.assert_allclose(Wd_loop, Wd_ref, atol=1e-7)
+
+
+# ----------------------------------------------------------------------------
 # units whose ReLU decision is within rounding distance of zero
 # ----------------------------------------------------------------------------
 def test_near_zero_units_are_listed_and_can_take_the_other_branch():
