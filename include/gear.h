@@ -17,6 +17,8 @@
  *                             image; every M-th arrival completes a group.
  *   gear_collect_ready        event 6: hand over the averaged gradient of
  *                             every completed group.
+ *   gear_refresh_dfv          Section 1 / Section 3: recomputed DFVs replace
+ *                             expired ones and restart their clocks.
  *   gear_collect_expired      Section 1 / Section 3: cached inference results
  *                             older than the inference-expired time.
  *
@@ -211,6 +213,22 @@ int gear_collect_ready(gear_ctx* ctx, int32_t* ids, int32_t* seq, float* avg, in
  */
 int gear_collect_expired(gear_ctx* ctx, int64_t now, int restamp, int32_t* ids, int64_t cap,
                          int64_t* d_n, int64_t* h_n, void* stream);
+
+/*
+ * Refresh of cached inference results (Section 1, second point; Section 3: a Dense Feature Vector whose cached
+ * copy has expired is computed again by the Dense Part).  For k < n:
+ *     dfv[ids[k]][c] = rows[k * ld + c] rounded to dfv_dtype (bf16: nearest even), c < dfv_dim;  dfv_ts[ids[k]] = now.
+ * The gradient store is not touched: gradients taken against the old vector keep accumulating.
+ * ids: device, distinct -- the list gear_collect_expired returns qualifies; if an ID repeats, one of its rows is
+ * stored, unspecified which.  rows: device fp32, 16-byte aligned, ld a multiple of 4.  An ID outside
+ * [0, img_vocab) is skipped and raises GEAR_DEV_BAD_ID.  d_n (device, optional): the call processes
+ * min(n, *d_n) entries, *d_n read on the device when the kernel runs, so that the count an expiry scan has just
+ * written can be used without a trip to the host (n is then the capacity of ids / rows).
+ * The call writes dfv and dfv_ts: the caller orders it after the training calls that should still see the old
+ * vectors and before the next expiry scan (same stream, or events between streams).
+ */
+int gear_refresh_dfv(gear_ctx* ctx, const int32_t* ids, const float* rows, int64_t ld, int64_t n,
+                     const int64_t* d_n, int64_t now, void* stream);
 
 /*
  * Synchronises the stream last used; returns the device status word (GEAR_DEV_* bits, then cleared) and

@@ -25,7 +25,7 @@ GEAR_TAG_USER, GEAR_TAG_URL, GEAR_TAG_DFV, GEAR_TAG_TS, GEAR_TAG_GRAD = 1, 2, 3,
 EXPORTS = ("gear_workspace_bytes", "gear_init_tables", "gear_forward_backward", "gear_accumulate_dfv_grad",
            "gear_collect_ready", "gear_collect_expired", "gear_status", "gear_destroy", "gear_fill_uniform",
            "gear_last_error", "gear_profile_enable", "gear_profile_read", "gear_launch_count",
-           "gear_collect_expired_static")
+           "gear_collect_expired_static", "gear_refresh_dfv")
 GEAR_STATIC_EXPIRY_MAX_VOCAB = 16777216
 
 
@@ -86,6 +86,8 @@ def load() -> C.CDLL:
     L.gear_collect_expired.restype = C.c_int
     L.gear_collect_expired.argtypes = [vp, i64, C.c_int, vp, i64, vp, C.POINTER(i64), vp]
     L.gear_status.restype = C.c_int
+    L.gear_refresh_dfv.restype = C.c_int
+    L.gear_refresh_dfv.argtypes = [vp, vp, vp, i64, i64, vp, i64, vp]
     L.gear_status.argtypes = [vp, C.POINTER(i32), C.POINTER(i64)]
     L.gear_destroy.restype = C.c_int
     L.gear_destroy.argtypes = [vp]
@@ -207,6 +209,13 @@ def gear_collect_expired(ctx, now: int, restamp: bool, ids, cap: int, d_n=None, 
     _check(load().gear_collect_expired(ctx, now, 1 if restamp else 0, _p(ids), cap, _p(d_n),
                                        C.byref(h) if sync else None, _stream(stream)), "gear_collect_expired")
     return h.value if sync else None
+
+
+def gear_refresh_dfv(ctx, ids, rows, n: int, now: int, d_n=None, stream=None):
+    """rows: fp32 [>= n][ld] device tensor (stride(0) = ld); processes min(n, *d_n) entries when d_n is given."""
+    assert rows.is_cuda and rows.dtype == torch.float32 and rows.dim() == 2 and rows.stride(1) == 1
+    _check(load().gear_refresh_dfv(ctx, _p(ids), C.c_void_p(rows.data_ptr()), rows.stride(0), n, _p(d_n), now, _stream(stream)),
+           "gear_refresh_dfv")
 
 
 def gear_status(ctx, raise_on_error: bool = False):

@@ -313,7 +313,8 @@ int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* 
 // stream of its own, that one too.
 static cudaError_t sync_streams(const gear_ctx_impl& c) {
     cudaError_t e = cudaStreamSynchronize(c.last_stream);
-    if (e == cudaSuccess && c.expiry_used && c.expiry_stream != c.last_stream) e = cudaStreamSynchronize(c.expiry_stream);
+    for (int i = 0; i < c.n_seen && e == cudaSuccess; ++i)
+        if (c.seen_stream[i] != c.last_stream) e = cudaStreamSynchronize(c.seen_stream[i]);
     return e;
 }
 
@@ -351,12 +352,26 @@ int gear_collect_expired(gear_ctx* ctx, int64_t now, int restamp, int32_t* ids, 
     gear_ctx_impl& c = ctx->impl;
     if (cap < 0 || (cap > 0 && !ids)) return arg_fail("NULL output with cap > 0");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    c.expiry_stream = st;          // may differ from the stream of the training calls: the scan shares nothing with them
-    c.expiry_used = true;
+    c.note_stream(st);             // may differ from the stream of the training calls: the scan shares nothing with them
     int64_t* d_cnt = d_n ? d_n : &c.state()->pad[1];
     cudaError_t e = launch_collect_expired(c, now, restamp, ids, cap, d_cnt, st);
     if (e != cudaSuccess) return cuda_fail(e, "collect_expired");
     return finish_count(c, d_cnt, cap, h_n, st);
+}
+
+int gear_refresh_dfv(gear_ctx* ctx, const int32_t* ids, const float* rows, int64_t ld, int64_t n, const int64_t* d_n,
+                     int64_t now, void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (n < 0) return arg_fail("n < 0");
+    if (n == 0) return GEAR_OK;
+    if (!ids || !rows) return arg_fail("NULL pointer");
+    if (ld < c.cfg.dfv_dim || (ld & 3) || !aligned16(rows)) return arg_fail("rows must be 16-byte aligned, ld >= dfv_dim and a multiple of 4");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.note_stream(st);
+    cudaError_t e = launch_refresh_dfv(c, ids, rows, ld, n, d_n, now, st);
+    if (e != cudaSuccess) return cuda_fail(e, "refresh_dfv");
+    return GEAR_OK;
 }
 
 int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready) {

@@ -53,8 +53,16 @@ struct gear_ctx_impl {
     int d_in;
     int64_t n_params;
     cudaStream_t last_stream;
-    cudaStream_t expiry_stream = nullptr;   // stream of the most recent gear_collect_expired
-    bool expiry_used = false;
+    // streams the calls were enqueued on (the expiry scan and the refresh may sit on streams of their own); the
+    // calls that wait for the ctx's work wait for all of them
+    static constexpr int MAX_STREAMS = 4;
+    cudaStream_t seen_stream[MAX_STREAMS] = {};
+    int n_seen = 0;
+    void note_stream(cudaStream_t st) {
+        for (int i = 0; i < n_seen; ++i) if (seen_stream[i] == st) return;
+        if (n_seen < MAX_STREAMS) seen_stream[n_seen++] = st;
+        else { cudaStreamSynchronize(seen_stream[0]); seen_stream[0] = st; }     // a fifth stream: retire the oldest
+    }
     bool alive;
     void* tc_state;     // tensor-core head state (tensor maps), owned by head_tc.cu; may be null
     cudaStream_t side_stream;          // runs the ID sort of a step beside the gather and the head
@@ -139,6 +147,8 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
                                  int64_t* d_n, cudaStream_t st);
 
 // expiry.cu
+cudaError_t launch_refresh_dfv(const gear_ctx_impl& c, const int32_t* ids, const float* rows, int64_t ld, int64_t n,
+                               const int64_t* d_n, int64_t now, cudaStream_t st);
 cudaError_t launch_collect_expired(const gear_ctx_impl& c, int64_t now, int restamp, int32_t* ids, int64_t cap,
                                    int64_t* d_n, cudaStream_t st);
 

@@ -125,6 +125,10 @@ class GearSession:
         return gb.gear_collect_expired(self.ctx, now, restamp, self.expired_ids, self.expired_cap,
                                        d_n=self.d_counts[1:2], sync=sync)
 
+    def refresh_dfv(self, ids: torch.Tensor, rows: torch.Tensor, now: int, n: Optional[int] = None, d_n=None):
+        """Recomputed DFVs replace cached ones (rows fp32) and restart their clocks."""
+        return gb.gear_refresh_dfv(self.ctx, ids, rows, int(ids.shape[0]) if n is None else n, now, d_n=d_n)
+
     def step(self, b: DeviceBatch, now: int, sync: bool = False, expiry_beside: bool = True):
         """One pass of the whole hot path over one batch.  The expiry scan depends on nothing the training calls
         produce: with expiry_beside it goes to a stream of its own, starts when the step starts and is joined

@@ -417,3 +417,93 @@ def test_step_with_expiry_on_its_own_stream_matches_step_on_one_stream(gb):
     finally:
         for sess in sessions:
             sess.close()
+
+
+# ------------------------------------------------------------------ refresh of cached DFVs
+@pytest.mark.parametrize("name", ["tiny", "medium"])
+def test_refresh_dfv_matches_oracle(gb, name):
+    """Rows, timestamps and the skipped-ID flag, bit for bit; fp32 table (tiny) and bf16 table (medium); source rows
+    with a leading dimension wider than the row; the device-side count bounds the call."""
+    from gpu_harness import _np
+    p = PRESETS[name].scaled(img_vocab=60_000) if name == "medium" else PRESETS[name]
+    rng = np.random.default_rng(5)
+    n = 3000
+    ids = rng.choice(p.img_vocab, n, replace=False).astype(np.int32)
+    ids[17], ids[1234] = -3, p.img_vocab                     # skipped, flagged
+    rows = rng.normal(0, 1, (n + 100, p.dfv_dim + 12)).astype(np.float32)
+    rows[5, :4] = [1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -0.0, 3.0e38]      # bf16 ties and edge values
+    pair = _pair(p, [], seed=2, dense=True)
+    g, cpu = pair.gpu, pair.cpu
+    try:
+        d_ids, d_rows = torch.from_numpy(ids).cuda(), torch.from_numpy(rows).cuda()
+        view = d_rows[:, :p.dfv_dim]                                          # ld = dfv_dim + 12
+        # first call: everything; second call: capacity n, the device count says 1000 (other rows, other time)
+        g.refresh_dfv(d_ids, view, now=77)
+        assert cpu.refresh_dfv(ids, rows[:n, :p.dfv_dim], now=77) == 2
+        d_n = torch.tensor([1000], dtype=torch.int64, device="cuda")
+        g.refresh_dfv(d_ids, view[100:], now=90, n=n, d_n=d_n)
+        assert cpu.refresh_dfv(ids[:1000], rows[100:1100, :p.dfv_dim], now=90) == 1
+        got = g.dfv.view(torch.int16).cpu().numpy().view(np.uint16) if p.dfv_dtype == BF16 else _np(g.dfv)
+        assert np.array_equal(got, cpu.dfv)
+        assert np.array_equal(_np(g.dfv_ts), cpu.ts)
+        assert not g.dfv_gsum.any().item() and not g.dfv_gcnt.any().item()
+        rc, bits, _ = g.status()
+        assert bits & gb.GEAR_DEV_BAD_ID
+        # argument checks: misaligned rows, short leading dimension
+        with pytest.raises(gb.GearError):
+            gb.gear_refresh_dfv(g.ctx, d_ids, d_rows[:, 1:1 + p.dfv_dim], n, 5)
+        # a refreshed image is gathered in its new form and not listed by the scan before now + expire
+        k = g.collect_expired(90 + p.expire - 1, restamp=False)
+        listed = set(_np(g.expired_ids[:k]).tolist())
+        assert not (set(ids[:1000].tolist()) - {-3, p.img_vocab}) & listed
+    finally:
+        g.close()
+
+
+def test_gear_loop_with_refresh_on_the_gpu_path_trains_a_linear_dense_part(gb):
+    """M = 1, expiry 0, a linear Dense Part DFV_i = raw_i . Wd kept by the test: every step the scan lists every
+    image, gear_refresh_dfv writes raw . Wd for the current Wd, and the emitted averages give dLoss/dWd (Eq. 1).
+    Two SGD steps on Wd through the GPU path against the same loop on the oracle."""
+    from gpu_harness import _np, assert_close
+    p = PRESETS["tiny"].scaled(M=1, expire=0, img_vocab=512, batch=128)
+    R = 24
+    rng = np.random.default_rng(9)
+    raw = rng.normal(0, 1, (p.img_vocab, R)).astype(np.float32)
+    Wd0 = rng.normal(0, 0.3, (R, p.dfv_dim)).astype(np.float32)
+    src = BatchSource(p, 4)
+    batches = [src.batch(s) for s in range(2)]
+    pair = _pair(p, batches, seed=4, dense=True)
+    g, cpu = pair.gpu, pair.cpu
+    try:
+        Wd_g, Wd_c, lr = Wd0.copy(), Wd0.astype(np.float64), 5.0
+        for step, b in enumerate(batches):
+            now = step + 1
+            from paper_1806_03925_b200.session import DeviceBatch
+            # --- GPU path
+            k = g.collect_expired(now, restamp=True)
+            assert k == p.img_vocab
+            ids = g.expired_ids[:k]
+            rows = torch.from_numpy(raw).cuda()[ids.long()] @ torch.from_numpy(Wd_g).cuda()
+            g.refresh_dfv(ids, rows.contiguous(), now)
+            db = DeviceBatch.from_host(b)
+            g.forward_backward(db, lr=0.0)
+            g.accumulate_from_step(db)
+            n_ready = g.collect_ready()
+            assert n_ready == b.nnz                                    # M = 1: every gradient row is emitted
+            eid, eavg = _np(g.ready_ids[:n_ready]), _np(g.ready_avg[:n_ready]).astype(np.float64)
+            G_g = raw[eid].astype(np.float64).T @ eavg
+            # --- oracle
+            exp_c = cpu.collect_expired(now, restamp=True)
+            cpu.refresh_dfv(exp_c, (raw[exp_c] @ Wd_c.astype(np.float32)).astype(np.float32), now)
+            r = cpu.forward_backward(pair.params.astype(np.float64), b.user_id, b.url_id, b.img_off, b.img_id, b.label)
+            cpu.accumulate(b.img_id, cpu.dfv_grad_rows(b.img_off, r.dX))
+            cid, _, cavg = cpu.collect_ready()
+            G_c = raw[cid].astype(np.float64).T @ cavg
+            assert_close(G_g, G_c, 1e-4, "dense-part gradient of step %d" % step)
+            Wd_g = (Wd_g - lr * G_g).astype(np.float32)
+            Wd_c = Wd_c - lr * G_c
+        assert_close(Wd_g.astype(np.float64), Wd_c, 1e-4, "dense-part weights after two steps")
+        assert np.abs(Wd_c - Wd0).max() > 1e-4                         # the steps did move the weights
+        assert g.status()[1] == 0
+    finally:
+        g.close()
