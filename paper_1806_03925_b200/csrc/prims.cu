@@ -122,11 +122,33 @@ coop_sort_kernel(const SortBatch batch) {
         }
         if (!(ok = sync_all())) break;
 
-        // ---- scan: per digit (one warp per row), exclusive scan of the per-tile counts; digit totals
+        // ---- scan: per digit, exclusive scan of the per-tile counts; digit totals.  Jobs of few tiles: one thread per
+        //      digit row (its loads are independent, so the rows of all digits cost one trip to the L2 together);
+        //      jobs of many tiles: one warp per row.
+        constexpr int RS_ROW_THREAD_TILES = 32;
+        for (int r = blockIdx.x * RS_THREADS + threadIdx.x; r < batch.n_jobs * RS_BUCKETS; r += nblk * RS_THREADS) {
+            const int jj = r / RS_BUCKETS, d = r % RS_BUCKETS;
+            const SortJob& j = batch.job[jj];
+            const int nt = live_tiles[jj];
+            if (d >= (1 << j.width) || nt > RS_ROW_THREAD_TILES) continue;
+            uint32_t* row = j.hist + (int64_t)d * j.n_tiles;
+            uint32_t carry = 0;
+            for (int b0 = 0; b0 < nt; b0 += 8) {
+                uint32_t v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = b0 + q < nt ? __ldcg(row + b0 + q) : 0u;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (b0 + q < nt) __stcg(row + b0 + q, carry);
+                    carry += v[q];
+                }
+            }
+            __stcg(j.tot + d, carry);
+        }
         for (int r = blockIdx.x * (RS_THREADS / 32) + warp; r < batch.n_jobs * RS_BUCKETS; r += nblk * (RS_THREADS / 32)) {
             const int jj = r / RS_BUCKETS, d = r % RS_BUCKETS;
             const SortJob& j = batch.job[jj];
-            if (d >= (1 << j.width)) continue;
+            if (d >= (1 << j.width) || live_tiles[jj] <= RS_ROW_THREAD_TILES) continue;
             uint32_t* row = j.hist + (int64_t)d * j.n_tiles;
             uint32_t carry = 0;
             for (int b0 = 0; b0 < live_tiles[jj]; b0 += 32) {
