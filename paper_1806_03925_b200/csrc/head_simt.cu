@@ -87,12 +87,177 @@ gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sam, int64_t 
     }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// The same product for fp32 operands of at least 128 x 128 outputs: 128 x 128 x 8 tiles, 8 x 8 outputs per
+// thread (two 4-wide strips in each direction, 64 apart, so that shared-memory reads are 128-bit and free of
+// bank conflicts), operand tiles fetched with 128-bit loads one tile ahead into registers and passed through two
+// shared-memory buffers (one __syncthreads per tile).  Either operand may be contiguous along the reduction
+// (K_FAST) or along its other index; leading dimensions must be multiples of 4 and the pointers 16-byte
+// aligned (the launcher falls back to the 64 x 64 kernel otherwise).  16 FMAs per 128-bit shared-memory read.
+// ---------------------------------------------------------------------------------------------------
+constexpr int BT = 128;   // tile edge in M and N
+constexpr int BK = 8;     // tile depth
+
+// The 128-bit piece of an operand tile that thread `tid` fetches: K_FAST: row (tid / 2) of the tile, reduction
+// indices 4 * (tid % 2) .. + 3; else reduction index tid / 32, rows 4 * (tid % 32) .. + 3.  Out-of-range parts are
+// zero (whole pieces: the extents are multiples of 4 where it matters, see the launcher).
+template <bool K_FAST>
+__device__ __forceinline__ float4 fetch_piece(const float* __restrict__ base, int64_t ld, int row0, int rows, int k0,
+                                              int k_end, int tid) {
+    if (K_FAST) {
+        const int r = row0 + (tid >> 1), k = k0 + 4 * (tid & 1);
+        if (r < rows && k + 3 < k_end) return __ldg(reinterpret_cast<const float4*>(base + (int64_t)r * ld + k));
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < rows) {
+            const float* p = base + (int64_t)r * ld;
+            if (k < k_end) v.x = __ldg(p + k);
+            if (k + 1 < k_end) v.y = __ldg(p + k + 1);
+            if (k + 2 < k_end) v.z = __ldg(p + k + 2);
+        }
+        return v;
+    } else {
+        const int k = k0 + (tid >> 5), r = row0 + 4 * (tid & 31);
+        if (k < k_end && r + 3 < rows) return __ldg(reinterpret_cast<const float4*>(base + (int64_t)k * ld + r));
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (k < k_end) {
+            const float* p = base + (int64_t)k * ld;
+            if (r < rows) v.x = __ldg(p + r);
+            if (r + 1 < rows) v.y = __ldg(p + r + 1);
+            if (r + 2 < rows) v.z = __ldg(p + r + 2);
+        }
+        return v;
+    }
+}
+// ... and where it goes in the [BK][BT + 4] shared-memory tile
+template <bool K_FAST>
+__device__ __forceinline__ void stash_piece(float (*tile)[BT + 4], const float4& v, int tid) {
+    if (K_FAST) {
+        const int r = tid >> 1, k = 4 * (tid & 1);
+        tile[k][r] = v.x; tile[k + 1][r] = v.y; tile[k + 2][r] = v.z; tile[k + 3][r] = v.w;
+    } else {
+        *reinterpret_cast<float4*>(&tile[tid >> 5][4 * (tid & 31)]) = v;
+    }
+}
+
+// C[m][n] (+)= epi( sum_k A(m,k) B(k,n) ).  A_KFAST: A(m,k) = A[m * lda + k], else A[k * lda + m];
+// B_KFAST: B(k,n) = B[n * ldb + k], else B[k * ldb + n].  blockIdx.z selects a k-range of k_chunk elements.
+template <bool A_KFAST, bool B_KFAST, int EPI>
+__global__ void __launch_bounds__(256, 2)
+gemm128_kernel(int M, int N, int K, const float* __restrict__ A, int64_t lda, const float* __restrict__ Bm, int64_t ldb,
+               float* __restrict__ C, int64_t ldc, const float* __restrict__ bias, const float* __restrict__ mask,
+               int64_t ldm, int k_chunk) {
+    wait_for_predecessor();
+    __shared__ __align__(16) float As[2][BK][BT + 4];
+    __shared__ __align__(16) float Bs[2][BK][BT + 4];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int m0 = blockIdx.y * BT, n0 = blockIdx.x * BT;
+    const int k_begin = blockIdx.z * k_chunk, k_end = min(K, k_begin + k_chunk);
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+
+    float4 pa = fetch_piece<A_KFAST>(A, lda, m0, M, k_begin, k_end, tid);
+    float4 pb = fetch_piece<B_KFAST>(Bm, ldb, n0, N, k_begin, k_end, tid);
+    stash_piece<A_KFAST>(As[0], pa, tid);
+    stash_piece<B_KFAST>(Bs[0], pb, tid);
+    __syncthreads();
+    int buf = 0;
+    for (int k0 = k_begin; k0 < k_end; k0 += BK) {
+        const bool more = k0 + BK < k_end;
+        if (more) {                                               // the next tile travels while this one is used
+            pa = fetch_piece<A_KFAST>(A, lda, m0, M, k0 + BK, k_end, tid);
+            pb = fetch_piece<B_KFAST>(Bm, ldb, n0, N, k0 + BK, k_end, tid);
+        }
+#pragma unroll
+        for (int k = 0; k < BK; ++k) {
+            const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][k][ty * 4]);
+            const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][k][64 + ty * 4]);
+            const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
+            const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][k][64 + tx * 4]);
+            const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        if (more) {
+            stash_piece<A_KFAST>(As[buf ^ 1], pa, tid);           // the other buffer: nobody reads it during this tile
+            stash_piece<B_KFAST>(Bs[buf ^ 1], pb, tid);
+            __syncthreads();
+            buf ^= 1;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int gm = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + i - 4);
+        if (gm >= M) continue;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int gn = n0 + 64 * h + tx * 4;
+            if (gn >= N) continue;                                // N is a multiple of 4 here: whole 4-wide strips
+            float v[4] = {acc[i][4 * h], acc[i][4 * h + 1], acc[i][4 * h + 2], acc[i][4 * h + 3]};
+            if (EPI == EPI_BIAS_RELU) {
+                const float4 bb = __ldg(reinterpret_cast<const float4*>(bias + gn));
+                v[0] = fmaxf(v[0] + bb.x, 0.f); v[1] = fmaxf(v[1] + bb.y, 0.f);
+                v[2] = fmaxf(v[2] + bb.z, 0.f); v[3] = fmaxf(v[3] + bb.w, 0.f);
+            }
+            if (EPI == EPI_MASK) {
+                const float4 mm = __ldg(reinterpret_cast<const float4*>(mask + (int64_t)gm * ldm + gn));
+                v[0] = mm.x > 0.f ? v[0] : 0.f; v[1] = mm.y > 0.f ? v[1] : 0.f;
+                v[2] = mm.z > 0.f ? v[2] : 0.f; v[3] = mm.w > 0.f ? v[3] : 0.f;
+            }
+            float* dst = C + (int64_t)gm * ldc + gn;
+            if (EPI == EPI_ATOMIC) red_add_f4(dst, make_float4(v[0], v[1], v[2], v[3]));
+            else st_f4(dst, make_float4(v[0], v[1], v[2], v[3]));
+        }
+    }
+}
+
+static bool ptr16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Tries the 128 x 128 kernel; false if the shapes, strides or alignments do not fit it.
+template <int EPI>
+static bool try_gemm128(int M, int N, int K, const float* A, int64_t sam, int64_t sak, const float* B, int64_t sbk,
+                        int64_t sbn, float* C, int64_t ldc, const float* bias, const float* mask, int64_t ldm, int splits,
+                        cudaStream_t st) {
+    if (M < 96 || N < 96 || (N & 3) || (ldc & 3) || !ptr16(C) || !ptr16(A) || !ptr16(B)) return false;
+    const bool a_kfast = sak == 1, b_kfast = sbk == 1;
+    if (!a_kfast && sam != 1) return false;
+    if (!b_kfast && sbn != 1) return false;
+    const int64_t lda = a_kfast ? sam : sak, ldb = b_kfast ? sbn : sbk;
+    if ((lda & 3) || (ldb & 3)) return false;
+    if (EPI == EPI_BIAS_RELU && !ptr16(bias)) return false;
+    if (EPI == EPI_MASK && ((ldm & 3) || !ptr16(mask))) return false;
+    // as many slices of the reduction as fill the GPU twice over (two blocks per SM), each a multiple of the tile depth
+    const int64_t tiles = ceil_div(M, BT) * ceil_div(N, BT);
+    int64_t s = splits > 1 ? ceil_div(2 * sm_count(), tiles) : 1;
+    const int64_t max_s = ceil_div(K, 256);
+    if (s > max_s) s = max_s;
+    if (s < 1) s = 1;
+    const int k_chunk = (int)ceil_div(ceil_div(K, s), BK) * BK;
+    const dim3 grid((unsigned)ceil_div(N, BT), (unsigned)ceil_div(M, BT), (unsigned)ceil_div(K, k_chunk));
+#define GEAR_G128(AK, BKF) launch_dependent(gemm128_kernel<AK, BKF, EPI>, grid, dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, bias, mask, ldm, k_chunk)
+    if (a_kfast && !b_kfast) GEAR_G128(true, false);
+    else if (!a_kfast && !b_kfast) GEAR_G128(false, false);
+    else if (a_kfast && b_kfast) GEAR_G128(true, true);
+    else GEAR_G128(false, true);
+#undef GEAR_G128
+    return true;
+}
+
 template <typename TA, typename TB, typename TC, typename TM, int EPI>
 static void launch_gemm(int M, int N, int K, const TA* A, int64_t sam, int64_t sak, const TB* B, int64_t sbk,
                         int64_t sbn, TC* C, int64_t ldc, const float* bias, const TM* mask, int64_t ldm,
                         int splits, cudaStream_t st, Profiler* prof, const char* name) {
     if (M <= 0 || N <= 0 || K <= 0) return;
     KernelScope ks(prof, name, st);
+    if constexpr (std::is_same<TA, float>::value && std::is_same<TB, float>::value && std::is_same<TC, float>::value &&
+                  std::is_same<TM, float>::value) {
+        if (try_gemm128<EPI>(M, N, K, A, sam, sak, B, sbk, sbn, C, ldc, bias, mask, ldm, splits, st)) return;
+    }
     int k_chunk = (int)ceil_div(ceil_div(K, splits), GK) * GK;
     splits = (int)ceil_div(K, k_chunk);
     dim3 grid((unsigned)ceil_div(N, GT), (unsigned)ceil_div(M, GT), (unsigned)splits);
