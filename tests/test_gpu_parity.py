@@ -78,6 +78,13 @@ def test_medium_shapes_ragged_batch(gb):
     _run_steps(p, 2, B=1237, want_emb_grad=True)
 
 
+def test_skew_shapes_ragged_batch(gb):
+    # fp32 head of 192-256-128-1 (the 128 x 128 product kernel) on a batch that ends inside a tile and inside a
+    # 16-byte piece of the batch-long reductions
+    p = PRESETS["skew"].scaled(M=8, img_vocab=50_000, user_vocab=50_000, url_vocab=50_000)
+    _run_steps(p, 2, B=1237, want_emb_grad=True)
+
+
 @pytest.mark.parametrize("M", [1, 64, 1024])
 def test_skew_config_reduced(gb, M):
     # skew shapes with a smaller batch and image table; Zipf 1.3 keeps most rows on a handful of images
