@@ -327,7 +327,9 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
     now = [0]
 
-    def one_step(db, expiry_beside=True):
+    expiry_beside_default = p.img_vocab >= (1 << 22)       # GearSession.step's own rule
+
+    def one_step(db, expiry_beside=None):
         now[0] += 1
         sess.step(db, now[0], sync=False, expiry_beside=expiry_beside)
 
@@ -476,8 +478,9 @@ def run_ours(args):
                        "M": p.M, "expire": p.expire, "mean_nnz": round(stats["nnz"], 1),
                        "l2": "tables far exceed the 126 MB L2 and rows are Zipf-random; %d pre-generated batches cycle; "
                              "no explicit flush" % N_BATCHES,
-                       "streams": "training calls on one stream, the expiry scan of the same step on a second one, "
-                                  "forked at the step's start and joined at its end (inside the timed region)",
+                       "streams": ("training calls on one stream, the expiry scan of the same step on a second one, "
+                                   "forked at the step's start and joined at its end (inside the timed region)")
+                       if expiry_beside_default else "all calls on one stream",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks,
             "e2e": {"value": round(reps.whole_job_rate(p.batch * K, ms_e2e), 1), "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,

@@ -78,10 +78,22 @@ coop_sort_kernel(const SortBatch batch) {
     __syncthreads();
     int total_tiles = 0;
     for (int j = 0; j < batch.n_jobs; ++j) total_tiles += live_tiles[j];
-    // small problems: block 0 alone, no grid barrier (it still advances the arrival counter on behalf of all)
-    const bool solo = total_tiles <= RS_SOLO_TILES;
-    if (solo && blockIdx.x != 0) return;
-    const int nblk = solo ? 1 : gridDim.x;
+    // Small problems need no grid barrier (block 0 still advances the arrival counter on behalf of all):
+    //   every array fits one tile -> block b sorts array b by itself;  a few tiles in all -> block 0 sorts everything.
+    bool one_tile_each = batch.n_jobs > 1 && (int)gridDim.x >= batch.n_jobs;
+    for (int j = 0; j < batch.n_jobs; ++j) one_tile_each = one_tile_each && live_tiles[j] <= 1;
+    const bool per_job = one_tile_each;
+    const bool solo = per_job || total_tiles <= RS_SOLO_TILES;          // this block works alone
+    if (solo && (int)blockIdx.x >= (per_job ? batch.n_jobs : 1)) return;
+    const int nblk = solo ? 1 : gridDim.x, blk = solo ? 0 : (int)blockIdx.x;
+    // the tiles and the digit rows this block walks (with stride nblk)
+    int w_begin = blk, w_end = total_tiles, r_begin = 0, r_end = batch.n_jobs * RS_BUCKETS;
+    if (per_job) {
+        w_begin = 0;
+        for (int j = 0; j < (int)blockIdx.x; ++j) w_begin += live_tiles[j];
+        w_end = w_begin + live_tiles[blockIdx.x];
+        r_begin = (int)blockIdx.x * RS_BUCKETS; r_end = r_begin + RS_BUCKETS;
+    }
     unsigned long long target = batch.barrier_base;
     auto sync_all = [&]() -> bool {
         if (solo) { __syncthreads(); return true; }
@@ -94,7 +106,7 @@ coop_sort_kernel(const SortBatch batch) {
         const int src = pass & 1, dst = src ^ 1;
 
         // ---- count: digit histogram of every live tile
-        for (int w = blockIdx.x; w < total_tiles; w += nblk) {
+        for (int w = w_begin; w < w_end; w += nblk) {
             int jj = 0, t = w;
             while (t >= live_tiles[jj]) { t -= live_tiles[jj]; ++jj; }
             const SortJob& j = batch.job[jj];
@@ -126,7 +138,7 @@ coop_sort_kernel(const SortBatch batch) {
         //      digit row (its loads are independent, so the rows of all digits cost one trip to the L2 together);
         //      jobs of many tiles: one warp per row.
         constexpr int RS_ROW_THREAD_TILES = 32;
-        for (int r = blockIdx.x * RS_THREADS + threadIdx.x; r < batch.n_jobs * RS_BUCKETS; r += nblk * RS_THREADS) {
+        for (int r = r_begin + blk * RS_THREADS + threadIdx.x; r < r_end; r += nblk * RS_THREADS) {
             const int jj = r / RS_BUCKETS, d = r % RS_BUCKETS;
             const SortJob& j = batch.job[jj];
             const int nt = live_tiles[jj];
@@ -145,7 +157,7 @@ coop_sort_kernel(const SortBatch batch) {
             }
             __stcg(j.tot + d, carry);
         }
-        for (int r = blockIdx.x * (RS_THREADS / 32) + warp; r < batch.n_jobs * RS_BUCKETS; r += nblk * (RS_THREADS / 32)) {
+        for (int r = r_begin + blk * (RS_THREADS / 32) + warp; r < r_end; r += nblk * (RS_THREADS / 32)) {
             const int jj = r / RS_BUCKETS, d = r % RS_BUCKETS;
             const SortJob& j = batch.job[jj];
             if (d >= (1 << j.width) || live_tiles[jj] <= RS_ROW_THREAD_TILES) continue;
@@ -163,7 +175,7 @@ coop_sort_kernel(const SortBatch batch) {
         if (!(ok = sync_all())) break;
 
         // ---- scatter
-        for (int w = blockIdx.x; w < total_tiles; w += nblk) {
+        for (int w = w_begin; w < w_end; w += nblk) {
             int jj = 0, t = w;
             while (t >= live_tiles[jj]) { t -= live_tiles[jj]; ++jj; }
             const SortJob& j = batch.job[jj];
@@ -245,7 +257,7 @@ coop_sort_kernel(const SortBatch batch) {
         }
         if (pass + 1 < batch.passes && !(ok = sync_all())) break;
     }
-    if (solo && threadIdx.x == 0) {
+    if (solo && blockIdx.x == 0 && threadIdx.x == 0) {
         // the host has already booked this launch's arrivals: deliver them
         __threadfence();
         atomicAdd(batch.barrier_ctr, (unsigned long long)gridDim.x * (unsigned long long)batch.n_barriers);

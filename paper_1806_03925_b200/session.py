@@ -129,10 +129,13 @@ class GearSession:
         """Recomputed DFVs replace cached ones (rows fp32) and restart their clocks."""
         return gb.gear_refresh_dfv(self.ctx, ids, rows, int(ids.shape[0]) if n is None else n, now, d_n=d_n)
 
-    def step(self, b: DeviceBatch, now: int, sync: bool = False, expiry_beside: bool = True):
+    def step(self, b: DeviceBatch, now: int, sync: bool = False, expiry_beside: Optional[bool] = None):
         """One pass of the whole hot path over one batch.  The expiry scan depends on nothing the training calls
         produce: with expiry_beside it goes to a stream of its own, starts when the step starts and is joined
-        at the step's end, so that it runs beside the gather and the head."""
+        at the step's end, so that it runs beside the gather and the head.  Default: beside for tables of 4M images
+        or more (the fork and join cost the host more than a scan of a small table takes on the device)."""
+        if expiry_beside is None:
+            expiry_beside = self.p.img_vocab >= (1 << 22)
         if not expiry_beside:
             self.forward_backward(b)
             self.accumulate_from_step(b)
