@@ -172,20 +172,37 @@ def gear_init_tables(cfg: gear_config, user_emb, url_emb, dfv, dfv_gsum, dfv_gcn
     return ctx
 
 
-def gear_forward_backward(ctx, user_id, url_id, img_off, img_id, label, lr: float, loss, head_grad, dX, prob=None,
-                          row_view=None, inv_n=None, x_debug=None, user_grad=None, url_grad=None, stream=None,
-                          B: Optional[int] = None, nnz: Optional[int] = None):
+def make_batch(user_id, url_id, img_off, img_id, label, B: Optional[int] = None, nnz: Optional[int] = None) -> gear_batch:
+    """The C struct of a batch whose arrays are device tensors (a caller that reuses the tensors may keep it)."""
     bt = gear_batch()
     bt.B = int(user_id.shape[0]) if B is None else B
     bt.nnz = int(img_id.shape[0]) if nnz is None else nnz
-    bt.user_id, bt.url_id, bt.img_off = user_id.data_ptr(), url_id.data_ptr(), img_off.data_ptr()
-    bt.img_id, bt.label = img_id.data_ptr(), label.data_ptr()
+    bt.user_id, bt.url_id, bt.img_off = _p(user_id).value, _p(url_id).value, _p(img_off).value
+    bt.img_id, bt.label = _p(img_id).value, _p(label).value
+    return bt
+
+
+def make_step_out(loss, head_grad, dX, prob=None, row_view=None, inv_n=None, x_debug=None, user_grad=None,
+                  url_grad=None) -> gear_step_out:
     o = gear_step_out()
     for name, t in (("loss", loss), ("prob", prob), ("head_grad", head_grad), ("dX", dX), ("row_view", row_view),
                     ("inv_n", inv_n), ("x_debug", x_debug), ("user_grad", user_grad), ("url_grad", url_grad)):
         setattr(o, name, None if t is None else _p(t).value)
+    return o
+
+
+def gear_forward_backward_structs(ctx, bt: gear_batch, lr: float, o: gear_step_out, stream=None):
+    """gear_forward_backward on structs made by make_batch / make_step_out."""
     return _check(load().gear_forward_backward(ctx, C.byref(bt), lr, C.byref(o), _stream(stream)),
                   "gear_forward_backward")
+
+
+def gear_forward_backward(ctx, user_id, url_id, img_off, img_id, label, lr: float, loss, head_grad, dX, prob=None,
+                          row_view=None, inv_n=None, x_debug=None, user_grad=None, url_grad=None, stream=None,
+                          B: Optional[int] = None, nnz: Optional[int] = None):
+    bt = make_batch(user_id, url_id, img_off, img_id, label, B, nnz)
+    o = make_step_out(loss, head_grad, dX, prob, row_view, inv_n, x_debug, user_grad, url_grad)
+    return gear_forward_backward_structs(ctx, bt, lr, o, stream)
 
 
 def gear_accumulate_dfv_grad(ctx, img_id, grads_ptr: int, ld: int, src_row, scale, n: int, stream=None):

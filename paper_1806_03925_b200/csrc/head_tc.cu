@@ -22,6 +22,8 @@
 // code, leaves its loops, frees its tensor memory and returns.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "internal.h"
 
@@ -537,9 +539,43 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// A step encodes the same eighteen maps every time (operands and outputs live at fixed places in the workspace): a
+// small table of the most recent encodings saves the driver calls.  A map depends on the key alone.
+struct MapKey { const void* ptr; int64_t rows, cols, ld; int box_rows, f32; };
+struct MapCache {
+    static constexpr int N = 64;
+    std::mutex mu;
+    MapKey key[N];
+    CUtensorMap map[N];
+    int used = 0, next = 0;
+    bool find(const MapKey& k, CUtensorMap* out) {
+        std::lock_guard<std::mutex> lock(mu);
+        for (int i = 0; i < used; ++i)
+            if (key[i].ptr == k.ptr && key[i].rows == k.rows && key[i].cols == k.cols && key[i].ld == k.ld &&
+                key[i].box_rows == k.box_rows && key[i].f32 == k.f32) { *out = map[i]; return true; }
+        return false;
+    }
+    void put(const MapKey& k, const CUtensorMap& m) {
+        std::lock_guard<std::mutex> lock(mu);
+        const int i = used < N ? used++ : (next = (next + 1) % N);
+        key[i] = k; map[i] = m;
+    }
+};
+static MapCache g_maps;
+
+static bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows);
+static bool encode_bf16(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows);
+
 // bf16 matrix [rows][cols] with leading dimension ld (elements); box = box_rows x 64 columns, 128-byte swizzle.
 // Out-of-range parts of a box read as zero.
 static bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    const MapKey k{ptr, rows, cols, ld, box_rows, 0};
+    if (g_maps.find(k, m)) return true;
+    if (!encode_bf16(m, ptr, rows, cols, ld, box_rows)) return false;
+    g_maps.put(k, *m);
+    return true;
+}
+static bool encode_bf16(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -553,15 +589,19 @@ static bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols
 
 // fp32 matrix [rows][cols] with leading dimension ld (elements); box = box_rows x 32 columns, 128-byte swizzle.
 static bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    const MapKey k{ptr, rows, cols, ld, box_rows, 1};
+    if (g_maps.find(k, m)) return true;
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
     cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return false;
+    g_maps.put(k, *m);
+    return true;
 }
 
 template <int BN, bool MN, int EPI, int EW>

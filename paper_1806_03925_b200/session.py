@@ -94,14 +94,20 @@ class GearSession:
         self.expired_ids = torch.zeros(self.expired_cap, dtype=torch.int32, device=dev)
         self.d_counts = self.scalars[1:3]
         self._expiry_stream = None
+        self._step_out = None
 
     # ---- the four calls of a step ---------------------------------------------------------------
     def forward_backward(self, b: DeviceBatch, lr: Optional[float] = None):
-        return gb.gear_forward_backward(self.ctx, b.user_id, b.url_id, b.img_off, b.img_id, b.label,
-                                        self.p.lr if lr is None else lr, self.loss, self.head_grad, self.dX,
-                                        prob=self.prob, row_view=self.row_view, inv_n=self.inv_n,
-                                        x_debug=self.x_debug, user_grad=self.user_grad, url_grad=self.url_grad,
-                                        B=b.B, nnz=b.nnz)
+        # the output struct never changes and a batch's struct only in its counts: both are made once
+        if self._step_out is None:
+            self._step_out = gb.make_step_out(self.loss, self.head_grad, self.dX, prob=self.prob, row_view=self.row_view,
+                                              inv_n=self.inv_n, x_debug=self.x_debug, user_grad=self.user_grad,
+                                              url_grad=self.url_grad)
+        bt = b.__dict__.get("_c_batch")
+        if bt is None:
+            bt = b.__dict__["_c_batch"] = gb.make_batch(b.user_id, b.url_id, b.img_off, b.img_id, b.label)
+        bt.B, bt.nnz = b.B, b.nnz
+        return gb.gear_forward_backward_structs(self.ctx, bt, self.p.lr if lr is None else lr, self._step_out)
 
     def accumulate_from_step(self, b: DeviceBatch, reuse_sorted_ids: bool = True):
         """Event 5 in its indirect form: row r of the batch is dX[row_view[r], 2E:] * inv_n[row_view[r]].
