@@ -10,7 +10,8 @@
 //              apply bias+ReLU / ReLU mask / nothing, and store; meanwhile the MMA warp already fills
 //              the other accumulator buffer with the next tile.  Two warps share each quarter of the
 //              tensor-memory lanes and split the tile's columns; the read of the next 32 columns and
-//              the loads of the bias / mask are in flight while the current 32 columns are processed.
+//              the loads of the bias are in flight while the current 32 columns are processed; the ReLU
+//              mask of a 32 x 32 block arrives by TMA, requested two blocks ahead of its use.
 //              The ReLU-mask epilogue also sums its output columns (the bias gradient of the layer
 //              below): each lane adds up two columns of the block staged for the store; per-CTA partials
 //              in shared memory.
@@ -34,8 +35,7 @@ constexpr int TC_BK = 64;                 // 64 bf16 = 128 bytes = one swizzle r
 // Epilogue warps per CTA (a multiple of four: each warp reaches one quarter of the tensor-memory lanes).
 constexpr int tc_threads(int ew) { return 64 + 32 * ew; }
 constexpr int TC_MAX_N = 1024;            // widest output the column-sum partials cover
-constexpr int TC_STAGE_PITCH = 80;        // bytes between rows of a warp's mask block in shared memory (64 of data + 16 of padding)
-constexpr int TC_STAGE_BYTES = 32 * TC_STAGE_PITCH;
+constexpr int TC_MASK_BLOCK = 32 * 64;    // a warp's ReLU-mask block for 32 columns: 32 rows of 64 bytes (two per warp)
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
 enum { TC_EPI_BIAS_RELU = 0, TC_EPI_MASK = 1, TC_EPI_F32 = 2, TC_EPI_RED = 3 };
@@ -49,8 +49,8 @@ template <int BN, int EW, int EPI> struct TcCfg {
     // output blocks per epilogue warp: the fp32 store sends one per 32 columns and alternates between two
     static constexpr int OUT_BUFS = EPI == TC_EPI_RED ? 0 : (EPI == TC_EPI_F32 && EW == 8 ? 2 : 1);
     static constexpr int OUT_BYTES = EW * OUT_BUFS * TC_OUT_BLOCK;
-    static constexpr int MASK_BYTES = EPI == TC_EPI_MASK ? EW * TC_STAGE_BYTES : 0;
-    static constexpr int FIXED = 1024 /*alignment slack*/ + 256 /*barriers*/ + TC_MAX_N * 4 /*column sums*/ + OUT_BYTES + MASK_BYTES;
+    static constexpr int MASK_BYTES = EPI == TC_EPI_MASK ? EW * 2 * TC_MASK_BLOCK : 0;
+    static constexpr int FIXED = 1024 /*alignment slack*/ + 512 /*barriers*/ + TC_MAX_N * 4 /*column sums*/ + OUT_BYTES + MASK_BYTES;
     static constexpr int ROOM = (227 * 1024 - FIXED) / STAGE_BYTES;
     static constexpr int STAGES = ROOM > (BN == 256 ? 4 : 6) ? (BN == 256 ? 4 : 6) : ROOM;
     static constexpr int SMEM = STAGES * STAGE_BYTES + FIXED;
@@ -199,9 +199,30 @@ __host__ __device__ constexpr uint32_t instr_desc(int bn, bool mn_major) {
 // (conflict-free 128-bit writes, and the layout a 128-byte-swizzle tensor map expects); one lane then hands the
 // block to a TMA store, which writes whole rows of it, drops what lies past the matrix edge and needs no register
 // or issue slot of the warp while it runs.  `out_buf` is the shared-memory address of this warp's block(s).
+// The ReLU mask of a warp's 32 x 32 blocks travels by TMA, two blocks ahead of their use: block c goes to the warp's
+// half-buffer c % 2 (32 rows of 64 bytes, 64-byte swizzle) and reports to that half's mbarrier; as soon as the lanes
+// have read a half, the block two further on (of this tile or the next) is requested into it.
+struct MaskPipe {
+    const CUtensorMap* map;
+    uint32_t buf, bar;         // shared-memory addresses of the warp's two half-buffers / two mbarriers
+    uint32_t parity;           // bit h: phase the next wait on half h looks for
+    uint32_t pending;          // bit h: a copy into half h has been issued and not yet waited for
+    int next_m0, next_col0;    // first row / column of this warp's part of the CTA's next tile (-1: there is none)
+};
+__device__ __forceinline__ void mask_request(MaskPipe& mp, int h, int x, int y, int lane) {
+    __syncwarp();                                             // every lane has read the half's previous contents
+    if (lane == 0) {
+        fence_async_smem();
+        const uint32_t bar = mp.bar + 8u * h;
+        mbar_expect_tx(bar, TC_MASK_BLOCK);
+        tma_load_2d(mp.buf + (uint32_t)h * TC_MASK_BLOCK, mp.map, bar, x, y);
+    }
+    mp.pending |= 1u << h;
+}
+
 template <int BN, int EPI, int EW>
 __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap* map_out, uint32_t tmem_base, int a, int mt,
-                                              int nt, int warp, int lane, float* s_colsum, uint4* s_mask, uint32_t out_buf,
+                                              int nt, int warp, int lane, float* s_colsum, MaskPipe& mp, uint32_t out_buf,
                                               uint32_t& out_turn, uint64_t keep_policy) {
     const int quarter = warp & 3;
     const int part = (warp - 2) >> 2;
@@ -213,7 +234,6 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
     const int m = m0 + lane;
     const bool row_ok = m < g.M;
     const int rows = min(32, max(0, g.M - m0));
-    uint4* stage = s_mask + (warp - 2) * (TC_STAGE_BYTES / 16);
     const int col0 = nt * BN + part * COLS;
     const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN + part * COLS);
     const uint32_t swz = (uint32_t)(lane & 7);
@@ -231,29 +251,26 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
             for (int j = 0; j < 8; ++j)
                 bias4[j] = (n0 + 4 * j < g.N) ? ldg_f4(g.bias + n0 + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        if (EPI == TC_EPI_MASK) {
-            // the 32 x 64-byte block of the mask, fetched as 64-byte row segments (eight rows per instruction);
-            // each lane picks up its own row from the shared-memory block once the loads have landed
-            const int piece = lane & 3;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int row = j * 8 + (lane >> 2);
-                mask4[j] = (row < rows && n0 + 8 * piece < g.N)
-                               ? ldg_u4(g.mask + (int64_t)(m0 + row) * g.ldm + n0 + 8 * piece) : make_uint4(0u, 0u, 0u, 0u);
-            }
-        }
         tc_wait_ld(r[c & 1]);
         if (c + 1 < CHUNKS) tc_ld32(t_row + (uint32_t)((c + 1) * 32), r[(c + 1) & 1]);
-        if (!chunk_ok || rows == 0) continue;
         if (EPI == TC_EPI_MASK) {
-            constexpr int P = TC_STAGE_PITCH / 16;
-            __syncwarp();                               // the previous block has left the buffer
+            // this block's mask has been on its way since two blocks ago; a lane reads its own row (rows and columns past
+            // the matrix edge arrive as zeros), then the half is free for the block two further on
+            const int h = c & 1;
+            mbar_wait(mp.bar + 8u * h, (mp.parity >> h) & 1u, g.err, 6);
+            mp.parity ^= 1u << h;
+            mp.pending &= ~(1u << h);
+            const uint32_t row_addr = mp.buf + (uint32_t)h * TC_MASK_BLOCK + (uint32_t)lane * 64u;
+            const uint32_t sw = ((uint32_t)lane >> 1) & 3u;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) stage[(j * 8 + (lane >> 2)) * P + (lane & 3)] = mask4[j];
-            __syncwarp();
-#pragma unroll
-            for (int j = 0; j < 4; ++j) mask4[j] = stage[lane * P + j];
+            for (int j = 0; j < 4; ++j)
+                asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(mask4[j].x), "=r"(mask4[j].y), "=r"(mask4[j].z), "=r"(mask4[j].w)
+                             : "r"(row_addr + ((((uint32_t)j) ^ sw) << 4)) : "memory");
+            if (c + 2 < CHUNKS) mask_request(mp, h, n0 + 64, m0, lane);
+            else if (mp.next_m0 >= 0) mask_request(mp, h, mp.next_col0 + (c + 2 - CHUNKS) * 32, mp.next_m0, lane);
         }
+        if (!chunk_ok || rows == 0) continue;
         uint32_t (&acc)[32] = r[c & 1];
         if (EPI == TC_EPI_BIAS_RELU || EPI == TC_EPI_MASK) {
             uint32_t pk[16];
@@ -354,14 +371,15 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
 // ---------------------------------------------------------------- the kernel
 template <int BN, bool MN_MAJOR, int EPI, int EW>
 __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out,
-                                             const TcArgs& g) {
+                                             const CUtensorMap& map_mask, const TcArgs& g) {
     using Cfg = TcCfg<BN, EW, EPI>;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;                  // operand stages, 1024-byte aligned
     const uint32_t out_blocks = tiles + STAGES * Cfg::STAGE_BYTES;  // output blocks of the epilogue warps, 1024-byte aligned
-    const uint32_t bars = out_blocks + Cfg::OUT_BYTES;              // mbarriers, then the tmem address word
+    const uint32_t mask_blocks = out_blocks + Cfg::OUT_BYTES;       // ReLU-mask blocks of the epilogue warps, 1024-byte aligned
+    const uint32_t bars = mask_blocks + Cfg::MASK_BYTES;            // mbarriers, then the tmem address word
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     auto acc_full = [&](int a) { return bars + 8u * (2 * STAGES + a); };
@@ -369,8 +387,8 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUt
     const uint32_t tmem_word = bars + 8u * (2 * STAGES + 4);
     volatile uint32_t* tmem_word_ptr =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_word - raw));
-    float* s_colsum = reinterpret_cast<float*>(smem_raw + (bars + 256u - raw));     // [TC_MAX_N] per-CTA column sums
-    uint4* s_mask = reinterpret_cast<uint4*>(smem_raw + (bars + 256u + TC_MAX_N * 4u - raw));    // [EW] mask blocks
+    auto mask_bar = [&](int w, int h) { return bars + 8u * (24 + 2 * w + h); };     // two per epilogue warp
+    float* s_colsum = reinterpret_cast<float*>(smem_raw + (bars + 512u - raw));     // [TC_MAX_N] per-CTA column sums
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles * g.k_splits;
@@ -379,10 +397,13 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUt
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 32 * EW); }
+        if (EPI == TC_EPI_MASK)
+            for (int w = 0; w < EW; ++w) { mbar_init(mask_bar(w, 0), 1); mbar_init(mask_bar(w, 1), 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" :: "l"(&map_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" :: "l"(&map_b) : "memory");
         if (EPI != TC_EPI_RED) asm volatile("prefetch.tensormap [%0];" :: "l"(&map_out) : "memory");
+        if (EPI == TC_EPI_MASK) asm volatile("prefetch.tensormap [%0];" :: "l"(&map_mask) : "memory");
     }
     if (EPI == TC_EPI_MASK && g.colsum != nullptr)
         for (int n = threadIdx.x; n < TC_MAX_N; n += tc_threads(EW)) s_colsum[n] = 0.f;
@@ -475,26 +496,38 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUt
         const uint64_t keep_policy = l2_policy_evict_last();
         uint32_t tile_it = 0, out_turn = 0;
         bool ok = true;
+        constexpr int COLS = BN / (EW / 4);
+        // where this warp's part of tile t starts
+        auto part_m0 = [&](int t) { return ((t / g.n_tiles) % g.m_tiles) * TC_BM + (warp & 3) * 32; };
+        auto part_col0 = [&](int t) { return (t % g.n_tiles) * BN + ((warp - 2) >> 2) * COLS; };
+        MaskPipe mp{&map_mask, mask_blocks + (uint32_t)((warp - 2) * 2 * TC_MASK_BLOCK), mask_bar(warp - 2, 0), 0u, 0u, -1, -1};
+        if (EPI == TC_EPI_MASK && (int)blockIdx.x < total_tiles) {
+            // the masks of the first tile's first two blocks (after the wait for the previous kernel, which wrote them)
+            mask_request(mp, 0, part_col0(blockIdx.x), part_m0(blockIdx.x), lane);
+            mask_request(mp, 1, part_col0(blockIdx.x) + 32, part_m0(blockIdx.x), lane);
+        }
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
             const int nt = t % g.n_tiles, mt = (t / g.n_tiles) % g.m_tiles;
             const int a = tile_it & 1;
             if (EPI == TC_EPI_MASK) {
-                // the rows of the ReLU mask this warp will need: ask the L2 for them now, the wait below covers the trip
-                constexpr int COLS = BN / (EW / 4);
-                const int m = mt * TC_BM + (warp & 3) * 32 + lane, c0 = nt * BN + ((warp - 2) >> 2) * COLS;
-                if (m < g.M)
-#pragma unroll
-                    for (int c = 0; c < COLS; c += 64)             // one 128-byte line per 64 bf16 columns
-                        if (c0 + c < g.N)
-                            asm volatile("prefetch.global.L2 [%0];" :: "l"(g.mask + (int64_t)m * g.ldm + c0 + c));
+                const int tn = t + (int)gridDim.x;
+                mp.next_m0 = tn < total_tiles ? part_m0(tn) : -1;
+                mp.next_col0 = tn < total_tiles ? part_col0(tn) : -1;
             }
             if (!(ok = mbar_wait(acc_full(a), (tile_it >> 1) & 1u, g.err, 4))) break;
             tc_fence_after();
-            epilogue_tile<BN, EPI, EW>(g, &map_out, tmem_base, a, mt, nt, warp, lane, s_colsum, s_mask, out_buf, out_turn, keep_policy);
+            epilogue_tile<BN, EPI, EW>(g, &map_out, tmem_base, a, mt, nt, warp, lane, s_colsum, mp, out_buf, out_turn, keep_policy);
             tc_fence_before();
             mbar_arrive_relaxed(acc_empty(a));                   // all epilogue threads arrive: the buffer returns to the MMA warp
         }
         if (EPI != TC_EPI_RED && lane == 0) tma_store_wait_all();   // this warp's stores have left shared memory and landed
+        if (EPI == TC_EPI_MASK && mp.pending) {
+            // leaving early: let the mask copies already issued land before the CTA gives its shared memory back
+            for (int h = 0; h < 2; ++h)
+                if (mp.pending & (1u << h))
+                    for (uint32_t spin = 0; spin < (1u << 16) && !mbar_try(mp.bar + 8u * h, (mp.parity >> h) & 1u); ++spin)
+                        __nanosleep(64);
+        }
     }
 
     tc_fence_before();
@@ -516,8 +549,8 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUt
 template <int BN, bool MN_MAJOR, int EPI>
 __global__ void __maxnreg__(128)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_out, const TcArgs g) {
-    tc_gemm_body<BN, MN_MAJOR, EPI, 8>(map_a, map_b, map_out, g);
+               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_mask, const TcArgs g) {
+    tc_gemm_body<BN, MN_MAJOR, EPI, 8>(map_a, map_b, map_out, map_mask, g);
 }
 
 // ---------------------------------------------------------------- host side
@@ -604,9 +637,26 @@ static bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int64_t 
     return true;
 }
 
+// bf16 matrix [rows][cols] read in boxes of 32 rows x 32 columns (64 bytes a row), 64-byte swizzle: the ReLU mask.
+static bool make_map_mask(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld) {
+    const MapKey k{ptr, rows, cols, ld, 32, 2};
+    if (g_maps.find(k, m)) return true;
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return false;
+    g_maps.put(k, *m);
+    return true;
+}
+
 template <int BN, bool MN, int EPI, int EW>
-static cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const TcArgs& g,
-                                  cudaStream_t st) {
+static cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const CUtensorMap& mm,
+                                  const TcArgs& g, cudaStream_t st) {
     using Cfg = TcCfg<BN, EW, EPI>;
     static_assert(EW == 8, "one kernel entry point: eight epilogue warps");
     auto kernel = tc_gemm_kernel<BN, MN, EPI>;
@@ -618,13 +668,14 @@ static cudaError_t launch_variant(const CUtensorMap& ma, const CUtensorMap& mb, 
     }
     const int tiles = g.m_tiles * g.n_tiles * g.k_splits;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    return launch_dependent(kernel, dim3(grid), dim3(tc_threads(EW)), (size_t)Cfg::SMEM, st, ma, mb, mo, g);
+    return launch_dependent(kernel, dim3(grid), dim3(tc_threads(EW)), (size_t)Cfg::SMEM, st, ma, mb, mo, mm, g);
 }
 
 template <bool MN, int EPI, int EW = 8>
-static cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const TcArgs& g,
-                             cudaStream_t st) {
-    return bn == 256 ? launch_variant<256, MN, EPI, EW>(ma, mb, mo, g, st) : launch_variant<128, MN, EPI, EW>(ma, mb, mo, g, st);
+static cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const CUtensorMap& mm,
+                             const TcArgs& g, cudaStream_t st) {
+    return bn == 256 ? launch_variant<256, MN, EPI, EW>(ma, mb, mo, mm, g, st)
+                     : launch_variant<128, MN, EPI, EW>(ma, mb, mo, mm, g, st);
 }
 
 cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K, const __nv_bfloat16* A, int64_t lda,
@@ -645,9 +696,13 @@ cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K
     if (epi == TC_EPI_MASK && colsum != nullptr && g.colsum == nullptr) return cudaErrorInvalidValue;
     KernelScope ks(prof, name, st);
     switch (epi) {
-    case TC_EPI_BIAS_RELU: return launch_bn<false, TC_EPI_BIAS_RELU>(bn, ma, mb, mo, g, st);
-    case TC_EPI_MASK: return launch_bn<false, TC_EPI_MASK>(bn, ma, mb, mo, g, st);
-    default: return launch_bn<false, TC_EPI_F32>(bn, ma, mb, mo, g, st);
+    case TC_EPI_BIAS_RELU: return launch_bn<false, TC_EPI_BIAS_RELU>(bn, ma, mb, mo, ma /*unused*/, g, st);
+    case TC_EPI_MASK: {
+        CUtensorMap mm;
+        if (!mask || !make_map_mask(&mm, mask, M, N, ldm)) return cudaErrorInvalidValue;
+        return launch_bn<false, TC_EPI_MASK>(bn, ma, mb, mo, mm, g, st);
+    }
+    default: return launch_bn<false, TC_EPI_F32>(bn, ma, mb, mo, ma /*unused*/, g, st);
     }
 }
 
@@ -670,7 +725,7 @@ cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int 
     g.k_splits = (int)ceil_div(total_kb, g.kb_per_split);
     g.out = out; g.ldo = ldo; g.bias = nullptr; g.mask = nullptr; g.ldm = 0; g.colsum = nullptr; g.err = err;
     KernelScope ks(prof, name, st);
-    return launch_bn<true, TC_EPI_RED>(bn, ma, mb, ma /*unused: partial tiles are added with red.global*/, g, st);
+    return launch_bn<true, TC_EPI_RED>(bn, ma, mb, ma /*unused: partial tiles are added with red.global*/, ma /*unused*/, g, st);
 }
 
 }  // namespace gear
