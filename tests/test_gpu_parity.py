@@ -85,6 +85,19 @@ def test_skew_shapes_ragged_batch(gb):
     _run_steps(p, 2, B=1237, want_emb_grad=True)
 
 
+@pytest.mark.parametrize("head,hidden,E,D,dfv,B", [
+    (BF16, (1024, 64), 4, 256, BF16, 3000),     # widest layer, narrowest layer, a batch that ends inside a row tile
+    (BF16, (192, 448), 64, 256, F32, 1),        # widths that are no multiple of a 256-column tile; one view
+    (BF16, (320,), 20, 200, BF16, 129),         # head input 240 wide: a partial reduction block and partial column tiles
+    (F32, (264,), 32, 8, F32, 2049),            # fp32 head: 128 x 128 product tiles with ragged edges on every side
+    (F32, (64, 96), 16, 8, F32, 33),            # fp32 head below the large-tile threshold
+])
+def test_odd_head_shapes(gb, head, hidden, E, D, dfv, B):
+    p = PRESETS["medium"].scaled(emb_dim=E, dfv_dim=D, dfv_dtype=dfv, head_dtype=head, hidden=hidden, M=3,
+                                 user_vocab=30_000, url_vocab=20_000, img_vocab=40_000, expire=2)
+    _run_steps(p, 2, B=B, want_emb_grad=True)
+
+
 @pytest.mark.parametrize("M", [1, 64, 1024])
 def test_skew_config_reduced(gb, M):
     # skew shapes with a smaller batch and image table; Zipf 1.3 keeps most rows on a handful of images
