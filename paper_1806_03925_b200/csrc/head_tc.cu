@@ -50,7 +50,8 @@ template <int BN, int EW, int EPI> struct TcCfg {
     static constexpr int OUT_BUFS = EPI == TC_EPI_RED ? 0 : (EPI == TC_EPI_F32 && EW == 8 ? 2 : 1);
     static constexpr int OUT_BYTES = EW * OUT_BUFS * TC_OUT_BLOCK;
     static constexpr int MASK_BYTES = EPI == TC_EPI_MASK ? EW * 2 * TC_MASK_BLOCK : 0;
-    static constexpr int FIXED = 1024 /*alignment slack*/ + 512 /*barriers*/ + TC_MAX_N * 4 /*column sums*/ + OUT_BYTES + MASK_BYTES;
+    static constexpr int COLSUM_BYTES = EPI == TC_EPI_MASK ? TC_MAX_N * 4 : 0;     // per-CTA column sums of the masked product
+    static constexpr int FIXED = 1024 /*alignment slack*/ + 512 /*barriers*/ + COLSUM_BYTES + OUT_BYTES + MASK_BYTES;
     static constexpr int ROOM = (227 * 1024 - FIXED) / STAGE_BYTES;
     static constexpr int STAGES = ROOM > (BN == 256 ? 4 : 6) ? (BN == 256 ? 4 : 6) : ROOM;
     static constexpr int SMEM = STAGES * STAGE_BYTES + FIXED;
