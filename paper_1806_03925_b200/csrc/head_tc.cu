@@ -46,9 +46,7 @@ template <int BN, int EW, int EPI> struct TcCfg {
     static constexpr int A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
     static constexpr int B_BYTES = BN * TC_BK * 2;               // 32 KB or 16 KB
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    // output blocks per epilogue warp: the fp32 store sends one per 32 columns and alternates between two
-    static constexpr int OUT_BUFS = EPI == TC_EPI_RED ? 0 : (EPI == TC_EPI_F32 && EW == 8 ? 2 : 1);
-    static constexpr int OUT_BYTES = EW * OUT_BUFS * TC_OUT_BLOCK;
+    static constexpr int OUT_BYTES = EPI == TC_EPI_RED ? 0 : EW * TC_OUT_BLOCK;       // one output block per epilogue warp
     static constexpr int MASK_BYTES = EPI == TC_EPI_MASK ? EW * 2 * TC_MASK_BLOCK : 0;
     static constexpr int COLSUM_BYTES = EPI == TC_EPI_MASK ? TC_MAX_N * 4 : 0;     // per-CTA column sums of the masked product
     static constexpr int FIXED = 1024 /*alignment slack*/ + 512 /*barriers*/ + COLSUM_BYTES + OUT_BYTES + MASK_BYTES;
@@ -224,12 +222,11 @@ __device__ __forceinline__ void mask_request(MaskPipe& mp, int h, int x, int y, 
 template <int BN, int EPI, int EW>
 __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap* map_out, uint32_t tmem_base, int a, int mt,
                                               int nt, int warp, int lane, float* s_colsum, MaskPipe& mp, uint32_t out_buf,
-                                              uint32_t& out_turn, uint64_t keep_policy) {
+                                              uint64_t keep_policy) {
     const int quarter = warp & 3;
     const int part = (warp - 2) >> 2;
     constexpr int COLS = BN / (EW / 4);                   // columns per warp and tile
     constexpr int CHUNKS = COLS / 32;                     // 32-column chunks per warp and tile
-    constexpr int OUT_BUFS = TcCfg<BN, EW, EPI>::OUT_BUFS;
     static_assert(EPI == TC_EPI_F32 || EPI == TC_EPI_RED || CHUNKS % 2 == 0, "bf16 output leaves in blocks of 64 columns");
     const int m0 = mt * TC_BM + quarter * 32;         // first row of this warp's block
     const int m = m0 + lane;
@@ -352,11 +349,10 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
                 }
             }
         } else {
-            // fp32 output (dX): one block per 32 columns, alternating between the warp's blocks; it is read again right
+            // fp32 output (dX): one block per 32 columns; it is read again right
             // after (embedding and DFV gradients): ask the L2 to keep it
-            const uint32_t buf = out_buf + (OUT_BUFS == 2 ? (out_turn & 1u) * (uint32_t)TC_OUT_BLOCK : 0u);
-            ++out_turn;
-            if (lane == 0) tma_store_wait_read<OUT_BUFS - 1>();       // at most the other block is still being read
+            const uint32_t buf = out_buf;
+            if (lane == 0) tma_store_wait_read<0>();                  // the block's previous contents have been read
             __syncwarp();
             const uint32_t row_addr = buf + (uint32_t)lane * 128u;
 #pragma unroll
@@ -493,9 +489,9 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUt
         }
     } else {
         // ---------------- epilogue warps
-        const uint32_t out_buf = out_blocks + (uint32_t)((warp - 2) * Cfg::OUT_BUFS * TC_OUT_BLOCK);
+        const uint32_t out_buf = out_blocks + (uint32_t)((warp - 2) * TC_OUT_BLOCK);
         const uint64_t keep_policy = l2_policy_evict_last();
-        uint32_t tile_it = 0, out_turn = 0;
+        uint32_t tile_it = 0;
         bool ok = true;
         constexpr int COLS = BN / (EW / 4);
         // where this warp's part of tile t starts
@@ -517,7 +513,7 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUt
             }
             if (!(ok = mbar_wait(acc_full(a), (tile_it >> 1) & 1u, g.err, 4))) break;
             tc_fence_after();
-            epilogue_tile<BN, EPI, EW>(g, &map_out, tmem_base, a, mt, nt, warp, lane, s_colsum, mp, out_buf, out_turn, keep_policy);
+            epilogue_tile<BN, EPI, EW>(g, &map_out, tmem_base, a, mt, nt, warp, lane, s_colsum, mp, out_buf, keep_policy);
             tc_fence_before();
             mbar_arrive_relaxed(acc_empty(a));                   // all epilogue threads arrive: the buffer returns to the MMA warp
         }
