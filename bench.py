@@ -163,7 +163,7 @@ def kernel_models(p, stats):
 NCU_TRAFFIC_LARGE_2M = {
     "gather_pool": (65.5e6, "work"), "acc_reduce": (239.7e6, "work"), "expiry_mark": (16.0e6, "vocab"),
     "head_out": (34.4e6, None), "collect_move": (5.9e6, "work"), "emb_reduce": (46.9e6, "work"),
-    "tc_gemm_fwd": (69.3e6, None), "tc_gemm_dw": (114.9e6, None), "tc_gemm_dh": (129.9e6, None), "tc_gemm_dx": (111.6e6, None),
+    "tc_gemm_fwd": (68.3e6, None), "tc_gemm_dw": (113.7e6, None), "tc_gemm_dh": (129.5e6, None), "tc_gemm_dx": (110.2e6, None),
 }
 # algorithmic bytes per launch of the table-bound kernels on large_2m (kernel_models on that workload's batches)
 NCU_WORK_LARGE_2M = {"gather_pool": 222.0e6, "acc_reduce": 224.5e6, "collect_move": 14.2e6, "emb_reduce": 58.9e6}
