@@ -71,26 +71,45 @@ struct GatherArgs {
     DevState* state;
 };
 
-// Adds rows j .. j + K - 1 of the view to acc, in order; their IDs sit in lanes (j + t) % 32 of my_id
-// (-1: the row counts as zeros).  All K loads are issued before the first addition.
-template <typename TD, int NQ, int K>
+// Adds rows j .. j + K - 1 of the view to acc, in order; their IDs, all valid, sit in lanes (j + t) % 32 of my_id.
+// All K loads are issued before the first addition.  FULL: every lane owns a chunk of every row (the row is NQ * 512
+// bytes), so the loads carry no predicate at all -- the kernel is bound by its integer instructions, and the
+// compare-and-clear around a guarded 128-bit load costs as much as the row's additions.
+template <typename TD, int NQ, int K, bool FULL>
 __device__ __forceinline__ void add_rows(float (&acc)[NQ][Chunk<TD>::PER], const TD* __restrict__ dfv, int D,
                                          int n_chunks, int my_id, int j, int lane) {
     uint4 v[K][NQ];
 #pragma unroll
     for (int t = 0; t < K; ++t) {
         const int id = __shfl_sync(0xffffffffu, my_id, (j + t) & 31);
-        const uint4* __restrict__ row = reinterpret_cast<const uint4*>(dfv + (int64_t)(id < 0 ? 0 : id) * D);
+        const uint4* __restrict__ row = reinterpret_cast<const uint4*>(dfv + (int64_t)id * D);
 #pragma unroll
         for (int q = 0; q < NQ; ++q) {
             const int ch = lane + 32 * q;
-            v[t][q] = (id >= 0 && ch < n_chunks) ? __ldg(row + ch) : make_uint4(0u, 0u, 0u, 0u);
+            v[t][q] = (FULL || ch < n_chunks) ? __ldg(row + ch) : make_uint4(0u, 0u, 0u, 0u);
         }
     }
 #pragma unroll
     for (int t = 0; t < K; ++t)
 #pragma unroll
         for (int q = 0; q < NQ; ++q) Chunk<TD>::add(acc[q], v[t][q]);
+}
+
+// The same for a stretch of the view that holds an invalid ID (-1: the row counts as zeros): one row at a time.
+template <typename TD, int NQ>
+__device__ __forceinline__ void add_rows_checked(float (&acc)[NQ][Chunk<TD>::PER], const TD* __restrict__ dfv, int D,
+                                              int n_chunks, int my_id, int j, int count, int lane) {
+#pragma unroll 1
+    for (int t = 0; t < count; ++t) {
+        const int id = __shfl_sync(0xffffffffu, my_id, (j + t) & 31);
+        const uint4* __restrict__ row = reinterpret_cast<const uint4*>(dfv + (int64_t)(id < 0 ? 0 : id) * D);
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const int ch = lane + 32 * q;
+            const uint4 v = (id >= 0 && ch < n_chunks) ? __ldg(row + ch) : make_uint4(0u, 0u, 0u, 0u);
+            Chunk<TD>::add(acc[q], v);
+        }
+    }
 }
 
 struct ViewRec { int uid, hid, s, n; };
@@ -111,7 +130,7 @@ __device__ __forceinline__ ViewRec load_view(const GatherArgs& a, int b) {
 // and keeps two stages of look-ahead in registers: the record of the view after next and the image IDs of
 // the next view are requested before the current view's rows are summed, so that per view only one memory
 // round trip (the rows themselves) is exposed.
-template <typename TD, typename TX, int NQ>
+template <typename TD, typename TX, int NQ, bool FULL>
 __global__ void __launch_bounds__(GP_WARPS * 32, NQ <= 2 ? 3 : 2)
 gather_pool_kernel(const GatherArgs a) {
     wait_for_predecessor();
@@ -150,6 +169,8 @@ gather_pool_kernel(const GatherArgs a) {
             if (my_id < 0 || my_id >= a.img_vocab) { my_id = -1; flags |= GEAR_DEV_BAD_ID; }
             if (a.row_view) a.row_view[s + lane] = b;
         } else my_id = -1;
+        // every ID among the (up to 32) held now is valid: the straight-line code may load without looking
+        bool clean = !__any_sync(0xffffffffu, lane < n && my_id < 0);
 
         // ---- user and URL-hash rows: the first 2E columns of X are the two rows end to end.  The common case
         //      (at most 32 chunks) is loaded here and stored after the DFV loads have been issued.
@@ -176,23 +197,26 @@ gather_pool_kernel(const GatherArgs a) {
                     if (my_id < 0 || my_id >= a.img_vocab) { my_id = -1; flags |= GEAR_DEV_BAD_ID; }
                     if (a.row_view) a.row_view[s + j + lane] = b;
                 } else my_id = -1;
+                clean = !__any_sync(0xffffffffu, j + lane < n && my_id < 0);
             }
         };
         while (n - j >= KMAX) {
             next_ids();
-            add_rows<TD, NQ, KMAX>(acc, dfv, a.D, n_chunks, my_id, j, lane);
+            if (clean) add_rows<TD, NQ, KMAX, FULL>(acc, dfv, a.D, n_chunks, my_id, j, lane);
+            else add_rows_checked<TD, NQ>(acc, dfv, a.D, n_chunks, my_id, j, KMAX, lane);
             j += KMAX;
         }
         if (KMAX > 1 && j < n) {
             next_ids();
-            switch (n - j) {                                       // 1 .. KMAX - 1 rows left: straight-line code for each count
-            case 1: add_rows<TD, NQ, 1>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
-            case 2: if constexpr (KMAX > 2) add_rows<TD, NQ, 2>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
-            case 3: if constexpr (KMAX > 3) add_rows<TD, NQ, 3>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
-            case 4: if constexpr (KMAX > 4) add_rows<TD, NQ, 4>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
-            case 5: if constexpr (KMAX > 5) add_rows<TD, NQ, 5>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
-            case 6: if constexpr (KMAX > 6) add_rows<TD, NQ, 6>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
-            default: if constexpr (KMAX > 7) add_rows<TD, NQ, 7>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            if (!clean) add_rows_checked<TD, NQ>(acc, dfv, a.D, n_chunks, my_id, j, n - j, lane);
+            else switch (n - j) {                                  // 1 .. KMAX - 1 rows left: straight-line code for each count
+            case 1: add_rows<TD, NQ, 1, FULL>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 2: if constexpr (KMAX > 2) add_rows<TD, NQ, 2, FULL>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 3: if constexpr (KMAX > 3) add_rows<TD, NQ, 3, FULL>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 4: if constexpr (KMAX > 4) add_rows<TD, NQ, 4, FULL>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 5: if constexpr (KMAX > 5) add_rows<TD, NQ, 5, FULL>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            case 6: if constexpr (KMAX > 6) add_rows<TD, NQ, 6, FULL>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
+            default: if constexpr (KMAX > 7) add_rows<TD, NQ, 7, FULL>(acc, dfv, a.D, n_chunks, my_id, j, lane); break;
             }
         }
 
@@ -240,10 +264,15 @@ static cudaError_t dispatch_nq(const GatherArgs& a, cudaStream_t st, Profiler* p
     const int64_t resident = (int64_t)sm_count() * (nq <= 2 ? 3 : 2);
     const int grid = (int)std::min<int64_t>(ceil_div(a.B, GP_WARPS), resident);
     KernelScope ks(prof, "gather_pool", st);
-    if (nq <= 1) launch_dependent(gather_pool_kernel<TD, TX, 1>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a);
-    else if (nq <= 2) launch_dependent(gather_pool_kernel<TD, TX, 2>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a);
-    else if (nq <= 4) launch_dependent(gather_pool_kernel<TD, TX, 4>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a);
-    else launch_dependent(gather_pool_kernel<TD, TX, 8>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a);
+    const bool full = n_chunks == nq * 32;                          // every lane owns a chunk of every DFV row
+#define GEAR_GATHER(NQ) do { \
+        if (full) launch_dependent(gather_pool_kernel<TD, TX, NQ, true>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a); \
+        else launch_dependent(gather_pool_kernel<TD, TX, NQ, false>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a); } while (0)
+    if (nq <= 1) GEAR_GATHER(1);
+    else if (nq <= 2) GEAR_GATHER(2);
+    else if (nq <= 4) GEAR_GATHER(4);
+    else GEAR_GATHER(8);
+#undef GEAR_GATHER
     return cudaGetLastError();
 }
 
