@@ -161,7 +161,7 @@ def kernel_models(p, stats):
 # re-reads that hit the L2 in a real step count as DRAM traffic here.  A kernel that has changed since its capture
 # must be taken out of this table (traffic is then reported as null).
 NCU_TRAFFIC_LARGE_2M = {
-    "gather_pool": (65.5e6, "work"), "acc_reduce": (239.7e6, "work"), "expiry_mark": (16.0e6, "vocab"),
+    "gather_pool": (64.4e6, "work"), "acc_reduce": (239.7e6, "work"), "expiry_mark": (16.0e6, "vocab"),
     "head_out": (34.4e6, None), "collect_move": (5.9e6, "work"), "emb_reduce": (46.9e6, "work"),
     "tc_gemm_fwd": (68.3e6, None), "tc_gemm_dw": (113.7e6, None), "tc_gemm_dh": (129.5e6, None), "tc_gemm_dx": (110.2e6, None),
 }
