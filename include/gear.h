@@ -57,7 +57,7 @@ enum {
     GEAR_ERR_CAPACITY = -2,  /* an output list or the ready queue is too small; nothing was consumed */
     GEAR_ERR_BAD_ID = -3,    /* an out-of-range ID was met (reported by gear_status; the row was skipped) */
     GEAR_ERR_CUDA = -4,      /* a CUDA runtime or driver call failed */
-    GEAR_ERR_STATE = -5      /* call order violated (e.g. ctx destroyed) */
+    GEAR_ERR_STATE = -5      /* call order violated (e.g. img_id == NULL without a preceding gear_forward_backward) */
 };
 
 /* element types of tables and of the head's matrix-product operands */
@@ -237,7 +237,8 @@ int gear_refresh_dfv(gear_ctx* ctx, const int32_t* ids, const float* rows, int64
  */
 int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready);
 
-/* Releases the ctx (host memory only).  Synchronises the stream last used. */
+/* Releases the ctx (host memory only).  Synchronises the stream last used.  The pointer is dangling afterwards:
+ * passing it to any call again, gear_destroy included, is undefined. */
 int gear_destroy(gear_ctx* ctx);
 
 /*

@@ -67,7 +67,7 @@ def lib():
         L.orc_forward_backward.restype = i64
         L.orc_forward_backward.argtypes = [C.POINTER(_Model), vp, C.c_int, vp, C.c_int, vp, C.c_int, vp,
                                            i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
-                                           dbl, vp, i64, vp, vp, i64]
+                                           dbl, dbl, vp, vp, i64, vp, vp, i64]
         L.orc_emb_apply.restype = i64
         L.orc_emb_apply.argtypes = [vp, C.c_int, i64, i32, vp, i32, vp, i32, i32, dbl, vp]
         L.orc_dfv_grad_rows.restype = None
@@ -137,6 +137,7 @@ class StepResult:
     dX: Optional[np.ndarray]
     bad_ids: int
     near_units: Optional[np.ndarray] = None   # coded (layer * B + view) * 1024 + column
+    near_abs: Optional[np.ndarray] = None     # |pre-activation| of each listed unit
 
 
 def decode_unit(code: int, B: int) -> Tuple[int, int, int]:
@@ -188,7 +189,10 @@ class GearOracle:
     # -- events 1, 3, 4 -----------------------------------------------------
     def forward_backward(self, params: np.ndarray, user_id, url_id, img_off, img_id, label,
                          backward: bool = True, relu_margin: Optional[float] = None,
-                         flip_units: Optional[Sequence[int]] = None) -> StepResult:
+                         flip_units: Optional[Sequence[int]] = None, relu_margin_rel: float = 0.0,
+                         near_cap: int = 65536) -> StepResult:
+        """relu_margin / relu_margin_rel: list the hidden units whose pre-activation a has
+        |a| <= relu_margin + relu_margin_rel * max|input row| * max|layer weights| (None: no list)."""
         B = int(len(user_id))
         params = _c(params, np.float64)
         assert params.shape[0] == self.n_params
@@ -200,7 +204,8 @@ class GearOracle:
         loss = C.c_double(0.0)
         hg = np.zeros(self.n_params, dtype=np.float64) if backward else None
         dX = np.zeros((B, self.d_in), dtype=np.float64) if backward else None
-        near = np.zeros(65536, dtype=np.int64) if relu_margin is not None else None
+        near = np.zeros(near_cap, dtype=np.int64) if relu_margin is not None else None
+        near_abs = np.zeros(near_cap, dtype=np.float64) if relu_margin is not None else None
         n_near = C.c_int64(0)
         flips = _c(flip_units, np.int64) if flip_units is not None and len(flip_units) else None
         bad = lib().orc_forward_backward(
@@ -208,12 +213,13 @@ class GearOracle:
             _ptr(self.url_emb), _dtype_tag(self.url_emb), _ptr(self.dfv), _dtype_tag(self.dfv),
             _ptr(params), B, _ptr(uid), _ptr(hid), _ptr(off), _ptr(img), _ptr(y),
             _ptr(X), _ptr(prob), C.byref(loss), _ptr(hg), _ptr(dX),
-            0.0 if relu_margin is None else float(relu_margin), _ptr(near), 0 if near is None else len(near),
-            C.byref(n_near), _ptr(flips), 0 if flips is None else len(flips))
+            0.0 if relu_margin is None else float(relu_margin), float(relu_margin_rel), _ptr(near), _ptr(near_abs),
+            0 if near is None else len(near), C.byref(n_near), _ptr(flips), 0 if flips is None else len(flips))
         if near is not None:
             assert n_near.value <= len(near), "near-zero unit list overflowed"
             near = near[:n_near.value].copy()
-        return StepResult(X, prob, loss.value, hg, dX, int(bad), near)
+            near_abs = near_abs[:n_near.value].copy()
+        return StepResult(X, prob, loss.value, hg, dX, int(bad), near, near_abs)
 
     def emb_grad(self, which: str, ids, dX: np.ndarray) -> np.ndarray:
         """Dense summed gradient G[vocab, E] of one embedding table."""
@@ -251,7 +257,8 @@ class GearOracle:
         n = len(ids)
         assert g.shape == (n, self.D)
         n0 = len(self._emit_id)
-        cap = n0 + n
+        # room for the emissions this call can add: every emission takes M arrivals, old (still open) or new
+        cap = n0 + (n + int(self.gcnt.sum(dtype=np.int64))) // self.M + 1
         eid = np.zeros(cap, dtype=np.int32); eid[:n0] = self._emit_id
         eseq = np.zeros(cap, dtype=np.int32); eseq[:n0] = self._emit_seq
         eavg = np.zeros((cap, self.D), dtype=np.float64); eavg[:n0] = self._emit_avg

@@ -182,10 +182,13 @@ int64_t orc_head_param_count(const orc_model* m) { return head_param_count(m); }
  * on a machine that sums in another order or precision, and either decision is
  * then a correct evaluation of the method.  So that a comparison can accept
  * both decisions there and nowhere else, the units (layer l, view b, column j)
- * with |pre-activation| <= relu_margin are listed in near_units (coded
- * (l * B + b) * 1024 + j; *n_near receives their number, near_cap bounds the
- * list; near_units may be NULL), and the units named in flip_units take the
- * other branch in the backward pass (their forward value is left as computed).
+ * with |pre-activation| <= relu_margin + relu_margin_rel * max_i|in_i| *
+ * max|W_l| (in: the unit's input row, W_l: the layer's weights as the product
+ * sees them) are listed in near_units (coded (l * B + b) * 1024 + j; *n_near
+ * receives their number, near_cap bounds the list; near_units may be NULL;
+ * near_abs, optional, receives |pre-activation| of every listed unit), and the
+ * units named in flip_units take the other branch in the backward pass (their
+ * forward value is left as computed).  The list reports; it changes no result.
  *
  * Returns the number of out-of-range IDs met (their rows count as zeros).
  */
@@ -198,7 +201,8 @@ int64_t orc_forward_backward(const orc_model* m,
                              const int32_t* img_off, const int32_t* img_id, const double* label,
                              double* X, double* prob, double* loss,
                              double* head_grad, double* dX,
-                             double relu_margin, int64_t* near_units, int64_t near_cap, int64_t* n_near,
+                             double relu_margin, double relu_margin_rel, int64_t* near_units, double* near_abs,
+                             int64_t near_cap, int64_t* n_near,
                              const int64_t* flip_units, int64_t n_flip) {
     const int E = m->emb_dim, D = m->dfv_dim, Din = 2 * E + D;
     const int L = m->n_hidden;
@@ -221,10 +225,14 @@ int64_t orc_forward_backward(const orc_model* m,
 
     /* rounded copies of the matrix-product operands (identity when rb == 0) */
     double* Wr[2] = {0, 0};
+    double w_amax[2] = {0.0, 0.0};
     for (int l = 0; l < L; ++l) {
         int64_t n = (int64_t)fan[l] * m->hidden[l];
         Wr[l] = (double*)malloc(sizeof(double) * n);
-        for (int64_t i = 0; i < n; ++i) Wr[l][i] = rb ? round_bf16(W[l][i]) : W[l][i];
+        for (int64_t i = 0; i < n; ++i) {
+            Wr[l][i] = rb ? round_bf16(W[l][i]) : W[l][i];
+            if (fabs(Wr[l][i]) > w_amax[l]) w_amax[l] = fabs(Wr[l][i]);
+        }
     }
 
     /* events 1-3: gather the embeddings, fetch and mean-pool the DFVs */
@@ -258,15 +266,21 @@ int64_t orc_forward_backward(const orc_model* m,
             const double* in = H[l] + (int64_t)b * K;
             double* out = H[l + 1] + (int64_t)b * N;
             for (int j = 0; j < N; ++j) out[j] = 0.0;
+            double in_amax = 0.0;
             for (int i = 0; i < K; ++i) {
                 const double xi = in[i];
                 const double* wrow = Wr[l] + (int64_t)i * N;
                 for (int j = 0; j < N; ++j) out[j] += xi * wrow[j];
+                if (fabs(xi) > in_amax) in_amax = fabs(xi);
             }
+            const double near = relu_margin + relu_margin_rel * in_amax * w_amax[l];
             for (int j = 0; j < N; ++j) {
                 double a = out[j] + bias[l][j];
-                if (near_units && fabs(a) <= relu_margin) {
-                    if (*n_near < near_cap) near_units[*n_near] = ((int64_t)l * B + b) * 1024 + j;
+                if (near_units && fabs(a) <= near) {
+                    if (*n_near < near_cap) {
+                        near_units[*n_near] = ((int64_t)l * B + b) * 1024 + j;
+                        if (near_abs) near_abs[*n_near] = fabs(a);
+                    }
                     ++*n_near;
                 }
                 a = a > 0.0 ? a : 0.0;

@@ -416,8 +416,9 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
 #pragma unroll
                     for (int q = 0; q < NQ; ++q) {
                         const float4 v = row[lane + 32 * q];
-                        acc[q].x = fmaf(scale, v.x, acc[q].x); acc[q].y = fmaf(scale, v.y, acc[q].y);
-                        acc[q].z = fmaf(scale, v.z, acc[q].z); acc[q].w = fmaf(scale, v.w, acc[q].w);
+                        // the gradient row is the rounded product (row * 1/n_b); it is then added: two roundings, no fused step
+                        acc[q].x = __fadd_rn(acc[q].x, __fmul_rn(scale, v.x)); acc[q].y = __fadd_rn(acc[q].y, __fmul_rn(scale, v.y));
+                        acc[q].z = __fadd_rn(acc[q].z, __fmul_rn(scale, v.z)); acc[q].w = __fadd_rn(acc[q].w, __fmul_rn(scale, v.w));
                     }
                     if (meta & 3) settle(meta >> 2, (meta & 1) != 0, (meta & 2) != 0);
                     cslot = advance(cslot);
@@ -522,10 +523,11 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
                                         c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id),
                                         c.at<float>(c.ws.q_avg), state);
     };
-    // ring depth: as many row slots as about 96 KB per block (two blocks per SM) allow, at most 8
-    const bool full = D == nq * 128;                              // every lane owns a chunk of every row
+    // ring depth: as many row slots as about 96 KB per block (two blocks per SM) allow, at most 8.
+    // FULL only when a row fills the instantiated width exactly (D == NQ * 128): every lane then owns a chunk of every
+    // row; any other width (also 384, 640, 768, 896, which round up to the next instantiation) keeps the per-chunk guard
 #define GEAR_ACC_LAUNCH(NQ, S) \
-    do { if (full) launch(acc_reduce_kernel<NQ, S, true>, NQ * 512, S); else launch(acc_reduce_kernel<NQ, S, false>, NQ * 512, S); } while (0)
+    do { if (D == NQ * 128) launch(acc_reduce_kernel<NQ, S, true>, NQ * 512, S); else launch(acc_reduce_kernel<NQ, S, false>, NQ * 512, S); } while (0)
     if (nq <= 1) GEAR_ACC_LAUNCH(1, 8);
     else if (nq <= 2) GEAR_ACC_LAUNCH(2, 8);
     else if (nq <= 4) GEAR_ACC_LAUNCH(4, 5);
@@ -738,6 +740,7 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     c.plan_ready = false;                                    // a plan made ahead counted on the queue length of before
     SortJob sb = c.sort_job(gear_ctx_impl::SORT_READY);
     const int64_t n_max = c.ws.ready_cap;
+    const int64_t resident = (int64_t)sm_count() * 8;       // blocks of 256 threads that fit the GPU at once
     const bool solo = c.acc_calls_pending <= 1;
     if (!solo) { KernelScope k(&c.prof, "collect_begin", st);
     launch_dependent(collect_begin_kernel, dim3(1), dim3(1), 0, st, state, cap, d_n); }
@@ -748,7 +751,7 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     if (c.acc_calls_pending > 1) {
         int64_t blocks = ceil_div(n_max, 256);
         { KernelScope k(&c.prof, "collect_keys", st);
-        launch_dependent(collect_keys_kernel, dim3((unsigned)(blocks > 1184 ? 1184 : blocks)), dim3(256), 0, st, c.at<int32_t>(c.ws.q_id), state,
+        launch_dependent(collect_keys_kernel, dim3((unsigned)(blocks > resident ? resident : blocks)), dim3(256), 0, st, c.at<int32_t>(c.ws.q_id), state,
                                                                                      sb.keys[0]); }
         SortBatch batch = c.sort_batch();
         batch.n_jobs = 1;
@@ -764,7 +767,7 @@ cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* 
     if (cap >= c.ws.ready_cap) c.acc_calls_pending = 0;      // this collect cannot be refused: the queue will be empty
     int64_t want = ceil_div(n_max, 8);
     { KernelScope k(&c.prof, "collect_move", st);
-    launch_dependent(collect_move_kernel, dim3((unsigned)(want > 1184 ? 1184 : want)), dim3(256), 0, st, sb.keys[cur], sb.vals[cur],
+    launch_dependent(collect_move_kernel, dim3((unsigned)(want > resident ? resident : want)), dim3(256), 0, st, sb.keys[cur], sb.vals[cur],
                                                                             c.at<int32_t>(c.ws.q_id),
                                                                             c.at<float>(c.ws.q_avg), c.cfg.dfv_dim,
                                                                             state, ids, seq, avg, solo ? 1 : 0, cap, d_n); }

@@ -260,8 +260,18 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
         }
     }
     c.plan_ready = false;
+    // A failure between the fork and the join must not leave the side stream unjoined or the sorted order marked as
+    // usable: the caller's stream waits for whatever the side stream was given, and the ctx forgets the batch.
+    auto abandon = [&](cudaError_t err, const char* where) {
+        if (joined_needed) {
+            if (cudaEventRecord(c.ev_join, c.side_stream) != cudaSuccess || cudaStreamWaitEvent(st, c.ev_join, 0) != cudaSuccess)
+                cudaStreamSynchronize(c.side_stream);
+        }
+        c.img_sorted = false; c.img_sort_valid = false; c.plan_ready = false;
+        return cuda_fail(err, where);
+    };
     cudaError_t e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
-    if (e != cudaSuccess) return cuda_fail(e, "gather");
+    if (e != cudaSuccess) return abandon(e, "gather");
     if (joined_needed) {
         // Still on the side stream, behind the sort: the plan of the accumulate call that usually follows (which rows
         // form which group, where every group's rows and queue slot are).  It needs the gather's row_view / inv_n.
@@ -269,22 +279,23 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
             e = cudaEventRecord(c.ev_gather, st);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(c.side_stream, c.ev_gather, 0);
             if (e == cudaSuccess) e = launch_accumulate_plan_ahead(c, b.nnz, o.row_view, o.inv_n, c.side_stream);
-            if (e != cudaSuccess) return cuda_fail(e, "accumulate plan");
+            if (e != cudaSuccess) return abandon(e, "accumulate plan");
         }
         e = cudaEventRecord(c.ev_join, c.side_stream);
-        if (e != cudaSuccess) return cuda_fail(e, "join");
+        if (e != cudaSuccess) return abandon(e, "join");
     }
     e = launch_head_simt(c, b, o, st);
-    if (e != cudaSuccess) return cuda_fail(e, "head");
+    if (e != cudaSuccess) return abandon(e, "head");
     if (joined_needed) {
         e = cudaStreamWaitEvent(st, c.ev_join, 0);
-        if (e != cudaSuccess) return cuda_fail(e, "join");
+        if (e != cudaSuccess) return abandon(e, "join");
+        joined_needed = false;
     }
     float* ut = o.user_grad ? o.user_grad : c.buf.user_emb;
     float* ht = o.url_grad ? o.url_grad : c.buf.url_emb;
     const float alpha = o.user_grad ? 1.0f : -lr;
     e = launch_emb_reduce(c, sorted_buf, b.B, ut, ht, o.dX, c.d_in, alpha, st);
-    if (e != cudaSuccess) return cuda_fail(e, "embedding scatter");
+    if (e != cudaSuccess) return abandon(e, "embedding scatter");
     return GEAR_OK;
 }
 
@@ -378,8 +389,10 @@ int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready) {
     if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
     gear_ctx_impl& c = ctx->impl;
     DevState h;
+    memset(&h, 0, sizeof(h));
     cudaError_t e = sync_streams(c);
     if (e == cudaSuccess) e = cudaMemcpy(&h, c.state(), sizeof(DevState), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "gear_status");      // h holds nothing to look at
     if (h.tc_error != 0) h.status |= GEAR_DEV_TIMEOUT;
     if (e == cudaSuccess && h.status != 0) e = cudaMemset(c.state(), 0, 2 * sizeof(int32_t));   // status, tc_error
     if (e == cudaSuccess && h.tc_error != 0) {
@@ -446,7 +459,8 @@ int gear_launch_count(gear_ctx* ctx, int64_t* n_launches) {
 
 int gear_destroy(gear_ctx* ctx) {
     if (!ctx) return GEAR_OK;
-    if (!ctx->impl.alive) return GEAR_ERR_STATE;
+    if (!ctx->impl.alive) return GEAR_ERR_STATE;     // a ctx that failed half-way through its set-up; a destroyed
+                                                     // ctx is freed memory and must not be passed in again
     sync_streams(ctx->impl);
     cudaStreamSynchronize(ctx->impl.side_stream);
     release_host_objects(ctx->impl);

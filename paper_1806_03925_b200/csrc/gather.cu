@@ -264,9 +264,10 @@ static cudaError_t dispatch_nq(const GatherArgs& a, cudaStream_t st, Profiler* p
     const int64_t resident = (int64_t)sm_count() * (nq <= 2 ? 3 : 2);
     const int grid = (int)std::min<int64_t>(ceil_div(a.B, GP_WARPS), resident);
     KernelScope ks(prof, "gather_pool", st);
-    const bool full = n_chunks == nq * 32;                          // every lane owns a chunk of every DFV row
+    // FULL only when a row fills the instantiated width exactly (n_chunks == NQ * 32): every lane then owns a chunk of
+    // every DFV row; widths that round up to the next instantiation (3, 5, 6, 7 chunks per lane) keep the guard
 #define GEAR_GATHER(NQ) do { \
-        if (full) launch_dependent(gather_pool_kernel<TD, TX, NQ, true>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a); \
+        if (n_chunks == NQ * 32) launch_dependent(gather_pool_kernel<TD, TX, NQ, true>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a); \
         else launch_dependent(gather_pool_kernel<TD, TX, NQ, false>, dim3(grid), dim3(GP_WARPS * 32), 0, st, a); } while (0)
     if (nq <= 1) GEAR_GATHER(1);
     else if (nq <= 2) GEAR_GATHER(2);

@@ -33,6 +33,9 @@ class DeviceBatch:
 class GearSession:
     """Tables + ctx + output buffers for one configuration on one GPU."""
 
+    GUARD_I = -7
+    GUARD_F = 12345.0
+
     def __init__(self, p: GearPreset, head_params: np.ndarray, max_batch: Optional[int] = None,
                  max_nnz: Optional[int] = None, seed: int = 0, fill: bool = True, now: int = 0,
                  tables: Optional[Dict[str, np.ndarray]] = None, ready_cap: int = 0, device: str = "cuda",
@@ -86,12 +89,17 @@ class GearSession:
                                     device=dev) if want_debug else None)
         self.user_grad = torch.zeros_like(self.user_emb) if want_emb_grad else None
         self.url_grad = torch.zeros_like(self.url_emb) if want_emb_grad else None
+        # every output list is followed by one guard entry the library must never write (guards_intact checks them)
         self.ready_cap = int(ready_cap or nnz)
-        self.ready_ids = torch.zeros(self.ready_cap, dtype=torch.int32, device=dev)
-        self.ready_seq = torch.zeros(self.ready_cap, dtype=torch.int32, device=dev)
-        self.ready_avg = torch.zeros((self.ready_cap, p.dfv_dim), dtype=torch.float32, device=dev)
+        self._ready_ids_g = torch.full((self.ready_cap + 1,), self.GUARD_I, dtype=torch.int32, device=dev)
+        self._ready_seq_g = torch.full((self.ready_cap + 1,), self.GUARD_I, dtype=torch.int32, device=dev)
+        self._ready_avg_g = torch.zeros((self.ready_cap + 1, p.dfv_dim), dtype=torch.float32, device=dev)
+        self._ready_avg_g[self.ready_cap].fill_(self.GUARD_F)
+        self.ready_ids, self.ready_seq = self._ready_ids_g[:self.ready_cap], self._ready_seq_g[:self.ready_cap]
+        self.ready_avg = self._ready_avg_g[:self.ready_cap]
         self.expired_cap = int(expired_cap if expired_cap is not None else p.img_vocab)
-        self.expired_ids = torch.zeros(self.expired_cap, dtype=torch.int32, device=dev)
+        self._expired_ids_g = torch.full((self.expired_cap + 1,), self.GUARD_I, dtype=torch.int32, device=dev)
+        self.expired_ids = self._expired_ids_g[:self.expired_cap]
         self.d_counts = self.scalars[1:3]
         self._expiry_stream = None
         self._step_out = None
@@ -165,6 +173,12 @@ class GearSession:
 
     def status(self):
         return gb.gear_status(self.ctx)
+
+    def guards_intact(self) -> bool:
+        """The entry after the end of each output list still holds the value it was created with."""
+        return bool(int(self._ready_ids_g[-1]) == self.GUARD_I and int(self._ready_seq_g[-1]) == self.GUARD_I and
+                    int(self._expired_ids_g[-1]) == self.GUARD_I and
+                    bool((self._ready_avg_g[-1] == self.GUARD_F).all()))
 
     def close(self):
         if self.ctx is not None:

@@ -25,6 +25,27 @@ from paper_1806_03925_b200.workloads import BF16, Batch, GearPreset
 TOL_F32 = 1e-5      # relative tolerance for fp32 configurations (normwise: against the largest reference entry)
 TOL_BF16 = 1e-2     # for configurations whose DFVs / head operands are bfloat16
 
+# How close to zero a hidden pre-activation a = sum_i in_i * w_ij + b_j has to be for the device's ReLU branch to be
+# allowed to differ from the oracle's, relative to max|in| * max|w| of the unit's layer:
+#   * both sides add the same K products, the device in fp32 in its own order, the oracle in fp64: the sums differ by
+#     about sqrt(K) * 2^-24 * (rms term) * sqrt(K) <= K * 2^-24 * max|in| * max|w|; eight times that is allowed;
+#   * bf16 heads: the operand in_i is itself a rounded fp32 value (pooled mean, or the layer below's activation); where
+#     the two sides' values straddle a rounding boundary the operands differ by one bf16 unit in the last place, at
+#     most 2^-7 |in_i|, which moves a by at most 2^-7 * max|in| * max|w|.
+# A unit outside this band must take the oracle's branch.
+def relu_margin_rel(p: GearPreset) -> float:
+    k_max = max((p.d_in,) + tuple(p.hidden))
+    accum = 8.0 * k_max * 2.0 ** -24
+    return accum + (2.0 ** -7 if p.head_dtype == BF16 else 0.0)
+
+
+MAX_FLIPS_PER_VIEW = 3      # branches of one view that may differ from the oracle's (each inside the band above)
+
+
+def max_views_with_flips(B: int) -> int:
+    """Views of a batch whose ReLU branches may validly differ from the oracle's before a test calls it a failure."""
+    return 2 + B // 512
+
 
 def tol_of(p: GearPreset) -> float:
     return TOL_BF16 if (p.head_dtype == BF16 or p.dfv_dtype == BF16) else TOL_F32
@@ -39,6 +60,15 @@ def assert_close(got, want, tol, what=""):
     scale = max(np.abs(want).max(), 1e-30)
     err = np.abs(got - want).max()
     assert err <= tol * scale, "%s: max abs error %.3e > %.1e * %.3e" % (what, err, tol, scale)
+
+
+def count_nonzero(t: torch.Tensor) -> int:
+    """Non-zero entries of a (possibly very large) tensor, counted in pieces so that no table-sized temporary is made."""
+    flat = t.reshape(-1)
+    step, total = 1 << 28, 0
+    for i in range(0, flat.numel(), step):
+        total += int(torch.count_nonzero(flat[i:i + step]).item())
+    return total
 
 
 def _rows(t: torch.Tensor, rows: np.ndarray) -> np.ndarray:
@@ -115,6 +145,8 @@ class Pair:
         self.updated_user = np.zeros(0, np.int32)
         self.updated_url = np.zeros(0, np.int32)
         self.relu_flips_accepted = 0
+        self.relu_views_flipped = 0
+        self.last_relu = dict(views=0, units=0, listed=0)
         self.status_bits = 0       # device status bits seen so far (reading the word clears it)
         self.status_rc = 0
 
@@ -134,8 +166,8 @@ class Pair:
         gpu.forward_backward(db, lr)
         uid, hid, img = self.ru(b.user_id), self.rh(b.url_id), self.ri(b.img_id)
         params64 = self.params.astype(np.float64)
-        margin = 2e-6 if tol == TOL_F32 else 1e-4
-        r = cpu.forward_backward(params64, uid, hid, b.img_off, img, b.label, relu_margin=margin)
+        r = cpu.forward_backward(params64, uid, hid, b.img_off, img, b.label, relu_margin=0.0,
+                                 relu_margin_rel=relu_margin_rel(p), near_cap=max(65536, 64 * b.B))
 
         B = b.B
         X = _np(gpu.x_debug[:B])
@@ -151,8 +183,7 @@ class Pair:
         assert_close(X, r.X, tol, "head input")
         assert_close(_np(gpu.prob[:B]), r.prob, tol, "prob")
         assert_close(_np(gpu.loss), [r.loss], tol, "loss")
-        r = self._resolve_relu_decisions(r, lambda flips: cpu.forward_backward(
-            params64, uid, hid, b.img_off, img, b.label, flip_units=flips), B)
+        r = self.resolve_relu_decisions(r, params64, uid, hid, b.img_off, img, b.label)
         assert_close(_np(gpu.head_grad), r.head_grad, tol, "head_grad")
         assert_close(_np(gpu.dX[:B]), r.dX, tol, "dX")
         view_of = np.repeat(np.arange(B, dtype=np.int32), n_b)
@@ -186,41 +217,65 @@ class Pair:
         n_exp = self.expire_and_compare(now)
         assert self.status() == 0
         out = dict(loss=r.loss, n_ready=n_ready, n_expired=n_exp, status=self.status_bits, rc=self.status_rc,
-                   bad=r.bad_ids)
+                   bad=r.bad_ids, relu=dict(self.last_relu))
         self.status_bits = self.status_rc = 0
         return out
 
-    def _resolve_relu_decisions(self, r, rerun, B):
+    def resolve_relu_decisions(self, r, params64, uid, hid, img_off, img, label):
         """The backward pass depends on the sign of every hidden pre-activation.  Where the oracle's own
-        pre-activation is within rounding distance of zero (r.near_units) the device may validly have taken
-        the other branch.  If the strict comparison fails, the expected values are recomputed BY THE ORACLE
-        with some of those units on the other branch; units outside that list are never touched."""
+        pre-activation lies inside the rounding band of relu_margin_rel (r.near_units) the device may validly have
+        taken the other branch; a unit's branch only affects its own view's row of dX (and, through the sums over
+        views, the head gradients).
+
+        Views whose dX row fails the strict comparison are looked at one by one: the candidates are that view's
+        listed units alone, smallest |pre-activation| first (the oracle's list, not the device's error, picks them);
+        the oracle is re-run on that single view with subsets of at most MAX_FLIPS_PER_VIEW of them on the other
+        branch until the row matches.  The expected values are then recomputed BY THE ORACLE over the whole batch
+        with the accepted units flipped.  The number of views that needed this is bounded by the caller."""
         import itertools
         from oracle import decode_unit
+        B = len(uid)
         got_dx, got_hg = _np(self.gpu.dX[:B]), _np(self.gpu.head_grad)
-
-        def ok(res):
-            try:
-                assert_close(got_hg, res.head_grad, self.tol)
-                assert_close(got_dx, res.dX, self.tol)
-                return True
-            except AssertionError:
-                return False
-
-        if ok(r) or r.near_units is None or len(r.near_units) == 0:
+        scale = max(np.abs(r.dX).max(), 1e-30)
+        bad_views = np.nonzero(np.abs(got_dx - r.dX).max(1) > self.tol * scale)[0]
+        self.last_relu = dict(views=0, units=0, listed=0 if r.near_units is None else len(r.near_units))
+        if len(bad_views) == 0 or r.near_units is None or len(r.near_units) == 0:
             return r
-        row_rel = np.abs(got_dx - r.dX).max(1) / np.maximum(np.abs(r.dX).max(1), 1e-30)
-        thr = 1e-4 if self.tol == TOL_F32 else 2e-2
-        cand = [int(c) for c in r.near_units if row_rel[decode_unit(c, B)[1]] > thr]
-        cand.sort(key=lambda c: -row_rel[decode_unit(c, B)[1]])
-        cand = cand[:10]
-        for k in range(1, min(3, len(cand)) + 1):
-            for flips in itertools.combinations(cand, k):
-                res = rerun(np.array(flips, dtype=np.int64))
-                if ok(res):
-                    self.relu_flips_accepted += k
-                    return res
-        return r        # the strict asserts that follow report the mismatch
+        if len(bad_views) > max_views_with_flips(B):
+            return r                                        # not a matter of a few branches: the strict asserts report
+        order = np.argsort(r.near_abs, kind="stable")
+        by_view = {}
+        for k in order:
+            l, v, j = decode_unit(r.near_units[k], B)
+            by_view.setdefault(v, []).append((l, j))
+        off = np.asarray(img_off)
+        all_flips = []
+        for v in bad_views:
+            cands = by_view.get(int(v), [])[:6]
+            lo, hi = int(off[v]), int(off[v + 1])
+            found = None
+            for k in range(1, min(MAX_FLIPS_PER_VIEW, len(cands)) + 1):
+                for subset in itertools.combinations(cands, k):
+                    codes = np.array([(l * 1 + 0) * 1024 + j for (l, j) in subset], dtype=np.int64)
+                    one = self.cpu.forward_backward(params64, uid[v:v + 1], hid[v:v + 1], np.array([0, hi - lo], np.int32),
+                                                    img[lo:hi], label[v:v + 1], flip_units=codes)
+                    # a batch of one view divides by 1 where the batch divides by B
+                    if np.abs(got_dx[v] - one.dX[0] / B).max() <= self.tol * scale:
+                        found = subset
+                        break
+                if found:
+                    break
+            if not found:
+                return r                                    # the strict asserts report the mismatch
+            all_flips += [(l * B + int(v)) * 1024 + j for (l, j) in found]
+        res = self.cpu.forward_backward(params64, uid, hid, img_off, img, label,
+                                        flip_units=np.array(all_flips, dtype=np.int64))
+        self.last_relu.update(views=len(bad_views), units=len(all_flips))
+        self.relu_flips_accepted += len(all_flips)
+        self.relu_views_flipped += len(bad_views)
+        print("ReLU branches taken the other way inside the rounding band: %d units in %d of %d views (%d units listed)"
+              % (len(all_flips), len(bad_views), B, self.last_relu["listed"]))
+        return res
 
     def compare_store(self, check_tables: bool = True):
         gpu, cpu = self.gpu, self.cpu
@@ -229,6 +284,9 @@ class Pair:
         assert int(gpu.dfv_gcnt.sum().item()) == int(cpu.gcnt.sum()), "counts outside the touched rows"
         if check_tables:
             assert_close(_np(gpu.dfv_gsum[rows]), cpu.gsum, self.tol, "open-group sums")
+            # nothing may land in the accumulator row of an image the batches never name (a row written too wide
+            # would spill into its neighbour): the table's non-zero entries are all inside the touched rows
+            assert count_nonzero(gpu.dfv_gsum) == count_nonzero(gpu.dfv_gsum[rows]), "sums outside the touched rows"
 
     def collect_and_compare(self) -> int:
         gpu, cpu = self.gpu, self.cpu
@@ -240,6 +298,7 @@ class Pair:
         assert np.array_equal(self.ri(gid), eid), "emitted ids"
         assert np.array_equal(_np(gpu.ready_seq[:n]), eseq), "emission numbers"
         assert_close(_np(gpu.ready_avg[:n]), eavg, self.tol, "averaged gradients")
+        assert gpu.guards_intact(), "an output list was written past its end"
         return n
 
     def expire_and_compare(self, now: int, restamp: bool = True) -> int:
@@ -249,6 +308,7 @@ class Pair:
         assert n == len(want), "number of expired entries"
         assert np.array_equal(_np(gpu.expired_ids[:n]), want), "expired ids"
         assert np.array_equal(_np(gpu.dfv_ts), cpu.ts), "timestamps after the scan"
+        assert gpu.guards_intact(), "an output list was written past its end"
         return n
 
     def close(self):

@@ -91,11 +91,49 @@ def test_skew_shapes_ragged_batch(gb):
     (BF16, (320,), 20, 200, BF16, 129),         # head input 240 wide: a partial reduction block and partial column tiles
     (F32, (264,), 32, 8, F32, 2049),            # fp32 head: 128 x 128 product tiles with ragged edges on every side
     (F32, (64, 96), 16, 8, F32, 33),            # fp32 head below the large-tile threshold
+    # DFV widths on either side of the row widths the gather and the reduce pass are instantiated for
+    # (1, 2, 4 or 8 sixteen-byte chunks per lane): 3, 5, 6 and 7 chunks per lane take the guarded path of the next
+    # instantiation up; 4 and 8 chunks per lane the unguarded one
+    (F32, (64,), 16, 384, F32, 257),
+    (F32, (64,), 16, 640, F32, 130),
+    (BF16, (128,), 32, 768, BF16, 300),
+    (F32, (64,), 16, 896, F32, 65),
+    (F32, (64,), 8, 512, F32, 100),
+    (F32, (64,), 8, 1024, F32, 40),
+    (BF16, (64,), 8, 1024, BF16, 40),
 ])
 def test_odd_head_shapes(gb, head, hidden, E, D, dfv, B):
     p = PRESETS["medium"].scaled(emb_dim=E, dfv_dim=D, dfv_dtype=dfv, head_dtype=head, hidden=hidden, M=3,
                                  user_vocab=30_000, url_vocab=20_000, img_vocab=40_000, expire=2)
     _run_steps(p, 2, B=B, want_emb_grad=True)
+
+
+def _soak_case(case: int):
+    """A random but reproducible configuration: head type and widths, embedding and DFV widths, DFV type, batch
+    size, M, image vocabulary and expiry time are all drawn from (case)."""
+    rng = np.random.default_rng(1000 + case)
+    bf = rng.random() < 0.65
+    if bf:
+        hidden = tuple(int(rng.choice([64, 128, 192, 256, 320, 448, 512, 1024])) for _ in range(int(rng.integers(1, 3))))
+        E = int(rng.choice([4, 8, 20, 32, 64]))
+        D = int(rng.choice([8, 24, 64, 128, 200, 256, 384, 512, 768]))
+        dfv_dtype = BF16 if rng.random() < 0.7 else F32
+    else:
+        hidden = tuple(int(rng.choice([8, 24, 64, 96, 136, 256, 264])) for _ in range(int(rng.integers(1, 3))))
+        E = int(rng.choice([4, 12, 16, 32]))
+        D = int(rng.choice([8, 40, 64, 128, 256, 640]))
+        dfv_dtype = F32
+    B = int(rng.choice([1, 7, 33, 129, 500, 1237, 2049, 3000]))
+    p = PRESETS["medium"].scaled(emb_dim=E, dfv_dim=D, dfv_dtype=dfv_dtype, head_dtype=BF16 if bf else F32,
+                                 hidden=hidden, M=int(rng.choice([1, 2, 5, 16])), user_vocab=30_000, url_vocab=20_000,
+                                 img_vocab=int(rng.choice([5_000, 40_000])), expire=int(rng.choice([0, 2, 50])))
+    return p, B, bool(rng.random() < 0.5)
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_shapes(gb, case):
+    p, B, want_emb_grad = _soak_case(case)
+    _run_steps(p, 2, seed=case, B=B, want_emb_grad=want_emb_grad)
 
 
 @pytest.mark.parametrize("M", [1, 64, 1024])

@@ -655,3 +655,9 @@ def test_near_zero_units_are_listed_and_can_take_the_other_branch():
     np.testing.assert_allclose(flipped.dX, X.grad.numpy(), atol=1e-15)
     assert np.any(flipped.dX != r.dX)
     assert len(orc.forward_backward(params, *args, relu_margin=0.5).near_units) == 1      # |0.25 + ...| unit stays out
+    # the relative form of the margin: |a| <= rel * max|input row| * max|weights| = rel * 2 * 1; unit 1 has a = 2.25
+    wide = orc.forward_backward(params, *args, relu_margin=0.0, relu_margin_rel=1.2)
+    assert [decode_unit(c, 1) for c in wide.near_units] == [(0, 0, 0), (0, 0, 1)]
+    assert wide.near_abs.tolist() == [0.0, 2.25]
+    assert len(orc.forward_backward(params, *args, relu_margin=0.0, relu_margin_rel=1.1).near_units) == 1
+    assert np.array_equal(wide.dX, r.dX) and np.array_equal(wide.head_grad, r.head_grad)   # listing changes no result

@@ -4,9 +4,10 @@ Some users of libgear run where cudaMalloc is not theirs to call (a serving proc
 plan, a plug-in that is only handed buffers), so they cannot give a gear_ctx its workspace.  This entry
 point keeps its scratch in a fixed array inside the library instead.  The test calls it through the C ABI,
 twice in a row on the same table, and checks each result against the ctx-based gear_collect_expired on an
-identical copy of the table: ID lists and restamped timestamps must be bit-identical (integer work, so the
-tolerance is zero, as in the other expiry tests).  The second call runs on whatever the first one left in
-the shared scratch and finds a different, smaller set of expired images.
+identical copy of the table and against the CPU oracle's scan of the same timestamps: ID lists and restamped
+timestamps must be bit-identical (integer work, so the tolerance is zero, as in the other expiry tests).  The
+second call runs on whatever the first one left in the shared scratch and finds a different, smaller set of
+expired images.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run every other test.
 """
@@ -37,6 +38,9 @@ def test_static_expiry_scan_matches_the_ctx_based_scan_twice_in_a_row(gb):
     tables = dict(user_emb=np.zeros((64, p.emb_dim), np.float32), url_emb=np.zeros((64, p.emb_dim), np.float32),
                   dfv=np.zeros((V, p.dfv_dim), np.float32), ts=ts0.copy())
     ref = GearSession(p, workloads.head_params(p, 0), max_batch=8, max_nnz=32, tables=tables)
+    from oracle import GearOracle
+    cpu = GearOracle(tables["user_emb"], tables["url_emb"], np.zeros((1, p.dfv_dim), np.float32), p.hidden, p.M, T,
+                     ts=ts0.copy())
     try:
         ts = torch.from_numpy(ts0.copy()).cuda()
         ids = torch.full((V,), -1, dtype=torch.int32, device="cuda")
@@ -48,6 +52,9 @@ def test_static_expiry_scan_matches_the_ctx_based_scan_twice_in_a_row(gb):
             assert n == n_ref and int(d_n.item()) == n_ref
             assert torch.equal(ids[:n], ref.expired_ids[:n])
             assert torch.equal(ts, ref.dfv_ts)
+            want = cpu.collect_expired(now, restamp=True)
+            assert n == len(want) and np.array_equal(ids[:n].cpu().numpy(), want)
+            assert np.array_equal(ts.cpu().numpy(), cpu.ts)
             seen.append(n)
         assert seen[0] > 0 and seen[1] > 0 and seen[0] != seen[1]
         # without restamping, and with the count read from the device only
@@ -55,6 +62,7 @@ def test_static_expiry_scan_matches_the_ctx_based_scan_twice_in_a_row(gb):
         assert gb.gear_collect_expired_static(ts, T, 60, False, ids, V, d_n=d_n, sync=False) is None
         assert int(d_n.item()) == n_ref and torch.equal(ids[:n_ref], ref.expired_ids[:n_ref])
         assert torch.equal(ts, ref.dfv_ts)
+        assert np.array_equal(ids[:n_ref].cpu().numpy(), cpu.collect_expired(60, restamp=False))
     finally:
         ref.close()
 
