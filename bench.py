@@ -35,6 +35,8 @@ sys.path.insert(0, ROOT)
 METRIC = "page views/sec per step (1 B200); gather+accumulate HBM GB/s vs ~8 TB/s peak"
 UNIT = "page views/s"
 N_BATCHES = 8          # distinct pre-generated batches the timed loop cycles through
+MIN_TIMED_MS = 1000.0  # device time measured per arm, whatever --steps is: the K-step region is repeated until then
+MAX_REGIONS = 400
 
 
 def measured_peaks():
@@ -161,7 +163,7 @@ def kernel_models(p, stats):
 # re-reads that hit the L2 in a real step count as DRAM traffic here.  A kernel that has changed since its capture
 # must be taken out of this table (traffic is then reported as null).
 NCU_TRAFFIC_LARGE_2M = {
-    "gather_pool": (64.4e6, "work"), "acc_reduce": (239.7e6, "work"), "expiry_mark": (16.0e6, "vocab"),
+    "gather_pool": (64.4e6, "l2"), "acc_reduce": (239.7e6, "work"), "expiry_mark": (16.0e6, "vocab"),
     "head_out": (34.4e6, None), "collect_move": (5.9e6, "work"), "emb_reduce": (46.9e6, "work"),
     "tc_gemm_fwd": (68.3e6, None), "tc_gemm_dw": (113.7e6, None), "tc_gemm_dh": (129.5e6, None), "tc_gemm_dx": (110.2e6, None),
 }
@@ -170,52 +172,72 @@ NCU_WORK_LARGE_2M = {"gather_pool": 222.0e6, "acc_reduce": 224.5e6, "collect_mov
 
 
 def ncu_traffic(name, p, work):
-    """DRAM traffic per launch of kernel `name` on workload p, scaled from the large_2m capture; None if unknown."""
-    if name not in NCU_TRAFFIC_LARGE_2M or not p.name.startswith("large"):
-        return None
+    """(DRAM traffic per launch of kernel `name` on workload p, where the figure comes from); (None, reason) if there
+    is no figure that holds for this workload."""
+    if name not in NCU_TRAFFIC_LARGE_2M:
+        return None, "no ncu capture of this kernel as it stands"
+    if not p.name.startswith("large"):
+        return None, "ncu captures exist for the large-table shapes only"
     bytes_2m, scales_with = NCU_TRAFFIC_LARGE_2M[name]
+    if p.name == "large_2m":
+        return round(bytes_2m), "ncu --set full on this workload (large_2m)"
     if scales_with == "vocab":
-        return round(bytes_2m * p.img_vocab / 2_000_000)
+        return round(bytes_2m * p.img_vocab / 2_000_000), "ncu on large_2m, scaled by the image vocabulary"
     if scales_with == "work":
         if not work or name not in NCU_WORK_LARGE_2M:
-            return None
-        return round(bytes_2m * work / NCU_WORK_LARGE_2M[name])
-    return round(bytes_2m)
+            return None, "no algorithmic-bytes figure to scale by"
+        return round(bytes_2m * work / NCU_WORK_LARGE_2M[name]), "ncu on large_2m, scaled by algorithmic bytes"
+    if scales_with == "l2":
+        return None, ("ncu on large_2m only: the L2 serves a share of the rows of a 2M-image table that it cannot "
+                      "serve of a 20M-image one, so the figure does not scale")
+    return round(bytes_2m), "ncu on large_2m, same shapes"
 
 
 def roofline_for(name, ms_per_launch, p, stats, peaks):
     """Roofline object of one kernel from its live per-launch time."""
     models = kernel_models(p, stats)
-    B = stats["B"]
-    fan = [p.d_in] + list(p.hidden)
     sec = ms_per_launch * 1e-3
     if name in models and isinstance(models[name], tuple):
         work = models[name][1]
         ach = work / sec / 1e9
+        traffic, source = ncu_traffic(name, p, work)
         return {"kernel": name, "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": ncu_traffic(name, p, work),
+                "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": traffic, "traffic_source": source,
                 "peak_source": peaks["source"], "work_per_launch": work}
     if name.startswith("simt_gemm") or name.startswith("tc_gemm"):
+        # The head's products are dense contractions: rated by their flops against the tensor peak (bf16 heads; the
+        # sustained figure, since they run inside a long step) or the fp32 FMA peak (fp32 heads).  memory_frac is
+        # the secondary figure: every operand and the output once, over the measured copy rate.
         flops, nbytes = models["gemm"][name.rsplit("_", 1)[1]]
         if name.startswith("tc_gemm"):
-            peak, bound, src = peaks["bf16_sustained"] or peaks["bf16_tflops"], "tensor", peaks["source"]
+            peak, bound, src = peaks["bf16_sustained"] or peaks["bf16_tflops"], "tensor", peaks["source"] + " (sustained bf16)"
         else:
             peak, bound, src = ALU_F32_TFLOPS, "alu", "148 SMs x 128 FMA lanes x 2 x 1.965 GHz"
-        # the roofline that binds: with reductions and outputs of a few hundred columns these products move a byte per
-        # ~100-200 flops, which is where a B200's tensor and memory rooflines cross
-        t_math, t_mem = flops / (peak * 1e12), nbytes / (peaks["hbm_gbs"] * 1e9)
-        if t_mem > t_math:
-            ach = nbytes / sec / 1e9
-            return {"kernel": name, "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": ncu_traffic(name, p, None),
-                    "peak_source": peaks["source"], "work_per_launch": nbytes,
-                    "math_frac": round(flops / sec / 1e12 / peak, 4)}
         ach = flops / sec / 1e12
+        traffic, source = ncu_traffic(name, p, None) if bound == "tensor" else (None, "fp32 head: no capture")
         return {"kernel": name, "bound": bound, "achieved": round(ach, 2), "peak": round(peak, 1), "unit": "TFLOP/s",
-                "frac": round(ach / peak, 4), "traffic": ncu_traffic(name, p, None) if bound == "tensor" else None,
+                "frac": round(ach / peak, 4), "traffic": traffic, "traffic_source": source,
                 "peak_source": src, "work_per_launch": flops, "memory_frac": round(nbytes / sec / 1e9 / peaks["hbm_gbs"], 4)}
     return {"kernel": name, "bound": "latency", "achieved": None, "peak": None, "unit": None, "frac": None,
-            "traffic": None}
+            "traffic": None, "traffic_source": None}
+
+
+def step_roofline(p, stats, ms_per_step, peaks):
+    """The whole step against both rooflines: the bytes the method has to move per step (gather, embedding scatter,
+    accumulate, emit, expiry scan; intermediates of the head not counted) and the head's flops, over the step time."""
+    m = kernel_models(p, stats)
+    nbytes = sum(m[k][1] for k in ("gather_pool", "acc_reduce", "expiry_mark", "emb_reduce"))
+    nbytes += stats.get("n_ready", 0.0) * (p.dfv_dim * 4 + 8) if not stats.get("emit_direct") else 0.0
+    fan = [p.d_in] + list(p.hidden)
+    flops = 6.0 * stats["B"] * (sum(fan[l] * fan[l + 1] for l in range(len(p.hidden))) + fan[-1])
+    sec = ms_per_step * 1e-3
+    tensor_peak = (peaks["bf16_sustained"] or peaks["bf16_tflops"]) if p.head_dtype == "bf16" else ALU_F32_TFLOPS
+    return {"bytes_per_step": round(nbytes), "flops_per_step": round(flops),
+            "hbm_GB/s": round(nbytes / sec / 1e9, 1), "hbm_frac": round(nbytes / sec / 1e9 / peaks["hbm_gbs"], 4),
+            "math_TFLOP/s": round(flops / sec / 1e12, 2), "math_frac": round(flops / sec / 1e12 / tensor_peak, 4),
+            "math_peak": round(tensor_peak, 1), "math_bound": "tensor" if p.head_dtype == "bf16" else "alu",
+            "lower_bound_ms": round(max(nbytes / (peaks["hbm_gbs"] * 1e9), flops / (tensor_peak * 1e12)) * 1e3, 4),
+            "peak_source": peaks["source"]}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -353,9 +375,20 @@ def run_ours(args):
     sampler.open_window()
     for s in range(W):
         one_step(dev_batches[s % N_BATCHES])
+    def regions_of(region_fn):
+        """Repeats the K-step timed region until MIN_TIMED_MS of device time have been measured (at least 3 regions):
+        a few steps alone are too short for the clock sampler to see and for the clocks to settle under load.  The
+        loop count follows from the max-over-ranks time, so every rank runs the same number of regions."""
+        out = []
+        while (sum(out) < MIN_TIMED_MS or len(out) < 3) and len(out) < MAX_REGIONS:
+            out.append(region_fn())
+        return out
+
     launches0 = gb.gear_launch_count(sess.ctx)
     ms = timed(lambda s: one_step(dev_batches[s % N_BATCHES]), K)
     launches = gb.gear_launch_count(sess.ctx) - launches0
+    region_ms = [ms] + regions_of(lambda: timed(lambda s: one_step(dev_batches[s % N_BATCHES]), K))
+    ms = float(np.median(region_ms))
     rc, status, _ = sess.status()
     n_ready_mean = None
 
@@ -432,7 +465,8 @@ def run_ours(args):
         return reps.max_over_ranks(ev0.elapsed_time(ev1), device="cuda")
 
     e2e_run(min(W, 3))
-    ms_e2e = timed_run(e2e_run, K)
+    e2e_region_ms = regions_of(lambda: timed_run(e2e_run, K))
+    ms_e2e = float(np.median(e2e_region_ms))
     sampler.close_window()
     clocks = sampler.stop()
     d2h_bytes = 24
@@ -469,8 +503,12 @@ def run_ours(args):
             hbm_kernels.append({"kernel": kd["name"], "GB/s": r["achieved"], "frac_of_measured": r["frac"],
                                 "frac_of_8TBs": round(r["achieved"] / 8000.0, 4), "ms": round(kd["ms_per_launch"], 4)})
 
+    stats["emit_direct"] = any(k["name"] == "acc_reduce" for k in kernels) and not any(k["name"] == "collect_move" for k in kernels)
+    spread = lambda xs: {"regions": len(xs), "min_ms_per_step": round(min(xs) / K, 4), "median_ms_per_step": round(float(np.median(xs)) / K, 4),
+                         "max_ms_per_step": round(max(xs) / K, 4), "timed_ms": round(sum(xs), 1)}
     line = {"metric": METRIC, "value": round(reps.whole_job_rate(p.batch * K, ms), 1), "unit": UNIT, "n_gpus": world, "steps": K,
-            "warmup": W, "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak",
+            "warmup": W, "ms_per_step": round(ms / K, 4), "regions": spread(region_ms),
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if p.head_dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": "large tables" if p.name == "large" else p.name, "batch": p.batch,
                        "tables_gb": round((p.user_vocab + p.url_vocab) * p.emb_dim * 4 / 1e9 + p.img_vocab * p.dfv_dim *
@@ -481,12 +519,18 @@ def run_ours(args):
                        "streams": ("training calls on one stream, the expiry scan of the same step on a second one, "
                                    "forked at the step's start and joined at its end (inside the timed region)")
                        if expiry_beside_default else "all calls on one stream",
+                       "outputs": "the averaged-gradient list (ids, seq, avg) and the expired-ID list of every step stay in "
+                                  "device memory, where a Dense Part on the same GPU would consume them; the end-to-end arm "
+                                  "reads back the loss and the two counts (24 bytes)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks,
             "e2e": {"value": round(reps.whole_job_rate(p.batch * K, ms_e2e), 1), "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,
-                    "d2h_bytes_per_step": d2h_bytes, "ms_per_step": round(ms_e2e / K, 4)},
+                    "d2h_bytes_per_step": d2h_bytes, "ms_per_step": round(ms_e2e / K, 4), "regions": spread(e2e_region_ms)},
             "gpu_launches": int(launches),
             "roofline": roof,
+            "roofline_step": step_roofline(p, stats, ms / K, peaks),
+            "products": [roofline_for(k["name"], k["ms_per_launch"], p, stats, peaks) for k in kernels
+                         if k["name"].startswith(("tc_gemm", "simt_gemm"))],
             "kernels": [{"name": k["name"], "ms_per_step": round(k["ms_per_step"], 4), "share": round(k["share"], 4),
                          "launches_per_step": round(k["launches_per_step"], 2)} for k in kernels],
             "hbm_kernels": hbm_kernels,
@@ -503,13 +547,94 @@ def run_ours(args):
     reps.close()
 
 
+# ---------------------------------------------------------------------------------------------
+# configurations 4 and 5: accumulate-only micro-benchmark, sort against atomics under skew
+# ---------------------------------------------------------------------------------------------
+def oracle_accumulate_sample(ids, V, D, M, n_sample, seed=5):
+    """The CPU oracle's accumulate + collect on the first n_sample rows of the case; returns seconds."""
+    import oracle
+    from oracle import GearOracle
+    n = min(n_sample, len(ids))
+    rows = oracle.fill_rows(seed, oracle.TAG_GRAD, D, None, n, np.float32, amp=1.0).astype(np.float64)
+    orc = GearOracle(np.zeros((1, 4), np.float32), np.zeros((1, 4), np.float32), np.zeros((V, D), np.uint16), (8,), M, 1 << 40)
+    t0 = time.perf_counter()
+    orc.accumulate(ids[:n], rows)
+    orc.collect_ready()
+    return time.perf_counter() - t0, n
+
+
+def accumulate_line(case, args, sampler_gpu, peaks, with_cpu=True):
+    """One JSON line for one accumulate-only case (a dict from microbench._run_case plus the keys of the contract)."""
+    acc_ms = case["kernel_ms"].get("acc_reduce")
+    total_ms = case["accumulate_ms"] + case["collect_ms"]
+    n, D, uniq, ready = case["rows"], case["dim"], case["distinct_images"], case["emissions_per_call"]
+    line = {"metric": METRIC, "value": case["rows_per_s"], "unit": "gradient rows/s", "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": case["case"], "mode": case["mode"], "rows": n, "img_vocab": case["img_vocab"], "dim": D,
+                       "M": case["M"], "distinct_images": uniq, "emissions_per_call": ready,
+                       "step": "one gear_accumulate_dfv_grad over all rows + one gear_collect_ready",
+                       "l2": "8.6 GB of gradient rows and a 2 GB store per call: far beyond the 126 MB L2"},
+            "clocks": sampler_gpu, "gpu_launches": case.get("launches_per_step"),
+            "e2e": None, "e2e_note": "the rows are produced on the device by the head's backward pass and never cross "
+                                     "PCIe in the method: no host-buffer arm for this kernel-level case",
+            "kernel_ms": case["kernel_ms"], "device_status": case["device_status"],
+            "roofline_step": {"bytes_per_step": round(case["algorithmic_GB"] * 1e9), "hbm_GB/s": case["GB/s"],
+                              "hbm_frac": case["frac_of_hbm_peak"], "frac_of_8TBs": case["frac_of_8TBs"],
+                              "peak_source": case["peak_source"]}}
+    if acc_ms:
+        work = n * D * 4 + n * 8 + uniq * (D * 4 + 4) * 2 + ready * (D * 4 + 4)
+        ach = work / (acc_ms * 1e-3) / 1e9
+        line["roofline"] = {"kernel": "acc_reduce", "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"],
+                            "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4), "traffic": None,
+                            "traffic_source": "no ncu capture at this size", "peak_source": peaks["source"],
+                            "work_per_launch": work}
+    return line
+
+
+def run_accumulate_cases(args, which):
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libgear has no CPU path")
+    from paper_1806_03925_b200 import microbench, workloads
+    from paper_1806_03925_b200.workloads import MICRO_PRESETS, PRESETS, BatchSource
+    peaks = measured_peaks()
+    cases = []
+    if which == "micro":
+        for name, mp in MICRO_PRESETS.items():
+            cases.append((name, workloads.micro_ids(mp, seed=0), mp.img_vocab, mp.dfv_dim, mp.M, "sort"))
+    else:
+        p = PRESETS["skew"]
+        ids = BatchSource(p, 0).batch(0).img_id
+        for M in (1, 64, 1024):
+            for mode in ("sort", "atomic"):
+                cases.append(("skew_M%d" % M, ids, p.img_vocab, p.dfv_dim, M, mode))
+    for name, ids, V, D, M, mode in cases:
+        sampler = ClockSampler(0)
+        sampler.start()
+        time.sleep(0.3)
+        sampler.open_window()
+        case = microbench._run_case(name, ids, V, D, M, mode, steps=max(args.steps, 5), warmup=max(args.warmup, 3))
+        sampler.close_window()
+        line = accumulate_line(case, args, sampler.stop(), peaks)
+        if not args.no_cpu_baseline:
+            sec, n_s = oracle_accumulate_sample(ids, V, D, M, 1 << 21)
+            line["cpu_baseline"] = {"value": round(n_s / sec, 1), "unit": "gradient rows/s", "cores": 1, "kind": "oracle",
+                                    "sample": "the first %d rows of the case through orc_accumulate and the hand-over, "
+                                              "%.1f s of CPU time" % (n_s, sec)}
+        print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="large", choices=["large", "large_2m", "medium", "tiny", "skew"])
+    ap.add_argument("--workload", default="large", choices=["large", "large_2m", "medium", "tiny", "skew", "micro", "skew_modes"],
+                    help="large (default): the configuration the metric is quoted on.  micro: the accumulate-only "
+                         "micro-benchmark, one line per case.  skew: the skew-stress step.  skew_modes: its accumulate call, "
+                         "sort against atomics, M in {1, 64, 1024}, one line per case")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     # defaults: a few hundred milliseconds of device time per timed region for the CUDA path (so that the
@@ -521,7 +646,13 @@ def main():
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
+        if args.workload in ("micro", "skew_modes"):
+            raise SystemExit("the reference arm times the whole step: use --workload large, medium, tiny or skew")
         run_reference(args)
+    elif args.workload in ("micro", "skew_modes"):
+        if args.steps == 400:
+            args.steps = 7
+        run_accumulate_cases(args, "micro" if args.workload == "micro" else "skew")
     else:
         run_ours(args)
 

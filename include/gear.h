@@ -17,6 +17,7 @@
  *                             image; every M-th arrival completes a group.
  *   gear_collect_ready        event 6: hand over the averaged gradient of
  *                             every completed group.
+ *   gear_accumulate_collect   events 5 and 6 as one call.
  *   gear_refresh_dfv          Section 1 / Section 3: recomputed DFVs replace
  *                             expired ones and restart their clocks.
  *   gear_collect_expired      Section 1 / Section 3: cached inference results
@@ -201,6 +202,19 @@ int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* 
  */
 int gear_collect_ready(gear_ctx* ctx, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
                        int64_t* d_n, int64_t* h_n, void* stream);
+
+/*
+ * Events 5 and 6 in one call (Section 3: the gradients arrive and, as soon as M of an image are there, their average
+ * goes on to the Dense Part): the same results as gear_accumulate_dfv_grad followed by gear_collect_ready with the
+ * same arguments.  When no average was waiting in the ready queue before the call and cap >= n, the averages of
+ * the groups this call completes are written straight into ids / seq / avg without passing through the queue;
+ * in every other case the library does the two steps one after the other.  Capacity behaviour as in
+ * gear_collect_ready (too small: the completed groups stay in the queue, nothing is handed over).
+ */
+int gear_accumulate_collect(gear_ctx* ctx, const int32_t* img_id, const float* grads, int64_t ld,
+                            const int32_t* src_row, const float* scale, int64_t n,
+                            int32_t* ids, int32_t* seq, float* avg, int64_t cap,
+                            int64_t* d_n, int64_t* h_n, void* stream);
 
 /*
  * Expiry scan.  Lists, in ascending order, every image with now - dfv_ts[id] >= expire; with

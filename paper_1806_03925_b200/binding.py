@@ -25,7 +25,7 @@ GEAR_TAG_USER, GEAR_TAG_URL, GEAR_TAG_DFV, GEAR_TAG_TS, GEAR_TAG_GRAD = 1, 2, 3,
 EXPORTS = ("gear_workspace_bytes", "gear_init_tables", "gear_forward_backward", "gear_accumulate_dfv_grad",
            "gear_collect_ready", "gear_collect_expired", "gear_status", "gear_destroy", "gear_fill_uniform",
            "gear_last_error", "gear_profile_enable", "gear_profile_read", "gear_launch_count",
-           "gear_collect_expired_static", "gear_refresh_dfv")
+           "gear_collect_expired_static", "gear_refresh_dfv", "gear_accumulate_collect")
 GEAR_STATIC_EXPIRY_MAX_VOCAB = 16777216
 
 
@@ -83,6 +83,8 @@ def load() -> C.CDLL:
     L.gear_accumulate_dfv_grad.argtypes = [vp, vp, vp, i64, vp, vp, i64, vp]
     L.gear_collect_ready.restype = C.c_int
     L.gear_collect_ready.argtypes = [vp, vp, vp, vp, i64, vp, C.POINTER(i64), vp]
+    L.gear_accumulate_collect.restype = C.c_int
+    L.gear_accumulate_collect.argtypes = [vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, i64, vp, C.POINTER(i64), vp]
     L.gear_collect_expired.restype = C.c_int
     L.gear_collect_expired.argtypes = [vp, i64, C.c_int, vp, i64, vp, C.POINTER(i64), vp]
     L.gear_status.restype = C.c_int
@@ -217,6 +219,16 @@ def gear_collect_ready(ctx, ids, seq, avg, cap: int, d_n=None, sync: bool = True
     h = C.c_int64(-1)
     _check(load().gear_collect_ready(ctx, _p(ids), _p(seq), _p(avg), cap, _p(d_n), C.byref(h) if sync else None,
                                      _stream(stream)), "gear_collect_ready")
+    return h.value if sync else None
+
+
+def gear_accumulate_collect(ctx, img_id, grads_ptr: int, ld: int, src_row, scale, n: int, ids, seq, avg, cap: int,
+                            d_n=None, sync: bool = True, stream=None) -> Optional[int]:
+    """gear_accumulate_dfv_grad and gear_collect_ready as one call; returns the number of entries when sync."""
+    h = C.c_int64(-1)
+    _check(load().gear_accumulate_collect(ctx, _p(img_id), C.c_void_p(grads_ptr), ld, _p(src_row), _p(scale), n,
+                                          _p(ids), _p(seq), _p(avg), cap, _p(d_n), C.byref(h) if sync else None,
+                                          _stream(stream)), "gear_accumulate_collect")
     return h.value if sync else None
 
 

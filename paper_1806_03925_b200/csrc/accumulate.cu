@@ -51,6 +51,7 @@ struct TileFlags {
     bool first[AF_ITEMS];      // ... and is the first row of its image in this call
     bool complete[AF_ITEMS];   // ... and the group reaches M
     int c0[AF_ITEMS];          // rows the image already holds in the table
+    int seq[AF_ITEMS];         // group heads: how many groups of the image this call completes before this one
     int64_t i0;                // first position owned by this thread
 };
 
@@ -109,7 +110,7 @@ __device__ __forceinline__ void tile_flags(TileFlags& f, const uint32_t* __restr
     for (int t = 0; t < AF_ITEMS; ++t) {
         const int64_t i = f.i0 + t;
         f.head[t] = f.first[t] = f.complete[t] = false;
-        f.c0[t] = 0;
+        f.c0[t] = 0; f.seq[t] = 0;
         if (i >= n || f.key[t] >= vocab) continue;
         uint32_t rs = max(run_start[t], before_thread);
         const int64_t start = rs ? (int64_t)rs - 1 : (int64_t)carry;
@@ -120,6 +121,7 @@ __device__ __forceinline__ void tile_flags(TileFlags& f, const uint32_t* __restr
         if (j == 0 || rem == 0) {
             f.head[t] = true;
             f.first[t] = (j == 0);
+            f.seq[t] = (int)((c0 + j) / M);          // c0 < M: the first group of the image gets 0
             const int64_t last = i + (M - rem) - 1;  // the row that brings the count to M
             f.complete[t] = last < n && ks[last] == f.key[t];
         }
@@ -172,9 +174,11 @@ acc_plan_kernel(const uint32_t* __restrict__ ks, int64_t n, uint32_t vocab, int 
         if (((f.i0 + t) % ACC_SPAN) == 0 && f.i0 + t < n && f.key[t] < vocab) blk_first[(f.i0 + t) / ACC_SPAN] = gi;
         if (!f.head[t]) continue;
         // one 16-byte record per group: start position (top bit: first group of its image in this call), image ID,
-        // ready-queue slot (-1: the group stays open), rows the image already held
+        // ready-queue slot (-1: the group stays open), and for the image's first group the rows the image already held,
+        // for a later one its number among the groups of the image that this call completes
         grp_rec[gi] = make_uint4((uint32_t)(f.i0 + t) | (f.first[t] ? 0x80000000u : 0u), f.key[t],
-                                 (uint32_t)(f.complete[t] ? (int32_t)(q_base + ci) : -1), (uint32_t)f.c0[t]);
+                                 (uint32_t)(f.complete[t] ? (int32_t)(q_base + ci) : -1),
+                                 (uint32_t)(f.first[t] ? f.c0[t] : f.seq[t]));
         ++gi;
         ci += f.complete[t];
     }
@@ -207,8 +211,13 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
 struct LaneGroup {
     uint32_t start, key, zstart;
     int slot, c0, len, zlen, items;      // items = rows the warp stages for the group (0: nothing to do)
+    int seq;                             // number of the group among those of its image that the call completes
     bool first;
 };
+
+// Where the averages of the groups a call completes go when they bypass the ready queue: the caller's own lists
+// (gear_accumulate_collect on a queue that is known to be empty).  All null: the groups join the queue.
+struct EmitTarget { int32_t* ids; int32_t* seq; float* avg; int64_t* d_n; };
 
 // One row to stage, as the copy side sees it (where the row starts; bit 0 of the address word is set if the item
 // exists) and as the adding side sees it (what the row is scaled by and
@@ -235,14 +244,20 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                   const uint2* __restrict__ tile_cnt, const uint4* __restrict__ grp_rec,
                   const uint32_t* __restrict__ blk_first, const uint32_t* __restrict__ run_end,
                   float* __restrict__ gsum, int32_t* __restrict__ gcnt,
-                  int32_t* __restrict__ q_id, float* __restrict__ q_avg, DevState* __restrict__ state) {
+                  int32_t* __restrict__ q_id, float* __restrict__ q_avg, const EmitTarget direct,
+                  DevState* __restrict__ state) {
     wait_for_predecessor();
     extern __shared__ float4 ring_mem[];                          // [warps][S][NQ * 32] float4
     const uint2 totals = tile_cnt[n_tiles];
     const int64_t n_groups = totals.x;
+    // Averages go to the ready queue, or (the queue being empty, so that queue slot k is also entry k of the hand-over)
+    // straight into the caller's lists, whose capacity the host has checked against the row count.
+    const bool to_caller = direct.avg != nullptr;
+    int32_t* __restrict__ e_id = to_caller ? direct.ids : q_id;
+    float* __restrict__ e_avg = to_caller ? direct.avg : q_avg;
     // Step 6 of the plan (commit) is done by whichever block finishes last: by then every block has read the queue
     // length it started from.  Every block, also one of a dropped call, leaves through this.
-    const bool dropped = state->q_count + (int64_t)totals.y > ready_cap;
+    const bool dropped = !to_caller && state->q_count + (int64_t)totals.y > ready_cap;
     auto leave = [&]() {
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -251,7 +266,8 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
             if (atomicInc(ticket, gridDim.x - 1) == gridDim.x - 1) {
                 state->n_groups = totals.x;
                 state->n_complete = totals.y;
-                if (dropped) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
+                if (to_caller) { if (direct.d_n) *direct.d_n = totals.y; }
+                else if (dropped) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
                 else if (totals.y > 0) { state->q_count += totals.y; state->q_calls += 1; }
             }
         }
@@ -277,13 +293,14 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
         return v;
     };
     auto load_group = [&](int64_t g_lo, int64_t g_hi) -> LaneGroup {
-        LaneGroup r{0u, 0u, 0u, -1, 0, 0, 0, 0, false};
+        LaneGroup r{0u, 0u, 0u, -1, 0, 0, 0, 0, 0, false};
         const int64_t g = g_lo + lane;
         if (g < g_hi) {
             const uint4 rec = __ldg(grp_rec + g);
             const uint32_t end = (g + 1 < n_groups) ? (__ldg(&grp_rec[g + 1].x) & 0x7fffffffu) : (uint32_t)n_valid;
             r.start = rec.x & 0x7fffffffu; r.first = rec.x >> 31; r.key = rec.y; r.slot = (int)rec.z;
             r.c0 = r.first ? (int)rec.w : 0;
+            r.seq = r.first ? 0 : (int)rec.w;
             r.len = (int)(end - r.start);
         }
         return r;
@@ -349,7 +366,7 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                 const int slot = __shfl_sync(0xffffffffu, G.slot, l);
                 float* srow = gsum + (int64_t)key * D;
                 if (own_done && slot >= 0) {                    // the group reached M: its average joins the queue
-                    float* qrow = q_avg + (int64_t)slot * D;
+                    float* qrow = e_avg + (int64_t)slot * D;
 #pragma unroll
                     for (int q = 0; q < NQ; ++q) {
                         const int ch = lane + 32 * q;
@@ -357,7 +374,11 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
                             st_f4(qrow + ch * 4, make_float4(acc[q].x / m_f, acc[q].y / m_f, acc[q].z / m_f, acc[q].w / m_f));
                         acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
-                    if (lane == 0) q_id[slot] = (int32_t)key;
+                    if (lane == 0) e_id[slot] = (int32_t)key;
+                    if (to_caller) {
+                        const int seq = __shfl_sync(0xffffffffu, G.seq, l);
+                        if (lane == 0) direct.seq[slot] = seq;
+                    }
                 }
                 if (all_done) {
                     const int c0 = __shfl_sync(0xffffffffu, G.c0, l), len = __shfl_sync(0xffffffffu, G.len, l);
@@ -416,9 +437,9 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
 #pragma unroll
                     for (int q = 0; q < NQ; ++q) {
                         const float4 v = row[lane + 32 * q];
-                        // the gradient row is the rounded product (row * 1/n_b); it is then added: two roundings, no fused step
-                        acc[q].x = __fadd_rn(acc[q].x, __fmul_rn(scale, v.x)); acc[q].y = __fadd_rn(acc[q].y, __fmul_rn(scale, v.y));
-                        acc[q].z = __fadd_rn(acc[q].z, __fmul_rn(scale, v.z)); acc[q].w = __fadd_rn(acc[q].w, __fmul_rn(scale, v.w));
+                        // in the indirect form the scaled row is never stored: the product joins the sum with one rounding
+                        acc[q].x = fmaf(scale, v.x, acc[q].x); acc[q].y = fmaf(scale, v.y, acc[q].y);
+                        acc[q].z = fmaf(scale, v.z, acc[q].z); acc[q].w = fmaf(scale, v.w, acc[q].w);
                     }
                     if (meta & 3) settle(meta >> 2, (meta & 1) != 0, (meta & 2) != 0);
                     cslot = advance(cslot);
@@ -468,8 +489,11 @@ cudaError_t launch_accumulate_plan_ahead(const gear_ctx_impl& c, int64_t n, cons
     return cudaSuccess;
 }
 
-cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
-                              const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st) {
+// to_caller (optional): the caller's lists; only valid while the ready queue is known to be empty and the lists hold
+// at least n entries (gear_accumulate_collect checks both on the host)
+static cudaError_t launch_accumulate_to(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
+                                        const int32_t* src_row, const float* scale, int64_t n, const EmitTarget& to_caller,
+                                        cudaStream_t st) {
     if (n <= 0) return cudaSuccess;
     const int64_t vocab = c.cfg.img_vocab;
     const int D = c.cfg.dfv_dim, M = c.cfg.M;
@@ -521,7 +545,7 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
         if (le != cudaSuccess) return;
         le = launch_dependent(kernel, dim3(grid), dim3(256), (size_t)smem, st, ks, rg, D, M, n_tiles, c.ws.ready_cap, tile_cnt, grp_rec, blk_first, run_end,
                                         c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id),
-                                        c.at<float>(c.ws.q_avg), state);
+                                        c.at<float>(c.ws.q_avg), to_caller, state);
     };
     // ring depth: as many row slots as about 96 KB per block (two blocks per SM) allow, at most 8.
     // FULL only when a row fills the instantiated width exactly (D == NQ * 128): every lane then owns a chunk of every
@@ -535,8 +559,31 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
 #undef GEAR_ACC_LAUNCH
     }
     if (le != cudaSuccess) return le;
-    ++c.acc_calls_pending;
+    if (!to_caller.avg) ++c.acc_calls_pending;                    // a call that bypasses the queue leaves it empty
     return cudaGetLastError();
+}
+
+cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
+                              const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st) {
+    return launch_accumulate_to(c, img_id, grads, ld, src_row, scale, n, EmitTarget{nullptr, nullptr, nullptr, nullptr}, st);
+}
+
+// Events 5 and 6 in one call.  When the host knows the ready queue to be empty (no accumulate call since a collect that
+// could not be refused) and the caller's lists can take every group the n rows could complete, the reduce pass writes
+// ids, emission numbers and averages straight into the caller's lists and its last block reports the count: no
+// hand-over pass, and the averages cross memory once.  Otherwise: accumulate into the queue, then hand the queue over.
+cudaError_t launch_accumulate_collect(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
+                                      const int32_t* src_row, const float* scale, int64_t n, int32_t* ids, int32_t* seq,
+                                      float* avg, int64_t cap, int64_t* d_n, cudaStream_t st) {
+    const bool direct = c.cfg.accum_mode == GEAR_ACC_SORT && c.acc_calls_pending == 0 && n > 0 && cap >= n;
+    if (direct) return launch_accumulate_to(c, img_id, grads, ld, src_row, scale, n, EmitTarget{ids, seq, avg, d_n}, st);
+    cudaError_t e = cudaSuccess;
+    if (n > 0)
+        e = c.cfg.accum_mode == GEAR_ACC_ATOMIC
+                ? launch_accumulate_atomic(c, img_id ? img_id : c.last_img_id, grads, ld, src_row, scale, n, st)
+                : launch_accumulate(c, img_id, grads, ld, src_row, scale, n, st);
+    if (e != cudaSuccess) return e;
+    return launch_collect_ready(c, ids, seq, avg, cap, d_n, st);
 }
 
 // ---------------------------------------------------------------- GEAR_ACC_ATOMIC: the store without arrival order

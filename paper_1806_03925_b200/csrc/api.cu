@@ -320,6 +320,32 @@ int gear_accumulate_dfv_grad(gear_ctx* ctx, const int32_t* img_id, const float* 
     return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "accumulate");
 }
 
+static int finish_count(gear_ctx_impl& c, const int64_t* d_src, int64_t cap, int64_t* h_n, cudaStream_t st);
+
+int gear_accumulate_collect(gear_ctx* ctx, const int32_t* img_id, const float* grads, int64_t ld, const int32_t* src_row,
+                            const float* scale, int64_t n, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
+                            int64_t* d_n, int64_t* h_n, void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (n < 0 || n > c.cfg.max_nnz) return arg_fail("n outside [0, max_nnz]");
+    if (n > 0 && !grads) return arg_fail("NULL pointer");
+    if (n > 0 && !img_id && (!c.img_sorted || c.img_sorted_n != n)) {
+        snprintf(g_last_error, sizeof(g_last_error),
+                 "img_id == NULL needs a preceding gear_forward_backward whose nnz equals n");
+        return GEAR_ERR_STATE;
+    }
+    if (n > 0 && (ld < c.cfg.dfv_dim || ld % 4 || !aligned16(grads)))
+        return arg_fail("grads rows must be 16-byte aligned, ld >= dfv_dim");
+    if (cap < 0 || (cap > 0 && (!ids || !seq || !avg))) return arg_fail("NULL output with cap > 0");
+    if (avg && !aligned16(avg)) return arg_fail("avg must be 16-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.last_stream = st;
+    int64_t* d_cnt = d_n ? d_n : &c.state()->pad[0];
+    cudaError_t e = launch_accumulate_collect(c, img_id, grads, ld, src_row, scale, n, ids, seq, avg, cap, d_cnt, st);
+    if (e != cudaSuccess) return cuda_fail(e, "accumulate_collect");
+    return finish_count(c, d_cnt, cap, h_n, st);
+}
+
 // Waits for everything the ctx has enqueued: the stream of the training calls and, if the expiry scan went to a
 // stream of its own, that one too.
 static cudaError_t sync_streams(const gear_ctx_impl& c) {

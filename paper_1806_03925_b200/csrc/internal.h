@@ -145,6 +145,10 @@ cudaError_t launch_accumulate_plan_ahead(const gear_ctx_impl& c, int64_t n, cons
                                          cudaStream_t st);
 cudaError_t launch_collect_ready(const gear_ctx_impl& c, int32_t* ids, int32_t* seq, float* avg, int64_t cap,
                                  int64_t* d_n, cudaStream_t st);
+// accumulate followed by the hand-over; averages bypass the queue when the host knows it to be empty and cap >= n
+cudaError_t launch_accumulate_collect(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
+                                      const int32_t* src_row, const float* scale, int64_t n, int32_t* ids, int32_t* seq,
+                                      float* avg, int64_t cap, int64_t* d_n, cudaStream_t st);
 
 // expiry.cu
 cudaError_t launch_refresh_dfv(const gear_ctx_impl& c, const int32_t* ids, const float* rows, int64_t ld, int64_t n,

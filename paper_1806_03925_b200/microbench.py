@@ -57,6 +57,7 @@ def _run_case(name, ids_np, V, D, M, mode, steps, warmup=2):
         gb.gear_fill_uniform(grads, seed=5, tag=gb.GEAR_TAG_GRAD, amp=1.0)
         stream = torch.cuda.current_stream()
         t_acc, t_col, n_ready = [], [], []
+        launches0 = gb.gear_launch_count(sess.ctx)
         for s in range(warmup + steps):
             e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
             e0.record(stream)
@@ -67,6 +68,7 @@ def _run_case(name, ids_np, V, D, M, mode, steps, warmup=2):
             torch.cuda.synchronize()
             if s >= warmup:
                 t_acc.append(e0.elapsed_time(e1)); t_col.append(e1.elapsed_time(e2)); n_ready.append(k)
+        launches_per_step = (gb.gear_launch_count(sess.ctx) - launches0) / (warmup + steps)
         # one more call with per-kernel events (serialised, so each kernel is timed alone)
         gb.gear_profile_enable(sess.ctx, True)
         sess.accumulate_rows(ids, grads)
@@ -85,7 +87,8 @@ def _run_case(name, ids_np, V, D, M, mode, steps, warmup=2):
                 "rows_per_s": round(n / ((acc_ms + col_ms) * 1e-3), 1),
                 "algorithmic_GB": round((bytes_acc + bytes_col) / 1e9, 3), "GB/s": round(gbs, 1),
                 "frac_of_hbm_peak": round(gbs / peak, 4), "hbm_peak_GB/s": peak, "peak_source": src,
-                "frac_of_8TBs": round(gbs / 8000.0, 4), "kernel_ms": kernels, "device_status": status, "dtype": "f32", "data": "synthetic"}
+                "frac_of_8TBs": round(gbs / 8000.0, 4), "kernel_ms": kernels, "launches_per_step": launches_per_step,
+                "device_status": status, "dtype": "f32", "data": "synthetic"}
     finally:
         sess.close()
 

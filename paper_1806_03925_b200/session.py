@@ -131,6 +131,20 @@ class GearSession:
         return gb.gear_accumulate_dfv_grad(self.ctx, img_id, grads.data_ptr(), grads.stride(0), None, None,
                                            int(img_id.shape[0]))
 
+    def accumulate_collect_from_step(self, b: DeviceBatch, sync: bool = True, reuse_sorted_ids: bool = True):
+        """Events 5 and 6 of a step as one call: the batch's gradient rows (indirect form, as in
+        accumulate_from_step) are added and the averages of the completed groups handed over."""
+        ptr = self.dX.data_ptr() + 4 * 2 * self.p.emb_dim
+        return gb.gear_accumulate_collect(self.ctx, None if (reuse_sorted_ids and b.nnz > 0) else b.img_id, ptr, self.d_in,
+                                          self.row_view, self.inv_n, b.nnz, self.ready_ids, self.ready_seq,
+                                          self.ready_avg, self.ready_cap, d_n=self.d_counts[0:1], sync=sync)
+
+    def accumulate_collect_rows(self, img_id: torch.Tensor, grads: torch.Tensor, sync: bool = True):
+        assert grads.dtype == torch.float32 and grads.shape[1] == self.p.dfv_dim
+        return gb.gear_accumulate_collect(self.ctx, img_id, grads.data_ptr(), grads.stride(0) if grads.shape[0] else
+                                          self.p.dfv_dim, None, None, int(img_id.shape[0]), self.ready_ids, self.ready_seq,
+                                          self.ready_avg, self.ready_cap, d_n=self.d_counts[0:1], sync=sync)
+
     def collect_ready(self, sync: bool = True):
         return gb.gear_collect_ready(self.ctx, self.ready_ids, self.ready_seq, self.ready_avg, self.ready_cap,
                                      d_n=self.d_counts[0:1], sync=sync)
@@ -152,8 +166,7 @@ class GearSession:
             expiry_beside = self.p.img_vocab >= (1 << 22)
         if not expiry_beside:
             self.forward_backward(b)
-            self.accumulate_from_step(b)
-            n_ready = self.collect_ready(sync=sync)
+            n_ready = self.accumulate_collect_from_step(b, sync=sync)
             n_exp = self.collect_expired(now, restamp=True, sync=sync)
             return n_ready, n_exp
         main = torch.cuda.current_stream()
@@ -166,8 +179,7 @@ class GearSession:
             n_exp = self.collect_expired(now, restamp=True, sync=sync)
             self._ev_join.record(self._expiry_stream)
         self.forward_backward(b)
-        self.accumulate_from_step(b)
-        n_ready = self.collect_ready(sync=sync)
+        n_ready = self.accumulate_collect_from_step(b, sync=sync)
         main.wait_event(self._ev_join)
         return n_ready, n_exp
 

@@ -113,9 +113,10 @@ class Pair:
 
     def __init__(self, p: GearPreset, batches: List[Batch], seed: int = 0, dense: Optional[bool] = None,
                  now0: int = 0, ready_cap: int = 0, want_emb_grad: bool = False, extra_img_ids=None,
-                 atomic: bool = False):
+                 atomic: bool = False, fused: bool = False):
         # atomic: GEAR_ACC_ATOMIC on the device against the oracle's order-free (pooled) store
-        self.p, self.seed, self.atomic = p, seed, atomic
+        # fused: a step's events 5 and 6 go through gear_accumulate_collect instead of the two separate calls
+        self.p, self.seed, self.atomic, self.fused = p, seed, atomic, fused
         if dense is None:
             dense = max(p.user_vocab, p.url_vocab, p.img_vocab) <= 200_000
         cat = lambda k: np.concatenate([getattr(b, k) for b in batches]) if batches else np.zeros(0, np.int32)
@@ -210,10 +211,13 @@ class Pair:
                 assert_close(_rows(gpu.url_emb, self.rh.rows), cpu.url_emb, tol, "url_emb after update")
 
         # event 5 + 6
-        gpu.accumulate_from_step(db)
+        if self.fused:
+            n_fused = gpu.accumulate_collect_from_step(db)
+        else:
+            gpu.accumulate_from_step(db)
         cpu.accumulate(img, cpu.dfv_grad_rows(b.img_off, r.dX), pooled=self.atomic)
         self.compare_store(check_tables)
-        n_ready = self.collect_and_compare()
+        n_ready = self.collect_and_compare(n_fused if self.fused else None)
         n_exp = self.expire_and_compare(now)
         assert self.status() == 0
         out = dict(loss=r.loss, n_ready=n_ready, n_expired=n_exp, status=self.status_bits, rc=self.status_rc,
@@ -288,10 +292,16 @@ class Pair:
             # would spill into its neighbour): the table's non-zero entries are all inside the touched rows
             assert count_nonzero(gpu.dfv_gsum) == count_nonzero(gpu.dfv_gsum[rows]), "sums outside the touched rows"
 
-    def collect_and_compare(self) -> int:
+    def collect_and_compare(self, n_handed_over: Optional[int] = None) -> int:
+        """n_handed_over: the count a gear_accumulate_collect call returned (the hand-over has happened already)."""
         gpu, cpu = self.gpu, self.cpu
-        assert self.status() == cpu.pending_ready, "pending ready count"
-        n = gpu.collect_ready()
+        if n_handed_over is None:
+            assert self.status() == cpu.pending_ready, "pending ready count"
+            n = gpu.collect_ready()
+        else:
+            assert self.status() == 0, "the queue is empty after a fused call"
+            n = n_handed_over
+            assert int(gpu.d_counts[0].item()) == n, "device-side count of the fused call"
         eid, eseq, eavg = oracle.sort_emissions(*cpu.collect_ready())
         assert n == len(eid), "number of emissions"
         gid = _np(gpu.ready_ids[:n])

@@ -42,10 +42,10 @@ def test_procedural_fill_is_bit_identical(gb):
 
 
 # ------------------------------------------------------------------ whole step, every configuration (reduced where needed)
-def _run_steps(p, steps, seed=0, want_emb_grad=False, B=None, dense=None):
+def _run_steps(p, steps, seed=0, want_emb_grad=False, B=None, dense=None, fused=False):
     src = BatchSource(p, seed)
     batches = [src.batch(s, B) for s in range(steps)]
-    pair = _pair(p, batches, seed=seed, want_emb_grad=want_emb_grad, dense=dense)
+    pair = _pair(p, batches, seed=seed, want_emb_grad=want_emb_grad, dense=dense, fused=fused)
     out = []
     try:
         for s, b in enumerate(batches):
@@ -55,9 +55,10 @@ def _run_steps(p, steps, seed=0, want_emb_grad=False, B=None, dense=None):
     return out
 
 
-def test_tiny_config_all_steps(gb):
+@pytest.mark.parametrize("fused", [False, True])
+def test_tiny_config_all_steps(gb, fused):
     p = PRESETS["tiny"]
-    out = _run_steps(p, p.steps)
+    out = _run_steps(p, p.steps, fused=fused)
     assert all(o["status"] == 0 for o in out)
     assert sum(o["n_ready"] for o in out) > 0 and sum(o["n_expired"] for o in out) > 0
 
@@ -70,6 +71,11 @@ def test_medium_config_two_steps(gb):
     # full medium shapes (1M-row tables, bf16 DFVs, 192-256-128-1 head); the oracle keeps the touched rows only
     p = PRESETS["medium"]
     out = _run_steps(p, 2, dense=False)
+    assert out[-1]["n_ready"] > 0
+
+
+def test_medium_config_two_steps_events_5_and_6_in_one_call(gb):
+    out = _run_steps(PRESETS["medium"], 2, dense=False, fused=True)
     assert out[-1]["n_ready"] > 0
 
 
@@ -133,7 +139,7 @@ def _soak_case(case: int):
 @pytest.mark.parametrize("case", range(24))
 def test_random_shapes(gb, case):
     p, B, want_emb_grad = _soak_case(case)
-    _run_steps(p, 2, seed=case, B=B, want_emb_grad=want_emb_grad)
+    _run_steps(p, 2, seed=case, B=B, want_emb_grad=want_emb_grad, fused=bool(case % 2))
 
 
 @pytest.mark.parametrize("M", [1, 64, 1024])
@@ -260,6 +266,44 @@ def test_plan_made_ahead_is_dropped_when_other_calls_come_first(gb):
         assert pair.status_bits == 0
     finally:
         pair.close()
+
+
+def test_fused_call_on_a_non_empty_queue_and_with_a_short_list(gb):
+    """gear_accumulate_collect must give the results of accumulate + collect also where it cannot bypass the queue:
+    when averages of an earlier call are still waiting, and when the caller's lists are shorter than the row count."""
+    from gpu_harness import _np, assert_close
+    p = PRESETS["tiny"].scaled(user_vocab=16, url_vocab=16, img_vocab=300, M=2)
+    rng = np.random.default_rng(11)
+    ids_a = rng.integers(0, 40, 500).astype(np.int32)
+    ids_b = rng.integers(0, 40, 300).astype(np.int32)
+    ga = rng.normal(0, 1, (500, p.dfv_dim)).astype(np.float32)
+    gb_ = rng.normal(0, 1, (300, p.dfv_dim)).astype(np.float32)
+    for cap in (None, 260):          # None: lists as long as the row count; 260 < 300 rows, but enough for the groups
+        pair = _pair(p, [], dense=True, extra_img_ids=np.concatenate([ids_a, ids_b]), ready_cap=cap or 0)
+        try:
+            g, cpu = pair.gpu, pair.cpu
+            if cap is None:
+                g.accumulate_rows(torch.from_numpy(ids_a).cuda(), torch.from_numpy(ga).cuda())     # stays in the queue
+                cpu.accumulate(ids_a, ga.astype(np.float64))
+            n = g.accumulate_collect_rows(torch.from_numpy(ids_b).cuda(), torch.from_numpy(gb_).cuda())
+            cpu.accumulate(ids_b, gb_.astype(np.float64))
+            pair.compare_store()
+            eid, eseq, eavg = oracle.sort_emissions(*cpu.collect_ready())
+            assert n == len(eid) and n > 0
+            assert np.array_equal(_np(g.ready_ids[:n]), eid) and np.array_equal(_np(g.ready_seq[:n]), eseq)
+            assert_close(_np(g.ready_avg[:n]), eavg, 1e-5, "averaged gradients")
+            assert g.status()[1:] == (0, 0) and g.guards_intact()
+            # and straight after, with the queue empty again, the same call bypasses the queue
+            n2 = g.accumulate_collect_rows(torch.from_numpy(ids_a[:200]).cuda(), torch.from_numpy(ga[:200]).cuda())
+            cpu.accumulate(ids_a[:200], ga[:200].astype(np.float64))
+            pair.compare_store()
+            eid, eseq, eavg = oracle.sort_emissions(*cpu.collect_ready())
+            assert n2 == len(eid)
+            assert np.array_equal(_np(g.ready_ids[:n2]), eid) and np.array_equal(_np(g.ready_seq[:n2]), eseq)
+            assert_close(_np(g.ready_avg[:n2]), eavg, 1e-5, "averaged gradients")
+            assert g.status()[1:] == (0, 0) and g.guards_intact()
+        finally:
+            pair.close()
 
 
 def test_zero_sized_calls_are_accepted(gb):
