@@ -82,6 +82,14 @@ def lib():
         L.orc_collect_expired.argtypes = [vp, i64, i64, i64, C.c_int, vp]
         L.orc_refresh_dfv.restype = i64
         L.orc_refresh_dfv.argtypes = [vp, C.c_int, i64, i32, vp, i64, vp, vp, vp, i64, i64, i64]
+        L.orc_dense_forward.restype = i64
+        L.orc_dense_forward.argtypes = [vp, C.c_int, i64, i32, vp, i32, vp, i64, vp]
+        L.orc_dense_backward.restype = i64
+        L.orc_dense_backward.argtypes = [vp, C.c_int, i64, i32, i32, vp, vp, i64, vp]
+        L.orc_adam_step.restype = None
+        L.orc_adam_step.argtypes = [vp, vp, vp, vp, i64, i64, dbl, dbl, dbl, dbl]
+        L.orc_emb_adam.restype = i64
+        L.orc_emb_adam.argtypes = [vp, C.c_int, vp, vp, i64, i32, vp, i32, vp, i32, i32, i64, dbl, dbl, dbl, dbl]
         _lib = L
     return _lib
 
@@ -310,6 +318,55 @@ class GearOracle:
         tid = None if ts_ids is None else _c(np.asarray(ts_ids), np.int32)
         return int(lib().orc_refresh_dfv(_ptr(self.dfv), _dtype_tag(self.dfv), self.V, self.D, _ptr(self.ts), len(self.ts),
                                          _ptr(ids), _ptr(tid), _ptr(rows), rows.shape[1], len(ids), int(now)))
+
+
+# -- a linear Dense Part and the optimiser ------------------------------------------
+def dense_forward(raw: np.ndarray, Wd: np.ndarray, ids) -> np.ndarray:
+    """DFV rows raw[ids] . Wd of a linear Dense Part (raw in its storage type, Wd float64 [R][D])."""
+    raw = np.ascontiguousarray(raw)
+    Wd = _c(Wd, np.float64)
+    ids = _c(np.asarray(ids), np.int32)
+    rows = np.zeros((len(ids), Wd.shape[1]), dtype=np.float64)
+    lib().orc_dense_forward(_ptr(raw), _dtype_tag(raw), raw.shape[0], raw.shape[1], _ptr(Wd), Wd.shape[1], _ptr(ids),
+                            len(ids), _ptr(rows))
+    return rows
+
+
+def dense_backward(raw: np.ndarray, ids, avg: np.ndarray) -> np.ndarray:
+    """dLoss/dWd [R][D] of a linear Dense Part from the emitted (id, averaged gradient) pairs."""
+    raw = np.ascontiguousarray(raw)
+    ids = _c(np.asarray(ids), np.int32)
+    avg = _c(avg, np.float64)
+    G = np.zeros((raw.shape[1], avg.shape[1] if avg.ndim == 2 else 0), dtype=np.float64)
+    lib().orc_dense_backward(_ptr(raw), _dtype_tag(raw), raw.shape[0], raw.shape[1], G.shape[1], _ptr(ids), _ptr(avg),
+                             len(ids), _ptr(G))
+    return G
+
+
+@dataclass
+class AdamConfig:
+    lr: float = 1e-4          # the paper's learning rate
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+
+
+def adam_step(p: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, t: int, cfg: AdamConfig) -> None:
+    """In place on float64 arrays of equal size."""
+    for a in (p, g, m, v):
+        assert a.dtype == np.float64 and a.flags.c_contiguous and a.size == p.size
+    lib().orc_adam_step(_ptr(p), _ptr(g), _ptr(m), _ptr(v), p.size, int(t), cfg.lr, cfg.beta1, cfg.beta2, cfg.eps)
+
+
+def emb_adam(table: np.ndarray, m: np.ndarray, v: np.ndarray, ids, dX: np.ndarray, col0: int, t: int,
+             cfg: AdamConfig) -> int:
+    """Adam on the rows of an embedding table that received a gradient (in place; m, v float64 [vocab][E])."""
+    ids = _c(np.asarray(ids), np.int32)
+    dX = _c(dX, np.float64)
+    assert table.flags.c_contiguous and m.dtype == np.float64 and v.dtype == np.float64
+    return int(lib().orc_emb_adam(_ptr(table), _dtype_tag(table), _ptr(m), _ptr(v), table.shape[0], table.shape[1],
+                                  _ptr(ids), len(ids), _ptr(dX), dX.shape[1], col0, int(t), cfg.lr, cfg.beta1,
+                                  cfg.beta2, cfg.eps))
 
 
 def sort_emissions(ids: np.ndarray, seq: np.ndarray, avg: np.ndarray):

@@ -31,6 +31,13 @@
  *   orc_refresh_dfv       Section 1 (second point) and Section 3: a refreshed
  *                         Dense Feature Vector replaces the expired cached one
  *                         and restarts its clock.
+ *   orc_dense_forward     Section 3, events 2 and 3, for a linear Dense Part
+ *                         (DFV = raw image row times a weight matrix).
+ *   orc_dense_backward    event 6, second half; right factor of Eq. 1: the
+ *                         averaged gradients go back through the Dense Part.
+ *   orc_adam_step         Section 4: the optimiser of the paper's experiments
+ *   orc_emb_adam          (Adam), dense and for the rows of an embedding
+ *                         table that received a gradient.
  *   orc_fill_*            not in the paper: counter-based table
  *                         initialisation (SplitMix64, Steele, Lea and Flood
  *                         2014) so that tables too large to ship can be
@@ -40,7 +47,9 @@
  * reverse-mode autodiff library for the head and the pooling; closed forms;
  * a literal keep-every-gradient-in-a-list store for the accumulate rule;
  * Eq. 1 with a linear dense part at M = 1 and zero expiry; count
- * conservation; expiry special cases.
+ * conservation; expiry special cases; the Dense Part's gradient by finite
+ * differences of the loss; Adam against an optimiser library in double
+ * precision and the closed form of its first step.
  * Parity unpinned: the training-trajectory effects the paper reports
  * (convergence against expiry time and M) -- figures and datasets are not
  * available, nothing here claims them.
@@ -550,3 +559,100 @@ int64_t orc_refresh_dfv(void* dfv, int dt, int64_t vocab, int32_t D, int64_t* ts
     return bad;
 }
 
+
+/* --------------------------------------------------- a linear Dense Part */
+
+/*
+ * Dense Part inference (Section 3, events 2 and 3) for the smallest Dense Part
+ * there is: a linear map of the image's raw feature row,
+ *     DFV[id] = raw[id] . Wd        raw [vocab][R] (storage type given), Wd [R][D].
+ * rows[k][D] receives the DFV of image ids[k]; an ID outside [0, vocab) gives a
+ * zero row and is counted in the return value.
+ */
+int64_t orc_dense_forward(const void* raw, int raw_dt, int64_t vocab, int32_t R, const double* Wd, int32_t D,
+                          const int32_t* ids, int64_t n, double* rows) {
+    int64_t bad = 0;
+    for (int64_t k = 0; k < n; ++k) {
+        double* out = rows + k * D;
+        for (int c = 0; c < D; ++c) out[c] = 0.0;
+        const int64_t id = ids[k];
+        if (id < 0 || id >= vocab) { ++bad; continue; }
+        for (int r = 0; r < R; ++r) {
+            const double x = load_elem(raw, raw_dt, id * (int64_t)R + r);
+            for (int c = 0; c < D; ++c) out[c] += x * Wd[(int64_t)r * D + c];
+        }
+    }
+    return bad;
+}
+
+/*
+ * Event 6, second half, and the right factor of Eq. 1: the averaged gradient
+ * of every completed group is back-propagated through the Dense Part.  For the
+ * linear Dense Part dDFV[id][c] / dWd[r][c] = raw[id][r], so
+ *     G[r][c] += sum over emissions e of raw[id_e][r] * avg_e[c].
+ * G [R][D] is accumulated into (the caller zeroes it).  Returns the number of
+ * out-of-range IDs (skipped).
+ */
+int64_t orc_dense_backward(const void* raw, int raw_dt, int64_t vocab, int32_t R, int32_t D,
+                           const int32_t* ids, const double* avg, int64_t n, double* G) {
+    int64_t bad = 0;
+    for (int64_t e = 0; e < n; ++e) {
+        const int64_t id = ids[e];
+        if (id < 0 || id >= vocab) { ++bad; continue; }
+        for (int r = 0; r < R; ++r) {
+            const double x = load_elem(raw, raw_dt, id * (int64_t)R + r);
+            for (int c = 0; c < D; ++c) G[(int64_t)r * D + c] += x * avg[e * D + c];
+        }
+    }
+    return bad;
+}
+
+/* ------------------------------------------------------------ optimiser */
+
+/*
+ * One step of Adam (Kingma and Ba 2015, Algorithm 1), the optimiser of the
+ * paper's Section 4 (learning rate 1e-4 there), on n parameters:
+ *     m = b1 m + (1 - b1) g;   v = b2 v + (1 - b2) g^2;
+ *     p -= lr * (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps),      t = 1, 2, ...
+ */
+void orc_adam_step(double* p, const double* g, double* m, double* v, int64_t n, int64_t t,
+                   double lr, double b1, double b2, double eps) {
+    const double c1 = 1.0 - pow(b1, (double)t), c2 = 1.0 - pow(b2, (double)t);
+    for (int64_t i = 0; i < n; ++i) {
+        m[i] = b1 * m[i] + (1.0 - b1) * g[i];
+        v[i] = b2 * v[i] + (1.0 - b2) * g[i] * g[i];
+        p[i] -= lr * (m[i] / c1) / (sqrt(v[i] / c2) + eps);
+    }
+}
+
+/*
+ * The same optimiser for an embedding table whose gradient is sparse (event 4,
+ * "push gradients of Sparse Part"): G[id] = sum over the views b (ascending)
+ * with ids[b] == id of dX[b][col0 .. col0+E); every row that received a
+ * gradient takes one Adam step with its own moment rows m[id], v[id] and the
+ * global step count t; rows without a gradient, and their moments, stay as they
+ * are.  table in its storage type; m, v doubles [vocab][E].  Returns the
+ * number of out-of-range IDs (skipped).
+ */
+int64_t orc_emb_adam(void* table, int dt, double* m, double* v, int64_t vocab, int32_t E,
+                     const int32_t* ids, int32_t B, const double* dX, int32_t ldx, int32_t col0,
+                     int64_t t, double lr, double b1, double b2, double eps) {
+    int64_t bad = 0;
+    double* G = (double*)calloc((size_t)vocab * E, sizeof(double));
+    uint8_t* seen = (uint8_t*)calloc((size_t)vocab, 1);
+    for (int32_t b = 0; b < B; ++b) {
+        int32_t id = ids[b];
+        if (id < 0 || id >= vocab) { ++bad; continue; }
+        seen[id] = 1;
+        for (int c = 0; c < E; ++c) G[(int64_t)id * E + c] += dX[(int64_t)b * ldx + col0 + c];
+    }
+    double* row = (double*)malloc(sizeof(double) * E);
+    for (int64_t id = 0; id < vocab; ++id) {
+        if (!seen[id]) continue;
+        for (int c = 0; c < E; ++c) row[c] = load_elem(table, dt, id * E + c);
+        orc_adam_step(row, G + id * E, m + id * E, v + id * E, E, t, lr, b1, b2, eps);
+        for (int c = 0; c < E; ++c) store_elem(table, dt, id * E + c, row[c]);
+    }
+    free(row); free(G); free(seen);
+    return bad;
+}

@@ -106,6 +106,9 @@ static void release_host_objects(gear_ctx_impl& c) {
     if (c.ev_fork) cudaEventDestroy(c.ev_fork);
     if (c.ev_join) cudaEventDestroy(c.ev_join);
     if (c.ev_gather) cudaEventDestroy(c.ev_gather);
+    if (c.ev_weights) cudaEventDestroy(c.ev_weights);
+    if (c.ev_dx) cudaEventDestroy(c.ev_dx);
+    c.ev_weights = c.ev_dx = nullptr;
     if (c.side_stream) cudaStreamDestroy(c.side_stream);
     c.ev_fork = c.ev_join = c.ev_gather = nullptr;
     c.side_stream = nullptr;
@@ -173,13 +176,15 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
     c.side_stream = nullptr;
-    c.ev_fork = c.ev_join = c.ev_gather = nullptr;
+    c.ev_fork = c.ev_join = c.ev_gather = c.ev_weights = c.ev_dx = nullptr;
     c.plan_ready = false; c.plan_n = 0; c.plan_src_row = nullptr; c.plan_scale = nullptr;
 
     cudaError_t e = cudaStreamCreateWithFlags(&c.side_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_gather, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_join, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_weights, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_dx, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemsetAsync(c.state(), 0, sizeof(DevState), st);
     if (e == cudaSuccess && fill) {
         const double amp = 0.17320508075688773;   // uniform half-width for standard deviation 0.1
@@ -219,12 +224,43 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
 
-    // The three ID arrays of the batch are key-sorted in one launch: the user and URL orders drive the embedding
-    // scatter below, the image order is kept for gear_accumulate_dfv_grad (img_id == NULL).
+    // What depends on the batch's ID arrays and on head_params alone runs on the ctx's side stream, beside the gather
+    // and the head: the bf16 copies of the weights, the key sort of the three ID arrays (the user and URL orders drive
+    // the embedding scatter, the image order is kept for gear_accumulate_dfv_grad with img_id == NULL) and, once the
+    // gather has written row_view / inv_n, the plan of that accumulate call.  The embedding scatter itself joins them
+    // there as soon as dX exists, beside the last weight-gradient product; the caller's stream waits for the side
+    // stream before the call returns.  With per-kernel timing on, everything stays on the caller's stream so that each
+    // kernel is timed alone.
     c.img_sorted = false;
     c.img_sort_valid = false;
+    c.plan_ready = false;
+    const bool forked = !c.prof.on && b.B > 0;
+    bool join_pending = false;          // the side stream holds work the caller's stream has not waited for
+    cudaStream_t side = forked ? c.side_stream : st;
+    // A failure between the fork and the join must not leave the side stream unjoined or the sorted order marked as
+    // usable: the caller's stream waits for whatever the side stream was given, and the ctx forgets the batch.
+    auto abandon = [&](cudaError_t err, const char* where) {
+        if (join_pending) {
+            if (cudaEventRecord(c.ev_join, c.side_stream) != cudaSuccess || cudaStreamWaitEvent(st, c.ev_join, 0) != cudaSuccess)
+                cudaStreamSynchronize(c.side_stream);
+        }
+        c.img_sorted = false; c.img_sort_valid = false; c.plan_ready = false;
+        return cuda_fail(err, where);
+    };
+    cudaError_t e = cudaSuccess;
+    if (forked) {
+        e = cudaEventRecord(c.ev_fork, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c.side_stream, c.ev_fork, 0);
+        if (e != cudaSuccess) return cuda_fail(e, "fork");
+        join_pending = true;
+    }
+    const bool weights_on_side = forked && c.cfg.head_dtype == GEAR_BF16;
+    if (weights_on_side) {
+        e = launch_round_weights(c, c.side_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(c.ev_weights, c.side_stream);
+        if (e != cudaSuccess) return abandon(e, "weight copies");
+    }
     int sorted_buf = 0;
-    bool joined_needed = false;
     if (b.B > 0) {
         SortBatch batch = c.sort_batch();
         batch.job[0] = c.sort_job(gear_ctx_impl::SORT_USER);
@@ -240,62 +276,57 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
             batch.job[2].n_max = b.nnz; batch.job[2].bits = bits_for(c.cfg.img_vocab);
             batch.n_jobs = 3;
         }
-        // The sort depends only on the ID arrays, so it runs on the ctx's side stream beside the gather and
-        // the head (fork here, join before the first consumer of a sorted order).  With per-kernel timing on,
-        // everything stays on the caller's stream so that each kernel is timed alone.
-        const bool forked = !c.prof.on;
         cudaError_t se = cudaSuccess;
-        if (forked) {
-            se = cudaEventRecord(c.ev_fork, st);
-            if (se == cudaSuccess) se = cudaStreamWaitEvent(c.side_stream, c.ev_fork, 0);
-            if (se != cudaSuccess) return cuda_fail(se, "fork");
-        }
         batch.name = "sort_ids";
-        sorted_buf = sort_jobs(batch, &c.gbs, forked ? c.side_stream : st, &c.prof, &se);
-        if (se != cudaSuccess) return cuda_fail(se, "id sort");
-        joined_needed = forked;
+        sorted_buf = sort_jobs(batch, &c.gbs, side, &c.prof, &se);
+        if (se != cudaSuccess) return abandon(se, "id sort");
         if (b.nnz > 0) {
             c.img_sorted = true; c.img_sorted_n = b.nnz; c.img_sorted_buf = sorted_buf; c.last_img_id = b.img_id;
             c.img_sort_valid = c.cfg.accum_mode == GEAR_ACC_SORT;
         }
     }
-    c.plan_ready = false;
-    // A failure between the fork and the join must not leave the side stream unjoined or the sorted order marked as
-    // usable: the caller's stream waits for whatever the side stream was given, and the ctx forgets the batch.
-    auto abandon = [&](cudaError_t err, const char* where) {
-        if (joined_needed) {
-            if (cudaEventRecord(c.ev_join, c.side_stream) != cudaSuccess || cudaStreamWaitEvent(st, c.ev_join, 0) != cudaSuccess)
-                cudaStreamSynchronize(c.side_stream);
-        }
-        c.img_sorted = false; c.img_sort_valid = false; c.plan_ready = false;
-        return cuda_fail(err, where);
-    };
-    cudaError_t e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
+    e = launch_gather(c, b, o.row_view, o.inv_n, o.x_debug, st);
     if (e != cudaSuccess) return abandon(e, "gather");
-    if (joined_needed) {
-        // Still on the side stream, behind the sort: the plan of the accumulate call that usually follows (which rows
-        // form which group, where every group's rows and queue slot are).  It needs the gather's row_view / inv_n.
-        if (b.nnz > 0 && o.row_view && o.inv_n && c.cfg.accum_mode == GEAR_ACC_SORT) {
-            e = cudaEventRecord(c.ev_gather, st);
-            if (e == cudaSuccess) e = cudaStreamWaitEvent(c.side_stream, c.ev_gather, 0);
-            if (e == cudaSuccess) e = launch_accumulate_plan_ahead(c, b.nnz, o.row_view, o.inv_n, c.side_stream);
-            if (e != cudaSuccess) return abandon(e, "accumulate plan");
+    if (forked && b.nnz > 0 && o.row_view && o.inv_n && c.cfg.accum_mode == GEAR_ACC_SORT) {
+        // behind the sort: the plan of the accumulate call that usually follows (which rows form which group, where every
+        // group's rows and queue slot are).  It needs the gather's row_view / inv_n.
+        e = cudaEventRecord(c.ev_gather, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c.side_stream, c.ev_gather, 0);
+        if (e == cudaSuccess) e = launch_accumulate_plan_ahead(c, b.nnz, o.row_view, o.inv_n, c.side_stream);
+        if (e != cudaSuccess) return abandon(e, "accumulate plan");
+    }
+    if (weights_on_side) {
+        e = cudaStreamWaitEvent(st, c.ev_weights, 0);
+        if (e != cudaSuccess) return abandon(e, "weight copies");
+    }
+    // the embedding scatter: enqueued by the head as soon as dX is on its way
+    struct Scatter {
+        gear_ctx_impl* c; const gear_step_out* o; int sorted_buf; int32_t B; float lr; cudaStream_t st; bool forked;
+    } sc{&c, &o, sorted_buf, b.B, lr, st, forked};
+    auto scatter = [](void* arg) -> cudaError_t {
+        Scatter& k = *static_cast<Scatter*>(arg);
+        gear_ctx_impl& c = *k.c;
+        float* ut = k.o->user_grad ? k.o->user_grad : c.buf.user_emb;
+        float* ht = k.o->url_grad ? k.o->url_grad : c.buf.url_emb;
+        const float alpha = k.o->user_grad ? 1.0f : -k.lr;
+        cudaStream_t where = k.st;
+        if (k.forked) {
+            cudaError_t e = cudaEventRecord(c.ev_dx, k.st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(c.side_stream, c.ev_dx, 0);
+            if (e != cudaSuccess) return e;
+            where = c.side_stream;
         }
-        e = cudaEventRecord(c.ev_join, c.side_stream);
-        if (e != cudaSuccess) return abandon(e, "join");
-    }
-    e = launch_head_simt(c, b, o, st);
+        return launch_emb_reduce(c, k.sorted_buf, k.B, ut, ht, k.o->dX, c.d_in, alpha, where);
+    };
+    const HeadHooks hooks{weights_on_side, scatter, &sc};
+    e = launch_head_simt(c, b, o, st, hooks);
     if (e != cudaSuccess) return abandon(e, "head");
-    if (joined_needed) {
-        e = cudaStreamWaitEvent(st, c.ev_join, 0);
+    if (forked) {
+        e = cudaEventRecord(c.ev_join, c.side_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c.ev_join, 0);
         if (e != cudaSuccess) return abandon(e, "join");
-        joined_needed = false;
+        join_pending = false;
     }
-    float* ut = o.user_grad ? o.user_grad : c.buf.user_emb;
-    float* ht = o.url_grad ? o.url_grad : c.buf.url_emb;
-    const float alpha = o.user_grad ? 1.0f : -lr;
-    e = launch_emb_reduce(c, sorted_buf, b.B, ut, ht, o.dX, c.d_in, alpha, st);
-    if (e != cudaSuccess) return abandon(e, "embedding scatter");
     return GEAR_OK;
 }
 

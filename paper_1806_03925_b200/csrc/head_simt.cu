@@ -565,8 +565,31 @@ static int splits_for(int M, int N, int K) {
     return (int)(s < 1 ? 1 : s);
 }
 
+// bf16 copies of the hidden layers' weights in both orientations (what the tensor-core products read).  Depends on
+// head_params only, so a step may run it on another stream beside the gather.
+cudaError_t launch_round_weights(const gear_ctx_impl& c, cudaStream_t st) {
+    if (c.cfg.head_dtype != GEAR_BF16) return cudaSuccess;
+    const int L = c.cfg.n_hidden;
+    RoundArgs ra;
+    int max_in = 0, max_out = 0, fan = c.d_in;
+    int64_t pos = 0;
+    for (int l = 0; l < L; ++l) {
+        const int h = c.cfg.hidden[l];
+        ra.fan_in[l] = fan; ra.fan_out[l] = h; ra.W[l] = c.buf.head_params + pos;
+        ra.wb[l] = c.at<__nv_bfloat16>(c.ws.wb[l]); ra.wbt[l] = c.at<__nv_bfloat16>(c.ws.wbt[l]);
+        if (fan > max_in) max_in = fan;
+        if (h > max_out) max_out = h;
+        pos += (int64_t)fan * h + h;
+        fan = h;
+    }
+    KernelScope ks(&c.prof, "round_weights", st);
+    return launch_dependent(round_weights_kernel, dim3((unsigned)ceil_div(max_out, 32), (unsigned)ceil_div(max_in, 32), (unsigned)L),
+                            dim3(256), 0, st, ra);
+}
+
 template <typename TX>
-static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const gear_step_out& o, cudaStream_t st) {
+static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const gear_step_out& o, cudaStream_t st,
+                            const HeadHooks& hooks) {
     constexpr bool BF = !std::is_same<TX, float>::value;
     const int L = c.cfg.n_hidden, B = bt.B;
     HeadParams p = split_params(c, o.head_grad);
@@ -585,18 +608,11 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
     // weights as the products see them
     const void* Wop[MAX_LAYERS];
     if (BF) {
-        RoundArgs ra;
-        int max_in = 0, max_out = 0;
-        for (int l = 0; l < L; ++l) {
-            ra.fan_in[l] = p.fan[l]; ra.fan_out[l] = p.fan[l + 1]; ra.W[l] = p.W[l];
-            ra.wb[l] = c.at<__nv_bfloat16>(c.ws.wb[l]); ra.wbt[l] = c.at<__nv_bfloat16>(c.ws.wbt[l]);
-            Wop[l] = ra.wb[l];
-            if (p.fan[l] > max_in) max_in = p.fan[l];
-            if (p.fan[l + 1] > max_out) max_out = p.fan[l + 1];
+        for (int l = 0; l < L; ++l) Wop[l] = c.at<__nv_bfloat16>(c.ws.wb[l]);
+        if (!hooks.weights_ready) {
+            cudaError_t re = launch_round_weights(c, st);
+            if (re != cudaSuccess) return re;
         }
-        KernelScope ks(&c.prof, "round_weights", st);
-        launch_dependent(round_weights_kernel, dim3((unsigned)ceil_div(max_out, 32), (unsigned)ceil_div(max_in, 32), (unsigned)L),
-                         dim3(256), 0, st, ra);
     } else {
         for (int l = 0; l < L; ++l) Wop[l] = p.W[l];
     }
@@ -632,16 +648,11 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
         else GEAR_HEAD_OUT(4, 1);
 #undef GEAR_HEAD_OUT
     }
-    // backward
+    // backward.  Per layer the gradient that the layers below wait for (dA_l, at the bottom dX) comes first, its weight
+    // gradient after it: once dX exists the caller's hook may start the embedding scatter on another stream, beside the
+    // last weight-gradient product.
     for (int l = L - 1; l >= 0; --l) {
         const int K = p.fan[l], N = p.fan[l + 1];
-        // dW_l = H_l^T dA_{l+1}
-        if constexpr (BF) {
-            tce = tc_gemm_mnmajor(&c.prof, "tc_gemm_dw", K, N, B, H[l], K, dA[l + 1], N, p.gW[l], N, tc_err, st);
-            if (tce != cudaSuccess) return tce;
-        } else
-        launch_gemm<TX, TX, float, TX, EPI_ATOMIC>(K, N, B, H[l], 1, K, dA[l + 1], N, 1, p.gW[l], N, nullptr,
-                                                   (const TX*)nullptr, 0, splits_for(K, N, B), st, &c.prof, "simt_gemm_dw");
         // bias gradient of a lower layer (the top layer's came out of head_out_kernel); the tensor-core path
         // sums the columns of dA inside the epilogue of the product that makes dA
         if (!BF && l < L - 1) {
@@ -663,13 +674,25 @@ static cudaError_t run_head(const gear_ctx_impl& c, const gear_batch& bt, const 
             launch_gemm<TX, TX, float, TX, EPI_NONE>(B, K, N, dA[l + 1], N, 1, static_cast<const TX*>(Wop[l]), 1, N,
                                                      o.dX, K, nullptr, (const TX*)nullptr, 0, 1, st, &c.prof, "simt_gemm_dx");
         }
+        if (l == 0 && hooks.after_dx) {
+            cudaError_t he = hooks.after_dx(hooks.arg);
+            if (he != cudaSuccess) return he;
+        }
+        // dW_l = H_l^T dA_{l+1}
+        if constexpr (BF) {
+            tce = tc_gemm_mnmajor(&c.prof, "tc_gemm_dw", K, N, B, H[l], K, dA[l + 1], N, p.gW[l], N, tc_err, st);
+            if (tce != cudaSuccess) return tce;
+        } else
+        launch_gemm<TX, TX, float, TX, EPI_ATOMIC>(K, N, B, H[l], 1, K, dA[l + 1], N, 1, p.gW[l], N, nullptr,
+                                                   (const TX*)nullptr, 0, splits_for(K, N, B), st, &c.prof, "simt_gemm_dw");
     }
     return cudaGetLastError();
 }
 
-cudaError_t launch_head_simt(const gear_ctx_impl& c, const gear_batch& b, const gear_step_out& o, cudaStream_t st) {
-    if (c.cfg.head_dtype == GEAR_BF16) return run_head<__nv_bfloat16>(c, b, o, st);
-    return run_head<float>(c, b, o, st);
+cudaError_t launch_head_simt(const gear_ctx_impl& c, const gear_batch& b, const gear_step_out& o, cudaStream_t st,
+                             const HeadHooks& hooks) {
+    if (c.cfg.head_dtype == GEAR_BF16) return run_head<__nv_bfloat16>(c, b, o, st, hooks);
+    return run_head<float>(c, b, o, st, hooks);
 }
 
 }  // namespace gear

@@ -82,6 +82,8 @@ struct gear_ctx_impl {
     mutable const int32_t* plan_src_row;
     mutable const float* plan_scale;
     cudaEvent_t ev_gather;              // the gather's outputs (row_view, inv_n) exist
+    cudaEvent_t ev_weights;             // the bf16 copies of the head's weights exist (made on the side stream)
+    cudaEvent_t ev_dx;                  // dX exists: the embedding scatter may start on the side stream
     mutable int acc_calls_pending;      // accumulate calls enqueued since a collect that was sure to drain the queue
 
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(static_cast<char*>(buf.workspace) + off); }
@@ -114,8 +116,13 @@ cudaError_t launch_fill_ts(int64_t* ts, int64_t n, uint64_t seed, int64_t expire
 cudaError_t launch_gather(const gear_ctx_impl& c, const gear_batch& b, int32_t* row_view, float* inv_n,
                           void* x_debug, cudaStream_t st);
 
-// head_simt.cu: forward + backward of the head with fp32 FMA products (operands fp32 or bf16)
-cudaError_t launch_head_simt(const gear_ctx_impl& c, const gear_batch& b, const gear_step_out& o, cudaStream_t st);
+// head_simt.cu: forward + backward of the head (fp32 FMA products, or the tensor-core products of head_tc.cu).
+// weights_ready: the bf16 copies of the weights have been made already (launch_round_weights on another stream, joined by
+// the caller).  after_dx(arg) is called once dX has been enqueued, before the last weight-gradient product.
+struct HeadHooks { bool weights_ready; cudaError_t (*after_dx)(void*); void* arg; };
+cudaError_t launch_head_simt(const gear_ctx_impl& c, const gear_batch& b, const gear_step_out& o, cudaStream_t st,
+                             const HeadHooks& hooks);
+cudaError_t launch_round_weights(const gear_ctx_impl& c, cudaStream_t st);
 
 // head_tc.cu: bf16 products on tcgen05 tensor cores.  epi: 0 bias+ReLU -> bf16, 1 ReLU mask -> bf16, 2 plain fp32.
 // colsum (epi 1 only, may be null): colsum[n] += sum over the rows of the stored (rounded) output.

@@ -522,7 +522,7 @@ def test_eq1_M1_zero_expiry_equals_direct_backprop():
     r = orc.forward_backward(params, **batch)
     orc.accumulate(batch["img_id"], orc.dfv_grad_rows(batch["img_off"], r.dX))
     eid, _, eavg = orc.collect_ready()
-    got = sum(np.outer(raw[i], a) for i, a in zip(eid, eavg))  # dLoss/dDFV . dDFV/dW_dense
+    got = oracle.dense_backward(raw, eid, eavg)              # dLoss/dDFV . dDFV/dW_dense, event 6's second half
     np.testing.assert_allclose(got, want, atol=1e-8)
 
 
@@ -532,8 +532,8 @@ def test_eq1_total_gradient_is_conserved_for_M3():
     r = orc.forward_backward(params, **batch)
     orc.accumulate(batch["img_id"], orc.dfv_grad_rows(batch["img_off"], r.dX))
     eid, _, eavg = orc.collect_ready()
-    got = sum((np.outer(raw[i], 3 * a) for i, a in zip(eid, eavg)), np.zeros_like(Wd))
-    got = got + sum(np.outer(raw[i], orc.gsum[i]) for i in range(orc.V))
+    got = oracle.dense_backward(raw, eid, 3 * eavg)
+    got = got + oracle.dense_backward(raw, np.arange(orc.V), orc.gsum)      # what is still waiting in the store
     np.testing.assert_allclose(got, want, atol=1e-8)
 
 
@@ -618,12 +618,12 @@ def test_gear_loop_with_refresh_every_step_is_ordinary_training_of_the_dense_par
     for step in range(2):
         expired = orc.collect_expired(now=step, restamp=True)
         assert len(expired) == orc.V
-        orc.refresh_dfv(expired, (raw[expired] @ Wd_loop).astype(np.float32), now=step)
+        orc.refresh_dfv(expired, oracle.dense_forward(raw, Wd_loop, expired).astype(np.float32), now=step)
         orc.dfv[:] = raw @ Wd_loop                                 # keep the fp64 table exact (refresh rows are fp32)
         r = orc.forward_backward(params, **batch)
         orc.accumulate(batch["img_id"], orc.dfv_grad_rows(batch["img_off"], r.dX))
         eid, _, eavg = orc.collect_ready()
-        Wd_loop = Wd_loop - lr * sum(np.outer(raw[i], a) for i, a in zip(eid, eavg))
+        Wd_loop = Wd_loop - lr * oracle.dense_backward(raw, eid, eavg)
         Wd_ref = Wd_ref - lr * _dense_grad_by_finite_differences(orc, params, batch, raw, Wd_ref)
         orc.dfv[:] = raw @ Wd_loop
     np.testing.assert_allclose(Wd_loop, Wd_ref, atol=1e-7)
@@ -661,3 +661,82 @@ def test_near_zero_units_are_listed_and_can_take_the_other_branch():
     assert wide.near_abs.tolist() == [0.0, 2.25]
     assert len(orc.forward_backward(params, *args, relu_margin=0.0, relu_margin_rel=1.1).near_units) == 1
     assert np.array_equal(wide.dX, r.dX) and np.array_equal(wide.head_grad, r.head_grad)   # listing changes no result
+
+
+# ----------------------------------------------------------------------------
+# the linear Dense Part and the optimiser
+# ----------------------------------------------------------------------------
+def test_dense_forward_special_cases():
+    raw = np.array([[1.0, 0.0, 0.0], [0.0, 0.0, 1.0], [2.0, -1.0, 0.5]])
+    Wd = np.array([[1.0, 2.0], [3.0, 4.0], [5.0, 6.0]])
+    rows = oracle.dense_forward(raw, Wd, [0, 1, 2, 1, 7])
+    assert rows[0].tolist() == [1.0, 2.0] and rows[1].tolist() == [5.0, 6.0]      # unit rows pick rows of Wd
+    assert rows[2].tolist() == [2 - 3 + 2.5, 4 - 4 + 3.0]                          # by hand
+    assert np.array_equal(rows[3], rows[1]) and not rows[4].any()                  # repeats; out-of-range id: zeros
+    assert np.array_equal(oracle.dense_forward(raw, np.eye(3), [2, 0]), raw[[2, 0]])   # identity Wd: the raw rows
+    # float32 storage is read exactly
+    assert np.array_equal(oracle.dense_forward(raw.astype(np.float32), Wd, [2]), rows[2:3])
+
+
+def test_dense_backward_is_the_gradient_of_the_dense_forward():
+    # L(Wd) = sum_e <avg_e, raw[id_e] . Wd> is linear in Wd, so its gradient is exact by finite differences
+    rng = np.random.default_rng(21)
+    raw, Wd = rng.normal(size=(6, 4)), rng.normal(size=(4, 3))
+    ids, avg = np.array([5, 0, 5, 2], np.int32), rng.normal(size=(4, 3))
+    G = oracle.dense_backward(raw, ids, avg)
+    f = lambda: float((oracle.dense_forward(raw, Wd, ids) * avg).sum())
+    want = np.array([central_diff(f, Wd, i, h=1e-3) for i in range(Wd.size)]).reshape(Wd.shape)
+    np.testing.assert_allclose(G, want, atol=1e-9)
+    # a repeated image counts once per emission; an out-of-range id is skipped
+    one = oracle.dense_backward(raw, np.array([5], np.int32), avg[:1] + avg[2:3])
+    two = oracle.dense_backward(raw, np.array([5, 5, 9], np.int32), np.vstack([avg[:1], avg[2:3], avg[:1]]))
+    np.testing.assert_allclose(one, two, atol=1e-15)
+
+
+def test_adam_matches_the_optimiser_library_and_the_closed_form_of_its_first_step():
+    from oracle import AdamConfig
+    rng = np.random.default_rng(22)
+    cfg = AdamConfig(lr=1e-2, beta1=0.8, beta2=0.95, eps=1e-6)
+    p0 = rng.normal(size=17)
+    p, m, v = p0.copy(), np.zeros(17), np.zeros(17)
+    tp = torch.tensor(p0.copy(), requires_grad=True)
+    opt = torch.optim.Adam([tp], lr=cfg.lr, betas=(cfg.beta1, cfg.beta2), eps=cfg.eps)
+    for t in range(1, 6):
+        g = rng.normal(size=17) * (10.0 ** rng.integers(-3, 2))
+        oracle.adam_step(p, g, m, v, t, cfg)
+        tp.grad = torch.tensor(g.copy())
+        opt.step()
+        np.testing.assert_allclose(p, tp.detach().numpy(), rtol=0, atol=1e-13)
+    # first step from zero moments: m_hat = g, v_hat = g^2, so the step is -lr * g / (|g| + eps), about -lr * sign(g)
+    g = np.array([3.0, -0.2, 1e-3, -50.0])
+    p, m, v = np.zeros(4), np.zeros(4), np.zeros(4)
+    oracle.adam_step(p, g, m, v, 1, cfg)
+    np.testing.assert_allclose(p, -cfg.lr * g / (np.abs(g) + cfg.eps), rtol=1e-12)
+    np.testing.assert_allclose(m, (1 - cfg.beta1) * g, rtol=1e-15)
+    np.testing.assert_allclose(v, (1 - cfg.beta2) * g * g, rtol=1e-15)
+    # a zero gradient with zero moments moves nothing
+    p, m, v = np.ones(3), np.zeros(3), np.zeros(3)
+    oracle.adam_step(p, np.zeros(3), m, v, 4, cfg)
+    assert p.tolist() == [1.0, 1.0, 1.0]
+
+
+def test_embedding_adam_steps_each_touched_row_once_with_the_summed_gradient():
+    from oracle import AdamConfig
+    rng = np.random.default_rng(23)
+    cfg = AdamConfig(lr=1e-2)
+    V, E = 6, 3
+    table = rng.normal(size=(V, E))
+    m, v = rng.normal(0, 0.1, (V, E)), rng.random((V, E)) * 0.01
+    ids = np.array([4, 1, 4, 9, 4], np.int32)                 # id 4 three times, id 9 out of range
+    dX = rng.normal(size=(5, 8))
+    t0, m0, v0 = table.copy(), m.copy(), v.copy()
+    assert oracle.emb_adam(table, m, v, ids, dX, col0=2, t=3, cfg=cfg) == 1
+    for i in (0, 2, 3, 5):                                    # untouched rows and their moments stay
+        assert np.array_equal(table[i], t0[i]) and np.array_equal(m[i], m0[i]) and np.array_equal(v[i], v0[i])
+    for i, views in ((4, [0, 2, 4]), (1, [1])):               # one step with the sum, not one step per view
+        g = dX[views, 2:5].sum(0)
+        pr, mr, vr = t0[i].copy(), m0[i].copy(), v0[i].copy()
+        oracle.adam_step(pr, g, mr, vr, 3, cfg)
+        np.testing.assert_allclose(table[i], pr, atol=1e-15)
+        np.testing.assert_allclose(m[i], mr, atol=1e-15)
+        np.testing.assert_allclose(v[i], vr, atol=1e-15)
