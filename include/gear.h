@@ -20,6 +20,9 @@
  *   gear_accumulate_collect   events 5 and 6 as one call.
  *   gear_refresh_dfv          Section 1 / Section 3: recomputed DFVs replace
  *                             expired ones and restart their clocks.
+ *   gear_dense_forward /      events 2-3 and the second half of event 6 for a
+ *   gear_dense_backward       linear Dense Part; gear_adam_dense and the adam
+ *                             fields of gear_step_out: Section 4's optimiser.
  *   gear_collect_expired      Section 1 / Section 3: cached inference results
  *                             older than the inference-expired time.
  *
@@ -105,8 +108,8 @@ typedef struct {
     int32_t hidden[2];     /* widths; multiples of 8 (GEAR_F32) or 64 (GEAR_BF16), <= 1024 */
     int32_t M;             /* gradients per image per emitted average, >= 1 */
     int64_t expire;        /* inference-expired time, >= 0, in the caller's time unit */
-    int32_t max_batch;     /* largest B of any gear_forward_backward call */
-    int64_t max_nnz;       /* largest number of rows of any forward_backward / accumulate call */
+    int32_t max_batch;     /* largest B of any gear_forward_backward call, < 2^30 */
+    int64_t max_nnz;       /* largest number of rows of any forward_backward / accumulate call, < 2^30 */
     int64_t ready_cap;     /* rows of the ready queue (averages waiting for gear_collect_ready);
                               0 = max_nnz, which can never overflow if every accumulate call is
                               followed by a collect */
@@ -126,6 +129,11 @@ typedef struct {
     void*     workspace;    /* scratch, 256-byte aligned, >= gear_workspace_bytes; contents belong to the ctx */
     size_t    workspace_bytes;
 } gear_buffers;
+
+/* Adam (Kingma and Ba 2015, Algorithm 1), the optimiser of the paper's experiments (Section 4: learning rate 1e-4):
+ *   m = beta1 m + (1 - beta1) g;  v = beta2 v + (1 - beta2) g^2;
+ *   p -= lr * (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps),   t = 1, 2, ... */
+typedef struct { float lr, beta1, beta2, eps; } gear_adam;
 
 /* One batch of page views (Table 1 of the paper) in CSR form; device pointers. */
 typedef struct {
@@ -151,6 +159,14 @@ typedef struct {
     void*  x_debug;     /* [B][2*emb_dim + dfv_dim] copy of the head input in head_dtype; optional */
     float* user_grad;   /* [user_vocab][emb_dim] optional: the summed embedding gradient is ADDED here and the */
     float* url_grad;    /* [url_vocab][emb_dim]  table is left untouched (both or neither) */
+    /* Optional: Section 4's optimiser for the embedding tables in place of the plain scaled scatter (adam != NULL; not
+     * together with user_grad / url_grad).  Every row that received a gradient in this step takes one Adam step with
+     * the step count adam_step (>= 1) and its own rows of the moment tables; rows without a gradient, and their
+     * moments, stay as they are.  lr of gear_forward_backward is ignored.  The struct is host memory. */
+    const gear_adam* adam;
+    int64_t adam_step;
+    float *user_m, *user_v;   /* [user_vocab][emb_dim] first and second moments, zero before the first step */
+    float *url_m, *url_v;     /* [url_vocab][emb_dim] */
 } gear_step_out;
 
 /* Bytes of workspace a ctx with this configuration needs.  Host-only. */
@@ -243,6 +259,33 @@ int gear_collect_expired(gear_ctx* ctx, int64_t now, int restamp, int32_t* ids, 
  */
 int gear_refresh_dfv(gear_ctx* ctx, const int32_t* ids, const float* rows, int64_t ld, int64_t n,
                      const int64_t* d_n, int64_t now, void* stream);
+
+/*
+ * The smallest Dense Part there is, for closing the loop on one device: DFV[id] = raw[id] . Wd, with raw
+ * [img_vocab][raw_dim] the images' raw feature rows and Wd [raw_dim][dfv_dim] the Dense Part's weights (fp32, device,
+ * row-major).
+ *
+ * gear_dense_forward   Section 3, events 2 and 3 (Dense Part inference): rows[k][c] = sum_r raw[ids[k]][r] Wd[r][c] for
+ *                      k < n (and k < *d_n when d_n, a device count such as the one an expiry scan wrote, is given);
+ *                      rows fp32 with leading dimension ld >= dfv_dim: the input gear_refresh_dfv takes.
+ * gear_dense_backward  Section 3, event 6, second half; Eq. 1, right factor: Wd_grad[r][c] += sum over the emissions
+ *                      e < n (e < *d_n) of raw[ids[e]][r] * avg[e][c]; ids / avg are the lists gear_collect_ready or
+ *                      gear_accumulate_collect returned (avg rows dfv_dim apart).  Wd_grad is added to: the caller
+ *                      zeroes it.  Sums are fp32 in an order the hardware picks.
+ * An ID outside [0, img_vocab) contributes a zero row / nothing and raises GEAR_DEV_BAD_ID.
+ */
+int gear_dense_forward(gear_ctx* ctx, const float* raw, int32_t raw_dim, const float* Wd, const int32_t* ids, int64_t n,
+                       const int64_t* d_n, float* rows, int64_t ld, void* stream);
+int gear_dense_backward(gear_ctx* ctx, const float* raw, int32_t raw_dim, const int32_t* ids, const float* avg,
+                        int64_t n, const int64_t* d_n, float* Wd_grad, void* stream);
+
+/*
+ * One Adam step (Section 4) on n parameters that all have a gradient: the head's parameters with the head_grad of a
+ * step, the Dense Part's weights with the Wd_grad of gear_dense_backward.  param, grad, m, v: device fp32 [n]; m and
+ * v zero before the first step; t >= 1 counts the steps.  cfg is host memory.
+ */
+int gear_adam_dense(float* param, const float* grad, float* m, float* v, int64_t n, int64_t t, const gear_adam* cfg,
+                    void* stream);
 
 /*
  * Synchronises the stream last used; returns the device status word (GEAR_DEV_* bits, then cleared) and

@@ -25,7 +25,8 @@ GEAR_TAG_USER, GEAR_TAG_URL, GEAR_TAG_DFV, GEAR_TAG_TS, GEAR_TAG_GRAD = 1, 2, 3,
 EXPORTS = ("gear_workspace_bytes", "gear_init_tables", "gear_forward_backward", "gear_accumulate_dfv_grad",
            "gear_collect_ready", "gear_collect_expired", "gear_status", "gear_destroy", "gear_fill_uniform",
            "gear_last_error", "gear_profile_enable", "gear_profile_read", "gear_launch_count",
-           "gear_collect_expired_static", "gear_refresh_dfv", "gear_accumulate_collect")
+           "gear_collect_expired_static", "gear_refresh_dfv", "gear_accumulate_collect", "gear_dense_forward",
+           "gear_dense_backward", "gear_adam_dense")
 GEAR_STATIC_EXPIRY_MAX_VOCAB = 16777216
 
 
@@ -53,10 +54,16 @@ class gear_batch(C.Structure):
                 ("img_off", C.c_void_p), ("img_id", C.c_void_p), ("label", C.c_void_p)]
 
 
+class gear_adam(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
+
+
 class gear_step_out(C.Structure):
     _fields_ = [("loss", C.c_void_p), ("prob", C.c_void_p), ("head_grad", C.c_void_p), ("dX", C.c_void_p),
                 ("row_view", C.c_void_p), ("inv_n", C.c_void_p), ("x_debug", C.c_void_p),
-                ("user_grad", C.c_void_p), ("url_grad", C.c_void_p)]
+                ("user_grad", C.c_void_p), ("url_grad", C.c_void_p),
+                ("adam", C.POINTER(gear_adam)), ("adam_step", C.c_int64),
+                ("user_m", C.c_void_p), ("user_v", C.c_void_p), ("url_m", C.c_void_p), ("url_v", C.c_void_p)]
 
 
 _lib = None
@@ -85,6 +92,12 @@ def load() -> C.CDLL:
     L.gear_collect_ready.argtypes = [vp, vp, vp, vp, i64, vp, C.POINTER(i64), vp]
     L.gear_accumulate_collect.restype = C.c_int
     L.gear_accumulate_collect.argtypes = [vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, i64, vp, C.POINTER(i64), vp]
+    L.gear_dense_forward.restype = C.c_int
+    L.gear_dense_forward.argtypes = [vp, vp, i32, vp, vp, i64, vp, vp, i64, vp]
+    L.gear_dense_backward.restype = C.c_int
+    L.gear_dense_backward.argtypes = [vp, vp, i32, vp, vp, i64, vp, vp, vp]
+    L.gear_adam_dense.restype = C.c_int
+    L.gear_adam_dense.argtypes = [vp, vp, vp, vp, i64, i64, C.POINTER(gear_adam), vp]
     L.gear_collect_expired.restype = C.c_int
     L.gear_collect_expired.argtypes = [vp, i64, C.c_int, vp, i64, vp, C.POINTER(i64), vp]
     L.gear_status.restype = C.c_int
@@ -184,12 +197,23 @@ def make_batch(user_id, url_id, img_off, img_id, label, B: Optional[int] = None,
     return bt
 
 
+def make_adam(lr: float = 1e-4, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8) -> gear_adam:
+    """The optimiser's constants (defaults: the paper's learning rate, Kingma and Ba's other constants)."""
+    return gear_adam(lr, beta1, beta2, eps)
+
+
 def make_step_out(loss, head_grad, dX, prob=None, row_view=None, inv_n=None, x_debug=None, user_grad=None,
-                  url_grad=None) -> gear_step_out:
+                  url_grad=None, adam: Optional[gear_adam] = None, adam_step: int = 0, user_m=None, user_v=None,
+                  url_m=None, url_v=None) -> gear_step_out:
     o = gear_step_out()
     for name, t in (("loss", loss), ("prob", prob), ("head_grad", head_grad), ("dX", dX), ("row_view", row_view),
-                    ("inv_n", inv_n), ("x_debug", x_debug), ("user_grad", user_grad), ("url_grad", url_grad)):
+                    ("inv_n", inv_n), ("x_debug", x_debug), ("user_grad", user_grad), ("url_grad", url_grad),
+                    ("user_m", user_m), ("user_v", user_v), ("url_m", url_m), ("url_v", url_v)):
         setattr(o, name, None if t is None else _p(t).value)
+    if adam is not None:
+        o.adam = C.pointer(adam)
+        o._adam_keepalive = adam
+    o.adam_step = adam_step
     return o
 
 
@@ -245,6 +269,27 @@ def gear_refresh_dfv(ctx, ids, rows, n: int, now: int, d_n=None, stream=None):
     assert rows.is_cuda and rows.dtype == torch.float32 and rows.dim() == 2 and rows.stride(1) == 1
     _check(load().gear_refresh_dfv(ctx, _p(ids), C.c_void_p(rows.data_ptr()), rows.stride(0), n, _p(d_n), now, _stream(stream)),
            "gear_refresh_dfv")
+
+
+def gear_dense_forward(ctx, raw, Wd, ids, n: int, rows, d_n=None, stream=None):
+    """rows[k] = raw[ids[k]] . Wd for k < n (and k < *d_n); rows fp32 [>= n][ld]."""
+    assert raw.dtype == torch.float32 and Wd.dtype == torch.float32 and rows.dtype == torch.float32 and rows.stride(1) == 1
+    _check(load().gear_dense_forward(ctx, _p(raw), raw.shape[1], _p(Wd), _p(ids), n, _p(d_n), C.c_void_p(rows.data_ptr()),
+                                     rows.stride(0), _stream(stream)), "gear_dense_forward")
+
+
+def gear_dense_backward(ctx, raw, ids, avg, n: int, Wd_grad, d_n=None, stream=None):
+    """Wd_grad[r][c] += sum_e raw[ids[e]][r] * avg[e][c] over the emissions e < n (and e < *d_n)."""
+    assert raw.dtype == torch.float32 and avg.dtype == torch.float32 and Wd_grad.dtype == torch.float32
+    _check(load().gear_dense_backward(ctx, _p(raw), raw.shape[1], _p(ids), _p(avg), n, _p(d_n), _p(Wd_grad),
+                                      _stream(stream)), "gear_dense_backward")
+
+
+def gear_adam_dense(param, grad, m, v, t: int, cfg: gear_adam, stream=None):
+    n = param.numel()
+    assert grad.numel() == n and m.numel() == n and v.numel() == n
+    _check(load().gear_adam_dense(_p(param), _p(grad), _p(m), _p(v), n, t, C.byref(cfg), _stream(stream)),
+           "gear_adam_dense")
 
 
 def gear_status(ctx, raise_on_error: bool = False):

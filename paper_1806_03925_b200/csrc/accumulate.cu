@@ -24,8 +24,6 @@
 //      complete groups (or the call is dropped whole if the queue would overflow).
 // HBM bound: the reduce pass reads every gradient row once and reads/writes one accumulator row per
 // distinct image; the sort and flag passes move 4-byte keys only.
-#include <cstdlib>
-
 #include "common.cuh"
 #include "internal.h"
 
@@ -457,192 +455,6 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
     leave();
 }
 
-// ---------------------------------------------------------------- the reduce pass, register version
-// Same plan, same results, other machinery: no shared-memory ring.  A warp takes spans of ACC_SPAN sorted positions and
-// walks the groups that start in its span one after the other; a lane owns NQ 16-byte chunks of a row and keeps the
-// group's sum in registers.  The rows of a group are fetched up to R = 8 / NQ at a time, all loads of a batch issued
-// before the first addition (straight-line code per batch size), together with the image's accumulator row where the
-// group continues one; memory-level parallelism comes from the number of resident warps, as in the gather.  Where
-// each sorted position's row lives and what it is scaled by (the 8-byte position records) sits in the lanes for a
-// window of 32 positions: the span's own window arrives with the group records, one span ahead; groups that reach
-// beyond it (long groups of hot images, an image's trailing open group) reload the window as they go.
-template <int NQ, int K, bool FULL>
-__device__ __forceinline__ void add_rows_from_window(float4 (&acc)[NQ], const float* __restrict__ grads, int64_t ld,
-                                                     int n_chunks, const int2& pm, int j, int lane) {
-    float4 v[K][NQ];
-    float sc[K];
-#pragma unroll
-    for (int t = 0; t < K; ++t) {
-        const int src = __shfl_sync(0xffffffffu, pm.x, j + t);
-        sc[t] = __int_as_float(__shfl_sync(0xffffffffu, pm.y, j + t));
-        const float* row = grads + (int64_t)src * ld;
-#pragma unroll
-        for (int q = 0; q < NQ; ++q) {
-            const int ch = lane + 32 * q;
-            v[t][q] = (FULL || ch < n_chunks) ? ld_stream_f4(row + ch * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-    }
-#pragma unroll
-    for (int t = 0; t < K; ++t)
-#pragma unroll
-        for (int q = 0; q < NQ; ++q) {
-            // in the indirect form the scaled row is never stored: the product joins the sum with one rounding
-            acc[q].x = fmaf(sc[t], v[t][q].x, acc[q].x); acc[q].y = fmaf(sc[t], v[t][q].y, acc[q].y);
-            acc[q].z = fmaf(sc[t], v[t][q].z, acc[q].z); acc[q].w = fmaf(sc[t], v[t][q].w, acc[q].w);
-        }
-}
-
-template <int NQ, bool FULL>
-__global__ void __launch_bounds__(256, NQ <= 2 ? 3 : 2)
-acc_reduce_reg_kernel(RowGather rg, int D, int M, int64_t n_tiles, int64_t ready_cap,
-                      const uint2* __restrict__ tile_cnt, const uint4* __restrict__ grp_rec,
-                      const uint32_t* __restrict__ blk_first, const uint32_t* __restrict__ run_end,
-                      float* __restrict__ gsum, int32_t* __restrict__ gcnt,
-                      int32_t* __restrict__ q_id, float* __restrict__ q_avg, const EmitTarget direct,
-                      DevState* __restrict__ state) {
-    wait_for_predecessor();
-    constexpr int R = NQ >= 8 ? 1 : 8 / NQ;                          // rows fetched per batch
-    const uint2 totals = tile_cnt[n_tiles];
-    const int64_t n_groups = totals.x;
-    const bool to_caller = direct.avg != nullptr;
-    int32_t* __restrict__ e_id = to_caller ? direct.ids : q_id;
-    float* __restrict__ e_avg = to_caller ? direct.avg : q_avg;
-    const bool dropped = !to_caller && state->q_count + (int64_t)totals.y > ready_cap;
-    auto leave = [&]() {
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            __threadfence();
-            unsigned int* ticket = reinterpret_cast<unsigned int*>(&state->pad[4]);
-            if (atomicInc(ticket, gridDim.x - 1) == gridDim.x - 1) {
-                state->n_groups = totals.x;
-                state->n_complete = totals.y;
-                if (to_caller) { if (direct.d_n) *direct.d_n = totals.y; }
-                else if (dropped) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
-                else if (totals.y > 0) { state->q_count += totals.y; state->q_calls += 1; }
-            }
-        }
-    };
-    if (dropped) { leave(); return; }
-    const int64_t n_valid = state->n_valid;
-    const int lane = (int)lane_id(), warp = (int)(threadIdx.x >> 5);
-    const int n_chunks = D / 4;
-    const float m_f = (float)M;
-    const int64_t W = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int64_t n_spans = ceil_div(n_valid, ACC_SPAN);
-
-    auto load_range = [&](int64_t span) -> uint32_t {              // lane 0: first group of the span, lane 1: one past its last
-        uint32_t v = 0;
-        if (span < n_spans && lane < 2) {
-            const int64_t w = span + lane;
-            v = w < n_spans ? __ldg(blk_first + w) : (uint32_t)n_groups;
-        }
-        return v;
-    };
-    struct Rec { uint32_t x, key, slot, w; int len; };
-    auto load_group = [&](int64_t g_lo, int64_t g_hi) -> Rec {
-        Rec r{0u, 0u, 0xffffffffu, 0u, 0};
-        const int64_t g = g_lo + lane;
-        if (g < g_hi) {
-            const uint4 rec = __ldg(grp_rec + g);
-            const uint32_t end = (g + 1 < n_groups) ? (__ldg(&grp_rec[g + 1].x) & 0x7fffffffu) : (uint32_t)n_valid;
-            r.x = rec.x; r.key = rec.y; r.slot = rec.z; r.w = rec.w;
-            r.len = (int)(end - (rec.x & 0x7fffffffu));
-        }
-        return r;
-    };
-    auto load_window = [&](int64_t p) -> int2 {                    // position records p .. p + 31, one per lane
-        return (p + lane < n_valid) ? __ldg(rg.pmeta + p + lane) : make_int2(0, 0);
-    };
-
-    int64_t span = (int64_t)blockIdx.x * (blockDim.x >> 5) + warp;
-    uint32_t range_cur = load_range(span), range_nxt = load_range(span + W);
-    Rec G = load_group(__shfl_sync(0xffffffffu, range_cur, 0), __shfl_sync(0xffffffffu, range_cur, 1));
-    int2 pm_span = load_window(span * ACC_SPAN);
-
-    for (; span < n_spans; span += W) {
-        // ---- look-ahead: group records and position records of the next span, group range of the one after it
-        const Rec G_nxt = load_group(__shfl_sync(0xffffffffu, range_nxt, 0), __shfl_sync(0xffffffffu, range_nxt, 1));
-        const int2 pm_nxt = load_window((span + W) * ACC_SPAN);
-        const uint32_t range_nxt2 = load_range(span + 2 * W);
-        const int n_here = (int)(__shfl_sync(0xffffffffu, range_cur, 1) - __shfl_sync(0xffffffffu, range_cur, 0));
-
-        uint32_t wbase = (uint32_t)(span * ACC_SPAN);
-        int2 pm = pm_span;
-        float4 acc[NQ];
-        // adds the rows at sorted positions pbeg .. pend - 1 to acc, in order
-        auto walk = [&](uint32_t pbeg, uint32_t pend) {
-            uint32_t p = pbeg;
-            while (p < pend) {
-                if (p < wbase || p >= wbase + 32u) { wbase = p; pm = load_window(p); }
-                const int j = (int)(p - wbase);
-                const int cnt = (int)min(min((uint32_t)R, pend - p), wbase + 32u - p);
-                switch (cnt) {
-                case 1: add_rows_from_window<NQ, 1, FULL>(acc, rg.grads, rg.ld, n_chunks, pm, j, lane); break;
-                case 2: if constexpr (R >= 2) add_rows_from_window<NQ, 2, FULL>(acc, rg.grads, rg.ld, n_chunks, pm, j, lane); break;
-                case 3: if constexpr (R >= 3) add_rows_from_window<NQ, 3, FULL>(acc, rg.grads, rg.ld, n_chunks, pm, j, lane); break;
-                case 4: if constexpr (R >= 4) add_rows_from_window<NQ, 4, FULL>(acc, rg.grads, rg.ld, n_chunks, pm, j, lane); break;
-                case 5: if constexpr (R >= 5) add_rows_from_window<NQ, 5, FULL>(acc, rg.grads, rg.ld, n_chunks, pm, j, lane); break;
-                case 6: if constexpr (R >= 6) add_rows_from_window<NQ, 6, FULL>(acc, rg.grads, rg.ld, n_chunks, pm, j, lane); break;
-                case 7: if constexpr (R >= 7) add_rows_from_window<NQ, 7, FULL>(acc, rg.grads, rg.ld, n_chunks, pm, j, lane); break;
-                default: if constexpr (R >= 8) add_rows_from_window<NQ, 8, FULL>(acc, rg.grads, rg.ld, n_chunks, pm, j, lane); break;
-                }
-                p += (uint32_t)cnt;
-            }
-        };
-
-        for (int gi = 0; gi < n_here; ++gi) {
-            const uint32_t gx = __shfl_sync(0xffffffffu, G.x, gi);
-            const int slot = (int)__shfl_sync(0xffffffffu, G.slot, gi);
-            const bool first = (gx >> 31) != 0u;
-            if (!first && slot < 0) continue;                     // an image's trailing open group: its first group's warp has it
-            const uint32_t start = gx & 0x7fffffffu;
-            const uint32_t key = __shfl_sync(0xffffffffu, G.key, gi);
-            const int w = (int)__shfl_sync(0xffffffffu, G.w, gi);
-            const int len = __shfl_sync(0xffffffffu, G.len, gi);
-            const int c0 = first ? w : 0;
-            float* srow = gsum + (int64_t)key * D;
-            // the sum starts from what the image's open group already holds
-#pragma unroll
-            for (int q = 0; q < NQ; ++q) {
-                const int ch = lane + 32 * q;
-                acc[q] = (c0 > 0 && (FULL || ch < n_chunks)) ? ld_f4(srow + ch * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            walk(start, start + (uint32_t)len);
-            int zlen = 0;
-            if (slot >= 0) {                                      // the group reached M: its average is handed on
-                float* qrow = e_avg + (int64_t)slot * D;
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    const int ch = lane + 32 * q;
-                    if (FULL || ch < n_chunks)
-                        st_f4(qrow + ch * 4, make_float4(acc[q].x / m_f, acc[q].y / m_f, acc[q].z / m_f, acc[q].w / m_f));
-                    acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-                if (lane == 0) {
-                    e_id[slot] = (int32_t)key;
-                    if (to_caller) direct.seq[slot] = first ? 0 : w;
-                }
-                if (first) {
-                    // what the image's remaining rows leave in the table: the rows of its trailing open group
-                    const uint32_t run_stop = __ldg(run_end + start);
-                    zlen = (int)(((int64_t)c0 + (int64_t)(run_stop - start)) % M);
-                    walk(run_stop - (uint32_t)zlen, run_stop);
-                }
-            }
-            if (first && (slot < 0 || zlen > 0 || c0 > 0)) {      // the table row: the image's open group after this call
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    const int ch = lane + 32 * q;
-                    if (FULL || ch < n_chunks) st_f4(srow + ch * 4, acc[q]);
-                }
-                if (lane == 0) gcnt[key] = slot < 0 ? c0 + len : zlen;
-            }
-        }
-        G = G_nxt; pm_span = pm_nxt; range_cur = range_nxt; range_nxt = range_nxt2;
-    }
-    leave();
-}
-
 // Steps 2-4 of the plan over the sorted keys ks / permutation perm (flag pass, scan, plan pass).
 static cudaError_t enqueue_plan(const gear_ctx_impl& c, const uint32_t* ks, const uint32_t* perm, int64_t n,
                                 const int32_t* src_row, const float* scale, cudaStream_t st) {
@@ -726,23 +538,6 @@ static cudaError_t launch_accumulate_to(const gear_ctx_impl& c, const int32_t* i
     const int resident = sm_count() * (nq <= 2 ? 3 : 2);          // every block stays resident
     const int grid = (int)(want < resident ? (want < 1 ? 1 : want) : resident);
     cudaError_t le = cudaSuccess;
-    static const bool use_ring = getenv("GEAR_ACC_RING") != nullptr;
-    if (!use_ring) {
-        KernelScope k(&c.prof, "acc_reduce", st);
-        const int64_t want_blocks = ceil_div(ceil_div(n, ACC_SPAN), 8);
-        const int grid_r = (int)(want_blocks < resident ? (want_blocks < 1 ? 1 : want_blocks) : resident);
-        auto launch_r = [&](auto kernel) {
-            le = launch_dependent(kernel, dim3(grid_r), dim3(256), 0, st, rg, D, M, n_tiles, c.ws.ready_cap, tile_cnt, grp_rec,
-                                  blk_first, run_end, c.buf.dfv_gsum, c.buf.dfv_gcnt, c.at<int32_t>(c.ws.q_id),
-                                  c.at<float>(c.ws.q_avg), to_caller, state);
-        };
-#define GEAR_ACC_REG(NQ) do { if (D == NQ * 128) launch_r(acc_reduce_reg_kernel<NQ, true>); else launch_r(acc_reduce_reg_kernel<NQ, false>); } while (0)
-        if (nq <= 1) GEAR_ACC_REG(1);
-        else if (nq <= 2) GEAR_ACC_REG(2);
-        else if (nq <= 4) GEAR_ACC_REG(4);
-        else GEAR_ACC_REG(8);
-#undef GEAR_ACC_REG
-    } else
     { KernelScope k(&c.prof, "acc_reduce", st);
     auto launch = [&](auto kernel, int slot_bytes, int slots) {
         const int smem = 8 * slots * slot_bytes;

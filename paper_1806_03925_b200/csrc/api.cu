@@ -37,9 +37,10 @@ static int validate_config(const gear_config& c) {
     }
     if (c.M < 1) return arg_fail("M >= 1");
     if (c.expire < 0) return arg_fail("expire >= 0");
-    if (c.max_batch < 1) return arg_fail("max_batch >= 1");
-    if (c.max_nnz < 1 || c.max_nnz > vmax) return arg_fail("max_nnz in [1, 2^31 - 2]");
-    if (c.ready_cap < 0 || c.ready_cap > vmax) return arg_fail("ready_cap in [0, 2^31 - 2]");
+    if (c.max_batch < 1 || c.max_batch > (1 << 30) - 1) return arg_fail("max_batch in [1, 2^30 - 1]");
+    const int64_t nmax = (1ll << 30) - 1;         // element counts of the key sort fit 30 bits
+    if (c.max_nnz < 1 || c.max_nnz > nmax) return arg_fail("max_nnz in [1, 2^30 - 1]");
+    if (c.ready_cap < 0 || c.ready_cap > nmax) return arg_fail("ready_cap in [0, 2^30 - 1]");
     if (c.accum_mode != GEAR_ACC_SORT && c.accum_mode != GEAR_ACC_ATOMIC) return arg_fail("accum_mode");
     if (c.accum_mode == GEAR_ACC_ATOMIC && c.M >= (1 << 29)) return arg_fail("GEAR_ACC_ATOMIC needs M < 2^29");
     return GEAR_OK;
@@ -77,8 +78,8 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
             p->sort_keys[s][i] = take((size_t)p->sort_n[s] * 4);
             p->sort_vals[s][i] = take((size_t)p->sort_n[s] * 4);
         }
-        p->sort_hist[s] = take((size_t)RS_BUCKETS * sort_tiles(p->sort_n[s]) * 4);
-        p->sort_tot[s] = take(RS_BUCKETS * 4);
+        p->sort_hist[s] = take((size_t)RS_MAX_PASSES * RS_BUCKETS * sort_tiles(p->sort_n[s]) * 4);
+        p->sort_tot[s] = take((size_t)RS_MAX_PASSES * RS_BUCKETS * 4);
     }
     p->tile_cnt = take((size_t)(ceil_div(c.max_nnz, 1024) + 1) * sizeof(uint2));
     p->grp_rec = take((size_t)c.max_nnz * 16);
@@ -87,6 +88,8 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
     p->run_end = take((size_t)c.max_nnz * 4);
     p->q_id = take((size_t)p->ready_cap * 4);
     p->q_avg = take((size_t)p->ready_cap * c.dfv_dim * 4);
+    p->emb_gsum[0] = take(B * c.emb_dim * 4);
+    p->emb_gsum[1] = take(B * c.emb_dim * 4);
     p->exp_bits = take((size_t)ceil_div(c.img_vocab, 32) * 4);
     p->exp_cnt = take((size_t)(ceil_div(c.img_vocab, EXP_MARK_TILE) + 1) * sizeof(uint2));
     p->total = off;
@@ -216,6 +219,17 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     if (b.nnz > 0 && !b.img_id) return arg_fail("NULL img_id");
     if (!o.loss || !o.head_grad || !o.dX) return arg_fail("loss, head_grad and dX are required outputs");
     if ((o.user_grad == nullptr) != (o.url_grad == nullptr)) return arg_fail("user_grad and url_grad: both or neither");
+    gear_adam adam_cfg = {0.f, 0.f, 0.f, 0.f};
+    if (o.adam) {
+        adam_cfg = *o.adam;
+        if (o.user_grad) return arg_fail("adam and user_grad / url_grad exclude each other");
+        if (!o.user_m || !o.user_v || !o.url_m || !o.url_v) return arg_fail("adam needs the four moment tables");
+        if (!aligned16(o.user_m) || !aligned16(o.user_v) || !aligned16(o.url_m) || !aligned16(o.url_v))
+            return arg_fail("moment tables must be 16-byte aligned");
+        if (o.adam_step < 1) return arg_fail("adam_step >= 1");
+        if (!(adam_cfg.beta1 >= 0.f && adam_cfg.beta1 < 1.f && adam_cfg.beta2 >= 0.f && adam_cfg.beta2 < 1.f && adam_cfg.eps >= 0.f))
+            return arg_fail("adam: beta1, beta2 in [0, 1), eps >= 0");
+    }
     if (c.cfg.head_dtype == GEAR_BF16 && (!aligned16(o.head_grad) || !aligned16(c.buf.head_params)))
         return arg_fail("bf16 head: head_params and head_grad must be 16-byte aligned");
     if (!aligned16(o.dX) || (o.x_debug && !aligned16(o.x_debug)) || (o.user_grad && !aligned16(o.user_grad)) ||
@@ -302,7 +316,8 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     // the embedding scatter: enqueued by the head as soon as dX is on its way
     struct Scatter {
         gear_ctx_impl* c; const gear_step_out* o; int sorted_buf; int32_t B; float lr; cudaStream_t st; bool forked;
-    } sc{&c, &o, sorted_buf, b.B, lr, st, forked};
+        const gear_adam* adam;
+    } sc{&c, &o, sorted_buf, b.B, lr, st, forked, o.adam ? &adam_cfg : nullptr};
     auto scatter = [](void* arg) -> cudaError_t {
         Scatter& k = *static_cast<Scatter*>(arg);
         gear_ctx_impl& c = *k.c;
@@ -316,6 +331,9 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
             if (e != cudaSuccess) return e;
             where = c.side_stream;
         }
+        if (k.adam)
+            return launch_emb_adam(c, k.sorted_buf, k.B, k.o->dX, c.d_in, *k.adam, k.o->adam_step, k.o->user_m, k.o->user_v,
+                                   k.o->url_m, k.o->url_v, where);
         return launch_emb_reduce(c, k.sorted_buf, k.B, ut, ht, k.o->dX, c.d_in, alpha, where);
     };
     const HeadHooks hooks{weights_on_side, scatter, &sc};
@@ -440,6 +458,43 @@ int gear_refresh_dfv(gear_ctx* ctx, const int32_t* ids, const float* rows, int64
     cudaError_t e = launch_refresh_dfv(c, ids, rows, ld, n, d_n, now, st);
     if (e != cudaSuccess) return cuda_fail(e, "refresh_dfv");
     return GEAR_OK;
+}
+
+int gear_dense_forward(gear_ctx* ctx, const float* raw, int32_t raw_dim, const float* Wd, const int32_t* ids, int64_t n,
+                       const int64_t* d_n, float* rows, int64_t ld, void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (n < 0 || raw_dim < 1) return arg_fail("n >= 0, raw_dim >= 1");
+    if (n == 0) return GEAR_OK;
+    if (!raw || !Wd || !ids || !rows || ld < c.cfg.dfv_dim) return arg_fail("NULL pointer or ld < dfv_dim");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.note_stream(st);
+    cudaError_t e = launch_dense_forward(c, raw, raw_dim, Wd, ids, n, d_n, rows, ld, st);
+    return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "dense_forward");
+}
+
+int gear_dense_backward(gear_ctx* ctx, const float* raw, int32_t raw_dim, const int32_t* ids, const float* avg, int64_t n,
+                        const int64_t* d_n, float* Wd_grad, void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (n < 0 || raw_dim < 1) return arg_fail("n >= 0, raw_dim >= 1");
+    if (n == 0) return GEAR_OK;
+    if (!raw || !ids || !avg || !Wd_grad) return arg_fail("NULL pointer");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.note_stream(st);
+    cudaError_t e = launch_dense_backward(c, raw, raw_dim, ids, avg, c.cfg.dfv_dim, n, d_n, Wd_grad, st);
+    return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "dense_backward");
+}
+
+int gear_adam_dense(float* param, const float* grad, float* m, float* v, int64_t n, int64_t t, const gear_adam* cfg,
+                    void* stream) {
+    if (n < 0 || t < 1 || !cfg) return arg_fail("n >= 0, t >= 1, cfg");
+    if (n == 0) return GEAR_OK;
+    if (!param || !grad || !m || !v) return arg_fail("NULL pointer");
+    if (!(cfg->beta1 >= 0.f && cfg->beta1 < 1.f && cfg->beta2 >= 0.f && cfg->beta2 < 1.f && cfg->eps >= 0.f))
+        return arg_fail("adam: beta1, beta2 in [0, 1), eps >= 0");
+    cudaError_t e = launch_adam_dense(nullptr, param, grad, m, v, n, t, *cfg, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "adam_dense");
 }
 
 int gear_status(gear_ctx* ctx, int32_t* device_status, int64_t* pending_ready) {

@@ -188,6 +188,7 @@ constexpr int RS_ITEMS = 16;
 constexpr int RS_TILE = RS_THREADS * RS_ITEMS;
 constexpr int RS_RADIX_BITS = 9;
 constexpr int RS_BUCKETS = 1 << RS_RADIX_BITS;
+constexpr int RS_MAX_PASSES = 4;          // 32-bit keys in digits of 9 bits
 
 inline int64_t sort_tiles(int64_t n_max) { return n_max > 0 ? ceil_div(n_max, RS_TILE) : 1; }
 
@@ -198,8 +199,9 @@ struct SortJob {
     int32_t* status;        // device status word that gets GEAR_DEV_BAD_ID when a sentinel key is met (may be null)
     uint32_t* keys[2];      // without ids the input keys are keys[0]
     uint32_t* vals[2];      // with identity_vals the value of element i is i, else vals[0][i]
-    uint32_t* hist;         // [RS_BUCKETS][n_tiles]
-    uint32_t* tot;          // [RS_BUCKETS]
+    uint32_t* hist;         // [RS_MAX_PASSES][n_tiles][RS_BUCKETS] tile descriptors: per pass and tile, how many of the
+                            // tile's elements (or of all tiles up to it) carry each digit; top two bits say which
+    uint32_t* tot;          // [RS_MAX_PASSES][RS_BUCKETS] digit histogram of every pass
     int64_t n_max;          // element count (or its upper bound when n_dev is given)
     const int64_t* n_dev;   // optional device-resident count, capped at n_max
     int bits;

@@ -17,7 +17,10 @@ constexpr int ES_SEG = 8;    // sorted positions walked by one lane group
 // One of the two tables of a launch (blockIdx.y picks it).
 struct EmbTable { const uint32_t* ks; const uint32_t* perm; uint32_t vocab; int col0; float* table; };
 
-template <int NQ>
+// COMPACT: the sums do not go to the table but to a buffer with one row per sorted position: an ID's sum lands in the
+// row of the position at which its run starts (table then points to that buffer, alpha is 1).  The optimiser's row
+// kernel (dense.cu) picks the sums up from there: a non-linear update needs an ID's whole sum before it can start.
+template <int NQ, bool COMPACT>
 __global__ void __launch_bounds__(256)
 emb_reduce_kernel(const EmbTable t0, const EmbTable t1, int n, int E, int lpr, const float* __restrict__ dX, int64_t ldx,
                   float alpha) {
@@ -54,6 +57,18 @@ emb_reduce_kernel(const EmbTable t0, const EmbTable t1, int n, int E, int lpr, c
     float4 acc[NQ];
 #pragma unroll
     for (int q = 0; q < NQ; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    // COMPACT: where the run that covers position p0 starts (it may start in an earlier segment: gallop back, then bisect)
+    int64_t head = p0;
+    if (COMPACT && p0 > 0 && key[0] < vocab && ks[p0 - 1] == key[0]) {
+        int64_t hi = p0 - 1, step = 1, lo = hi - 1;            // ks[hi] == key[0]
+        while (lo >= 0 && ks[lo] == key[0]) { hi = lo; step <<= 1; lo = max(hi - step, (int64_t)-1); }
+        int64_t l = lo + 1, h = hi;                            // answer in [l, h]; ks[h] == key[0], ks[lo] != key[0]
+        while (l < h) {
+            const int64_t mid = (l + h) >> 1;
+            if (ks[mid] == key[0]) h = mid; else l = mid + 1;
+        }
+        head = l;
+    }
 #pragma unroll
     for (int t = 0; t < ES_SEG; ++t) {
         if (key[t] >= vocab) break;
@@ -67,10 +82,11 @@ emb_reduce_kernel(const EmbTable t0, const EmbTable t1, int n, int E, int lpr, c
             for (int q = 0; q < NQ; ++q) {
                 const int ch = c + q * lpr;
                 if (ch < n_chunks)
-                    red_add_f4(table + (int64_t)key[t] * E + ch * 4,
+                    red_add_f4(table + (COMPACT ? head : (int64_t)key[t]) * E + ch * 4,
                                make_float4(alpha * acc[q].x, alpha * acc[q].y, alpha * acc[q].z, alpha * acc[q].w));
                 acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
+            head = p0 + t + 1;                                 // the next position starts a run
         }
     }
 }
@@ -88,7 +104,7 @@ cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int cur, int32_t B, float*
     const dim3 grid((unsigned)ceil_div(groups * lpr, 256), 2);
     const EmbTable t0{su.keys[cur], su.vals[cur], (uint32_t)c.cfg.user_vocab, 0, user_table};
     const EmbTable t1{sh.keys[cur], sh.vals[cur], (uint32_t)c.cfg.url_vocab, E, url_table};
-#define GEAR_ES_LAUNCH(NQ) launch_dependent(emb_reduce_kernel<NQ>, grid, dim3(256), 0, st, t0, t1, B, E, lpr, dX, (int64_t)ldx, alpha)
+#define GEAR_ES_LAUNCH(NQ) launch_dependent(emb_reduce_kernel<NQ, false>, grid, dim3(256), 0, st, t0, t1, B, E, lpr, dX, (int64_t)ldx, alpha)
     KernelScope ks(&c.prof, "emb_reduce", st);
     if (nq <= 1) GEAR_ES_LAUNCH(1);
     else if (nq <= 2) GEAR_ES_LAUNCH(2);
@@ -96,6 +112,41 @@ cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int cur, int32_t B, float*
     else GEAR_ES_LAUNCH(8);
 #undef GEAR_ES_LAUNCH
     return cudaGetLastError();
+}
+
+// Section 4's optimiser on the rows of both embedding tables that the batch touched: the per-ID sums go to the compact
+// buffers (zeroed first), then every distinct ID's row takes one Adam step.
+cudaError_t launch_emb_adam(const gear_ctx_impl& c, int cur, int32_t B, const float* dX, int ldx, const gear_adam& cfg,
+                            int64_t t, float* user_m, float* user_v, float* url_m, float* url_v, cudaStream_t st) {
+    if (B <= 0) return cudaSuccess;
+    SortJob su = c.sort_job(gear_ctx_impl::SORT_USER), sh = c.sort_job(gear_ctx_impl::SORT_URL);
+    const int E = c.cfg.emb_dim, n_chunks = E / 4;
+    float* gu = c.at<float>(c.ws.emb_gsum[0]);
+    float* gh = c.at<float>(c.ws.emb_gsum[1]);
+    cudaError_t e = cudaMemsetAsync(gu, 0, sizeof(float) * (size_t)B * E, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(gh, 0, sizeof(float) * (size_t)B * E, st);
+    if (e != cudaSuccess) return e;
+    int lpr = 1;
+    while (lpr < n_chunks && lpr < 32) lpr <<= 1;
+    const int nq = (int)ceil_div(n_chunks, lpr);
+    const int64_t groups = ceil_div(B, ES_SEG);
+    const dim3 grid((unsigned)ceil_div(groups * lpr, 256), 2);
+    const EmbTable t0{su.keys[cur], su.vals[cur], (uint32_t)c.cfg.user_vocab, 0, gu};
+    const EmbTable t1{sh.keys[cur], sh.vals[cur], (uint32_t)c.cfg.url_vocab, E, gh};
+    {
+#define GEAR_ES_LAUNCH(NQ) launch_dependent(emb_reduce_kernel<NQ, true>, grid, dim3(256), 0, st, t0, t1, B, E, lpr, dX, (int64_t)ldx, 1.0f)
+        KernelScope ks(&c.prof, "emb_reduce", st);
+        if (nq <= 1) GEAR_ES_LAUNCH(1);
+        else if (nq <= 2) GEAR_ES_LAUNCH(2);
+        else if (nq <= 4) GEAR_ES_LAUNCH(4);
+        else GEAR_ES_LAUNCH(8);
+#undef GEAR_ES_LAUNCH
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const EmbAdamTable a0{su.keys[cur], (uint32_t)c.cfg.user_vocab, c.buf.user_emb, user_m, user_v, gu};
+    const EmbAdamTable a1{sh.keys[cur], (uint32_t)c.cfg.url_vocab, c.buf.url_emb, url_m, url_v, gh};
+    return launch_emb_adam_rows(c, a0, a1, B, t, cfg, st);
 }
 
 }  // namespace gear

@@ -37,6 +37,8 @@ struct WsPlan {
     size_t pmeta;                       // [max_nnz] int2: source row and scale (fp32 bits) of every sorted position
     size_t q_id;                        // [ready_cap] int32
     size_t q_avg;                       // [ready_cap][dfv_dim] fp32
+    size_t emb_gsum[2];                 // [max_batch][emb_dim] fp32 per table: summed gradient of every distinct ID of the
+                                        // batch, in the row of the sorted position where the ID's run starts (Adam only)
     size_t exp_bits;                    // [ceil(img_vocab / 32)] uint32 expired bitmap
     size_t exp_cnt;                     // [expiry mark tiles + 1] uint2
     size_t total;
@@ -139,6 +141,20 @@ cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int 
 // sorted (id, view) pairs of buffer sets SORT_USER / SORT_URL
 cudaError_t launch_emb_reduce(const gear_ctx_impl& c, int buf, int32_t B, float* user_table, float* url_table,
                               const float* dX, int ldx, float alpha, cudaStream_t st);
+
+// dense.cu: a linear Dense Part (DFV = raw row . Wd) and Adam
+struct EmbAdamTable { const uint32_t* ks; uint32_t vocab; float* table; float* m; float* v; const float* gsum; };
+cudaError_t launch_dense_forward(const gear_ctx_impl& c, const float* raw, int R, const float* Wd, const int32_t* ids,
+                                 int64_t n, const int64_t* d_n, float* rows, int64_t ld, cudaStream_t st);
+cudaError_t launch_dense_backward(const gear_ctx_impl& c, const float* raw, int R, const int32_t* ids, const float* avg,
+                                  int64_t ld_avg, int64_t n, const int64_t* d_n, float* G, cudaStream_t st);
+cudaError_t launch_adam_dense(Profiler* prof, float* p, const float* g, float* m, float* v, int64_t n, int64_t t,
+                              const gear_adam& cfg, cudaStream_t st);
+cudaError_t launch_emb_adam_rows(const gear_ctx_impl& c, const EmbAdamTable& t0, const EmbAdamTable& t1, int32_t B,
+                                 int64_t t, const gear_adam& cfg, cudaStream_t st);
+// emb_scatter.cu: Adam on the embedding rows the batch touched (per-ID sums into compact buffers, then the row steps)
+cudaError_t launch_emb_adam(const gear_ctx_impl& c, int buf, int32_t B, const float* dX, int ldx, const gear_adam& cfg,
+                            int64_t t, float* user_m, float* user_v, float* url_m, float* url_v, cudaStream_t st);
 
 // accumulate.cu
 // img_id == nullptr: use the image IDs sorted by the last gear_forward_backward (buffer set SORT_IMG)

@@ -40,7 +40,7 @@ class GearSession:
                  max_nnz: Optional[int] = None, seed: int = 0, fill: bool = True, now: int = 0,
                  tables: Optional[Dict[str, np.ndarray]] = None, ready_cap: int = 0, device: str = "cuda",
                  want_emb_grad: bool = False, want_debug: bool = False, expired_cap: Optional[int] = None,
-                 accum_mode: int = gb.GEAR_ACC_SORT):
+                 accum_mode: int = gb.GEAR_ACC_SORT, adam: Optional["gb.gear_adam"] = None):
         gb.load()
         self.p = p
         self.dev = torch.device(device)
@@ -89,6 +89,13 @@ class GearSession:
                                     device=dev) if want_debug else None)
         self.user_grad = torch.zeros_like(self.user_emb) if want_emb_grad else None
         self.url_grad = torch.zeros_like(self.url_emb) if want_emb_grad else None
+        # Section 4's optimiser for the embedding tables: first and second moments per table row
+        self.adam = adam
+        self.adam_step = 0
+        self.user_m = torch.zeros_like(self.user_emb) if adam is not None else None
+        self.user_v = torch.zeros_like(self.user_emb) if adam is not None else None
+        self.url_m = torch.zeros_like(self.url_emb) if adam is not None else None
+        self.url_v = torch.zeros_like(self.url_emb) if adam is not None else None
         # every output list is followed by one guard entry the library must never write (guards_intact checks them)
         self.ready_cap = int(ready_cap or nnz)
         self._ready_ids_g = torch.full((self.ready_cap + 1,), self.GUARD_I, dtype=torch.int32, device=dev)
@@ -110,7 +117,11 @@ class GearSession:
         if self._step_out is None:
             self._step_out = gb.make_step_out(self.loss, self.head_grad, self.dX, prob=self.prob, row_view=self.row_view,
                                               inv_n=self.inv_n, x_debug=self.x_debug, user_grad=self.user_grad,
-                                              url_grad=self.url_grad)
+                                              url_grad=self.url_grad, adam=self.adam, user_m=self.user_m,
+                                              user_v=self.user_v, url_m=self.url_m, url_v=self.url_v)
+        if self.adam is not None:
+            self.adam_step += 1
+            self._step_out.adam_step = self.adam_step
         bt = b.__dict__.get("_c_batch")
         if bt is None:
             bt = b.__dict__["_c_batch"] = gb.make_batch(b.user_id, b.url_id, b.img_off, b.img_id, b.label)
@@ -156,6 +167,14 @@ class GearSession:
     def refresh_dfv(self, ids: torch.Tensor, rows: torch.Tensor, now: int, n: Optional[int] = None, d_n=None):
         """Recomputed DFVs replace cached ones (rows fp32) and restart their clocks."""
         return gb.gear_refresh_dfv(self.ctx, ids, rows, int(ids.shape[0]) if n is None else n, now, d_n=d_n)
+
+    # ---- a linear Dense Part on the same device ---------------------------------------------------
+    def dense_forward(self, raw: torch.Tensor, Wd: torch.Tensor, ids: torch.Tensor, rows: torch.Tensor, n=None, d_n=None):
+        return gb.gear_dense_forward(self.ctx, raw, Wd, ids, int(ids.shape[0]) if n is None else n, rows, d_n=d_n)
+
+    def dense_backward(self, raw: torch.Tensor, n: int, Wd_grad: torch.Tensor, d_n=None):
+        """Back-propagation of the averages just handed over (ready_ids, ready_avg) through the Dense Part."""
+        return gb.gear_dense_backward(self.ctx, raw, self.ready_ids, self.ready_avg, n, Wd_grad, d_n=d_n)
 
     def step(self, b: DeviceBatch, now: int, sync: bool = False, expiry_beside: Optional[bool] = None):
         """One pass of the whole hot path over one batch.  The expiry scan depends on nothing the training calls

@@ -562,50 +562,157 @@ def test_refresh_dfv_matches_oracle(gb, name):
         g.close()
 
 
-def test_gear_loop_with_refresh_on_the_gpu_path_trains_a_linear_dense_part(gb):
-    """M = 1, expiry 0, a linear Dense Part DFV_i = raw_i . Wd kept by the test: every step the scan lists every
-    image, gear_refresh_dfv writes raw . Wd for the current Wd, and the emitted averages give dLoss/dWd (Eq. 1).
-    Two SGD steps on Wd through the GPU path against the same loop on the oracle."""
+def test_gear_loop_on_the_gpu_path_trains_a_linear_dense_part(gb):
+    """The whole loop of the paper's Section 3 on the device, with the smallest Dense Part there is (DFV_i = raw_i . Wd):
+    M = 1 and expiry 0, so every step the scan lists every image, gear_dense_forward recomputes every DFV from the current
+    Wd, gear_refresh_dfv stores them, the step's averaged gradients go back through the Dense Part
+    (gear_dense_backward: Eq. 1) and Wd takes an Adam step (gear_adam_dense, Section 4).  Three steps against the same
+    loop on the oracle; no product, sum or optimiser arithmetic happens in the test."""
     from gpu_harness import _np, assert_close
+    from oracle import AdamConfig
+    from paper_1806_03925_b200.session import DeviceBatch
     p = PRESETS["tiny"].scaled(M=1, expire=0, img_vocab=512, batch=128)
     R = 24
     rng = np.random.default_rng(9)
     raw = rng.normal(0, 1, (p.img_vocab, R)).astype(np.float32)
     Wd0 = rng.normal(0, 0.3, (R, p.dfv_dim)).astype(np.float32)
     src = BatchSource(p, 4)
-    batches = [src.batch(s) for s in range(2)]
+    batches = [src.batch(s) for s in range(3)]
     pair = _pair(p, batches, seed=4, dense=True)
     g, cpu = pair.gpu, pair.cpu
+    acfg = AdamConfig(lr=2e-2, beta1=0.9, beta2=0.99, eps=1e-8)
+    adam = gb.make_adam(acfg.lr, acfg.beta1, acfg.beta2, acfg.eps)
     try:
-        Wd_g, Wd_c, lr = Wd0.copy(), Wd0.astype(np.float64), 5.0
+        d_raw = torch.from_numpy(raw).cuda()
+        Wd = torch.from_numpy(Wd0.copy()).cuda()
+        Wd_m, Wd_v, Wd_grad = torch.zeros_like(Wd), torch.zeros_like(Wd), torch.zeros_like(Wd)
+        rows = torch.zeros((p.img_vocab, p.dfv_dim), device="cuda")
+        Wc, mc, vc = Wd0.astype(np.float64), np.zeros(Wd0.shape), np.zeros(Wd0.shape)
         for step, b in enumerate(batches):
-            now = step + 1
-            from paper_1806_03925_b200.session import DeviceBatch
-            # --- GPU path
+            now, t = step + 1, step + 1
+            # --- device
             k = g.collect_expired(now, restamp=True)
             assert k == p.img_vocab
-            ids = g.expired_ids[:k]
-            rows = torch.from_numpy(raw).cuda()[ids.long()] @ torch.from_numpy(Wd_g).cuda()
-            g.refresh_dfv(ids, rows.contiguous(), now)
+            g.dense_forward(d_raw, Wd, g.expired_ids, rows, n=p.img_vocab, d_n=g.d_counts[1:2])
+            g.refresh_dfv(g.expired_ids, rows, now, n=p.img_vocab, d_n=g.d_counts[1:2])
             db = DeviceBatch.from_host(b)
             g.forward_backward(db, lr=0.0)
-            g.accumulate_from_step(db)
-            n_ready = g.collect_ready()
-            assert n_ready == b.nnz                                    # M = 1: every gradient row is emitted
-            eid, eavg = _np(g.ready_ids[:n_ready]), _np(g.ready_avg[:n_ready]).astype(np.float64)
-            G_g = raw[eid].astype(np.float64).T @ eavg
+            n_ready = g.accumulate_collect_from_step(db)
+            assert n_ready == b.nnz                                    # M = 1: every gradient row is handed over
+            Wd_grad.zero_()
+            g.dense_backward(d_raw, b.nnz, Wd_grad, d_n=g.d_counts[0:1])
+            gb.gear_adam_dense(Wd, Wd_grad, Wd_m, Wd_v, t, adam)
             # --- oracle
             exp_c = cpu.collect_expired(now, restamp=True)
-            cpu.refresh_dfv(exp_c, (raw[exp_c] @ Wd_c.astype(np.float32)).astype(np.float32), now)
+            cpu.refresh_dfv(exp_c, oracle.dense_forward(raw, Wc, exp_c).astype(np.float32), now)
             r = cpu.forward_backward(pair.params.astype(np.float64), b.user_id, b.url_id, b.img_off, b.img_id, b.label)
             cpu.accumulate(b.img_id, cpu.dfv_grad_rows(b.img_off, r.dX))
             cid, _, cavg = cpu.collect_ready()
-            G_c = raw[cid].astype(np.float64).T @ cavg
-            assert_close(G_g, G_c, 1e-4, "dense-part gradient of step %d" % step)
-            Wd_g = (Wd_g - lr * G_g).astype(np.float32)
-            Wd_c = Wd_c - lr * G_c
-        assert_close(Wd_g.astype(np.float64), Wd_c, 1e-4, "dense-part weights after two steps")
-        assert np.abs(Wd_c - Wd0).max() > 1e-4                         # the steps did move the weights
+            G_c = oracle.dense_backward(raw, cid, cavg)
+            assert_close(_np(Wd_grad), G_c, 1e-5, "dense-part gradient of step %d" % step)
+            oracle.adam_step(Wc, G_c, mc, vc, t, acfg)
+            assert_close(_np(Wd) - Wd0, Wc - Wd0, 1e-4, "movement of the dense-part weights after step %d" % step)
+            assert_close(_np(Wd_m), mc, 1e-5, "first moments")
+            assert_close(_np(Wd_v), vc, 1e-5, "second moments")
+            got = _np(g.dfv)
+            assert_close(got, cpu.dfv, 1e-5, "refreshed DFV table")
+        assert np.abs(Wc - Wd0).max() > 1e-2                           # the steps did move the weights
+        assert g.status()[1] == 0
+    finally:
+        g.close()
+
+
+def test_dense_part_calls_edge_cases(gb):
+    """Ragged sizes on every side of the tiles, a device-side count below the capacity, a leading dimension wider than
+    the row, an out-of-range ID (zero row / skipped, flagged), repeated IDs in the emission list."""
+    from gpu_harness import _np, assert_close
+    p = PRESETS["tiny"].scaled(user_vocab=64, url_vocab=64, img_vocab=1000, dfv_dim=72)
+    pair = _pair(p, [], dense=True)
+    g = pair.gpu
+    try:
+        rng = np.random.default_rng(31)
+        R, n = 37, 333
+        raw = rng.normal(0, 1, (p.img_vocab, R)).astype(np.float32)
+        Wd = rng.normal(0, 0.3, (R, p.dfv_dim)).astype(np.float32)
+        ids = rng.integers(0, p.img_vocab, n).astype(np.int32)
+        ids[5] = p.img_vocab + 3
+        ids[77] = ids[78] = ids[200]
+        d_raw, d_Wd, d_ids = torch.from_numpy(raw).cuda(), torch.from_numpy(Wd).cuda(), torch.from_numpy(ids).cuda()
+        rows = torch.full((n, p.dfv_dim + 8), 7.0, device="cuda")
+        d_n = torch.tensor([300], dtype=torch.int64, device="cuda")
+        gb.gear_dense_forward(g.ctx, d_raw, d_Wd, d_ids, n, rows[:, :p.dfv_dim], d_n=d_n)
+        want = oracle.dense_forward(raw, Wd.astype(np.float64), ids[:300])
+        assert_close(_np(rows[:300, :p.dfv_dim]), want, 1e-5, "dense forward")
+        assert not _np(rows[5, :p.dfv_dim]).any()
+        assert (_np(rows[300:]) == 7.0).all() and (_np(rows[:, p.dfv_dim:]) == 7.0).all()       # nothing beyond the count / the row
+        rc, bits, _ = g.status()
+        assert bits & gb.GEAR_DEV_BAD_ID
+        avg = rng.normal(0, 1, (n, p.dfv_dim)).astype(np.float32)
+        G = torch.zeros((R, p.dfv_dim), device="cuda")
+        gb.gear_dense_backward(g.ctx, d_raw, d_ids, torch.from_numpy(avg).cuda(), n, G, d_n=d_n)
+        assert_close(_np(G), oracle.dense_backward(raw, ids[:300], avg[:300].astype(np.float64)), 1e-5, "dense backward")
+        gb.gear_dense_backward(g.ctx, d_raw, d_ids, torch.from_numpy(avg).cuda(), n, G)          # adds to what is there
+        want2 = oracle.dense_backward(raw, ids[:300], avg[:300].astype(np.float64)) + oracle.dense_backward(raw, ids, avg.astype(np.float64))
+        assert_close(_np(G), want2, 1e-5, "dense backward, accumulated")
+        g.status()
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "medium"])
+def test_adam_on_the_embedding_rows_and_the_head(gb, name):
+    """Section 4's optimiser through the library: the embedding rows a step touches (the adam fields of gear_step_out)
+    and the head's parameters (gear_adam_dense on head_grad) against the oracle, three steps, so that the second and
+    third start from non-zero moments and revisit rows.  Tables, both moment tables and the parameters are compared.
+
+    The moments are linear / quadratic in the gradient and are held to the configuration's tolerance.  The step itself
+    divides by sqrt(v) + eps, which turns a gradient entry's RELATIVE error into an error of the step: an entry far
+    below the largest one carries an absolute error of tol * max|g| like every other, so its sign and size, and with
+    them its step, are only as good as tol * max|g| / (|g| + eps).  The fp32 configuration runs with the usual
+    eps = 1e-8 (entry errors around 1e-10: steps good to 1e-2 of the learning rate in the worst entry); the bf16
+    configuration, whose gradient entries are good to about 1e-6, with eps = 1e-4, which keeps the same bound."""
+    from gpu_harness import _np, _rows, assert_close, Remap, tol_of
+    from oracle import AdamConfig, GearOracle
+    from paper_1806_03925_b200.session import DeviceBatch, GearSession
+    p = PRESETS[name].scaled(user_vocab=3000, url_vocab=2000, img_vocab=5000, batch=1500)
+    tol = tol_of(p)
+    acfg = AdamConfig(lr=1e-2, beta1=0.9, beta2=0.99, eps=1e-8 if p.head_dtype == F32 else 1e-4)
+    step_tol = 2e-2 if p.head_dtype == F32 else 5e-2          # of the largest movement, which is about lr
+    adam = gb.make_adam(acfg.lr, acfg.beta1, acfg.beta2, acfg.eps)
+    src = BatchSource(p, 6)
+    batches = [src.batch(s) for s in range(3)]
+    params = workloads.head_params(p, 6)
+    g = GearSession(p, params, max_batch=p.batch, max_nnz=max(b.nnz for b in batches), seed=6, fill=True, adam=adam)
+    dfv_np = np.uint16 if p.dfv_dtype == BF16 else np.float32
+    cpu = GearOracle(oracle.fill_rows(6, oracle.TAG_USER, p.emb_dim, None, p.user_vocab, np.float32),
+                     oracle.fill_rows(6, oracle.TAG_URL, p.emb_dim, None, p.url_vocab, np.float32),
+                     oracle.fill_rows(6, oracle.TAG_DFV, p.dfv_dim, None, p.img_vocab, dfv_np),
+                     p.hidden, p.M, p.expire, round_bf16=(p.head_dtype == BF16))
+    try:
+        u0, h0 = cpu.user_emb.copy(), cpu.url_emb.copy()
+        mom = {k: np.zeros(t.shape) for k, t in (("um", u0), ("uv", u0), ("hm", h0), ("hv", h0))}
+        pc, pm, pv = params.astype(np.float64), np.zeros(len(params)), np.zeros(len(params))
+        hp_m, hp_v = torch.zeros_like(g.head_params), torch.zeros_like(g.head_params)
+        for step, b in enumerate(batches):
+            t = step + 1
+            g.forward_backward(DeviceBatch.from_host(b))
+            gb.gear_adam_dense(g.head_params, g.head_grad, hp_m, hp_v, t, adam)
+            r = cpu.forward_backward(pc.copy(), b.user_id, b.url_id, b.img_off, b.img_id, b.label)
+            assert_close(_np(g.head_grad), r.head_grad, tol, "head_grad of step %d" % step)
+            oracle.emb_adam(cpu.user_emb, mom["um"], mom["uv"], b.user_id, r.dX, 0, t, acfg)
+            oracle.emb_adam(cpu.url_emb, mom["hm"], mom["hv"], b.url_id, r.dX, p.emb_dim, t, acfg)
+            oracle.adam_step(pc, r.head_grad, pm, pv, t, acfg)
+            # what moved, against what should have moved (the tables themselves are 0.17 wide, a step 0.01)
+            assert_close(_np(g.user_emb) - u0, cpu.user_emb.astype(np.float64) - u0, step_tol, "user table movement")
+            assert_close(_np(g.url_emb) - h0, cpu.url_emb.astype(np.float64) - h0, step_tol, "url table movement")
+            assert_close(_np(g.user_m), mom["um"], tol, "user first moments")
+            assert_close(_np(g.user_v), mom["uv"], tol, "user second moments")
+            assert_close(_np(g.url_m), mom["hm"], tol, "url first moments")
+            assert_close(_np(g.url_v), mom["hv"], tol, "url second moments")
+            assert_close(_np(g.head_params) - params, pc - params, step_tol, "head parameter movement")
+            # rows no view named stay bit for bit, moments included
+            idle = np.setdiff1d(np.arange(p.user_vocab), np.concatenate([x.user_id for x in batches[:step + 1]]))
+            assert np.array_equal(_np(g.user_emb)[idle], u0[idle]) and not _np(g.user_m)[idle].any() and not _np(g.user_v)[idle].any()
         assert g.status()[1] == 0
     finally:
         g.close()
