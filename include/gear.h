@@ -90,6 +90,9 @@ enum {
     GEAR_DEV_TIMEOUT = 16        /* a bounded wait inside a kernel gave up; the step's results are invalid */
 };
 
+/* the three tables a request for rows can name (gear_fetch_rows, gear_apply_emb_grad) */
+enum { GEAR_TABLE_USER = 0, GEAR_TABLE_URL = 1, GEAR_TABLE_DFV = 2 };
+
 /* tags of the procedural table fill (SplitMix64 streams, see gear_fill_uniform) */
 enum { GEAR_TAG_USER = 1, GEAR_TAG_URL = 2, GEAR_TAG_DFV = 3, GEAR_TAG_TS = 4, GEAR_TAG_GRAD = 5 };
 
@@ -157,6 +160,9 @@ typedef struct {
     int32_t* row_view;  /* [nnz] view index of every image occurrence (the src_row of accumulate); optional */
     float*   inv_n;     /* [B]   1/n_b, the mean-pool weight (the scale of accumulate); optional */
     void*  x_debug;     /* [B][2*emb_dim + dfv_dim] copy of the head input in head_dtype; optional */
+    float* dfv_grad;    /* [nnz][dfv_dim] optional: event 5 in its materialised form, one gradient row per image
+                           occurrence (view-major, slot-minor): dX[view][2*emb_dim ..] * 1/n_view.  Needs row_view and
+                           inv_n.  These are the rows a worker sends to the owners of the images */
     float* user_grad;   /* [user_vocab][emb_dim] optional: the summed embedding gradient is ADDED here and the */
     float* url_grad;    /* [url_vocab][emb_dim]  table is left untouched (both or neither) */
     /* Optional: Section 4's optimiser for the embedding tables in place of the plain scaled scatter (adam != NULL; not
@@ -259,6 +265,25 @@ int gear_collect_expired(gear_ctx* ctx, int64_t now, int restamp, int32_t* ids, 
  */
 int gear_refresh_dfv(gear_ctx* ctx, const int32_t* ids, const float* rows, int64_t ld, int64_t n,
                      const int64_t* d_n, int64_t now, void* stream);
+
+/*
+ * Tables partitioned by ID across devices (Section 3: the Slowgear Workers serve the Fastgear Workers' requests "by
+ * partition of Image ID"; Section 4 runs N of each).  The exchange itself is the caller's (any all-to-all); these two
+ * calls are what the owner of a table shard does with what arrives.
+ *
+ * gear_fetch_rows      event 3, the owner's answer to a request: out[k] = row ids[k] of table `which`
+ *                      (GEAR_TABLE_USER / URL: emb_dim fp32; GEAR_TABLE_DFV: dfv_dim values in dfv_dtype), k < n, dense,
+ *                      bit-exact copies; an ID outside the table gives a zero row and raises GEAR_DEV_BAD_ID.
+ *                      out: device, 16-byte aligned.
+ * gear_apply_emb_grad  event 4's push, at the owner: table[id] -= lr * (sum of the rows[k], k < n, with ids[k] == id) for
+ *                      `which` = GEAR_TABLE_USER or GEAR_TABLE_URL; rows fp32 [n][ld >= emb_dim], 16-byte aligned, ld a
+ *                      multiple of 4; n <= max_batch.  What gear_forward_backward does with its own batch's rows.
+ * Gradient rows for the image store arrive the same way and go to gear_accumulate_dfv_grad / gear_accumulate_collect
+ * with explicit img_id (rows are taken to arrive in index order: sender by sender, each in its own row order).
+ */
+int gear_fetch_rows(gear_ctx* ctx, int32_t which, const int32_t* ids, int64_t n, void* out, void* stream);
+int gear_apply_emb_grad(gear_ctx* ctx, int32_t which, const int32_t* ids, const float* rows, int64_t ld, int64_t n,
+                        float lr, void* stream);
 
 /*
  * The smallest Dense Part there is, for closing the loop on one device: DFV[id] = raw[id] . Wd, with raw

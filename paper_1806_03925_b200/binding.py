@@ -21,12 +21,13 @@ GEAR_F32, GEAR_BF16 = 0, 1
 GEAR_ACC_SORT, GEAR_ACC_ATOMIC = 0, 1
 GEAR_DEV_BAD_ID, GEAR_DEV_READY_OVERFLOW, GEAR_DEV_OUT_CAPACITY, GEAR_DEV_BAD_CSR = 1, 2, 4, 8
 GEAR_TAG_USER, GEAR_TAG_URL, GEAR_TAG_DFV, GEAR_TAG_TS, GEAR_TAG_GRAD = 1, 2, 3, 4, 5
+GEAR_TABLE_USER, GEAR_TABLE_URL, GEAR_TABLE_DFV = 0, 1, 2
 
 EXPORTS = ("gear_workspace_bytes", "gear_init_tables", "gear_forward_backward", "gear_accumulate_dfv_grad",
            "gear_collect_ready", "gear_collect_expired", "gear_status", "gear_destroy", "gear_fill_uniform",
            "gear_last_error", "gear_profile_enable", "gear_profile_read", "gear_launch_count",
            "gear_collect_expired_static", "gear_refresh_dfv", "gear_accumulate_collect", "gear_dense_forward",
-           "gear_dense_backward", "gear_adam_dense")
+           "gear_dense_backward", "gear_adam_dense", "gear_fetch_rows", "gear_apply_emb_grad")
 GEAR_STATIC_EXPIRY_MAX_VOCAB = 16777216
 
 
@@ -60,7 +61,7 @@ class gear_adam(C.Structure):
 
 class gear_step_out(C.Structure):
     _fields_ = [("loss", C.c_void_p), ("prob", C.c_void_p), ("head_grad", C.c_void_p), ("dX", C.c_void_p),
-                ("row_view", C.c_void_p), ("inv_n", C.c_void_p), ("x_debug", C.c_void_p),
+                ("row_view", C.c_void_p), ("inv_n", C.c_void_p), ("x_debug", C.c_void_p), ("dfv_grad", C.c_void_p),
                 ("user_grad", C.c_void_p), ("url_grad", C.c_void_p),
                 ("adam", C.POINTER(gear_adam)), ("adam_step", C.c_int64),
                 ("user_m", C.c_void_p), ("user_v", C.c_void_p), ("url_m", C.c_void_p), ("url_v", C.c_void_p)]
@@ -92,6 +93,10 @@ def load() -> C.CDLL:
     L.gear_collect_ready.argtypes = [vp, vp, vp, vp, i64, vp, C.POINTER(i64), vp]
     L.gear_accumulate_collect.restype = C.c_int
     L.gear_accumulate_collect.argtypes = [vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, i64, vp, C.POINTER(i64), vp]
+    L.gear_fetch_rows.restype = C.c_int
+    L.gear_fetch_rows.argtypes = [vp, i32, vp, i64, vp, vp]
+    L.gear_apply_emb_grad.restype = C.c_int
+    L.gear_apply_emb_grad.argtypes = [vp, i32, vp, vp, i64, i64, C.c_float, vp]
     L.gear_dense_forward.restype = C.c_int
     L.gear_dense_forward.argtypes = [vp, vp, i32, vp, vp, i64, vp, vp, i64, vp]
     L.gear_dense_backward.restype = C.c_int
@@ -204,10 +209,11 @@ def make_adam(lr: float = 1e-4, beta1: float = 0.9, beta2: float = 0.999, eps: f
 
 def make_step_out(loss, head_grad, dX, prob=None, row_view=None, inv_n=None, x_debug=None, user_grad=None,
                   url_grad=None, adam: Optional[gear_adam] = None, adam_step: int = 0, user_m=None, user_v=None,
-                  url_m=None, url_v=None) -> gear_step_out:
+                  url_m=None, url_v=None, dfv_grad=None) -> gear_step_out:
     o = gear_step_out()
     for name, t in (("loss", loss), ("prob", prob), ("head_grad", head_grad), ("dX", dX), ("row_view", row_view),
                     ("inv_n", inv_n), ("x_debug", x_debug), ("user_grad", user_grad), ("url_grad", url_grad),
+                    ("dfv_grad", dfv_grad),
                     ("user_m", user_m), ("user_v", user_v), ("url_m", url_m), ("url_v", url_v)):
         setattr(o, name, None if t is None else _p(t).value)
     if adam is not None:
@@ -269,6 +275,18 @@ def gear_refresh_dfv(ctx, ids, rows, n: int, now: int, d_n=None, stream=None):
     assert rows.is_cuda and rows.dtype == torch.float32 and rows.dim() == 2 and rows.stride(1) == 1
     _check(load().gear_refresh_dfv(ctx, _p(ids), C.c_void_p(rows.data_ptr()), rows.stride(0), n, _p(d_n), now, _stream(stream)),
            "gear_refresh_dfv")
+
+
+def gear_fetch_rows(ctx, which: int, ids, n: int, out, stream=None):
+    """out[k] = row ids[k] of table `which` (bit-exact copies, the table's storage type), k < n."""
+    _check(load().gear_fetch_rows(ctx, which, _p(ids), n, _p(out), _stream(stream)), "gear_fetch_rows")
+
+
+def gear_apply_emb_grad(ctx, which: int, ids, rows, n: int, lr: float, stream=None):
+    """table[id] -= lr * sum of the rows that carry id (rows fp32 [>= n][ld])."""
+    assert rows.dtype == torch.float32 and rows.stride(1) == 1
+    _check(load().gear_apply_emb_grad(ctx, which, _p(ids), C.c_void_p(rows.data_ptr()), rows.stride(0), n, lr,
+                                      _stream(stream)), "gear_apply_emb_grad")
 
 
 def gear_dense_forward(ctx, raw, Wd, ids, n: int, rows, d_n=None, stream=None):

@@ -232,6 +232,8 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     }
     if (c.cfg.head_dtype == GEAR_BF16 && (!aligned16(o.head_grad) || !aligned16(c.buf.head_params)))
         return arg_fail("bf16 head: head_params and head_grad must be 16-byte aligned");
+    if (o.dfv_grad && (!o.row_view || !o.inv_n || !aligned16(o.dfv_grad)))
+        return arg_fail("dfv_grad needs row_view and inv_n and 16-byte alignment");
     if (!aligned16(o.dX) || (o.x_debug && !aligned16(o.x_debug)) || (o.user_grad && !aligned16(o.user_grad)) ||
         (o.url_grad && !aligned16(o.url_grad)))
         return arg_fail("dX, x_debug, user_grad, url_grad must be 16-byte aligned");
@@ -339,6 +341,10 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     const HeadHooks hooks{weights_on_side, scatter, &sc};
     e = launch_head_simt(c, b, o, st, hooks);
     if (e != cudaSuccess) return abandon(e, "head");
+    if (o.dfv_grad && b.B > 0) {
+        e = launch_dfv_grad_rows(c, o.dX, o.row_view, o.inv_n, b.nnz, o.dfv_grad, st);
+        if (e != cudaSuccess) return abandon(e, "gradient rows");
+    }
     if (forked) {
         e = cudaEventRecord(c.ev_join, c.side_stream);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c.ev_join, 0);
@@ -458,6 +464,33 @@ int gear_refresh_dfv(gear_ctx* ctx, const int32_t* ids, const float* rows, int64
     cudaError_t e = launch_refresh_dfv(c, ids, rows, ld, n, d_n, now, st);
     if (e != cudaSuccess) return cuda_fail(e, "refresh_dfv");
     return GEAR_OK;
+}
+
+int gear_fetch_rows(gear_ctx* ctx, int32_t which, const int32_t* ids, int64_t n, void* out, void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (which != GEAR_TABLE_USER && which != GEAR_TABLE_URL && which != GEAR_TABLE_DFV) return arg_fail("which");
+    if (n < 0) return arg_fail("n < 0");
+    if (n == 0) return GEAR_OK;
+    if (!ids || !out || !aligned16(out)) return arg_fail("NULL or misaligned pointer");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.note_stream(st);
+    cudaError_t e = launch_fetch_rows(c, which, ids, n, out, st);
+    return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "fetch_rows");
+}
+
+int gear_apply_emb_grad(gear_ctx* ctx, int32_t which, const int32_t* ids, const float* rows, int64_t ld, int64_t n, float lr,
+                        void* stream) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    gear_ctx_impl& c = ctx->impl;
+    if (which != GEAR_TABLE_USER && which != GEAR_TABLE_URL) return arg_fail("which: GEAR_TABLE_USER or GEAR_TABLE_URL");
+    if (n < 0 || n > c.cfg.max_batch) return arg_fail("n outside [0, max_batch]");
+    if (n == 0) return GEAR_OK;
+    if (!ids || !rows || !aligned16(rows) || ld < c.cfg.emb_dim || (ld & 3)) return arg_fail("rows: 16-byte aligned, ld >= emb_dim, multiple of 4");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    c.last_stream = st;
+    cudaError_t e = launch_apply_emb_grad(c, which, ids, rows, ld, n, -lr, st);
+    return e == cudaSuccess ? GEAR_OK : cuda_fail(e, "apply_emb_grad");
 }
 
 int gear_dense_forward(gear_ctx* ctx, const float* raw, int32_t raw_dim, const float* Wd, const int32_t* ids, int64_t n,

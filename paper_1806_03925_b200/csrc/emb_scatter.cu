@@ -150,3 +150,40 @@ cudaError_t launch_emb_adam(const gear_ctx_impl& c, int cur, int32_t B, const fl
 }
 
 }  // namespace gear
+
+namespace gear {
+
+// The owner of a table shard applies gradient rows that arrive with their IDs (from its own step or from other devices):
+// stable key sort of the IDs, then the segmented sum and scatter above on that one table.
+cudaError_t launch_apply_emb_grad(const gear_ctx_impl& c, int which, const int32_t* ids, const float* rows, int64_t ld,
+                                  int64_t n, float alpha, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    const bool user = which == GEAR_TABLE_USER;
+    const int64_t vocab = user ? c.cfg.user_vocab : c.cfg.url_vocab;
+    SortBatch batch = c.sort_batch();
+    batch.n_jobs = 1;
+    batch.job[0] = c.sort_job(user ? gear_ctx_impl::SORT_USER : gear_ctx_impl::SORT_URL);
+    batch.job[0].ids = ids; batch.job[0].sentinel = (uint32_t)vocab;
+    batch.job[0].n_max = n; batch.job[0].bits = bits_for(vocab);
+    batch.name = "sort_emb";
+    cudaError_t se;
+    const int cur = sort_jobs(batch, &c.gbs, st, &c.prof, &se);
+    if (se != cudaSuccess) return se;
+    const int E = c.cfg.emb_dim, n_chunks = E / 4;
+    int lpr = 1;
+    while (lpr < n_chunks && lpr < 32) lpr <<= 1;
+    const int nq = (int)ceil_div(n_chunks, lpr);
+    const int64_t groups = ceil_div(n, ES_SEG);
+    const dim3 grid((unsigned)ceil_div(groups * lpr, 256), 1);
+    const EmbTable t0{batch.job[0].keys[cur], batch.job[0].vals[cur], (uint32_t)vocab, 0, user ? c.buf.user_emb : c.buf.url_emb};
+#define GEAR_ES_LAUNCH(NQ) launch_dependent(emb_reduce_kernel<NQ, false>, grid, dim3(256), 0, st, t0, t0, (int)n, E, lpr, rows, ld, alpha)
+    KernelScope ks(&c.prof, "emb_reduce", st);
+    if (nq <= 1) GEAR_ES_LAUNCH(1);
+    else if (nq <= 2) GEAR_ES_LAUNCH(2);
+    else if (nq <= 4) GEAR_ES_LAUNCH(4);
+    else GEAR_ES_LAUNCH(8);
+#undef GEAR_ES_LAUNCH
+    return cudaGetLastError();
+}
+
+}  // namespace gear

@@ -156,6 +156,14 @@ cudaError_t launch_emb_adam_rows(const gear_ctx_impl& c, const EmbAdamTable& t0,
 cudaError_t launch_emb_adam(const gear_ctx_impl& c, int buf, int32_t B, const float* dX, int ldx, const gear_adam& cfg,
                             int64_t t, float* user_m, float* user_v, float* url_m, float* url_v, cudaStream_t st);
 
+// shard.cu: row fetch for a table shard's owner; event 5's gradient rows in materialised form
+cudaError_t launch_fetch_rows(const gear_ctx_impl& c, int which, const int32_t* ids, int64_t n, void* out, cudaStream_t st);
+cudaError_t launch_dfv_grad_rows(const gear_ctx_impl& c, const float* dX, const int32_t* row_view, const float* inv_n,
+                                 int64_t nnz, float* out, cudaStream_t st);
+// emb_scatter.cu: table[id] += alpha * (sum of the rows with that id), ids given explicitly (sorted here)
+cudaError_t launch_apply_emb_grad(const gear_ctx_impl& c, int which, const int32_t* ids, const float* rows, int64_t ld,
+                                  int64_t n, float alpha, cudaStream_t st);
+
 // accumulate.cu
 // img_id == nullptr: use the image IDs sorted by the last gear_forward_backward (buffer set SORT_IMG)
 cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,

@@ -87,6 +87,8 @@ class GearSession:
         self.inv_n = torch.zeros(B, dtype=torch.float32, device=dev)
         self.x_debug = (torch.zeros((B, self.d_in), dtype=torch.bfloat16 if p.head_dtype == BF16 else torch.float32,
                                     device=dev) if want_debug else None)
+        # event 5's rows in materialised form (what a worker would send to the owners of the images); with want_debug
+        self.dfv_grad = torch.zeros((nnz, p.dfv_dim), dtype=torch.float32, device=dev) if want_debug else None
         self.user_grad = torch.zeros_like(self.user_emb) if want_emb_grad else None
         self.url_grad = torch.zeros_like(self.url_emb) if want_emb_grad else None
         # Section 4's optimiser for the embedding tables: first and second moments per table row
@@ -117,7 +119,7 @@ class GearSession:
         if self._step_out is None:
             self._step_out = gb.make_step_out(self.loss, self.head_grad, self.dX, prob=self.prob, row_view=self.row_view,
                                               inv_n=self.inv_n, x_debug=self.x_debug, user_grad=self.user_grad,
-                                              url_grad=self.url_grad, adam=self.adam, user_m=self.user_m,
+                                              url_grad=self.url_grad, dfv_grad=self.dfv_grad, adam=self.adam, user_m=self.user_m,
                                               user_v=self.user_v, url_m=self.url_m, url_v=self.url_v)
         if self.adam is not None:
             self.adam_step += 1

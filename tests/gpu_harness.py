@@ -191,6 +191,8 @@ class Pair:
         assert np.array_equal(_np(gpu.row_view[:b.nnz]), view_of), "row_view"
         inv = np.where(n_b > 0, 1.0 / np.maximum(n_b, 1), 0.0)
         assert_close(_np(gpu.inv_n[:B]), inv, 1e-7, "inv_n")
+        # event 5 in its materialised form: one gradient row per image occurrence
+        assert_close(_np(gpu.dfv_grad[:b.nnz]), cpu.dfv_grad_rows(b.img_off, r.dX), tol, "DFV gradient rows")
 
         # embedding gradients / in-place update
         if self.want_emb_grad:

@@ -716,3 +716,89 @@ def test_adam_on_the_embedding_rows_and_the_head(gb, name):
         assert g.status()[1] == 0
     finally:
         g.close()
+
+
+# ------------------------------------------------------------------ tables partitioned by ID over several ranks
+@pytest.mark.parametrize("name,world", [("tiny", 2), ("tiny", 3), ("medium", 2)])
+def test_step_with_tables_partitioned_by_id(gb, name, world):
+    """Every rank holds the table rows whose ID is congruent to its rank and works on its own page views: IDs travel
+    to the owners, rows come back, gradient rows travel to the owners (paper, Section 3: "by partition of Image ID").
+    All ranks run in this process, one after the other, over an in-process exchange (no kernel of one rank waits for
+    another's), and the result is compared with the oracle doing the same thing on whole tables: every worker's
+    forward and backward pass on the tables as they stood at the start of the step, then all embedding gradients
+    applied, then all (Image ID, gradient) pairs fed to the store rank by rank in row order.  Two steps."""
+    from gpu_harness import _np, assert_close, tol_of
+    from oracle import GearOracle
+    from paper_1806_03925_b200.sharded import LoopbackExchange, ShardedGear
+    p = PRESETS[name].scaled(user_vocab=1501, url_vocab=1200, img_vocab=2003, batch=700, expire=3)
+    tol = tol_of(p)
+    dfv_np = np.uint16 if p.dfv_dtype == BF16 else np.float32
+    tables = dict(user_emb=oracle.fill_rows(2, oracle.TAG_USER, p.emb_dim, None, p.user_vocab, np.float32),
+                  url_emb=oracle.fill_rows(2, oracle.TAG_URL, p.emb_dim, None, p.url_vocab, np.float32),
+                  dfv=oracle.fill_rows(2, oracle.TAG_DFV, p.dfv_dim, None, p.img_vocab, dfv_np),
+                  ts=oracle.fill_ts(2, p.expire, 0, None, p.img_vocab))
+    params = workloads.head_params(p, 2)
+    src = BatchSource(p, 2)
+    # rank r takes batches r, world + r, ... ; the ranks' batches differ in size
+    sizes = [p.batch - 37 * r for r in range(world)]
+    steps = [[src.batch(s * world + r, sizes[r]) for r in range(world)] for s in range(2)]
+    sg = ShardedGear(p, params, LoopbackExchange(world), max_batch_local=p.batch, max_nnz_local=p.batch * p.img_hi,
+                     tables=tables)
+    cpu = GearOracle(tables["user_emb"].copy(), tables["url_emb"].copy(), tables["dfv"].copy(), p.hidden, p.M, p.expire,
+                     round_bf16=(p.head_dtype == BF16), ts=tables["ts"].copy())
+
+    def gather_shards(attr):
+        out = None
+        for r, ow in enumerate(sg.owners):
+            t = _np(getattr(ow, attr))
+            if out is None:
+                out = np.zeros((getattr(p, {"user_emb": "user_vocab", "url_emb": "url_vocab"}.get(attr, "img_vocab")),) + t.shape[1:], t.dtype)
+            out[r::world] = t
+        return out
+    try:
+        for s, batches in enumerate(steps):
+            now = s + 1
+            out = sg.step(batches, now, mean_head_grad=False)
+            res = [cpu.forward_backward(params.astype(np.float64), b.user_id, b.url_id, b.img_off, b.img_id, b.label)
+                   for b in batches]
+            for wk, b, r in zip(sg.workers, batches, res):
+                assert_close(_np(wk.loss), [r.loss], tol, "loss")
+                assert_close(_np(wk.prob[:b.B]), r.prob, tol, "prob")
+                assert_close(_np(wk.dX[:b.B]), r.dX, tol, "dX")
+                assert_close(_np(wk.head_grad), r.head_grad, tol, "head_grad")
+            uid = np.concatenate([b.user_id for b in batches]); hid = np.concatenate([b.url_id for b in batches])
+            dX = np.concatenate([r.dX for r in res])
+            cpu.emb_apply("user", uid, dX, -p.lr)
+            cpu.emb_apply("url", hid, dX, -p.lr)
+            assert_close(gather_shards("user_emb"), cpu.user_emb, tol, "user table")
+            assert_close(gather_shards("url_emb"), cpu.url_emb, tol, "url table")
+            img = np.concatenate([b.img_id for b in batches])
+            rows = np.concatenate([cpu.dfv_grad_rows(b.img_off, r.dX) for b, r in zip(batches, res)])
+            cpu.accumulate(img, rows)
+            assert np.array_equal(gather_shards("dfv_gcnt"), cpu.gcnt), "open-group counts"
+            assert_close(gather_shards("dfv_gsum"), cpu.gsum, tol, "open-group sums")
+            eid, eseq, eavg = oracle.sort_emissions(*cpu.collect_ready())
+            got = []
+            for r, (ow, (n_ready, _)) in enumerate(zip(sg.owners, out)):
+                got.append((_np(ow.ready_ids[:n_ready]).astype(np.int64) * world + r, _np(ow.ready_seq[:n_ready]),
+                            _np(ow.ready_avg[:n_ready])))
+            gid = np.concatenate([g[0] for g in got]); gseq = np.concatenate([g[1] for g in got])
+            gavg = np.concatenate([g[2] for g in got])
+            order = np.lexsort((gseq, gid))
+            assert np.array_equal(gid[order], eid) and np.array_equal(gseq[order], eseq), "emitted (id, seq) pairs"
+            assert_close(gavg[order], eavg, tol, "averaged gradients")
+            want_exp = cpu.collect_expired(now, True)
+            got_exp = np.sort(np.concatenate([_np(ow.expired_ids[:n_exp]).astype(np.int64) * world + r
+                                              for r, (ow, (_, n_exp)) in enumerate(zip(sg.owners, out))]))
+            assert np.array_equal(got_exp, want_exp), "expired ids"
+            assert np.array_equal(gather_shards("dfv_ts"), cpu.ts)
+        assert sum(n for n, _ in out) > 0
+        for s_ in sg.owners + sg.workers:
+            assert s_.status()[1] == 0
+        # the head's gradient averaged over the ranks, as the collective would leave it on every rank
+        want = np.mean([r.head_grad for r in res], axis=0)
+        sg.ex.mean_over_ranks([wk.head_grad for wk in sg.workers])
+        for wk in sg.workers:
+            assert_close(_np(wk.head_grad), want, tol, "head_grad, mean over the ranks")
+    finally:
+        sg.close()
