@@ -625,6 +625,78 @@ def run_accumulate_cases(args, which):
         print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------------------
+# tables partitioned by ID over the ranks (opt-in; the default multi-GPU arm runs independent replicas)
+# ---------------------------------------------------------------------------------------------
+def run_sharded(args):
+    """Every rank owns the table rows whose ID is congruent to its rank and works on its own batch of the workload's
+    size; IDs, rows and gradient rows cross between the ranks by all-to-all (NCCL).  A step includes the host->device
+    copy of the batch's ID arrays, so the one figure reported is an end-to-end one."""
+    import torch
+    from paper_1806_03925_b200 import binding as gb, workloads
+    from paper_1806_03925_b200.replicas import Replicas
+    from paper_1806_03925_b200.sharded import DistExchange, ShardedGear
+    from paper_1806_03925_b200.workloads import BatchSource
+    reps = Replicas.from_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libgear has no CPU path")
+    torch.cuda.set_device(reps.local_rank)
+    reps.init("nccl", torch.device("cuda", reps.local_rank))
+    gb.load()
+    p = preset_for(args.workload)
+    K, W = args.steps, max(args.warmup, 3)
+    sampler = ClockSampler(reps.local_rank)
+    sampler.start()
+    src = BatchSource(p, reps.rank)
+    batches = [src.batch(s) for s in range(N_BATCHES)]
+    sg = ShardedGear(p, workloads.head_params(p, 0), DistExchange(reps.rank, reps.world), max_batch_local=p.batch,
+                     max_nnz_local=max(b.nnz for b in batches), seed=0)
+    stream = torch.cuda.current_stream()
+    now = [0]
+
+    def one(s):
+        now[0] += 1
+        sg.step([batches[s % N_BATCHES]], now[0])
+
+    for s in range(W):
+        one(s)
+    launches0 = sum(gb.gear_launch_count(x.ctx) for x in sg.owners + sg.workers)
+    region_ms = []
+    sampler.open_window()
+    while (sum(region_ms) < MIN_TIMED_MS or len(region_ms) < 3) and len(region_ms) < MAX_REGIONS:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(); reps.barrier(); torch.cuda.synchronize()
+        ev0.record(stream)
+        for s in range(K):
+            one(s)
+        ev1.record(stream)
+        torch.cuda.synchronize(); reps.barrier(); torch.cuda.synchronize()
+        region_ms.append(reps.max_over_ranks(ev0.elapsed_time(ev1), device="cuda"))
+    sampler.close_window()
+    launches = (sum(gb.gear_launch_count(x.ctx) for x in sg.owners + sg.workers) - launches0) / len(region_ms)
+    ms = float(np.median(region_ms))
+    h2d = int(np.mean([b.user_id.nbytes + b.url_id.nbytes + b.img_id.nbytes + b.img_off.nbytes + b.label.nbytes for b in batches]))
+    value = round(reps.whole_job_rate(p.batch * K, ms), 1)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": reps.world, "steps": K, "warmup": W,
+            "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if p.head_dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": "large tables" if p.name == "large" else p.name, "batch": p.batch,
+                       "parallelism": "tables partitioned by ID over %d ranks, a batch per rank, three all-to-all "
+                                      "exchanges per table and step" % reps.world,
+                       "l2": "tables far exceed the 126 MB L2; %d pre-generated batches cycle" % N_BATCHES},
+            "regions": {"regions": len(region_ms), "min_ms_per_step": round(min(region_ms) / K, 4),
+                        "max_ms_per_step": round(max(region_ms) / K, 4)},
+            "clocks": sampler.stop(), "gpu_launches": int(launches),
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 16,
+                    "note": "the timed step itself copies the batch in and reads the two counts back"},
+            "roofline": None, "cpu_baseline": None,
+            "device_status": [x.status()[1] for x in sg.owners + sg.workers]}
+    if reps.rank == 0:
+        print(json.dumps(line), flush=True)
+    sg.close()
+    reps.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -636,6 +708,9 @@ def main():
                          "micro-benchmark, one line per case.  skew: the skew-stress step.  skew_modes: its accumulate call, "
                          "sort against atomics, M in {1, 64, 1024}, one line per case")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sharded", action="store_true",
+                    help="tables partitioned by ID over the ranks instead of independent replicas (not the default: this "
+                         "arm has only ever run on one GPU)")
     args = ap.parse_args()
     # defaults: a few hundred milliseconds of device time per timed region for the CUDA path (so that the
     # clock sampler sees it), a couple of minutes of host time for the CPU oracle
@@ -649,6 +724,10 @@ def main():
         if args.workload in ("micro", "skew_modes"):
             raise SystemExit("the reference arm times the whole step: use --workload large, medium, tiny or skew")
         run_reference(args)
+    elif args.sharded:
+        if args.steps == 400:
+            args.steps = 50
+        run_sharded(args)
     elif args.workload in ("micro", "skew_modes"):
         if args.steps == 400:
             args.steps = 7

@@ -117,6 +117,9 @@ typedef struct {
                               0 = max_nnz, which can never overflow if every accumulate call is
                               followed by a collect */
     int32_t accum_mode;    /* GEAR_ACC_SORT | GEAR_ACC_ATOMIC */
+    int32_t fast_dim;      /* columns of dense input the Fastgear side brings along per view (Section 4: the part of the
+                              image that is fed to the Fastgear Worker directly), appended to the head input after the
+                              pooled DFV; 0 = none; multiple of 8, <= 4096 */
 } gear_config;
 
 /* Caller-owned device buffers that persist across calls. */
@@ -147,6 +150,7 @@ typedef struct {
     const int32_t* img_off;    /* [B+1] img_off[0] = 0, non-decreasing, img_off[B] = nnz */
     const int32_t* img_id;     /* [nnz] view-major, slot-minor */
     const float*   label;      /* [B]  0 or 1 */
+    const float*   fast;       /* [B][fast_dim] fp32, 16-byte aligned: the views' own dense input; NULL when fast_dim = 0 */
 } gear_batch;
 
 /* Outputs of one step; device pointers.  "optional" ones may be NULL. */
@@ -154,12 +158,12 @@ typedef struct {
     float* loss;        /* [1]  mean binary cross-entropy over the batch */
     float* prob;        /* [B]  sigmoid of the logit; optional */
     float* head_grad;   /* packed like head_params: dLoss/dparams (not applied by the library) */
-    float* dX;          /* [B][2*emb_dim + dfv_dim] dLoss/d(head input).  Columns [2*emb_dim, ...) are
-                           dLoss/d(pooled DFV) of each view: pass dX + 2*emb_dim with ld = 2*emb_dim + dfv_dim
-                           to gear_accumulate_dfv_grad */
+    float* dX;          /* [B][d_in] dLoss/d(head input), d_in = 2*emb_dim + dfv_dim + fast_dim.  Columns
+                           [2*emb_dim, 2*emb_dim + dfv_dim) are dLoss/d(pooled DFV) of each view: pass dX + 2*emb_dim
+                           with ld = d_in to gear_accumulate_dfv_grad */
     int32_t* row_view;  /* [nnz] view index of every image occurrence (the src_row of accumulate); optional */
     float*   inv_n;     /* [B]   1/n_b, the mean-pool weight (the scale of accumulate); optional */
-    void*  x_debug;     /* [B][2*emb_dim + dfv_dim] copy of the head input in head_dtype; optional */
+    void*  x_debug;     /* [B][d_in] copy of the head input in head_dtype; optional */
     float* dfv_grad;    /* [nnz][dfv_dim] optional: event 5 in its materialised form, one gradient row per image
                            occurrence (view-major, slot-minor): dX[view][2*emb_dim ..] * 1/n_view.  Needs row_view and
                            inv_n.  These are the rows a worker sends to the owners of the images */
@@ -190,8 +194,8 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
                      uint64_t seed, int fill, int64_t now, void* stream);
 
 /*
- * Events 1, 3, 4.  X[b] = [user_emb[user_id[b]] | url_emb[url_id[b]] | mean_j DFV[img_id[j]]] (fp32 sum
- * in slot order, divided by n_b; zeros for n_b = 0); hidden layers h = ReLU(h W + b); z = h . w_out + b_out;
+ * Events 1, 3, 4.  X[b] = [user_emb[user_id[b]] | url_emb[url_id[b]] | mean_j DFV[img_id[j]] | fast[b]] (fp32 sum
+ * in slot order, divided by n_b; zeros for n_b = 0; the last part only when fast_dim > 0); hidden layers h = ReLU(h W + b); z = h . w_out + b_out;
  * p = sigmoid(z); loss = mean_b BCE(p_b, label_b).  Backward yields head_grad and dX.  Then, per
  * embedding table, rows of views sharing an ID are summed and table[id] -= lr * sum (or the sums are
  * added to user_grad / url_grad when those are given).

@@ -41,7 +41,7 @@ def build(force: bool = False) -> str:
 class _Model(C.Structure):
     _fields_ = [("user_vocab", C.c_int64), ("url_vocab", C.c_int64), ("img_vocab", C.c_int64),
                 ("emb_dim", C.c_int32), ("dfv_dim", C.c_int32), ("n_hidden", C.c_int32),
-                ("hidden", C.c_int32 * 2), ("round_bf16", C.c_int32)]
+                ("hidden", C.c_int32 * 2), ("round_bf16", C.c_int32), ("fast_dim", C.c_int32)]
 
 
 _lib = None
@@ -66,7 +66,7 @@ def lib():
         L.orc_head_param_count.argtypes = [C.POINTER(_Model)]
         L.orc_forward_backward.restype = i64
         L.orc_forward_backward.argtypes = [C.POINTER(_Model), vp, C.c_int, vp, C.c_int, vp, C.c_int, vp,
-                                           i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                           i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                            dbl, dbl, vp, vp, i64, vp, vp, i64]
         L.orc_emb_apply.restype = i64
         L.orc_emb_apply.argtypes = [vp, C.c_int, i64, i32, vp, i32, vp, i32, i32, dbl, vp]
@@ -164,7 +164,7 @@ class GearOracle:
 
     def __init__(self, user_emb: np.ndarray, url_emb: np.ndarray, dfv: np.ndarray,
                  hidden: Sequence[int], M: int, expire: int, round_bf16: bool = False,
-                 ts: Optional[np.ndarray] = None):
+                 ts: Optional[np.ndarray] = None, fast_dim: int = 0):
         """ts may be longer than the DFV table: a test that keeps only the touched rows of a huge
         table still scans every timestamp."""
         self.user_emb = np.ascontiguousarray(user_emb)
@@ -183,8 +183,9 @@ class GearOracle:
         for i, h in enumerate(self.hidden):
             m.hidden[i] = h
         m.round_bf16 = 1 if round_bf16 else 0
+        m.fast_dim = self.F = int(fast_dim)
         self.model = m
-        self.d_in = 2 * self.E + self.D
+        self.d_in = 2 * self.E + self.D + self.F
         self.n_params = int(lib().orc_head_param_count(C.byref(m)))
         self.gsum = np.zeros((self.V, self.D), dtype=np.float64)
         self.gcnt = np.zeros(self.V, dtype=np.int32)
@@ -198,7 +199,7 @@ class GearOracle:
     def forward_backward(self, params: np.ndarray, user_id, url_id, img_off, img_id, label,
                          backward: bool = True, relu_margin: Optional[float] = None,
                          flip_units: Optional[Sequence[int]] = None, relu_margin_rel: float = 0.0,
-                         near_cap: int = 65536) -> StepResult:
+                         near_cap: int = 65536, fast: Optional[np.ndarray] = None) -> StepResult:
         """relu_margin / relu_margin_rel: list the hidden units whose pre-activation a has
         |a| <= relu_margin + relu_margin_rel * max|input row| * max|layer weights| (None: no list)."""
         B = int(len(user_id))
@@ -207,6 +208,10 @@ class GearOracle:
         uid, hid = _c(user_id, np.int32), _c(url_id, np.int32)
         off, img = _c(img_off, np.int32), _c(img_id, np.int32)
         y = _c(label, np.float64)
+        fast64 = None
+        if self.F:
+            fast64 = _c(fast, np.float64)
+            assert fast64.shape == (B, self.F)
         X = np.zeros((B, self.d_in), dtype=np.float64)
         prob = np.zeros(B, dtype=np.float64)
         loss = C.c_double(0.0)
@@ -219,7 +224,7 @@ class GearOracle:
         bad = lib().orc_forward_backward(
             C.byref(self.model), _ptr(self.user_emb), _dtype_tag(self.user_emb),
             _ptr(self.url_emb), _dtype_tag(self.url_emb), _ptr(self.dfv), _dtype_tag(self.dfv),
-            _ptr(params), B, _ptr(uid), _ptr(hid), _ptr(off), _ptr(img), _ptr(y),
+            _ptr(params), B, _ptr(uid), _ptr(hid), _ptr(off), _ptr(img), _ptr(y), _ptr(fast64),
             _ptr(X), _ptr(prob), C.byref(loss), _ptr(hg), _ptr(dX),
             0.0 if relu_margin is None else float(relu_margin), float(relu_margin_rel), _ptr(near), _ptr(near_abs),
             0 if near is None else len(near), C.byref(n_near), _ptr(flips), 0 if flips is None else len(flips))

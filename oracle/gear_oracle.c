@@ -67,6 +67,8 @@ typedef struct {
     int32_t n_hidden;      /* 1 or 2 hidden ReLU layers, then one logistic unit */
     int32_t hidden[2];
     int32_t round_bf16;    /* 1: operands of the head's matrix products are rounded to bfloat16 */
+    int32_t fast_dim;      /* dense input columns the Fastgear side brings along per view (Section 4: the part of
+                              the image fed to the Fastgear Worker directly); appended to the head input */
 } orc_model;
 
 /* ---------------------------------------------------------------- storage */
@@ -166,7 +168,7 @@ int orc_fill_ts(uint64_t seed, uint64_t tag, int64_t expire, int64_t now,
 /* ----------------------------------------------------------------- head */
 
 static int64_t head_param_count(const orc_model* m) {
-    int64_t n = 0, fan = 2 * m->emb_dim + m->dfv_dim;
+    int64_t n = 0, fan = 2 * m->emb_dim + m->dfv_dim + m->fast_dim;
     for (int l = 0; l < m->n_hidden; ++l) { n += fan * m->hidden[l] + m->hidden[l]; fan = m->hidden[l]; }
     return n + fan + 1;
 }
@@ -179,7 +181,8 @@ int64_t orc_head_param_count(const orc_model* m) { return head_param_count(m); }
  * Inputs : the three tables (storage type given per table), packed head
  *          parameters (doubles: per hidden layer W[in][out] then b[out]; then
  *          w_out[in], b_out), and the batch in CSR form.
- * Outputs: X[B][Din]   head input = [user row | url row | mean of the view's DFVs]
+ *          fast[B][fast_dim] (fast_dim > 0): dense input the view brings itself.
+ * Outputs: X[B][Din]   head input = [user row | url row | mean of the view's DFVs | fast row]
  *          prob[B]     sigmoid(z)
  *          *loss       mean binary cross-entropy
  *          head_grad   dLoss/dparams, packed like params
@@ -208,12 +211,13 @@ int64_t orc_forward_backward(const orc_model* m,
                              const double* params,
                              int32_t B, const int32_t* user_id, const int32_t* url_id,
                              const int32_t* img_off, const int32_t* img_id, const double* label,
+                             const double* fast,
                              double* X, double* prob, double* loss,
                              double* head_grad, double* dX,
                              double relu_margin, double relu_margin_rel, int64_t* near_units, double* near_abs,
                              int64_t near_cap, int64_t* n_near,
                              const int64_t* flip_units, int64_t n_flip) {
-    const int E = m->emb_dim, D = m->dfv_dim, Din = 2 * E + D;
+    const int E = m->emb_dim, D = m->dfv_dim, F = m->fast_dim, Din = 2 * E + D + F;
     const int L = m->n_hidden;
     const int rb = m->round_bf16;
     int64_t bad = 0;
@@ -261,6 +265,7 @@ int64_t orc_forward_backward(const orc_model* m,
             for (int c = 0; c < D; ++c) pool[c] += load_elem(dfv, dfv_dt, (int64_t)id * D + c);
         }
         if (n_b > 0) for (int c = 0; c < D; ++c) pool[c] /= (double)n_b;
+        for (int c = 0; c < F; ++c) x[2 * E + D + c] = fast[(int64_t)b * F + c];     /* the view's own dense input */
         if (rb) for (int c = 0; c < Din; ++c) x[c] = round_bf16(x[c]);
     }
 

@@ -41,7 +41,8 @@ class gear_config(C.Structure):
     _fields_ = [("user_vocab", C.c_int64), ("url_vocab", C.c_int64), ("img_vocab", C.c_int64),
                 ("emb_dim", C.c_int32), ("dfv_dim", C.c_int32), ("dfv_dtype", C.c_int32), ("head_dtype", C.c_int32),
                 ("n_hidden", C.c_int32), ("hidden", C.c_int32 * 2), ("M", C.c_int32), ("expire", C.c_int64),
-                ("max_batch", C.c_int32), ("max_nnz", C.c_int64), ("ready_cap", C.c_int64), ("accum_mode", C.c_int32)]
+                ("max_batch", C.c_int32), ("max_nnz", C.c_int64), ("ready_cap", C.c_int64), ("accum_mode", C.c_int32),
+                ("fast_dim", C.c_int32)]
 
 
 class gear_buffers(C.Structure):
@@ -52,7 +53,7 @@ class gear_buffers(C.Structure):
 
 class gear_batch(C.Structure):
     _fields_ = [("B", C.c_int32), ("nnz", C.c_int64), ("user_id", C.c_void_p), ("url_id", C.c_void_p),
-                ("img_off", C.c_void_p), ("img_id", C.c_void_p), ("label", C.c_void_p)]
+                ("img_off", C.c_void_p), ("img_id", C.c_void_p), ("label", C.c_void_p), ("fast", C.c_void_p)]
 
 
 class gear_adam(C.Structure):
@@ -150,7 +151,7 @@ def _stream(stream: Optional[torch.cuda.Stream]):
 
 
 def make_config(user_vocab, url_vocab, img_vocab, emb_dim, dfv_dim, dfv_dtype, head_dtype, hidden, M, expire,
-                max_batch, max_nnz, ready_cap=0, accum_mode=GEAR_ACC_SORT) -> gear_config:
+                max_batch, max_nnz, ready_cap=0, accum_mode=GEAR_ACC_SORT, fast_dim=0) -> gear_config:
     c = gear_config()
     c.user_vocab, c.url_vocab, c.img_vocab = user_vocab, url_vocab, img_vocab
     c.emb_dim, c.dfv_dim, c.dfv_dtype, c.head_dtype = emb_dim, dfv_dim, dfv_dtype, head_dtype
@@ -158,6 +159,7 @@ def make_config(user_vocab, url_vocab, img_vocab, emb_dim, dfv_dim, dfv_dtype, h
     for i, h in enumerate(hidden):
         c.hidden[i] = h
     c.M, c.expire, c.max_batch, c.max_nnz, c.ready_cap, c.accum_mode = M, expire, max_batch, max_nnz, ready_cap, accum_mode
+    c.fast_dim = fast_dim
     return c
 
 
@@ -192,13 +194,15 @@ def gear_init_tables(cfg: gear_config, user_emb, url_emb, dfv, dfv_gsum, dfv_gcn
     return ctx
 
 
-def make_batch(user_id, url_id, img_off, img_id, label, B: Optional[int] = None, nnz: Optional[int] = None) -> gear_batch:
+def make_batch(user_id, url_id, img_off, img_id, label, B: Optional[int] = None, nnz: Optional[int] = None,
+               fast=None) -> gear_batch:
     """The C struct of a batch whose arrays are device tensors (a caller that reuses the tensors may keep it)."""
     bt = gear_batch()
     bt.B = int(user_id.shape[0]) if B is None else B
     bt.nnz = int(img_id.shape[0]) if nnz is None else nnz
     bt.user_id, bt.url_id, bt.img_off = _p(user_id).value, _p(url_id).value, _p(img_off).value
     bt.img_id, bt.label = _p(img_id).value, _p(label).value
+    bt.fast = None if fast is None else _p(fast).value
     return bt
 
 

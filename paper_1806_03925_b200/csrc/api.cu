@@ -43,6 +43,7 @@ static int validate_config(const gear_config& c) {
     if (c.ready_cap < 0 || c.ready_cap > nmax) return arg_fail("ready_cap in [0, 2^30 - 1]");
     if (c.accum_mode != GEAR_ACC_SORT && c.accum_mode != GEAR_ACC_ATOMIC) return arg_fail("accum_mode");
     if (c.accum_mode == GEAR_ACC_ATOMIC && c.M >= (1 << 29)) return arg_fail("GEAR_ACC_ATOMIC needs M < 2^29");
+    if (c.fast_dim < 0 || c.fast_dim % 8 || c.fast_dim > 4096) return arg_fail("fast_dim: multiple of 8 in [0, 4096]");
     return GEAR_OK;
 }
 
@@ -51,7 +52,7 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
     const size_t hsz = c.head_dtype == GEAR_BF16 ? 2 : 4;
-    const int d_in = 2 * c.emb_dim + c.dfv_dim;
+    const int d_in = 2 * c.emb_dim + c.dfv_dim + c.fast_dim;
     const size_t B = (size_t)c.max_batch;
     p->ready_cap = c.ready_cap > 0 ? c.ready_cap : c.max_nnz;
     p->loss_blocks = (int)ceil_div(c.max_batch, 8);
@@ -97,7 +98,7 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
 }
 
 static int64_t param_count(const gear_config& c) {
-    int64_t n = 0, fan = 2 * c.emb_dim + c.dfv_dim;
+    int64_t n = 0, fan = 2 * c.emb_dim + c.dfv_dim + c.fast_dim;
     for (int l = 0; l < c.n_hidden; ++l) { n += fan * c.hidden[l] + c.hidden[l]; fan = c.hidden[l]; }
     return n + fan + 1;
 }
@@ -164,7 +165,7 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
     c.buf = *buf;
     plan_workspace(*cfg, &c.ws);
     if (buf->workspace_bytes < c.ws.total) { delete ctx; return arg_fail("workspace too small"); }
-    c.d_in = 2 * cfg->emb_dim + cfg->dfv_dim;
+    c.d_in = 2 * cfg->emb_dim + cfg->dfv_dim + cfg->fast_dim;
     c.n_params = param_count(*cfg);
     c.alive = true;
     c.tc_state = nullptr;
@@ -217,6 +218,7 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     if (b.nnz < 0 || b.nnz > c.cfg.max_nnz) return arg_fail("nnz outside [0, max_nnz]");
     if (b.B > 0 && (!b.user_id || !b.url_id || !b.img_off || !b.label)) return arg_fail("NULL batch array");
     if (b.nnz > 0 && !b.img_id) return arg_fail("NULL img_id");
+    if (b.B > 0 && c.cfg.fast_dim > 0 && (!b.fast || !aligned16(b.fast))) return arg_fail("fast: needed (16-byte aligned) when fast_dim > 0");
     if (!o.loss || !o.head_grad || !o.dX) return arg_fail("loss, head_grad and dX are required outputs");
     if ((o.user_grad == nullptr) != (o.url_grad == nullptr)) return arg_fail("user_grad and url_grad: both or neither");
     gear_adam adam_cfg = {0.f, 0.f, 0.f, 0.f};

@@ -63,7 +63,8 @@ __device__ __forceinline__ float div_by_count(float x, float nf, float rinv) {
 struct GatherArgs {
     const float* user_emb; const float* url_emb; const void* dfv;
     int64_t user_vocab, url_vocab, img_vocab;
-    int E, D, B;
+    int E, D, B, F;
+    const float* fast;          // [B][F] the views' own dense input (F > 0)
     int64_t nnz;
     const int32_t* user_id; const int32_t* url_id; const int32_t* img_off; const int32_t* img_id;
     void* X; void* x_debug;
@@ -138,7 +139,7 @@ gather_pool_kernel(const GatherArgs a) {
     constexpr int KMAX = NQ >= 8 ? 1 : 8 / NQ;               // rows in flight per warp
     const int lane = (int)lane_id();
     const int W = gridDim.x * GP_WARPS;
-    const int Din = 2 * a.E + a.D;
+    const int Din = 2 * a.E + a.D + a.F;
     const int n_chunks = a.D / PER;
     const int ce = a.E / 4;                                    // 16-byte chunks per embedding row
     const TD* __restrict__ dfv = static_cast<const TD*>(a.dfv);
@@ -249,6 +250,13 @@ gather_pool_kernel(const GatherArgs a) {
             }
         }
         if (a.inv_n && lane == 0) a.inv_n[b] = rinv;
+        // ---- the view's own dense input (the part of the image the Fastgear side keeps), eight columns per lane and pass
+        for (int c = lane * 8; c < a.F; c += 256) {
+            const float4 f0 = ld_stream_f4(a.fast + (int64_t)b * a.F + c), f1 = ld_stream_f4(a.fast + (int64_t)b * a.F + c + 4);
+            const float f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+            store_x<8>(x + 2 * a.E + a.D + c, f);
+            if (xd) store_x<8>(xd + 2 * a.E + a.D + c, f);
+        }
 
         cur = nxt; nxt = nxt2; ids_cur = ids_nxt;
     }
@@ -283,7 +291,7 @@ cudaError_t launch_gather(const gear_ctx_impl& c, const gear_batch& b, int32_t* 
     GatherArgs a;
     a.user_emb = c.buf.user_emb; a.url_emb = c.buf.url_emb; a.dfv = c.buf.dfv;
     a.user_vocab = c.cfg.user_vocab; a.url_vocab = c.cfg.url_vocab; a.img_vocab = c.cfg.img_vocab;
-    a.E = c.cfg.emb_dim; a.D = c.cfg.dfv_dim; a.B = b.B; a.nnz = b.nnz;
+    a.E = c.cfg.emb_dim; a.D = c.cfg.dfv_dim; a.B = b.B; a.nnz = b.nnz; a.F = c.cfg.fast_dim; a.fast = b.fast;
     a.user_id = b.user_id; a.url_id = b.url_id; a.img_off = b.img_off; a.img_id = b.img_id;
     a.X = c.at<void>(c.ws.x); a.x_debug = x_debug; a.row_view = row_view; a.inv_n = inv_n;
     a.state = c.state();

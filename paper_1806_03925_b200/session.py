@@ -23,11 +23,13 @@ class DeviceBatch:
     label: torch.Tensor
     B: int
     nnz: int
+    fast: Optional[torch.Tensor] = None       # [B][fast_dim] fp32: the views' own dense input
 
     @staticmethod
     def from_host(b: Batch, device="cuda") -> "DeviceBatch":
         f = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
-        return DeviceBatch(f(b.user_id), f(b.url_id), f(b.img_off), f(b.img_id), f(b.label), b.B, b.nnz)
+        return DeviceBatch(f(b.user_id), f(b.url_id), f(b.img_off), f(b.img_id), f(b.label), b.B, b.nnz,
+                           None if b.fast is None else f(b.fast))
 
 
 class GearSession:
@@ -51,7 +53,8 @@ class GearSession:
         self.cfg = gb.make_config(p.user_vocab, p.url_vocab, p.img_vocab, p.emb_dim, p.dfv_dim,
                                   gb.GEAR_BF16 if p.dfv_dtype == BF16 else gb.GEAR_F32,
                                   gb.GEAR_BF16 if p.head_dtype == BF16 else gb.GEAR_F32,
-                                  list(p.hidden), p.M, p.expire, self.max_batch, self.max_nnz, ready_cap, accum_mode)
+                                  list(p.hidden), p.M, p.expire, self.max_batch, self.max_nnz, ready_cap, accum_mode,
+                                  fast_dim=p.fast_dim)
         dev = self.dev
         if tables is None:
             self.user_emb = torch.empty((p.user_vocab, p.emb_dim), dtype=torch.float32, device=dev)
@@ -126,7 +129,7 @@ class GearSession:
             self._step_out.adam_step = self.adam_step
         bt = b.__dict__.get("_c_batch")
         if bt is None:
-            bt = b.__dict__["_c_batch"] = gb.make_batch(b.user_id, b.url_id, b.img_off, b.img_id, b.label)
+            bt = b.__dict__["_c_batch"] = gb.make_batch(b.user_id, b.url_id, b.img_off, b.img_id, b.label, fast=b.fast)
         bt.B, bt.nnz = b.B, b.nnz
         return gb.gear_forward_backward_structs(self.ctx, bt, self.p.lr if lr is None else lr, self._step_out)
 

@@ -56,10 +56,11 @@ class GearPreset:
     img_lambda: float = 0.0
     label_rate: float = 0.05
     lr: float = 0.05
+    fast_dim: int = 0         # dense input columns a view brings itself (the Fastgear side's share of the image)
 
     @property
     def d_in(self) -> int:
-        return 2 * self.emb_dim + self.dfv_dim
+        return 2 * self.emb_dim + self.dfv_dim + self.fast_dim
 
     @property
     def n_params(self) -> int:
@@ -97,6 +98,13 @@ PRESETS: Dict[str, GearPreset] = {
         hidden=(512, 256), M=32, expire=100,
         zipf_user=1.05, zipf_url=1.05, zipf_img=1.05, img_dist="poisson", img_lo=1, img_hi=16,
         img_lambda=4.0),
+    # the shape of the paper's CIFAR100 experiment (Section 4): every 32x32x3 image is cut in two, the top half
+    # (16x32x3 = 1536 values) goes to the Fastgear side as a dense input of its own, the bottom half is the Slowgear
+    # side's image (one image per view, its DFV cached).  Values are synthetic.
+    "split_image": GearPreset(
+        name="split_image", batch=1024, steps=8, user_vocab=10_000, url_vocab=10_000, img_vocab=50_000,
+        emb_dim=16, dfv_dim=64, dfv_dtype=F32, head_dtype=F32, hidden=(256, 64), M=4, expire=20,
+        zipf_user=1.1, zipf_url=1.1, zipf_img=1.05, img_dist="uniform", img_lo=1, img_hi=1, fast_dim=1536),
     "skew": GearPreset(
         name="skew", batch=32768, steps=30, user_vocab=1_000_000, url_vocab=1_000_000,
         img_vocab=4_000_000, emb_dim=32, dfv_dim=128, dfv_dtype=F32, head_dtype=F32,
@@ -178,6 +186,7 @@ class Batch:
     img_off: np.ndarray   # int32 [B+1], img_off[0] == 0, non-decreasing
     img_id: np.ndarray    # int32 [nnz]
     label: np.ndarray     # float32 [B], 0.0 or 1.0
+    fast: Optional[np.ndarray] = None   # float32 [B, fast_dim]: the views' own dense input (presets with fast_dim > 0)
 
     @property
     def B(self) -> int:
@@ -222,6 +231,7 @@ class BatchSource:
             img_off=off.astype(np.int32),
             img_id=self.imgs.sample(rng, nnz),
             label=(rng.random(B) < p.label_rate).astype(np.float32),
+            fast=(rng.random((B, p.fast_dim), dtype=np.float32) - 0.5) if p.fast_dim > 0 else None,   # "pixels" in [-0.5, 0.5)
         )
 
 

@@ -140,7 +140,7 @@ class Pair:
             oracle.fill_rows(seed, oracle.TAG_URL, p.emb_dim, self.rh.rows, self.rh.n, np.float32),
             oracle.fill_rows(seed, oracle.TAG_DFV, p.dfv_dim, self.ri.rows, self.ri.n, dfv_np),
             p.hidden, p.M, p.expire, round_bf16=(p.head_dtype == BF16),
-            ts=oracle.fill_ts(seed, p.expire, now0, None, p.img_vocab))
+            ts=oracle.fill_ts(seed, p.expire, now0, None, p.img_vocab), fast_dim=p.fast_dim)
         self.tol = tol_of(p)
         self.want_emb_grad = want_emb_grad
         self.updated_user = np.zeros(0, np.int32)
@@ -168,7 +168,7 @@ class Pair:
         uid, hid, img = self.ru(b.user_id), self.rh(b.url_id), self.ri(b.img_id)
         params64 = self.params.astype(np.float64)
         r = cpu.forward_backward(params64, uid, hid, b.img_off, img, b.label, relu_margin=0.0,
-                                 relu_margin_rel=relu_margin_rel(p), near_cap=max(65536, 64 * b.B))
+                                 relu_margin_rel=relu_margin_rel(p), near_cap=max(65536, 64 * b.B), fast=b.fast)
 
         B = b.B
         X = _np(gpu.x_debug[:B])
@@ -181,10 +181,12 @@ class Pair:
         n_b = np.diff(b.img_off)
         single = (n_b == 1)
         assert np.array_equal(X[single, 2 * E:].astype(np.float64), r.X[single, 2 * E:]), "single-image pooled rows"
+        if p.fast_dim:      # the view's own dense input is a copy (rounded once for bf16 heads)
+            assert np.array_equal(X[:, 2 * E + D:].astype(np.float64), r.X[:, 2 * E + D:]), "fast-side dense input"
         assert_close(X, r.X, tol, "head input")
         assert_close(_np(gpu.prob[:B]), r.prob, tol, "prob")
         assert_close(_np(gpu.loss), [r.loss], tol, "loss")
-        r = self.resolve_relu_decisions(r, params64, uid, hid, b.img_off, img, b.label)
+        r = self.resolve_relu_decisions(r, params64, uid, hid, b.img_off, img, b.label, b.fast)
         assert_close(_np(gpu.head_grad), r.head_grad, tol, "head_grad")
         assert_close(_np(gpu.dX[:B]), r.dX, tol, "dX")
         view_of = np.repeat(np.arange(B, dtype=np.int32), n_b)
@@ -227,7 +229,7 @@ class Pair:
         self.status_bits = self.status_rc = 0
         return out
 
-    def resolve_relu_decisions(self, r, params64, uid, hid, img_off, img, label):
+    def resolve_relu_decisions(self, r, params64, uid, hid, img_off, img, label, fast=None):
         """The backward pass depends on the sign of every hidden pre-activation.  Where the oracle's own
         pre-activation lies inside the rounding band of relu_margin_rel (r.near_units) the device may validly have
         taken the other branch; a unit's branch only affects its own view's row of dX (and, through the sums over
@@ -264,7 +266,8 @@ class Pair:
                 for subset in itertools.combinations(cands, k):
                     codes = np.array([(l * 1 + 0) * 1024 + j for (l, j) in subset], dtype=np.int64)
                     one = self.cpu.forward_backward(params64, uid[v:v + 1], hid[v:v + 1], np.array([0, hi - lo], np.int32),
-                                                    img[lo:hi], label[v:v + 1], flip_units=codes)
+                                                    img[lo:hi], label[v:v + 1], flip_units=codes,
+                                                    fast=None if fast is None else fast[v:v + 1])
                     # a batch of one view divides by 1 where the batch divides by B
                     if np.abs(got_dx[v] - one.dX[0] / B).max() <= self.tol * scale:
                         found = subset
@@ -275,7 +278,7 @@ class Pair:
                 return r                                    # the strict asserts report the mismatch
             all_flips += [(l * B + int(v)) * 1024 + j for (l, j) in found]
         res = self.cpu.forward_backward(params64, uid, hid, img_off, img, label,
-                                        flip_units=np.array(all_flips, dtype=np.int64))
+                                        flip_units=np.array(all_flips, dtype=np.int64), fast=fast)
         self.last_relu.update(views=len(bad_views), units=len(all_flips))
         self.relu_flips_accepted += len(all_flips)
         self.relu_views_flipped += len(bad_views)

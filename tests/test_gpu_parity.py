@@ -79,6 +79,16 @@ def test_medium_config_two_steps_events_5_and_6_in_one_call(gb):
     assert out[-1]["n_ready"] > 0
 
 
+@pytest.mark.parametrize("head", [F32, BF16])
+def test_split_image_workload_with_a_dense_input_on_the_fast_side(gb, head):
+    """The shape of the paper's CIFAR100 experiment (Section 4): half of every image (1536 values) stays on the Fastgear
+    side as a dense input of its own, appended to the head input; the other half is the cached DFV."""
+    p = PRESETS["split_image"].scaled(head_dtype=head, dfv_dtype=head)
+    out = _run_steps(p, 3, want_emb_grad=True)
+    assert out[-1]["n_ready"] > 0
+    _run_steps(p, 2, B=333, fused=True)
+
+
 def test_medium_shapes_ragged_batch(gb):
     p = PRESETS["medium"].scaled(user_vocab=50_000, url_vocab=30_000, img_vocab=20_000)
     _run_steps(p, 2, B=1237, want_emb_grad=True)

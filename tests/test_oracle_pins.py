@@ -740,3 +740,38 @@ def test_embedding_adam_steps_each_touched_row_once_with_the_summed_gradient():
         np.testing.assert_allclose(table[i], pr, atol=1e-15)
         np.testing.assert_allclose(m[i], mr, atol=1e-15)
         np.testing.assert_allclose(v[i], vr, atol=1e-15)
+
+
+# ----------------------------------------------------------------------------
+# a dense input of the view's own (the Fastgear side's share of the image)
+# ----------------------------------------------------------------------------
+def test_fast_side_dense_input_is_appended_to_the_head_input():
+    rng = np.random.default_rng(41)
+    B, E, D, F, Vi = 4, 2, 3, 5, 6
+    orc = GearOracle(rng.normal(size=(3, E)), rng.normal(size=(3, E)), rng.normal(size=(Vi, D)), (4, 3), 1, 0, fast_dim=F)
+    assert orc.d_in == 2 * E + D + F
+    params = rng.normal(0, 0.5, orc.n_params)
+    n = np.array([2, 1, 0, 3])
+    off = np.concatenate([[0], np.cumsum(n)]).astype(np.int32)
+    fast = rng.normal(size=(B, F))
+    batch = dict(user_id=rng.integers(0, 3, B).astype(np.int32), url_id=rng.integers(0, 3, B).astype(np.int32), img_off=off,
+                 img_id=rng.integers(0, Vi, off[-1]).astype(np.int32), label=np.array([1.0, 0.0, 0.0, 1.0]), fast=fast)
+    r = orc.forward_backward(params, **batch)
+    assert np.array_equal(r.X[:, 2 * E + D:], fast)                       # a copy, after the pooled DFV
+    assert np.array_equal(r.X[2, 2 * E:2 * E + D], np.zeros(D))          # the empty view still pools to zeros
+    # dLoss/d(fast) and dLoss/d(DFV table) by central differences: the new columns moved nothing else
+    want = np.array([central_diff(lambda: loss_of(orc, params, batch), fast, i) for i in range(fast.size)]).reshape(fast.shape)
+    np.testing.assert_allclose(r.dX[:, 2 * E + D:], want, atol=1e-8)
+    g_tab = np.zeros_like(orc.dfv)
+    rows = orc.dfv_grad_rows(off, r.dX)
+    for k, i in enumerate(batch["img_id"]):
+        g_tab[i] += rows[k]
+    want_tab = np.array([central_diff(lambda: loss_of(orc, params, batch), orc.dfv, i) for i in range(orc.dfv.size)]).reshape(orc.dfv.shape)
+    np.testing.assert_allclose(g_tab, want_tab, atol=1e-8)
+    # with zero weights on the new columns the network is the one without them
+    plain = GearOracle(orc.user_emb, orc.url_emb, orc.dfv, (4, 3), 1, 0)
+    W1 = params[:orc.d_in * 4].reshape(orc.d_in, 4).copy()
+    p0 = params.copy(); p0[:orc.d_in * 4] = np.vstack([W1[:2 * E + D], np.zeros((F, 4))]).ravel()
+    pp = np.concatenate([W1[:2 * E + D].ravel(), params[orc.d_in * 4:]])
+    b2 = {k: v for k, v in batch.items() if k != "fast"}
+    assert abs(orc.forward_backward(p0, **batch).loss - plain.forward_backward(pp, **b2).loss) < 1e-15
