@@ -163,12 +163,12 @@ def kernel_models(p, stats):
 # re-reads that hit the L2 in a real step count as DRAM traffic here.  A kernel that has changed since its capture
 # must be taken out of this table (traffic is then reported as null).
 NCU_TRAFFIC_LARGE_2M = {
-    "gather_pool": (64.4e6, "l2"), "acc_reduce": (239.7e6, "work"), "expiry_mark": (16.0e6, "vocab"),
-    "head_out": (34.4e6, None), "collect_move": (5.9e6, "work"), "emb_reduce": (46.9e6, "work"),
-    "tc_gemm_fwd": (68.3e6, None), "tc_gemm_dw": (113.7e6, None), "tc_gemm_dh": (129.5e6, None), "tc_gemm_dx": (110.2e6, None),
+    "gather_pool": (64.1e6, "l2"), "acc_reduce": (238.3e6, "work"), "expiry_mark": (16.0e6, "vocab"),
+    "head_out": (34.5e6, None), "emb_reduce": (46.9e6, "work"),
+    "tc_gemm_fwd": (68.6e6, None), "tc_gemm_dw": (113.2e6, None), "tc_gemm_dh": (130.3e6, None), "tc_gemm_dx": (110.1e6, None),
 }
 # algorithmic bytes per launch of the table-bound kernels on large_2m (kernel_models on that workload's batches)
-NCU_WORK_LARGE_2M = {"gather_pool": 222.0e6, "acc_reduce": 224.5e6, "collect_move": 14.2e6, "emb_reduce": 58.9e6}
+NCU_WORK_LARGE_2M = {"gather_pool": 222.0e6, "acc_reduce": 224.5e6, "emb_reduce": 58.9e6}
 
 
 def ncu_traffic(name, p, work):
@@ -380,7 +380,7 @@ def run_ours(args):
         a few steps alone are too short for the clock sampler to see and for the clocks to settle under load.  The
         loop count follows from the max-over-ranks time, so every rank runs the same number of regions."""
         out = []
-        while (sum(out) < MIN_TIMED_MS or len(out) < 3) and len(out) < MAX_REGIONS:
+        while (sum(out) < args.min_timed_ms or len(out) < 3) and len(out) < MAX_REGIONS:
             out.append(region_fn())
         return out
 
@@ -663,7 +663,7 @@ def run_sharded(args):
     launches0 = sum(gb.gear_launch_count(x.ctx) for x in sg.owners + sg.workers)
     region_ms = []
     sampler.open_window()
-    while (sum(region_ms) < MIN_TIMED_MS or len(region_ms) < 3) and len(region_ms) < MAX_REGIONS:
+    while (sum(region_ms) < args.min_timed_ms or len(region_ms) < 3) and len(region_ms) < MAX_REGIONS:
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize(); reps.barrier(); torch.cuda.synchronize()
         ev0.record(stream)
@@ -708,6 +708,9 @@ def main():
                          "micro-benchmark, one line per case.  skew: the skew-stress step.  skew_modes: its accumulate call, "
                          "sort against atomics, M in {1, 64, 1024}, one line per case")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-timed-ms", type=float, default=MIN_TIMED_MS,
+                    help="device time to measure per arm: the K-step region is repeated until then (default 1000; a "
+                         "profiler capture passes 0 to keep the run to three short regions)")
     ap.add_argument("--sharded", action="store_true",
                     help="tables partitioned by ID over the ranks instead of independent replicas (not the default: this "
                          "arm has only ever run on one GPU)")
