@@ -573,7 +573,7 @@ def accumulate_line(case, args, sampler_gpu, peaks, with_cpu=True):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": case["case"], "mode": case["mode"], "rows": n, "img_vocab": case["img_vocab"], "dim": D,
                        "M": case["M"], "distinct_images": uniq, "emissions_per_call": ready,
-                       "step": "one gear_accumulate_dfv_grad over all rows + one gear_collect_ready",
+                       "step": "one gear_accumulate_collect over all rows (accumulate + hand-over of the completed groups)",
                        "l2": "8.6 GB of gradient rows and a 2 GB store per call: far beyond the 126 MB L2"},
             "clocks": sampler_gpu, "gpu_launches": case.get("launches_per_step"),
             "e2e": None, "e2e_note": "the rows are produced on the device by the head's backward pass and never cross "

@@ -67,18 +67,35 @@ __device__ __forceinline__ void tile_flags(TileFlags& f, const uint32_t* __restr
 #pragma unroll
     for (int t = 0; t < AF_ITEMS; ++t) f.key[t] = (f.i0 + t < n) ? ks[f.i0 + t] : vocab;
 
-    // start of the image's run that covers the tile's first position (the run may begin in an earlier tile)
-    if (threadIdx.x == 0) {
-        uint32_t carry = (uint32_t)tile0;
-        if (tile0 > 0 && tile0 < n && ks[tile0 - 1] == f.key[0]) {
-            int64_t lo = 0, hi = tile0 - 1;       // first index whose key is >= key[0]; ks[hi] == key[0]
-            while (lo < hi) {
-                const int64_t mid = (lo + hi) >> 1;
-                if (ks[mid] < f.key[0]) lo = mid + 1; else hi = mid;
+    // start of the image's run that covers the tile's first position (the run may begin in an earlier tile).  Warp 0
+    // searches backwards with all its lanes at once: first one round of probes at distances 1, 2, 4, ... brackets the
+    // start, then rounds of 32 evenly spaced probes narrow the bracket by a factor of 32 each, so that even a run of
+    // millions of rows (a hot image) costs a handful of trips to memory, and the usual short run one.
+    if (threadIdx.x < 32) {
+        const int lane0 = (int)threadIdx.x;
+        const uint32_t key0 = __shfl_sync(0xffffffffu, f.key[0], 0);
+        int64_t start = tile0;
+        const bool spans = tile0 > 0 && tile0 < n && ks[tile0 - 1] == key0;      // the same words for every lane
+        if (spans) {
+            int64_t hi = tile0 - 1;                                  // ks[hi] == key0
+            const int64_t far = hi - ((int64_t)1 << lane0);
+            const bool same = lane0 < 31 && far >= 0 && ks[far] == key0;
+            const int k = __popc(__ballot_sync(0xffffffffu, same));  // probes 0 .. k-1 still lie inside the run
+            int64_t lo = hi - ((int64_t)1 << k);                     // ks[lo] != key0, or lo < 0
+            if (lo < -1) lo = -1;
+            if (k > 0) hi -= (int64_t)1 << (k - 1);
+            while (hi - lo > 1) {
+                const int64_t step = (hi - lo + 31) / 32;
+                const int64_t p = hi - (int64_t)(lane0 + 1) * step;
+                const bool in = p > lo && ks[p] == key0;
+                const int m = __popc(__ballot_sync(0xffffffffu, in));
+                hi -= (int64_t)m * step;
+                const int64_t below = hi - step;
+                if (below > lo) lo = below;                          // the first probe that failed (it lies above the old lo)
             }
-            carry = (uint32_t)lo;
+            start = hi;
         }
-        smem[33] = carry;
+        if (lane0 == 0) smem[33] = (uint32_t)start;
     }
     // run start of every position: inclusive max-scan of "index if run head"
     uint32_t local_max = 0;
@@ -216,8 +233,11 @@ struct LaneGroup {
 };
 
 // Where the averages of the groups a call completes go when they bypass the ready queue: the caller's own lists
-// (gear_accumulate_collect on a queue that is known to be empty).  All null: the groups join the queue.
-struct EmitTarget { int32_t* ids; int32_t* seq; float* avg; int64_t* d_n; };
+// (gear_accumulate_collect).  All null: the groups join the queue.  cap < 0: the host has checked that the queue is empty
+// and that the lists can take every group the call could complete.  cap >= 0: the kernel decides: the lists are used if
+// the queue is empty and the call completes at most cap groups, else the groups join the queue and the hand-over pass
+// that the host has enqueued behind this kernel deals with them.
+struct EmitTarget { int32_t* ids; int32_t* seq; float* avg; int64_t* d_n; int64_t cap; };
 
 // One row to stage, as the copy side sees it (where the row starts; bit 0 of the address word is set if the item
 // exists) and as the adding side sees it (what the row is scaled by and
@@ -252,7 +272,8 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
     const int64_t n_groups = totals.x;
     // Averages go to the ready queue, or (the queue being empty, so that queue slot k is also entry k of the hand-over)
     // straight into the caller's lists, whose capacity the host has checked against the row count.
-    const bool to_caller = direct.avg != nullptr;
+    const bool to_caller = direct.avg != nullptr &&
+                           (direct.cap < 0 || (state->q_count == 0 && (int64_t)totals.y <= direct.cap));
     int32_t* __restrict__ e_id = to_caller ? direct.ids : q_id;
     float* __restrict__ e_avg = to_caller ? direct.avg : q_avg;
     // Step 6 of the plan (commit) is done by whichever block finishes last: by then every block has read the queue
@@ -264,8 +285,8 @@ acc_reduce_kernel(const uint32_t* __restrict__ ks, RowGather rg, int D, int M, i
             __threadfence();
             unsigned int* ticket = reinterpret_cast<unsigned int*>(&state->pad[4]);
             if (atomicInc(ticket, gridDim.x - 1) == gridDim.x - 1) {
-                state->n_groups = totals.x;
                 state->n_complete = totals.y;
+                state->direct_done = (to_caller && direct.cap >= 0) ? 1 : 0;
                 if (to_caller) { if (direct.d_n) *direct.d_n = totals.y; }
                 else if (dropped) atomicOr(&state->status, GEAR_DEV_READY_OVERFLOW);
                 else if (totals.y > 0) { state->q_count += totals.y; state->q_calls += 1; }
@@ -559,13 +580,14 @@ static cudaError_t launch_accumulate_to(const gear_ctx_impl& c, const int32_t* i
 #undef GEAR_ACC_LAUNCH
     }
     if (le != cudaSuccess) return le;
-    if (!to_caller.avg) ++c.acc_calls_pending;                    // a call that bypasses the queue leaves it empty
+    if (!to_caller.avg) ++c.acc_calls_pending;                    // a call that bypasses the queue leaves it empty (a call
+                                                                  // that may or may not bypass it: see launch_accumulate_collect)
     return cudaGetLastError();
 }
 
 cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
                               const int32_t* src_row, const float* scale, int64_t n, cudaStream_t st) {
-    return launch_accumulate_to(c, img_id, grads, ld, src_row, scale, n, EmitTarget{nullptr, nullptr, nullptr, nullptr}, st);
+    return launch_accumulate_to(c, img_id, grads, ld, src_row, scale, n, EmitTarget{nullptr, nullptr, nullptr, nullptr, -1}, st);
 }
 
 // Events 5 and 6 in one call.  When the host knows the ready queue to be empty (no accumulate call since a collect that
@@ -575,8 +597,17 @@ cudaError_t launch_accumulate(const gear_ctx_impl& c, const int32_t* img_id, con
 cudaError_t launch_accumulate_collect(const gear_ctx_impl& c, const int32_t* img_id, const float* grads, int64_t ld,
                                       const int32_t* src_row, const float* scale, int64_t n, int32_t* ids, int32_t* seq,
                                       float* avg, int64_t cap, int64_t* d_n, cudaStream_t st) {
-    const bool direct = c.cfg.accum_mode == GEAR_ACC_SORT && c.acc_calls_pending == 0 && n > 0 && cap >= n;
-    if (direct) return launch_accumulate_to(c, img_id, grads, ld, src_row, scale, n, EmitTarget{ids, seq, avg, d_n}, st);
+    const bool queue_empty = c.cfg.accum_mode == GEAR_ACC_SORT && c.acc_calls_pending == 0 && n > 0;
+    if (queue_empty && cap >= n)
+        return launch_accumulate_to(c, img_id, grads, ld, src_row, scale, n, EmitTarget{ids, seq, avg, d_n, -1}, st);
+    if (queue_empty && cap > 0) {
+        // the lists may or may not be long enough for what this call completes: the reduce pass finds out, and the
+        // hand-over pass behind it moves the queue only if the reduce pass had to use it
+        cudaError_t de = launch_accumulate_to(c, img_id, grads, ld, src_row, scale, n, EmitTarget{ids, seq, avg, d_n, cap}, st);
+        if (de != cudaSuccess) return de;
+        c.acc_calls_pending = 1;
+        return launch_collect_ready(c, ids, seq, avg, cap, d_n, st);
+    }
     cudaError_t e = cudaSuccess;
     if (n > 0)
         e = c.cfg.accum_mode == GEAR_ACC_ATOMIC
@@ -722,6 +753,18 @@ collect_move_kernel(const uint32_t* __restrict__ sorted_keys, const uint32_t* __
     // the caller's capacity itself and the last block to finish empties the queue
     const int64_t n = solo ? state->q_count : state->collect_n;
     if (solo) {
+        if (state->direct_done != 0) {
+            // the reduce pass in front of this launch has written the caller's lists and the count itself: nothing to
+            // move; the block that leaves last takes the mark down
+            __shared__ int last_out;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                __threadfence();
+                last_out = atomicInc(&state->pad32, gridDim.x - 1) == gridDim.x - 1;
+                if (last_out) state->direct_done = 0;
+            }
+            return;
+        }
         if (blockIdx.x == 0 && threadIdx.x == 0) {
             if (d_n) *d_n = n;
             if (n > cap) atomicOr(&state->status, GEAR_DEV_OUT_CAPACITY);

@@ -19,7 +19,8 @@ struct DevState {
     int32_t tc_error;      // non-zero: a bounded wait of the tensor-core head gave up (code of the wait)
     int64_t q_count;       // averages waiting in the ready queue
     int64_t n_valid;       // accumulate: rows with an in-range ID (sorted prefix length)
-    int64_t n_groups;      // accumulate: groups found in this call
+    int64_t direct_done;   // accumulate + collect as one call: 1 while the hand-over pass that follows has nothing to do
+                           // (the reduce pass wrote the averages straight into the caller's lists)
     int64_t n_complete;    // accumulate: groups of this call that reached M
     int64_t exp_total;     // expiry scan: entries found
     int64_t collect_n;     // collect_ready: entries moved by the running call

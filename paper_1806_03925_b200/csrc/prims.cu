@@ -22,6 +22,7 @@
 // earlier launch contributes).  The kernel is launched cooperatively, so all blocks are resident and a tile's
 // predecessors are always being worked on; the spins (barrier and look-back) are bounded all the same, and a block
 // that gives up records an error and makes every later wait of the launch fall through.
+#include <cstdlib>
 #include "common.cuh"
 
 namespace gear {
@@ -80,6 +81,7 @@ coop_sort_kernel(const SortBatch batch) {
     __shared__ uint32_t base[RS_BUCKETS];              // where each digit of this tile starts in the output
     __shared__ uint32_t lstart[RS_BUCKETS];            // ... and in the tile's own digit order
     __shared__ uint32_t wcnt[RS_THREADS / 32][RS_BUCKETS];
+    __shared__ uint32_t gstart[3][RS_BUCKETS];        // per job: where each digit of the current pass starts in the output
     __shared__ int live_tiles[3];
     __shared__ int64_t live_n[3];
     __shared__ int give_up;
@@ -140,11 +142,17 @@ coop_sort_kernel(const SortBatch batch) {
                     __stcg(j.hist + ((int64_t)p * j.n_tiles + t) * RS_BUCKETS + d, 0u);
             const int64_t tile0 = (int64_t)t * RS_TILE;
             bool bad = false;
-#pragma unroll 4
+            uint32_t hk[RS_ITEMS];
+#pragma unroll
+            for (int it = 0; it < RS_ITEMS; ++it) {                 // all loads of the tile in flight before the first is used
+                const int64_t i = tile0 + it * RS_THREADS + threadIdx.x;
+                hk[it] = i < n ? load_key(j, 0, i, 0) : 0u;
+            }
+#pragma unroll
             for (int it = 0; it < RS_ITEMS; ++it) {
                 const int64_t i = tile0 + it * RS_THREADS + threadIdx.x;
                 if (i < n) {
-                    const uint32_t k = load_key(j, 0, i, 0);
+                    const uint32_t k = hk[it];
                     bad |= (k == j.sentinel);
                     for (int p = 0; p < batch.passes; ++p)
                         atomicAdd(&hist[(jj * RS_MAX_PASSES + p) * RS_BUCKETS + ((k >> (p * j.width)) & mask)], 1u);
@@ -164,6 +172,22 @@ coop_sort_kernel(const SortBatch batch) {
 
     for (int pass = 0; pass < batch.passes && ok; ++pass) {
         const int src = pass & 1, dst = src ^ 1;
+        // where each digit starts in the output: digits before it, all tiles (the histogram of the pass), per job
+        for (int jj = 0; jj < batch.n_jobs; ++jj) {
+            const SortJob& j = batch.job[jj];
+            const uint32_t mask = (1u << j.width) - 1u;
+            uint32_t gtot[DPT], mine = 0;
+#pragma unroll
+            for (int q = 0; q < DPT; ++q) {
+                const int d = threadIdx.x * DPT + q;
+                gtot[q] = d <= (int)mask ? __ldcg(j.tot + pass * RS_BUCKETS + d) : 0u;
+                mine += gtot[q];
+            }
+            uint32_t ex = block_exclusive_scan(mine, scratch, nullptr);
+#pragma unroll
+            for (int q = 0; q < DPT; ++q) { gstart[jj][threadIdx.x * DPT + q] = ex; ex += gtot[q]; }
+        }
+        __syncthreads();
         for (int w = w_begin; w < w_end && ok; w += nblk) {
             int t;
             const int jj = job_of(w, t);
@@ -173,30 +197,18 @@ coop_sort_kernel(const SortBatch batch) {
             const int shift = pass * j.width;
             const uint32_t mask = (1u << j.width) - 1u;
             uint32_t* desc = j.hist + ((int64_t)pass * j.n_tiles) * RS_BUCKETS;      // [tile][digit] of this pass
-            // where each digit starts in the output: digits before it, all tiles (the histogram of the pass)
-            uint32_t gtot[DPT], gbase[DPT];
-            {
-                uint32_t mine = 0;
-#pragma unroll
-                for (int q = 0; q < DPT; ++q) {
-                    const int d = threadIdx.x * DPT + q;
-                    gtot[q] = d <= (int)mask ? __ldcg(j.tot + pass * RS_BUCKETS + d) : 0u;
-                    mine += gtot[q];
-                }
-                uint32_t ex = block_exclusive_scan(mine, scratch, nullptr);
-#pragma unroll
-                for (int q = 0; q < DPT; ++q) { gbase[q] = ex; ex += gtot[q]; }
-            }
             for (int d = threadIdx.x; d < RS_BUCKETS; d += RS_THREADS)
 #pragma unroll
                 for (int w2 = 0; w2 < RS_THREADS / 32; ++w2) wcnt[w2][d] = 0;
             __syncthreads();
-            uint32_t key[RS_ITEMS], rank[RS_ITEMS];
+            uint32_t key[RS_ITEMS], rank[RS_ITEMS], val[RS_ITEMS];
             const int64_t seg0 = tile0 + (int64_t)warp * (32 * RS_ITEMS);
+            const bool identity = (pass == 0 && j.identity_vals);
 #pragma unroll
-            for (int it = 0; it < RS_ITEMS; ++it) {
+            for (int it = 0; it < RS_ITEMS; ++it) {                 // keys and values of the tile: one trip to memory
                 const int64_t i = seg0 + it * 32 + lane;
                 key[it] = i < n ? load_key(j, pass, i, src) : 0u;
+                val[it] = identity ? (uint32_t)i : (i < n ? __ldcg(j.vals[src] + i) : 0u);
             }
 #pragma unroll
             for (int it = 0; it < RS_ITEMS; ++it) {
@@ -278,14 +290,13 @@ coop_sort_kernel(const SortBatch batch) {
                     }
                     __stcg(desc + (int64_t)t * RS_BUCKETS + d, DESC_UPTO | (before + tot[q]));
                 }
-                base[d] = gbase[q] + before;
+                base[d] = gstart[jj][d] + before;
             }
             __syncthreads();
             if (give_up) { ok = false; break; }
             // The pairs are first put in digit order inside the tile (shared memory), then written out position by
             // position: neighbouring threads write neighbouring words of a digit's run, so the stores of a warp fall
             // into a few full sectors instead of 32 different ones.
-            const bool identity = (pass == 0 && j.identity_vals);
             uint32_t* skey = stage;
             uint32_t* sval = stage + RS_TILE;
 #pragma unroll
@@ -295,7 +306,7 @@ coop_sort_kernel(const SortBatch batch) {
                     const uint32_t d = (key[it] >> shift) & mask;
                     const uint32_t lp = lstart[d] + wcnt[warp][d] + rank[it];
                     skey[lp] = key[it];
-                    sval[lp] = identity ? (uint32_t)i : __ldcg(j.vals[src] + i);
+                    sval[lp] = val[it];
                 }
             }
             __syncthreads();
@@ -329,6 +340,7 @@ static int coop_grid_limit() {
         if (sms <= 0) sms = 148;
         if (per_sm <= 0) per_sm = 1;
         if (per_sm > 3) per_sm = 3;
+        if (getenv("GEAR_SORT_PER_SM")) per_sm = atoi(getenv("GEAR_SORT_PER_SM"));
         limit = sms * per_sm;
     }
     return limit;

@@ -4,8 +4,8 @@
     python -m paper_1806_03925_b200.microbench [--config micro|skew|refresh|all] [--steps K] [--rows N]
 
 micro   n gradient rows of dim 128 fp32 (IDs uniform or Zipf 1.1) into a 4M-image sum+count table, followed by
-        the count >= M compaction (gear_collect_ready), M in {8, 64}: time and bytes-moved rate of
-        gear_accumulate_dfv_grad + gear_collect_ready against the measured HBM copy rate.
+        the count >= M compaction and hand-over, M in {8, 64}: time and bytes-moved rate of
+        gear_accumulate_collect (events 5 and 6 as one call) against the measured HBM copy rate.
 skew    the skew-stress shapes (32768 views, 4M images, Zipf 1.3, dim 128 fp32), M in {1, 64, 1024}:
         sort + segmented reduction (GEAR_ACC_SORT) against fp32 reductions (GEAR_ACC_ATOMIC) under contention.
 
@@ -61,9 +61,8 @@ def _run_case(name, ids_np, V, D, M, mode, steps, warmup=2):
         for s in range(warmup + steps):
             e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
             e0.record(stream)
-            sess.accumulate_rows(ids, grads)
+            k = sess.accumulate_collect_rows(ids, grads, sync=True)     # events 5 and 6 as one call
             e1.record(stream)
-            k = sess.collect_ready(sync=True)
             e2.record(stream)
             torch.cuda.synchronize()
             if s >= warmup:
@@ -71,15 +70,14 @@ def _run_case(name, ids_np, V, D, M, mode, steps, warmup=2):
         launches_per_step = (gb.gear_launch_count(sess.ctx) - launches0) / (warmup + steps)
         # one more call with per-kernel events (serialised, so each kernel is timed alone)
         gb.gear_profile_enable(sess.ctx, True)
-        sess.accumulate_rows(ids, grads)
-        sess.collect_ready(sync=True)
+        sess.accumulate_collect_rows(ids, grads, sync=True)
         prof = gb.gear_profile_read(sess.ctx, 64)
         gb.gear_profile_enable(sess.ctx, False)
         kernels = {k: round(v[0], 4) for k, v in sorted(prof.items(), key=lambda kv: -kv[1][0])}
         rc, status, _ = sess.status()
         acc_ms, col_ms, ready = float(np.median(t_acc)), float(np.median(t_col)), float(np.mean(n_ready))
         bytes_acc = n * D * 4 + n * 4 + uniq * (D * 4 + 4) * 2 + ready * (D * 4 + 4)
-        bytes_col = ready * (2 * D * 4 + 16)
+        bytes_col = 0.0 if "collect_move" not in prof else ready * (2 * D * 4 + 16)      # a separate hand-over pass, if one ran
         peak, src = _peak_gbs()
         gbs = (bytes_acc + bytes_col) / ((acc_ms + col_ms) * 1e-3) / 1e9
         return {"case": name, "mode": mode, "rows": n, "img_vocab": V, "dim": D, "M": M, "distinct_images": uniq,

@@ -316,6 +316,43 @@ def test_fused_call_on_a_non_empty_queue_and_with_a_short_list(gb):
             pair.close()
 
 
+def test_fused_call_whose_lists_cannot_take_the_completed_groups(gb):
+    """Lists shorter than what the call completes: the reduce pass must notice on the device, leave the averages in the
+    ready queue, report the required count and hand nothing over; a later hand-over into long enough lists gets all."""
+    from gpu_harness import _np, assert_close
+    p = PRESETS["tiny"].scaled(user_vocab=16, url_vocab=16, img_vocab=300, M=1)
+    rng = np.random.default_rng(12)
+    ids = rng.integers(0, 300, 500).astype(np.int32)
+    g_rows = rng.normal(0, 1, (500, p.dfv_dim)).astype(np.float32)
+    pair = _pair(p, [], dense=True, extra_img_ids=ids, ready_cap=1000)
+    try:
+        g, cpu = pair.gpu, pair.cpu
+        d_ids, d_rows = torch.from_numpy(ids).cuda(), torch.from_numpy(g_rows).cuda()
+        with pytest.raises(gb.GearError) as e:          # M = 1: 500 groups, lists of 100
+            gb.gear_accumulate_collect(g.ctx, d_ids, d_rows.data_ptr(), p.dfv_dim, None, None, 500, g.ready_ids, g.ready_seq,
+                                       g.ready_avg, 100, d_n=g.d_counts[0:1])
+        assert e.value.code == gb.GEAR_ERR_CAPACITY and int(g.d_counts[0].item()) == 500
+        rc, bits, pending = g.status()
+        assert pending == 500 and bits & gb.GEAR_DEV_OUT_CAPACITY
+        cpu.accumulate(ids, g_rows.astype(np.float64))
+        pair.compare_store()
+        # a second fused call with lists of 100 that DO suffice (2 new groups) must not bypass the non-empty queue
+        with pytest.raises(gb.GearError):
+            gb.gear_accumulate_collect(g.ctx, d_ids[:2], d_rows.data_ptr(), p.dfv_dim, None, None, 2, g.ready_ids, g.ready_seq,
+                                       g.ready_avg, 100, d_n=g.d_counts[0:1])
+        assert int(g.d_counts[0].item()) == 502
+        g.status()
+        cpu.accumulate(ids[:2], g_rows[:2].astype(np.float64))
+        n = g.collect_ready()
+        eid, eseq, eavg = oracle.sort_emissions(*cpu.collect_ready())
+        assert n == 502 == len(eid)
+        assert np.array_equal(_np(g.ready_ids[:n]), eid) and np.array_equal(_np(g.ready_seq[:n]), eseq)
+        assert_close(_np(g.ready_avg[:n]), eavg, 1e-5, "averaged gradients")
+        assert g.status()[1:] == (0, 0) and g.guards_intact()
+    finally:
+        pair.close()
+
+
 def test_zero_sized_calls_are_accepted(gb):
     b = _manual_batch([3], [4], [[8]], [1])
     p, pair = _tiny_pair([b])
