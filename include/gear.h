@@ -377,8 +377,13 @@ int gear_collect_expired_static(int64_t* dfv_ts, int64_t img_vocab, int64_t expi
  * its work on the caller's stream (no side stream), so that every kernel is timed alone: do not time
  * throughput with profiling on.
  * gear_launch_count returns the number of kernels this ctx has launched since it was created.
+ * on = 2 is the timeline mode: the events are recorded, but the library keeps its side stream, so that
+ * gear_profile_timeline can show what ran beside what: start and stop of every launch since the mode was switched on,
+ * in milliseconds after the first launch's start, in launch order (cap entries at most; names as in gear_profile_read).
+ * A kernel's start event completes when the stream reaches it, which may be well before the kernel's blocks get an SM.
  */
 int gear_profile_enable(gear_ctx* ctx, int on);
+int gear_profile_timeline(gear_ctx* ctx, char* names, float* start_ms, float* stop_ms, int32_t cap, int32_t* n_out);
 int gear_profile_read(gear_ctx* ctx, char* names, float* total_ms, int32_t* launches, int32_t cap, int32_t* n_out);
 int gear_launch_count(gear_ctx* ctx, int64_t* n_launches);
 

@@ -27,7 +27,7 @@ EXPORTS = ("gear_workspace_bytes", "gear_init_tables", "gear_forward_backward", 
            "gear_collect_ready", "gear_collect_expired", "gear_status", "gear_destroy", "gear_fill_uniform",
            "gear_last_error", "gear_profile_enable", "gear_profile_read", "gear_launch_count",
            "gear_collect_expired_static", "gear_refresh_dfv", "gear_accumulate_collect", "gear_dense_forward",
-           "gear_dense_backward", "gear_adam_dense", "gear_fetch_rows", "gear_apply_emb_grad")
+           "gear_dense_backward", "gear_adam_dense", "gear_fetch_rows", "gear_apply_emb_grad", "gear_profile_timeline")
 GEAR_STATIC_EXPIRY_MAX_VOCAB = 16777216
 
 
@@ -118,6 +118,8 @@ def load() -> C.CDLL:
     L.gear_profile_enable.argtypes = [vp, C.c_int]
     L.gear_profile_read.restype = C.c_int
     L.gear_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_float), C.POINTER(i32), i32, C.POINTER(i32)]
+    L.gear_profile_timeline.restype = C.c_int
+    L.gear_profile_timeline.argtypes = [vp, C.c_char_p, C.POINTER(C.c_float), C.POINTER(C.c_float), i32, C.POINTER(i32)]
     L.gear_launch_count.restype = C.c_int
     L.gear_launch_count.argtypes = [vp, C.POINTER(i64)]
     L.gear_collect_expired_static.restype = C.c_int
@@ -327,8 +329,18 @@ def gear_destroy(ctx):
     return _check(load().gear_destroy(ctx), "gear_destroy")
 
 
-def gear_profile_enable(ctx, on: bool):
-    return _check(load().gear_profile_enable(ctx, 1 if on else 0), "gear_profile_enable")
+def gear_profile_enable(ctx, on):
+    """on: False / True (every kernel alone on the caller's stream) / 2 (timeline mode: the side stream stays)."""
+    return _check(load().gear_profile_enable(ctx, int(on)), "gear_profile_enable")
+
+
+def gear_profile_timeline(ctx, cap: int = 256):
+    """[(kernel name, start ms, stop ms)] of every launch since timeline mode was switched on; synchronises."""
+    names = C.create_string_buffer(64 * cap)
+    t0, t1 = (C.c_float * cap)(), (C.c_float * cap)()
+    n = C.c_int32(0)
+    _check(load().gear_profile_timeline(ctx, names, t0, t1, cap, C.byref(n)), "gear_profile_timeline")
+    return [(names.raw[64 * k:64 * (k + 1)].split(b"\0", 1)[0].decode(), float(t0[k]), float(t1[k])) for k in range(n.value)]
 
 
 def gear_profile_read(ctx, cap: int = 64):

@@ -110,9 +110,8 @@ static void release_host_objects(gear_ctx_impl& c) {
     if (c.ev_fork) cudaEventDestroy(c.ev_fork);
     if (c.ev_join) cudaEventDestroy(c.ev_join);
     if (c.ev_gather) cudaEventDestroy(c.ev_gather);
-    if (c.ev_weights) cudaEventDestroy(c.ev_weights);
     if (c.ev_dx) cudaEventDestroy(c.ev_dx);
-    c.ev_weights = c.ev_dx = nullptr;
+    c.ev_dx = nullptr;
     if (c.side_stream) cudaStreamDestroy(c.side_stream);
     c.ev_fork = c.ev_join = c.ev_gather = nullptr;
     c.side_stream = nullptr;
@@ -180,14 +179,13 @@ int gear_init_tables(gear_ctx** out_ctx, const gear_config* cfg, const gear_buff
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c.last_stream = st;
     c.side_stream = nullptr;
-    c.ev_fork = c.ev_join = c.ev_gather = c.ev_weights = c.ev_dx = nullptr;
+    c.ev_fork = c.ev_join = c.ev_gather = c.ev_dx = nullptr;
     c.plan_ready = false; c.plan_n = 0; c.plan_src_row = nullptr; c.plan_scale = nullptr;
 
     cudaError_t e = cudaStreamCreateWithFlags(&c.side_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_gather, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_join, cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_weights, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c.ev_dx, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemsetAsync(c.state(), 0, sizeof(DevState), st);
     if (e == cudaSuccess && fill) {
@@ -252,7 +250,7 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
     c.img_sorted = false;
     c.img_sort_valid = false;
     c.plan_ready = false;
-    const bool forked = !c.prof.on && b.B > 0;
+    const bool forked = (!c.prof.on || c.prof.keep_streams) && b.B > 0;
     bool join_pending = false;          // the side stream holds work the caller's stream has not waited for
     cudaStream_t side = forked ? c.side_stream : st;
     // A failure between the fork and the join must not leave the side stream unjoined or the sorted order marked as
@@ -272,10 +270,12 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
         if (e != cudaSuccess) return cuda_fail(e, "fork");
         join_pending = true;
     }
-    const bool weights_on_side = forked && c.cfg.head_dtype == GEAR_BF16;
-    if (weights_on_side) {
-        e = launch_round_weights(c, c.side_stream);
-        if (e == cudaSuccess) e = cudaEventRecord(c.ev_weights, c.side_stream);
+    // bf16 copies of the head's weights: first on the caller's stream, ahead of the gather.  The gather keeps every SM
+    // busy for its whole duration, so a small kernel on another stream would get its blocks placed only when the gather
+    // ends, and the first product of the head would wait for it.
+    const bool weights_early = b.B > 0 && c.cfg.head_dtype == GEAR_BF16;
+    if (weights_early) {
+        e = launch_round_weights(c, st);
         if (e != cudaSuccess) return abandon(e, "weight copies");
     }
     int sorted_buf = 0;
@@ -313,10 +313,6 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
         if (e == cudaSuccess) e = launch_accumulate_plan_ahead(c, b.nnz, o.row_view, o.inv_n, c.side_stream);
         if (e != cudaSuccess) return abandon(e, "accumulate plan");
     }
-    if (weights_on_side) {
-        e = cudaStreamWaitEvent(st, c.ev_weights, 0);
-        if (e != cudaSuccess) return abandon(e, "weight copies");
-    }
     // the embedding scatter: enqueued by the head as soon as dX is on its way
     struct Scatter {
         gear_ctx_impl* c; const gear_step_out* o; int sorted_buf; int32_t B; float lr; cudaStream_t st; bool forked;
@@ -340,7 +336,7 @@ int gear_forward_backward(gear_ctx* ctx, const gear_batch* batch, float lr, cons
                                    k.o->url_m, k.o->url_v, where);
         return launch_emb_reduce(c, k.sorted_buf, k.B, ut, ht, k.o->dX, c.d_in, alpha, where);
     };
-    const HeadHooks hooks{weights_on_side, scatter, &sc};
+    const HeadHooks hooks{weights_early, scatter, &sc};
     e = launch_head_simt(c, b, o, st, hooks);
     if (e != cudaSuccess) return abandon(e, "head");
     if (o.dfv_grad && b.B > 0) {
@@ -565,6 +561,31 @@ int gear_profile_enable(gear_ctx* ctx, int on) {
     sync_streams(ctx->impl);
     ctx->impl.prof.clear();
     ctx->impl.prof.on = on != 0;
+    ctx->impl.prof.keep_streams = on == 2;
+    return GEAR_OK;
+}
+
+int gear_profile_timeline(gear_ctx* ctx, char* names, float* start_ms, float* stop_ms, int32_t cap, int32_t* n_out) {
+    if (!ctx || !ctx->impl.alive) return GEAR_ERR_STATE;
+    if (!n_out || cap < 0 || (cap > 0 && (!names || !start_ms || !stop_ms))) return arg_fail("gear_profile_timeline");
+    gear_ctx_impl& c = ctx->impl;
+    cudaError_t e = sync_streams(c);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c.side_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "gear_profile_timeline");
+    int n = 0;
+    for (const auto& r : c.prof.recs) {
+        if (n >= cap) break;
+        float a = 0.f, b = 0.f;
+        e = cudaEventElapsedTime(&a, c.prof.recs[0].start, r.start);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&b, c.prof.recs[0].start, r.stop);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventElapsedTime");
+        strncpy(names + 64 * n, r.name, 63);
+        names[64 * n + 63] = 0;
+        start_ms[n] = a; stop_ms[n] = b;
+        ++n;
+    }
+    *n_out = n;
+    c.prof.clear();
     return GEAR_OK;
 }
 

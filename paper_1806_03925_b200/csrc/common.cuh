@@ -149,6 +149,7 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 struct Profiler {
     struct Rec { const char* name; cudaEvent_t start, stop; };
     bool on = false;
+    bool keep_streams = false;     // timeline mode: events are recorded but the library keeps its side stream
     int64_t launches = 0;
     std::vector<Rec> recs;
     std::vector<cudaEvent_t> pool;

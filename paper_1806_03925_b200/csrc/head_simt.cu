@@ -566,7 +566,7 @@ static int splits_for(int M, int N, int K) {
 }
 
 // bf16 copies of the hidden layers' weights in both orientations (what the tensor-core products read).  Depends on
-// head_params only, so a step may run it on another stream beside the gather.
+// head_params only, so a step runs it ahead of the gather.
 cudaError_t launch_round_weights(const gear_ctx_impl& c, cudaStream_t st) {
     if (c.cfg.head_dtype != GEAR_BF16) return cudaSuccess;
     const int L = c.cfg.n_hidden;

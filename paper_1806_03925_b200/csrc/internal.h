@@ -84,7 +84,6 @@ struct gear_ctx_impl {
     mutable const int32_t* plan_src_row;
     mutable const float* plan_scale;
     cudaEvent_t ev_gather;              // the gather's outputs (row_view, inv_n) exist
-    cudaEvent_t ev_weights;             // the bf16 copies of the head's weights exist (made on the side stream)
     cudaEvent_t ev_dx;                  // dX exists: the embedding scatter may start on the side stream
     mutable int acc_calls_pending;      // accumulate calls enqueued since a collect that was sure to drain the queue
 
@@ -119,8 +118,7 @@ cudaError_t launch_gather(const gear_ctx_impl& c, const gear_batch& b, int32_t* 
                           void* x_debug, cudaStream_t st);
 
 // head_simt.cu: forward + backward of the head (fp32 FMA products, or the tensor-core products of head_tc.cu).
-// weights_ready: the bf16 copies of the weights have been made already (launch_round_weights on another stream, joined by
-// the caller).  after_dx(arg) is called once dX has been enqueued, before the last weight-gradient product.
+// weights_ready: the bf16 copies of the weights have been made already (launch_round_weights earlier on the same stream).  after_dx(arg) is called once dX has been enqueued, before the last weight-gradient product.
 struct HeadHooks { bool weights_ready; cudaError_t (*after_dx)(void*); void* arg; };
 cudaError_t launch_head_simt(const gear_ctx_impl& c, const gear_batch& b, const gear_step_out& o, cudaStream_t st,
                              const HeadHooks& hooks);

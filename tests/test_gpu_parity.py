@@ -568,6 +568,53 @@ def test_step_with_expiry_on_its_own_stream_matches_step_on_one_stream(gb):
             sess.close()
 
 
+def test_profiling_modes_leave_the_results_alone(gb):
+    """Per-kernel timing (every kernel alone on the caller's stream) and the timeline mode (the side stream stays)
+    bracket the same launches with events: the step's outputs are those of an unprofiled step, bit for bit where the
+    sums are taken in a fixed order, and the timeline lists every launch once, each with stop >= start >= 0."""
+    from gpu_harness import assert_close, _np
+    from paper_1806_03925_b200.session import DeviceBatch, GearSession
+    p = PRESETS["medium"].scaled(batch=2048, user_vocab=50_000, url_vocab=50_000, img_vocab=300_001, M=4)
+    src = BatchSource(p, 5)
+    batches = [src.batch(s) for s in range(3)]
+    max_nnz = max(b.nnz for b in batches)
+    sessions = [GearSession(p, workloads.head_params(p, 5), max_batch=p.batch, max_nnz=max_nnz, seed=5, fill=True, now=0,
+                            expired_cap=p.img_vocab) for _ in range(3)]
+    try:
+        gb.gear_profile_enable(sessions[1].ctx, True)
+        gb.gear_profile_enable(sessions[2].ctx, 2)
+        for s, b in enumerate(batches):
+            out = []
+            before = [gb.gear_launch_count(sess.ctx) for sess in sessions]
+            for sess in sessions:
+                n_ready, n_exp = sess.step(DeviceBatch.from_host(b), s + 1, sync=True, expiry_beside=False)
+                torch.cuda.synchronize()
+                out.append((n_ready, n_exp, _np(sess.ready_ids[:n_ready]), _np(sess.ready_seq[:n_ready]),
+                            _np(sess.ready_avg[:n_ready]), _np(sess.loss), _np(sess.head_grad), _np(sess.prob)))
+            launches = [gb.gear_launch_count(sess.ctx) - n0 for sess, n0 in zip(sessions, before)]
+            assert launches[0] == launches[1] == launches[2] > 0
+            for c in out[1:]:
+                a = out[0]
+                assert a[0] == c[0] and a[1] == c[1]
+                assert np.array_equal(a[2], c[2]) and np.array_equal(a[3], c[3]) and np.array_equal(a[7], c[7])
+                assert_close(c[4], a[4], 1e-5, "averaged gradients")
+                assert_close(c[5], a[5], 1e-5, "loss")
+                assert_close(c[6], a[6], 1e-4, "head gradient")          # split sums arrive in any order
+            per_kernel = gb.gear_profile_read(sessions[1].ctx, 64)
+            assert sum(v[1] for v in per_kernel.values()) == launches[1]
+            assert all(v[0] >= 0.0 for v in per_kernel.values())
+            timeline = gb.gear_profile_timeline(sessions[2].ctx, 256)
+            assert len(timeline) == launches[2]
+            assert sorted(k for k, _, _ in timeline) == sorted(k for k, v in per_kernel.items() for _ in range(v[1]))
+            assert all(t1 >= t0 >= 0.0 for _, t0, t1 in timeline)
+            assert gb.gear_profile_timeline(sessions[2].ctx, 256) == []         # reading clears the records
+        for sess in sessions:
+            assert sess.status()[1] == 0
+    finally:
+        for sess in sessions:
+            sess.close()
+
+
 # ------------------------------------------------------------------ refresh of cached DFVs
 @pytest.mark.parametrize("name", ["tiny", "medium"])
 def test_refresh_dfv_matches_oracle(gb, name):
