@@ -215,15 +215,6 @@ struct RowGather {
     const float* grads; int64_t ld; const int2* pmeta;      // pmeta[p] = (source row, scale bits) of sorted position p
 };
 
-// 16-byte asynchronous copy global -> shared; src_bytes = 0 reads nothing and fills the 16 bytes with zeros
-__device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void* gsrc, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(smem_dst), "l"(gsrc), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory");
-}
-
 // What a lane knows about "its" group of a span: own rows [start, start + len), then zlen rows from zstart.
 struct LaneGroup {
     uint32_t start, key, zstart;

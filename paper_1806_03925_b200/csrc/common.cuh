@@ -123,6 +123,15 @@ __device__ __forceinline__ void st_f4_hint(float* p, float4 v, uint64_t policy) 
                  :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy) : "memory");
 }
 
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 reads nothing and fills the 16 bytes with zeros
+__device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void* gsrc, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(smem_dst), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory");
+}
+
 // ---------------------------------------------------------------- programmatic dependent launch
 // The step is a chain of two dozen short kernels on one stream.  Launched this way, the blocks of a kernel may be
 // set up on SMs that the previous kernel in the stream has already left while its last blocks still run; every

@@ -350,6 +350,8 @@ head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict_
     __syncthreads();
     for (int b0 = (blockIdx.x * 8 + warp) * ROWS; b0 < B; b0 += gridDim.x * 8 * ROWS) {
         Raw8<TX> raw[ROWS][NQ];
+        // the label of this lane's view: asked for first, so that its latency passes while the rows are summed
+        const float y = b0 + my_row < B ? __ldg(label + b0 + my_row) : 0.f;
 #pragma unroll
         for (int j = 0; j < ROWS; ++j)
 #pragma unroll
@@ -388,7 +390,6 @@ head_out_kernel(int B, int H, const TX* __restrict__ h, const float* __restrict_
         zz += bias;
         const int b = b0 + my_row;
         const bool live = b < B;
-        const float y = live ? label[b] : 0.f;
         const float p = 1.0f / (1.0f + expf(-zz));
         const float g = live ? (p - y) / (float)B : 0.f;
         if (live && my_first) {
