@@ -32,7 +32,6 @@ namespace gear {
 constexpr int AF_THREADS = 256;
 constexpr int AF_ITEMS = 4;
 constexpr int AF_TILE = AF_THREADS * AF_ITEMS;
-constexpr int ACC_SPAN = 16;         // sorted positions per unit of work of the reduce pass (at most 32)
 
 __device__ __forceinline__ uint32_t warp_inclusive_max(uint32_t v) {
     const unsigned lane = lane_id();

@@ -85,7 +85,7 @@ int plan_workspace(const gear_config& c, WsPlan* p) {
     p->tile_cnt = take((size_t)(ceil_div(c.max_nnz, 1024) + 1) * sizeof(uint2));
     p->grp_rec = take((size_t)c.max_nnz * 16);
     p->pmeta = take((size_t)c.max_nnz * 8);
-    p->blk_first = take((size_t)(ceil_div(c.max_nnz, 16) + 2) * 4);
+    p->blk_first = take((size_t)(ceil_div(c.max_nnz, ACC_SPAN) + 2) * 4);
     p->run_end = take((size_t)c.max_nnz * 4);
     p->q_id = take((size_t)p->ready_cap * 4);
     p->q_avg = take((size_t)p->ready_cap * c.dfv_dim * 4);

@@ -193,6 +193,9 @@ struct KernelScope {
     ~KernelScope() { if (stop) cudaEventRecord(stop, st); }
 };
 
+// sorted positions per unit of work of the accumulate's reduce pass (at most 32); the workspace holds one word per span
+constexpr int ACC_SPAN = 16;
+
 // ---------------------------------------------------------------- radix sort / scans (prims.cu)
 constexpr int RS_THREADS = 256;
 constexpr int RS_ITEMS = 16;
