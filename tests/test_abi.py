@@ -66,3 +66,43 @@ def test_binding_refuses_host_tensors(gb):
     import torch
     with pytest.raises(TypeError):
         gb.gear_fill_uniform(torch.zeros((4, 4)), 0, 1)
+
+
+def test_struct_layouts_of_the_binding_match_the_header(gb, tmp_path):
+    """The ctypes structures of the binding against the C compiler's view of include/gear.h: same size, and every
+    field at the same offset (a field added to the header and not to the binding would shift everything behind it)."""
+    import shutil
+    import subprocess
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if cc is None:
+        pytest.skip("no C compiler")
+    structs = {"gear_config": gb.gear_config, "gear_buffers": gb.gear_buffers, "gear_batch": gb.gear_batch,
+               "gear_adam": gb.gear_adam, "gear_step_out": gb.gear_step_out}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "gear.h"', 'int main(void) {']
+    for name, st in structs.items():
+        lines.append('  printf("%s %%zu\\n", sizeof(%s));' % (name, name))
+        for field, _ in st._fields_:
+            lines.append('  printf("%s.%s %%zu\\n", offsetof(%s, %s));' % (name, field, name, field))
+    lines += ['  return 0;', '}']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines) + "\n")
+    exe = tmp_path / "layout"
+    subprocess.check_call([cc, "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    seen = dict(line.split() for line in subprocess.check_output([str(exe)], text=True).splitlines())
+    for name, st in structs.items():
+        assert int(seen[name]) == C.sizeof(st), name
+        for field, _ in st._fields_:
+            assert int(seen["%s.%s" % (name, field)]) == getattr(st, field).offset, "%s.%s" % (name, field)
+    # every field of the header's structures is known to the binding
+    text = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "gear.h")).read(), flags=re.S)
+    for name, st in structs.items():
+        body = re.search(r"typedef struct \{([^}]*)\}\s*%s;" % name, text).group(1)
+        fields = []
+        for decl in body.split(";"):
+            decl = decl.strip()
+            if not decl:
+                continue
+            names = decl.split(",")
+            names[0] = names[0].split()[-1]                      # drop the type of the first declarator
+            fields += [re.sub(r"\[.*\]", "", n).strip().lstrip("*").strip() for n in names]
+        assert fields == [f for f, _ in st._fields_], (name, fields)
