@@ -18,7 +18,9 @@
 // Two operand layouts:
 //   K-major   C[M][N] = A[M][K] . W[N][K]^T     (activations x weights; K contiguous in both)
 //   MN-major  C[M][N] += A[K][M]^T . B[K][N]    (weight gradients: the reduction runs over the batch,
-//                                                split across CTAs, partial tiles added with red.global)
+//                                                split across CTAs; a CTA's partial tile leaves like any
+//                                                fp32 output, in 32 x 32 blocks through shared memory, but
+//                                                as a TMA reduction: the copy engine adds it to the matrix)
 // No cluster launch and no multicast.  Every wait is bounded: on a timeout the kernel records an error
 // code, leaves its loops, frees its tensor memory and returns.
 #include <cuda.h>
@@ -46,7 +48,7 @@ template <int BN, int EW, int EPI> struct TcCfg {
     static constexpr int A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
     static constexpr int B_BYTES = BN * TC_BK * 2;               // 32 KB or 16 KB
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int OUT_BYTES = EPI == TC_EPI_RED ? 0 : EW * TC_OUT_BLOCK;       // one output block per epilogue warp
+    static constexpr int OUT_BYTES = EW * TC_OUT_BLOCK;       // one output block per epilogue warp
     static constexpr int MASK_BYTES = EPI == TC_EPI_MASK ? EW * 2 * TC_MASK_BLOCK : 0;
     static constexpr int COLSUM_BYTES = EPI == TC_EPI_MASK ? TC_MAX_N * 4 : 0;     // per-CTA column sums of the masked product
     static constexpr int FIXED = 1024 /*alignment slack*/ + 512 /*barriers*/ + COLSUM_BYTES + OUT_BYTES + MASK_BYTES;
@@ -122,6 +124,12 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, uint32_t src, int x, int y, uint64_t policy) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
                  :: "l"(map), "r"(src), "r"(x), "r"(y), "l"(policy) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// The same box added to the matrix instead of stored (fp32 adds by the copy engine, whole rows of the box at a time).
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 :: "l"(map), "r"(src), "r"(x), "r"(y) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 template <int PENDING>
@@ -230,7 +238,6 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
     static_assert(EPI == TC_EPI_F32 || EPI == TC_EPI_RED || CHUNKS % 2 == 0, "bf16 output leaves in blocks of 64 columns");
     const int m0 = mt * TC_BM + quarter * 32;         // first row of this warp's block
     const int m = m0 + lane;
-    const bool row_ok = m < g.M;
     const int rows = min(32, max(0, g.M - m0));
     const int col0 = nt * BN + part * COLS;
     const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN + part * COLS);
@@ -338,16 +345,6 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
                     }
                 }
             }
-        } else if (EPI == TC_EPI_RED) {
-            if (row_ok) {
-                float* dst = static_cast<float*>(g.out) + (int64_t)m * g.ldo + n0;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (n0 + 4 * j >= g.N) continue;
-                    red_add_f4(dst + 4 * j, make_float4(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1]),
-                                                        __uint_as_float(acc[4 * j + 2]), __uint_as_float(acc[4 * j + 3])));
-                }
-            }
         } else {
             // fp32 output (dX): one block per 32 columns; it is read again right
             // after (embedding and DFV gradients): ask the L2 to keep it
@@ -360,7 +357,11 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& g, const CUtensorMap
                 sts_u4(row_addr + (((uint32_t)j ^ swz) << 4), make_uint4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]));
             fence_async_smem();
             __syncwarp();
-            if (lane == 0) tma_store_2d_hint(map_out, buf, n0, m0, keep_policy);
+            if (lane == 0) {
+                // a slice's partial tile of a weight gradient is added to the matrix by the copy engine
+                if (EPI == TC_EPI_RED) tma_reduce_add_2d(map_out, buf, n0, m0);
+                else tma_store_2d_hint(map_out, buf, n0, m0, keep_policy);
+            }
         }
     }
 }
@@ -399,7 +400,7 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUt
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" :: "l"(&map_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" :: "l"(&map_b) : "memory");
-        if (EPI != TC_EPI_RED) asm volatile("prefetch.tensormap [%0];" :: "l"(&map_out) : "memory");
+        asm volatile("prefetch.tensormap [%0];" :: "l"(&map_out) : "memory");
         if (EPI == TC_EPI_MASK) asm volatile("prefetch.tensormap [%0];" :: "l"(&map_mask) : "memory");
     }
     if (EPI == TC_EPI_MASK && g.colsum != nullptr)
@@ -517,7 +518,7 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& map_a, const CUt
             tc_fence_before();
             mbar_arrive_relaxed(acc_empty(a));                   // all epilogue threads arrive: the buffer returns to the MMA warp
         }
-        if (EPI != TC_EPI_RED && lane == 0) tma_store_wait_all();   // this warp's stores have left shared memory and landed
+        if (lane == 0) tma_store_wait_all();   // this warp's stores have left shared memory and landed
         if (EPI == TC_EPI_MASK && mp.pending) {
             // leaving early: let the mask copies already issued land before the CTA gives its shared memory back
             for (int h = 0; h < 2; ++h)
@@ -708,8 +709,9 @@ cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int 
                             cudaStream_t st) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     const int bn = N > 128 ? 256 : 128;
-    CUtensorMap ma, mb;
-    if (!make_map(&ma, A, K, M, lda, 64) || !make_map(&mb, Bm, K, N, ldb, 64)) return cudaErrorInvalidValue;
+    CUtensorMap ma, mb, mo;
+    if (!make_map(&ma, A, K, M, lda, 64) || !make_map(&mb, Bm, K, N, ldb, 64) || !make_map_f32(&mo, out, M, N, ldo, 32))
+        return cudaErrorInvalidValue;
     TcArgs g;
     g.M = M; g.N = N; g.K = K;
     g.m_tiles = (int)ceil_div(M, TC_BM); g.n_tiles = (int)ceil_div(N, bn);
@@ -722,7 +724,7 @@ cudaError_t tc_gemm_mnmajor(Profiler* prof, const char* name, int M, int N, int 
     g.k_splits = (int)ceil_div(total_kb, g.kb_per_split);
     g.out = out; g.ldo = ldo; g.bias = nullptr; g.mask = nullptr; g.ldm = 0; g.colsum = nullptr; g.err = err;
     KernelScope ks(prof, name, st);
-    return launch_bn<true, TC_EPI_RED>(bn, ma, mb, ma /*unused: partial tiles are added with red.global*/, ma /*unused*/, g, st);
+    return launch_bn<true, TC_EPI_RED>(bn, ma, mb, mo, ma /*unused*/, g, st);
 }
 
 }  // namespace gear
