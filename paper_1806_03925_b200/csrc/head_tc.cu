@@ -55,7 +55,7 @@ template <int BN, int EW, int EPI> struct TcCfg {
     static constexpr int ROOM = (227 * 1024 - FIXED) / STAGE_BYTES;
     static constexpr int STAGES = ROOM > (BN == 256 ? 4 : 6) ? (BN == 256 ? 4 : 6) : ROOM;
     static constexpr int SMEM = STAGES * STAGE_BYTES + FIXED;
-    static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
+    static constexpr int TMEM_COLS = BN == 192 ? 512 : 2 * BN;   // two accumulator buffers (a power of two is allocated)
     static_assert(STAGES >= 3, "operand ring too short");
     static_assert(SMEM > 116 * 1024, "one CTA per SM: two CTAs would both ask for tensor memory");
     static_assert(SMEM <= 227 * 1024, "shared memory budget");
@@ -680,7 +680,9 @@ cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K
                            const __nv_bfloat16* W, int64_t ldw, int epi, void* out, int64_t ldo, const float* bias,
                            const __nv_bfloat16* mask, int64_t ldm, float* colsum, int32_t* err, cudaStream_t st) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
-    const int bn = N > 128 ? 256 : 128;
+    // column tiles of 256 or 128; the fp32 output (dX) also has 192, which fits a width like 384 without a half-empty tile
+    int bn = N > 128 ? 256 : 128;
+    if (epi == TC_EPI_F32 && N > 128 && ceil_div(N, 192) * 192 < ceil_div(N, 256) * 256) bn = 192;
     CUtensorMap ma, mb, mo;
     if (!make_map(&ma, A, M, K, lda, TC_BM) || !make_map(&mb, W, N, K, ldw, bn)) return cudaErrorInvalidValue;
     // the output leaves in boxes of 32 rows x 128 bytes
@@ -700,7 +702,9 @@ cudaError_t tc_gemm_kmajor(Profiler* prof, const char* name, int M, int N, int K
         if (!mask || !make_map_mask(&mm, mask, M, N, ldm)) return cudaErrorInvalidValue;
         return launch_bn<false, TC_EPI_MASK>(bn, ma, mb, mo, mm, g, st);
     }
-    default: return launch_bn<false, TC_EPI_F32>(bn, ma, mb, mo, ma /*unused*/, g, st);
+    default:
+        if (bn == 192) return launch_variant<192, false, TC_EPI_F32, 8>(ma, mb, mo, ma /*unused*/, g, st);
+        return launch_bn<false, TC_EPI_F32>(bn, ma, mb, mo, ma /*unused*/, g, st);
     }
 }
 
