@@ -165,7 +165,7 @@ def kernel_models(p, stats):
 NCU_TRAFFIC_LARGE_2M = {
     "gather_pool": (64.1e6, "l2"), "acc_reduce": (238.0e6, "work"), "expiry_mark": (16.0e6, "vocab"),
     "head_out": (34.5e6, None), "emb_reduce": (46.9e6, "work"),
-    "tc_gemm_fwd": (69.0e6, None), "tc_gemm_dw": (113.6e6, None), "tc_gemm_dh": (130.4e6, None), "tc_gemm_dx": (110.1e6, None),
+    "tc_gemm_fwd": (69.0e6, None), "tc_gemm_dw": (113.6e6, None), "tc_gemm_dh": (130.4e6, None), "tc_gemm_dx": (110.3e6, None),
 }
 # algorithmic bytes per launch of the table-bound kernels on large_2m (kernel_models on that workload's batches)
 NCU_WORK_LARGE_2M = {"gather_pool": 222.0e6, "acc_reduce": 224.5e6, "emb_reduce": 58.9e6}
