@@ -117,6 +117,8 @@ def test_skew_shapes_ragged_batch(gb):
     (F32, (64,), 8, 512, F32, 100),
     (F32, (64,), 8, 1024, F32, 40),
     (BF16, (64,), 8, 1024, BF16, 40),
+    # a 1024-wide layer on top of a 320-wide one, 3000 views: thousands of units inside the ReLU rounding band
+    (BF16, (320, 1024), 20, 512, BF16, 3000),
 ])
 def test_odd_head_shapes(gb, head, hidden, E, D, dfv, B):
     p = PRESETS["medium"].scaled(emb_dim=E, dfv_dim=D, dfv_dtype=dfv, head_dtype=head, hidden=hidden, M=3,
